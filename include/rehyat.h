@@ -1,0 +1,153 @@
+/*
+ * rehyat.h - C ABI of the ReHyAt recurrent hybrid attention operator for NVIDIA B200 (sm_100a).
+ *
+ * The operator (paper Section 3.2 "Hybrid Attention Formulation" and Section 3.3 "Recurrent
+ * HyAt"): N = frames*H*W tokens of a video latent are cut into temporal chunks of `chunk`
+ * frames.  A query i of chunk t attends
+ *   - with exact softmax weights exp(q_i.k_j/sqrt(head_dim) - c_i) to the keys of its window
+ *     TS_t = [max(t*N' - overlap*H*W, 0), min((t+1)*N', N)),  N' = chunk*H*W       (Eq. 12/13)
+ *   - with linear-attention weights phi_q(q_i).phi_k(k_j) to every earlier key
+ *     TL_t = [0, max(t*N' - overlap*H*W, 0))                                          (Eq. 13)
+ * and the output is  y_i = (aS_i + aL_i) / (nS_i + nL_i)                          (Eq. 5-9),
+ * the linear sums being carried from chunk to chunk as the state
+ *   s_t = sum_{j in TL_t} phi_k(k_j) v_j^T,   z_t = sum_{j in TL_t} phi_k(k_j)    (Eq. 14-18).
+ * phi_q, phi_k (Section 3.2 "Characterization of phi", Appendix "Training Details"): per-head
+ * two-layer MLP u = act_out(W2 act_hidden(W1 x + b1) + b2), u split into poly_degree equal
+ * contiguous parts, part p (1-based) raised element-wise to the power p, parts concatenated.
+ *
+ * Conventions
+ *   - All functions return REHYAT_OK (0) or a negative REHYAT_ERR_* code; nothing throws.
+ *   - Unless a parameter says "host", tensor pointers are DEVICE pointers owned by the caller,
+ *     16-byte aligned, and `out` must not alias an input.
+ *   - rehyat_forward only enqueues work on the given stream: no host synchronisation and no
+ *     allocation.  A context serves one stream at a time (it owns the workspace).
+ *   - There is no CPU fallback: on a machine without an sm_100 device rehyat_create fails.
+ */
+#ifndef REHYAT_H
+#define REHYAT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define REHYAT_OK                   0
+#define REHYAT_ERR_INVALID_ARG     -1   /* null / misaligned pointer, size out of range        */
+#define REHYAT_ERR_UNSUPPORTED     -2   /* legal request this build has no kernel for          */
+#define REHYAT_ERR_CUDA            -3   /* a CUDA runtime or driver call failed                */
+#define REHYAT_ERR_ARCH            -4   /* the device is not compute capability 10.x           */
+#define REHYAT_ERR_ALLOC           -5   /* workspace allocation failed                         */
+#define REHYAT_ERR_DEVICE_TIMEOUT  -6   /* a bounded wait inside a kernel ran out (see status) */
+
+typedef enum { REHYAT_DTYPE_BF16 = 0, REHYAT_DTYPE_FP32 = 1 } rehyat_dtype;
+
+/* Activations of the phi MLP.  The paper names none; ReLU/ReLU is the default reading. */
+typedef enum {
+  REHYAT_ACT_RELU = 0, REHYAT_ACT_IDENTITY = 1, REHYAT_ACT_SOFTPLUS = 2,
+  REHYAT_ACT_ELU1 = 3 /* 1 + elu(x) */, REHYAT_ACT_GELU = 4 /* erf form */
+} rehyat_act;
+
+/* The stabilising constant c of Eq. 6 and 8.  It is NOT applied to the linear terms (Eq. 7, 9),
+ * so the result depends on it.  ROWMAX: c_i = max over the window of the scaled logits of row i
+ * ("typically the maximum exponent").  ZERO: c = 0 (evaluated stably). */
+typedef enum { REHYAT_C_ROWMAX = 0, REHYAT_C_ZERO = 1 } rehyat_c_mode;
+
+/* Kernel family.  AUTO: tensor-core (tcgen05) kernels when dtype is bf16 and the shape is one
+ * they cover, SIMT fp32 kernels otherwise.  SIMT / TENSOR force one (TENSOR fails with
+ * REHYAT_ERR_UNSUPPORTED where it does not apply). */
+typedef enum { REHYAT_IMPL_AUTO = 0, REHYAT_IMPL_SIMT = 1, REHYAT_IMPL_TENSOR = 2 } rehyat_impl;
+
+typedef struct rehyat_config {
+  int32_t device;               /* CUDA device ordinal                                        */
+  int32_t dtype;                /* rehyat_dtype of q, k, v, out and the phi parameters        */
+  int32_t n_heads;
+  int32_t head_dim;             /* d: 64 or 128                                               */
+  int32_t phi_hidden;           /* D_h, hidden width of the phi MLP (<= 256, multiple of 8)   */
+  int32_t phi_dim;              /* D', output width of phi (<= 256, divisible by poly_degree) */
+  int32_t poly_degree;          /* P in 1..4                                                  */
+  int32_t act_hidden;           /* rehyat_act                                                 */
+  int32_t act_out;              /* rehyat_act                                                 */
+  int32_t c_mode;               /* rehyat_c_mode                                              */
+  int32_t impl;                 /* rehyat_impl                                                */
+  int32_t max_batch;            /* largest `batch` a forward call may pass                    */
+  int32_t max_tokens_per_frame; /* largest H*W                                                */
+  int32_t max_chunk_frames;     /* largest `chunk`                                            */
+  int32_t group_tokens;         /* 0 = default.  Queries per (batch, head) that one pass over
+                                   a group of chunks handles; the workspace grows with it and
+                                   with max_chunk_frames*max_tokens_per_frame, never with
+                                   `frames`.                                                  */
+} rehyat_config;
+
+/* Element strides of q, k, v and out (all four share them); the head_dim axis is contiguous.
+ * [B, n_heads, N, d] contiguous: {n_heads*N*d, N*d, d};  [B, N, n_heads, d]: {N*n_heads*d, d,
+ * n_heads*d}.  Each stride times the element size must be a multiple of 16 bytes. */
+typedef struct rehyat_layout {
+  int64_t stride_batch;
+  int64_t stride_head;
+  int64_t stride_token;
+} rehyat_layout;
+
+/* Device pointers to the parameters of phi_q and phi_k in the operator dtype, row-major:
+ * W1 [n_heads, D_h, d], b1 [n_heads, D_h], W2 [n_heads, D', D_h], b2 [n_heads, D']. */
+typedef struct rehyat_phi_params {
+  const void* q_W1; const void* q_b1; const void* q_W2; const void* q_b2;
+  const void* k_W1; const void* k_b1; const void* k_W2; const void* k_b2;
+} rehyat_phi_params;
+
+typedef struct rehyat_ctx rehyat_ctx;
+
+/* Creates a context on cfg->device and allocates its fixed workspace (chunk states, partial
+ * state sums, the linear read-out of one chunk group, a status word).  The workspace size is a
+ * function of the config only (Section 3.3, note 3: memory constant in the video length).
+ * Errors: INVALID_ARG (null, sizes out of range), UNSUPPORTED, ARCH, CUDA, ALLOC. */
+int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg);
+
+/* Enqueues the operator of Eq. 5-9 with the causal sets of Eq. 13 on `cuda_stream`
+ * (a cudaStream_t passed as void*; NULL is the default stream).
+ *   q, k, v  device, [batch, n_heads, frames*H*W, head_dim] through `lay`, read only
+ *   out      device, same shape and strides, written
+ *   H, W     the latent patch grid (tokens per frame = H*W), not attention heads
+ *   chunk    T_c >= 1 frames per chunk; frames need not be a multiple (the last chunk is short)
+ *   overlap  T_o >= 0 frames of overlap; any value is legal, the window is clamped at token 0
+ * Validation failures return INVALID_ARG before anything is enqueued.  Asynchronous errors
+ * (a bounded device wait that ran out) are reported by rehyat_status. */
+int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void* out,
+                   const rehyat_layout* lay, const rehyat_phi_params* phi,
+                   int32_t batch, int32_t frames, int32_t H, int32_t W,
+                   int32_t chunk, int32_t overlap, void* cuda_stream);
+
+/* Same operator with q, k, v, out in HOST memory as contiguous [batch, n_heads, N, head_dim]
+ * (pinned memory makes the copies asynchronous).  Copies the inputs to device staging buffers
+ * owned by the context (grown on demand: the one allocation whose size follows N, because it
+ * holds the tensors themselves), runs rehyat_forward, copies `out` back and synchronises the
+ * stream.  `phi` stays device-resident. */
+int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host,
+                        const void* v_host, void* out_host, const rehyat_phi_params* phi,
+                        int32_t batch, int32_t frames, int32_t H, int32_t W,
+                        int32_t chunk, int32_t overlap, void* cuda_stream);
+
+/* Frees the workspace.  NULL is a no-op returning REHYAT_OK. */
+int rehyat_destroy(rehyat_ctx* ctx);
+
+/* Bytes of device workspace the context holds (staging of rehyat_forward_host excluded). */
+size_t rehyat_workspace_bytes(const rehyat_ctx* ctx);
+
+/* Synchronises `cuda_stream`, reads the device status word and clears it.  Returns REHYAT_OK,
+ * REHYAT_ERR_DEVICE_TIMEOUT or REHYAT_ERR_CUDA. */
+int rehyat_status(rehyat_ctx* ctx, void* cuda_stream);
+
+/* Number of kernel launches the last rehyat_forward on this context enqueued. */
+int rehyat_last_launches(const rehyat_ctx* ctx);
+
+/* 1 if the last forward ran the tensor-core kernels, 0 for the SIMT kernels. */
+int rehyat_last_impl(const rehyat_ctx* ctx);
+
+const char* rehyat_strerror(int code);
+int rehyat_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REHYAT_H */

@@ -1,0 +1,167 @@
+"""Thin ctypes binding of librehyat.so (include/rehyat.h).  Argument marshalling only: every step
+of the operator runs inside the library's CUDA kernels.  PyTorch supplies device memory and
+streams, nothing else.  There is no fallback: a missing library raises."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "librehyat.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_ARCH, ERR_ALLOC, ERR_DEVICE_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
+DTYPE = {"bf16": 0, "fp32": 1}
+ACT = {"relu": 0, "identity": 1, "softplus": 2, "elu1": 3, "gelu": 4}
+C_MODE = {"rowmax": 0, "zero": 1}
+IMPL = {"auto": 0, "simt": 1, "tensor": 2}
+
+EXPORTS = ["rehyat_create", "rehyat_forward", "rehyat_forward_host", "rehyat_destroy",
+           "rehyat_workspace_bytes", "rehyat_status", "rehyat_last_launches", "rehyat_last_impl",
+           "rehyat_strerror", "rehyat_version"]
+
+
+class Config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "device", "dtype", "n_heads", "head_dim", "phi_hidden", "phi_dim", "poly_degree", "act_hidden",
+        "act_out", "c_mode", "impl", "max_batch", "max_tokens_per_frame", "max_chunk_frames", "group_tokens")]
+
+
+class Layout(C.Structure):
+    _fields_ = [("stride_batch", C.c_int64), ("stride_head", C.c_int64), ("stride_token", C.c_int64)]
+
+
+class PhiParams(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("q_W1", "q_b1", "q_W2", "q_b2", "k_W1", "k_b1", "k_W2", "k_b2")]
+
+
+_lib = None
+
+
+def lib():
+    """Loads librehyat.so on first use.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2601_04342_b200.build`; "
+                               "there is no fallback path")
+        L = C.CDLL(LIB_PATH)
+        L.rehyat_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(Config)]
+        L.rehyat_forward.argtypes = [C.c_void_p] + [C.c_void_p] * 4 + [C.POINTER(Layout), C.POINTER(PhiParams)] + \
+            [C.c_int32] * 6 + [C.c_void_p]
+        L.rehyat_forward_host.argtypes = [C.c_void_p] + [C.c_void_p] * 4 + [C.POINTER(PhiParams)] + \
+            [C.c_int32] * 6 + [C.c_void_p]
+        L.rehyat_destroy.argtypes = [C.c_void_p]
+        L.rehyat_workspace_bytes.argtypes = [C.c_void_p]
+        L.rehyat_workspace_bytes.restype = C.c_size_t
+        L.rehyat_status.argtypes = [C.c_void_p, C.c_void_p]
+        L.rehyat_last_launches.argtypes = [C.c_void_p]
+        L.rehyat_last_impl.argtypes = [C.c_void_p]
+        L.rehyat_strerror.argtypes = [C.c_int]
+        L.rehyat_strerror.restype = C.c_char_p
+        for name in EXPORTS:
+            if getattr(L, name).restype is None:
+                getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+class RehyatError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {lib().rehyat_strerror(code).decode()} ({code})")
+
+
+def _check(code, where):
+    if code != OK:
+        raise RehyatError(code, where)
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p(None)
+
+
+class Rehyat:
+    """One operator context (rehyat_create ... rehyat_destroy)."""
+
+    def __init__(self, *, n_heads, head_dim, dtype="bf16", phi_hidden=None, phi_dim=None, poly_degree=2,
+                 act_hidden="relu", act_out="relu", c_mode="rowmax", impl="auto", max_batch=1,
+                 max_tokens_per_frame=1560, max_chunk_frames=3, group_tokens=0, device=0):
+        self.cfg = Config(device, DTYPE[dtype], n_heads, head_dim, phi_hidden or 2 * head_dim,
+                          phi_dim or 2 * head_dim, poly_degree, ACT[act_hidden], ACT[act_out], C_MODE[c_mode],
+                          IMPL[impl], max_batch, max_tokens_per_frame, max_chunk_frames, group_tokens)
+        self.dtype = dtype
+        self._h = C.c_void_p(None)
+        _check(lib().rehyat_create(C.byref(self._h), C.byref(self.cfg)), "rehyat_create")
+
+    def close(self):
+        if self._h:
+            lib().rehyat_destroy(self._h)
+            self._h = C.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def workspace_bytes(self):
+        return lib().rehyat_workspace_bytes(self._h)
+
+    @property
+    def last_launches(self):
+        return lib().rehyat_last_launches(self._h)
+
+    @property
+    def last_impl(self):
+        return "tensor" if lib().rehyat_last_impl(self._h) else "simt"
+
+    @staticmethod
+    def phi_struct(phi_q, phi_k):
+        return PhiParams(*[_ptr(phi_q[n]) for n in ("W1", "b1", "W2", "b2")],
+                         *[_ptr(phi_k[n]) for n in ("W1", "b1", "W2", "b2")])
+
+    def forward(self, q, k, v, phi_q, phi_k, frames, H, W, chunk, overlap, out=None, layout="bhnd", stream=None):
+        """q, k, v: CUDA tensors [B, n_heads, N, d] ("bhnd") or [B, N, n_heads, d] ("bnhd"), contiguous.
+        Returns `out` (same shape).  Asynchronous on `stream` (default: torch's current stream)."""
+        if out is None:
+            out = torch.empty_like(q)
+        if layout == "bhnd":
+            B, nh, N, d = q.shape
+            lay = Layout(nh * N * d, N * d, d)
+        elif layout == "bnhd":
+            B, N, nh, d = q.shape
+            lay = Layout(N * nh * d, d, nh * d)
+        else:
+            raise ValueError(layout)
+        for t in (q, k, v, out):
+            if not (t.is_cuda and t.is_contiguous() and t.shape == q.shape):
+                raise ValueError("q, k, v, out must be contiguous CUDA tensors of one shape")
+        st = stream if stream is not None else torch.cuda.current_stream(q.device)
+        phi = self.phi_struct(phi_q, phi_k)
+        _check(lib().rehyat_forward(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), C.byref(lay), C.byref(phi),
+                                    B, frames, H, W, chunk, overlap, C.c_void_p(st.cuda_stream)), "rehyat_forward")
+        return out
+
+    def forward_host(self, q, k, v, out, phi_q, phi_k, frames, H, W, chunk, overlap, stream=None):
+        """q, k, v, out: CPU tensors [B, n_heads, N, d] (pinned for asynchronous copies); phi on the device.
+        Returns after `out` has been filled."""
+        B = q.shape[0]
+        st = stream if stream is not None else torch.cuda.current_stream(self.cfg.device)
+        phi = self.phi_struct(phi_q, phi_k)
+        _check(lib().rehyat_forward_host(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), C.byref(phi), B, frames, H,
+                                         W, chunk, overlap, C.c_void_p(st.cuda_stream)), "rehyat_forward_host")
+        return out
+
+    def status(self, stream=None):
+        st = stream if stream is not None else torch.cuda.current_stream(self.cfg.device)
+        return lib().rehyat_status(self._h, C.c_void_p(st.cuda_stream))
+
+
+def for_workload(wl, **kw):
+    """A context sized for a synth.Workload."""
+    args = dict(n_heads=wl.n_heads, head_dim=wl.head_dim, dtype=wl.dtype, phi_hidden=wl.D_h, phi_dim=wl.D_out,
+                poly_degree=wl.P, max_batch=wl.B, max_tokens_per_frame=wl.HW, max_chunk_frames=min(wl.Tc, wl.T))
+    args.update(kw)
+    return Rehyat(**args)

@@ -1,0 +1,320 @@
+// Host side of the C ABI declared in include/rehyat.h: argument validation, the fixed
+// workspace, the chunk-group schedule and the kernel launches.
+//
+// Schedule of one forward call.  The T' chunks are walked in groups of G consecutive chunks
+// (G*N' <= the read-out rows the workspace holds), so the workspace does not grow with the
+// number of frames (Section 3.3, note 3).  Per group:
+//   1. state increments: sum of phi_k(k_j)[v_j|1] over the keys each chunk newly admits (Eq. 17-18)
+//   2. scan along the chunk axis, carrying the last state of the previous group (Eq. 14-15)
+//   3. linear read-out phi_q(Q_t) s_t, phi_q(Q_t) z_t of the group's queries (Eq. 7, 9, 16)
+//   4. softmax window (Eq. 6, 8) and the joint normalisation (Eq. 5), writing y.
+#include <cuda_runtime.h>
+
+#include <climits>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "../../include/rehyat.h"
+#include "rehyat_common.cuh"
+#include "rehyat_simt.cuh"
+#include "rehyat_tc.cuh"
+
+using namespace rehyat;
+
+struct rehyat_ctx {
+  rehyat_config cfg;
+  float* state = nullptr;      // [Gmax][BHmax][Dp][d+4]
+  float* partial = nullptr;    // [partial_units][BHmax][Dp][d+4]
+  float* readout = nullptr;    // [BHmax][rd_rows][d+4]
+  int* status_dev = nullptr;
+  TcWorkspace tc;              // extra buffers of the tensor-core path
+  size_t ws_bytes = 0;
+  int Gmax = 0, partial_units = 0, rd_rows = 0, bh_max = 0;
+  void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
+  size_t stage_bytes = 0;
+  int last_launches = 0, last_impl = 0;
+  bool tensor_ok = false;
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+inline size_t elem_size(int dtype) { return dtype == REHYAT_DTYPE_FP32 ? 4 : 2; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_config(const rehyat_config* c) {
+  if (c->dtype != REHYAT_DTYPE_BF16 && c->dtype != REHYAT_DTYPE_FP32) return REHYAT_ERR_INVALID_ARG;
+  if (c->n_heads < 1 || c->n_heads > 1024) return REHYAT_ERR_INVALID_ARG;
+  if (c->max_batch < 1 || (long long)c->max_batch * c->n_heads > 65535) return REHYAT_ERR_INVALID_ARG;
+  if (c->poly_degree < 1 || c->poly_degree > 4) return REHYAT_ERR_INVALID_ARG;
+  if (c->phi_hidden < 8 || c->phi_hidden > 256 || c->phi_hidden % 8) return REHYAT_ERR_INVALID_ARG;
+  if (c->phi_dim < 8 || c->phi_dim > 256 || c->phi_dim % 8 || c->phi_dim % c->poly_degree)
+    return REHYAT_ERR_INVALID_ARG;
+  if (c->act_hidden < 0 || c->act_hidden > 4 || c->act_out < 0 || c->act_out > 4) return REHYAT_ERR_INVALID_ARG;
+  if (c->c_mode != REHYAT_C_ROWMAX && c->c_mode != REHYAT_C_ZERO) return REHYAT_ERR_INVALID_ARG;
+  if (c->impl < REHYAT_IMPL_AUTO || c->impl > REHYAT_IMPL_TENSOR) return REHYAT_ERR_INVALID_ARG;
+  if (c->max_tokens_per_frame < 1 || c->max_chunk_frames < 1 || c->group_tokens < 0) return REHYAT_ERR_INVALID_ARG;
+  if ((long long)c->max_tokens_per_frame * c->max_chunk_frames > (1 << 24)) return REHYAT_ERR_INVALID_ARG;
+  if (c->head_dim < 1) return REHYAT_ERR_INVALID_ARG;
+  if (c->head_dim != 64 && c->head_dim != 128) return REHYAT_ERR_UNSUPPORTED;
+  return REHYAT_OK;
+}
+
+template <typename T, int D>
+int set_simt_attributes(const rehyat_config& c) {
+  const int smem_state = SIMT_TM * (2 * D + c.phi_hidden + c.phi_dim) * (int)sizeof(float);
+  const int smem_rd = SIMT_TM * (D + c.phi_hidden + c.phi_dim) * (int)sizeof(float);
+  const int smem_win = (WIN_BM * (D + 4) + WIN_BN * (D + 4) + WIN_BN * D + WIN_BM * (WIN_BN + 4)) * (int)sizeof(float);
+  if (cudaFuncSetAttribute(state_partial_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_state) != cudaSuccess ||
+      cudaFuncSetAttribute(readout_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_rd) != cudaSuccess ||
+      cudaFuncSetAttribute(window_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_win) != cudaSuccess)
+    return REHYAT_ERR_CUDA;
+  return REHYAT_OK;
+}
+
+template <typename T, int D>
+int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* out, const rehyat_phi_params* phi,
+                      const Geo& g, int n_split, int carry_slot, bool any_linear, cudaStream_t st) {
+  const rehyat_config& c = ctx->cfg;
+  PhiDims pd = {D, c.phi_hidden, c.phi_dim, c.poly_degree, c.act_hidden, c.act_out};
+  constexpr int SD = D + 4;
+  const int tiles = (g.Np + SIMT_TM - 1) / SIMT_TM;
+  if (any_linear) {
+    PhiPtrs<T> wk = {(const T*)phi->k_W1, (const T*)phi->k_b1, (const T*)phi->k_W2, (const T*)phi->k_b2};
+    PhiPtrs<T> wq = {(const T*)phi->q_W1, (const T*)phi->q_b1, (const T*)phi->q_W2, (const T*)phi->q_b2};
+    const size_t smem_state = (size_t)SIMT_TM * (2 * D + pd.Dh + pd.Dp) * sizeof(float);
+    state_partial_simt<T, D><<<dim3(n_split, g.G, g.BH), SIMT_PHI_THREADS, smem_state, st>>>(
+        k, v, wk, pd, g, n_split, ctx->partial);
+    const size_t per_slot = (size_t)g.BH * pd.Dp * SD;
+    scan_states<<<(unsigned)((per_slot + 255) / 256), 256, 0, st>>>(ctx->partial, ctx->state, per_slot, g.G,
+                                                                     n_split, carry_slot);
+    const size_t smem_rd = (size_t)SIMT_TM * (D + pd.Dh + pd.Dp) * sizeof(float);
+    readout_simt<T, D><<<dim3(tiles, g.G, g.BH), SIMT_PHI_THREADS, smem_rd, st>>>(q, wq, pd, g, ctx->state,
+                                                                                 ctx->readout, ctx->rd_rows);
+    ctx->last_launches += 3;
+  }
+  const size_t smem_win = (size_t)(WIN_BM * (D + 4) + WIN_BN * (D + 4) + WIN_BN * D + WIN_BM * (WIN_BN + 4)) * sizeof(float);
+  const int wtiles = (g.Np + WIN_BM - 1) / WIN_BM;
+  window_simt<T, D><<<dim3(wtiles, g.G, g.BH), WIN_THREADS, smem_win, st>>>(
+      q, k, v, out, g, ctx->readout, ctx->rd_rows, 1.0f / sqrtf((float)D), c.c_mode);
+  ctx->last_launches += 1;
+  return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int rehyat_version(void) { return 100; }
+
+const char* rehyat_strerror(int code) {
+  switch (code) {
+    case REHYAT_OK: return "ok";
+    case REHYAT_ERR_INVALID_ARG: return "invalid argument";
+    case REHYAT_ERR_UNSUPPORTED: return "unsupported shape or mode";
+    case REHYAT_ERR_CUDA: return "CUDA call failed";
+    case REHYAT_ERR_ARCH: return "device is not compute capability 10.x (sm_100)";
+    case REHYAT_ERR_ALLOC: return "device allocation failed";
+    case REHYAT_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    default: return "unknown error code";
+  }
+}
+
+int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
+  if (!out || !cfg) return REHYAT_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = check_config(cfg);
+  if (rc != REHYAT_OK) return rc;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess) { cudaGetLastError(); return REHYAT_ERR_CUDA; }
+  if (cfg->device < 0 || cfg->device >= ndev) return REHYAT_ERR_INVALID_ARG;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return REHYAT_ERR_CUDA;
+  if (prop.major != 10) return REHYAT_ERR_ARCH;
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) return REHYAT_ERR_CUDA;
+
+  rehyat_ctx* ctx = new (std::nothrow) rehyat_ctx();
+  if (!ctx) return REHYAT_ERR_ALLOC;
+  ctx->cfg = *cfg;
+  const rehyat_config& c = ctx->cfg;
+  ctx->tensor_ok = tc_shape_supported(c.dtype == REHYAT_DTYPE_BF16, c.head_dim, c.phi_hidden, c.phi_dim,
+                                      c.poly_degree, c.act_hidden, c.act_out);
+  if (c.impl == REHYAT_IMPL_TENSOR && !ctx->tensor_ok) { delete ctx; return REHYAT_ERR_UNSUPPORTED; }
+  if (c.impl == REHYAT_IMPL_SIMT) ctx->tensor_ok = false;
+
+  const int np_max = c.max_tokens_per_frame * c.max_chunk_frames;
+  const int want = c.group_tokens > 0 ? c.group_tokens : 32768;
+  ctx->rd_rows = ((want > np_max ? want : np_max) + 127) / 128 * 128 + 128;
+  ctx->Gmax = 16;
+  ctx->partial_units = 32;
+  ctx->bh_max = c.max_batch * c.n_heads;
+  const size_t SD = c.head_dim + 4;
+  const size_t slot = (size_t)ctx->bh_max * c.phi_dim * SD * sizeof(float);
+  const size_t b_state = slot * ctx->Gmax, b_partial = slot * ctx->partial_units;
+  const size_t b_rd = (size_t)ctx->bh_max * ctx->rd_rows * SD * sizeof(float);
+  bool ok = cudaMalloc(&ctx->state, b_state) == cudaSuccess && cudaMalloc(&ctx->partial, b_partial) == cudaSuccess &&
+            cudaMalloc(&ctx->readout, b_rd) == cudaSuccess && cudaMalloc(&ctx->status_dev, 256) == cudaSuccess;
+  ctx->ws_bytes = b_state + b_partial + b_rd + 256;
+  if (ok && ctx->tensor_ok) {
+    size_t extra = 0;
+    ok = tc_workspace_create(&ctx->tc, ctx->bh_max, ctx->Gmax, c.head_dim, c.phi_dim, &extra);
+    ctx->ws_bytes += extra;
+  }
+  if (!ok) { cudaGetLastError(); rehyat_destroy(ctx); return REHYAT_ERR_ALLOC; }
+  if (cudaMemset(ctx->status_dev, 0, 256) != cudaSuccess) { rehyat_destroy(ctx); return REHYAT_ERR_CUDA; }
+
+  if (c.dtype == REHYAT_DTYPE_FP32)
+    rc = c.head_dim == 64 ? set_simt_attributes<float, 64>(c) : set_simt_attributes<float, 128>(c);
+  else
+    rc = c.head_dim == 64 ? set_simt_attributes<__nv_bfloat16, 64>(c) : set_simt_attributes<__nv_bfloat16, 128>(c);
+  if (rc == REHYAT_OK && ctx->tensor_ok) rc = tc_set_attributes();
+  if (rc != REHYAT_OK) { rehyat_destroy(ctx); return rc; }
+  *out = ctx;
+  return REHYAT_OK;
+}
+
+int rehyat_destroy(rehyat_ctx* ctx) {
+  if (!ctx) return REHYAT_OK;
+  DeviceGuard guard(ctx->cfg.device);
+  cudaFree(ctx->state); cudaFree(ctx->partial); cudaFree(ctx->readout); cudaFree(ctx->status_dev);
+  tc_workspace_destroy(&ctx->tc);
+  for (void* p : ctx->stage) cudaFree(p);
+  delete ctx;
+  return REHYAT_OK;
+}
+
+size_t rehyat_workspace_bytes(const rehyat_ctx* ctx) { return ctx ? ctx->ws_bytes : 0; }
+int rehyat_last_launches(const rehyat_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
+int rehyat_last_impl(const rehyat_ctx* ctx) { return ctx ? ctx->last_impl : 0; }
+
+int rehyat_status(rehyat_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return REHYAT_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->cfg.device);
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int word = 0;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
+  if (cudaMemcpy(&word, ctx->status_dev, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return REHYAT_ERR_CUDA;
+  if (word != 0) {
+    cudaMemset(ctx->status_dev, 0, 256);
+    return REHYAT_ERR_DEVICE_TIMEOUT;
+  }
+  return REHYAT_OK;
+}
+
+int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void* out,
+                   const rehyat_layout* lay, const rehyat_phi_params* phi, int32_t batch, int32_t frames,
+                   int32_t H, int32_t W, int32_t chunk, int32_t overlap, void* cuda_stream) {
+  if (!ctx || !q || !k || !v || !out || !lay || !phi) return REHYAT_ERR_INVALID_ARG;
+  const rehyat_config& c = ctx->cfg;
+  if (batch < 1 || batch > c.max_batch || frames < 1 || H < 1 || W < 1 || chunk < 1 || overlap < 0)
+    return REHYAT_ERR_INVALID_ARG;
+  const long long HW = (long long)H * W;
+  if (HW > c.max_tokens_per_frame) return REHYAT_ERR_INVALID_ARG;
+  const long long N = HW * frames;
+  if (N > INT_MAX / 2) return REHYAT_ERR_INVALID_ARG;
+  const int chunk_eff = chunk < frames ? chunk : frames;      // one chunk covers everything beyond that
+  if (chunk_eff > c.max_chunk_frames) return REHYAT_ERR_INVALID_ARG;
+  const int overlap_eff = overlap < frames ? overlap : frames; // the window is clamped at token 0 anyway
+  if (out == q || out == k || out == v) return REHYAT_ERR_INVALID_ARG;
+  const void* ptrs[] = {q, k, v, out, phi->q_W1, phi->q_b1, phi->q_W2, phi->q_b2,
+                        phi->k_W1, phi->k_b1, phi->k_W2, phi->k_b2};
+  for (const void* p : ptrs)
+    if (!p || !aligned16(p)) return REHYAT_ERR_INVALID_ARG;
+  const size_t es = elem_size(c.dtype);
+  const long long strides[] = {lay->stride_batch, lay->stride_head, lay->stride_token};
+  for (long long s : strides)
+    if (s < 0 || (s * (long long)es) % 16 != 0) return REHYAT_ERR_INVALID_ARG;
+  if (lay->stride_token < c.head_dim) return REHYAT_ERR_INVALID_ARG;
+
+  DeviceGuard guard(c.device);
+  if (!guard.ok) return REHYAT_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+
+  Geo g;
+  g.N = (int)N;
+  g.Np = (int)(chunk_eff * HW);
+  g.ToHW = (int)(overlap_eff * HW);
+  g.n_heads = c.n_heads;
+  g.BH = batch * c.n_heads;
+  g.stride_b = lay->stride_batch; g.stride_h = lay->stride_head; g.stride_n = lay->stride_token;
+  const int n_chunks = (frames + chunk_eff - 1) / chunk_eff;
+  int G = ctx->rd_rows / g.Np;
+  if (G < 1) return REHYAT_ERR_INVALID_ARG;   // cannot happen: rd_rows >= max chunk size
+  if (G > ctx->Gmax) G = ctx->Gmax;
+  int n_split = ctx->partial_units / G;
+  if (n_split > 8) n_split = 8;
+
+  ctx->last_launches = 0;
+  ctx->last_impl = ctx->tensor_ok ? 1 : 0;
+  int carry_slot = -1;
+  for (int t0 = 0; t0 < n_chunks; t0 += G) {
+    g.t0 = t0;
+    g.G = (n_chunks - t0) < G ? (n_chunks - t0) : G;
+    const bool any_linear = geo_lo(g, t0 + g.G - 1) > 0;
+    int rc;
+    if (ctx->tensor_ok) {
+      int launches = 0;
+      rc = tc_launch_group(&ctx->tc, q, k, v, out, phi, g, c.phi_hidden, c.phi_dim, c.c_mode, n_split, carry_slot,
+                           any_linear, ctx->state, ctx->partial, ctx->readout, ctx->rd_rows, ctx->status_dev, st,
+                           &launches);
+      ctx->last_launches += launches;
+    } else if (c.dtype == REHYAT_DTYPE_FP32) {
+      rc = c.head_dim == 64
+               ? launch_group_simt<float, 64>(ctx, (const float*)q, (const float*)k, (const float*)v, (float*)out, phi, g, n_split, carry_slot, any_linear, st)
+               : launch_group_simt<float, 128>(ctx, (const float*)q, (const float*)k, (const float*)v, (float*)out, phi, g, n_split, carry_slot, any_linear, st);
+    } else {
+      using B = __nv_bfloat16;
+      rc = c.head_dim == 64
+               ? launch_group_simt<B, 64>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot, any_linear, st)
+               : launch_group_simt<B, 128>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot, any_linear, st);
+    }
+    if (rc != REHYAT_OK) return rc;
+    if (any_linear) carry_slot = g.G - 1;
+  }
+  return REHYAT_OK;
+}
+
+int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
+                        void* out_host, const rehyat_phi_params* phi, int32_t batch, int32_t frames, int32_t H,
+                        int32_t W, int32_t chunk, int32_t overlap, void* cuda_stream) {
+  if (!ctx || !q_host || !k_host || !v_host || !out_host || !phi) return REHYAT_ERR_INVALID_ARG;
+  if (batch < 1 || frames < 1 || H < 1 || W < 1) return REHYAT_ERR_INVALID_ARG;
+  const rehyat_config& c = ctx->cfg;
+  const long long N = (long long)H * W * frames;
+  if (N > INT_MAX / 2 || batch > c.max_batch) return REHYAT_ERR_INVALID_ARG;
+  const size_t bytes = (size_t)batch * c.n_heads * N * c.head_dim * elem_size(c.dtype);
+  DeviceGuard guard(c.device);
+  if (!guard.ok) return REHYAT_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (bytes > ctx->stage_bytes) {
+    if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
+    for (void*& p : ctx->stage) { cudaFree(p); p = nullptr; }
+    ctx->stage_bytes = 0;
+    for (void*& p : ctx->stage)
+      if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return REHYAT_ERR_ALLOC; }
+    ctx->stage_bytes = bytes;
+  }
+  const void* src[3] = {q_host, k_host, v_host};
+  for (int i = 0; i < 3; ++i)
+    if (cudaMemcpyAsync(ctx->stage[i], src[i], bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return REHYAT_ERR_CUDA;
+  rehyat_layout lay = {(int64_t)c.n_heads * N * c.head_dim, (int64_t)N * c.head_dim, (int64_t)c.head_dim};
+  int rc = rehyat_forward(ctx, ctx->stage[0], ctx->stage[1], ctx->stage[2], ctx->stage[3], &lay, phi, batch, frames,
+                          H, W, chunk, overlap, cuda_stream);
+  if (rc != REHYAT_OK) return rc;
+  if (cudaMemcpyAsync(out_host, ctx->stage[3], bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return REHYAT_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
+  return REHYAT_OK;
+}
+
+}  // extern "C"

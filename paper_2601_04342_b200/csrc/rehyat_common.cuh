@@ -1,0 +1,76 @@
+// Shared device-side definitions of the ReHyAt kernels: geometry of one chunk group, element
+// load/store helpers, the phi activations.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace rehyat {
+
+// Activations of the phi MLP (same numbering as rehyat_act in the public header).
+enum Act : int { ACT_RELU = 0, ACT_IDENTITY = 1, ACT_SOFTPLUS = 2, ACT_ELU1 = 3, ACT_GELU = 4 };
+enum CMode : int { C_ROWMAX = 0, C_ZERO = 1 };
+
+// Everything a kernel needs to find chunk t = t0 + (chunk index inside the group).
+// Chunk t (Section 3.3, Eq. 13): queries [t*Np, min((t+1)*Np, N)), softmax window [lo_t, hi_t),
+// lo_t = max(t*Np - ToHW, 0), hi_t = end of the queries; linear prefix [0, lo_t).
+struct Geo {
+  int N;        // tokens per (batch, head)
+  int Np;       // tokens per chunk, chunk*H*W
+  int ToHW;     // overlap*H*W (clamped to N by the host so that it cannot overflow)
+  int t0;       // first chunk of the group
+  int G;        // chunks in the group
+  int n_heads;
+  int BH;       // batch * n_heads
+  long long stride_b, stride_h, stride_n;   // element strides of q, k, v, out
+};
+
+__host__ __device__ inline int geo_q0(const Geo& g, int t) { return t * g.Np; }
+__host__ __device__ inline int geo_q1(const Geo& g, int t) {
+  long long e = (long long)(t + 1) * g.Np;
+  return e < g.N ? (int)e : g.N;
+}
+__host__ __device__ inline int geo_lo(const Geo& g, int t) {
+  long long a = (long long)t * g.Np - g.ToHW;
+  return a > 0 ? (int)a : 0;
+}
+
+__device__ __forceinline__ long long head_offset(const Geo& g, int bh) {
+  return (long long)(bh / g.n_heads) * g.stride_b + (long long)(bh % g.n_heads) * g.stride_h;
+}
+
+__device__ __forceinline__ float ldf(const float* p) { return *p; }
+__device__ __forceinline__ float ldf(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void stf(float* p, float x) { *p = x; }
+__device__ __forceinline__ void stf(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+
+// Four consecutive elements as floats (pointer must be aligned to four elements).
+__device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 ld4(const __nv_bfloat16* p) {
+  uint2 u = *reinterpret_cast<const uint2*>(p);
+  __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&u.x);
+  __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162*>(&u.y);
+  float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+  return make_float4(fa.x, fa.y, fb.x, fb.y);
+}
+
+__device__ __forceinline__ float apply_act(float x, int act) {
+  switch (act) {
+    case ACT_RELU: return fmaxf(x, 0.f);
+    case ACT_IDENTITY: return x;
+    case ACT_SOFTPLUS: return x > 20.f ? x : log1pf(expf(x));
+    case ACT_ELU1: return x > 0.f ? x + 1.f : expf(x);
+    default: return 0.5f * x * (1.f + erff(x * 0.70710678118654752f));
+  }
+}
+
+// Element-wise power of the polynomial expansion: output feature j of D' belongs to part
+// j / (D'/P) (0-based) and is raised to that index plus one.
+__device__ __forceinline__ float poly_power(float u, int part) {
+  float r = u;
+  for (int i = 0; i < part; ++i) r *= u;
+  return r;
+}
+
+}  // namespace rehyat
