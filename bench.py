@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the ReHyAt hybrid attention operator on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference] [--workload NAME]
+
+One step = one pass of the whole operator (state increments, scan, linear read-out, softmax
+window + joint normaliser) over one synthetic layer input.  At N=1 the workload is the
+Wan2.1-1.3B-shaped layer (B=1, 12 heads of 128, 21 latent frames of 30x52 = 32,760 tokens,
+chunk 3, overlap 1, bf16).  With N>1 (one process per GPU under torchrun) every rank runs its
+own layer input of that shape: the (batch, head) problems are independent, so there is no
+collective on the data path and scaling is weak.
+
+`value` is algorithmic TFLOP/s of the whole job with inputs resident in HBM; `e2e` is the same
+metric through the host-buffer entry point (pinned host tensors, copies inside the timed
+region).  `--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2601_04342_b200 import geometry, synth  # noqa: E402
+
+METRIC = "hybrid-attention TFLOP/s (algorithmic) per layer at 32,760 tokens"
+UNIT = "TFLOP/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the ncu
+# capture summarised under profiles/; None until a capture exists for the kernel in use.
+NCU_TRAFFIC_BYTES = {"window_simt": None, "window_tc": None}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"bf16_burst": p["bf16_tflops"], "bf16_sustained": p["bf16_tflops_sustained"],
+                "hbm_gbs": p["hbm_gbs"], "source": "measured"}
+    return {"bf16_burst": 1590.0, "bf16_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            tok = [t.strip() for t in line.split(",")]
+            if len(tok) < 9:
+                continue
+            try:
+                sm.append(float(tok[1])); smax.append(float(tok[2])); power.append(float(tok[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, tok[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p["num_threads"] for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def oracle_sample(wl, inputs, heads):
+    """Times the fp64 oracle (recurrent form, as it stands) on `heads` of batch 0 of the workload."""
+    from oracle import rehyat_oracle as orc
+    sel = lambda t: t[:1, heads].to(torch.float64).numpy()
+    q, k, v = sel(inputs["q"]), sel(inputs["k"]), sel(inputs["v"])
+    pq = {n: t[heads].to(torch.float64).numpy() for n, t in inputs["phi_q"].items()}
+    pk = {n: t[heads].to(torch.float64).numpy() for n, t in inputs["phi_k"].items()}
+    t0 = time.perf_counter()
+    orc.hybrid_rnn(q, k, v, pq, pk, wl.T, wl.HW, wl.Tc, wl.To, P=wl.P)
+    dt = time.perf_counter() - t0
+    flops = geometry.flop_model(1, len(heads), wl.head_dim, wl.T, wl.HW, wl.Tc, wl.To, wl.D_h, wl.D_out)["total"]
+    return dt, flops
+
+
+def config_of(wl, extra=None):
+    cfg = {"workload": wl.name, "batch": wl.B, "heads": wl.n_heads, "head_dim": wl.head_dim,
+           "latent_frames": wl.T, "patch_grid": [wl.H, wl.W], "tokens": wl.N, "chunk_frames": wl.Tc,
+           "overlap_frames": wl.To, "phi": {"hidden": wl.D_h, "dim": wl.D_out, "degree": wl.P, "act": "relu/relu",
+                                            "param_std": 0.02},
+           "c_mode": "rowmax", "qk_rms_norm": wl.rms_norm_qk,
+           "l2": "inputs (q,k,v,out = %.0f MB) exceed the 126 MB L2; no flush" %
+                 (geometry.io_bytes(wl.B, wl.n_heads, wl.head_dim, wl.N, 2) / 1e6)}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inputs = synth.make_inputs(wl)
+    heads = list(range(args.ref_heads))
+    times = []
+    flops = 0
+    for i in range(args.warmup + args.steps):
+        dt, flops = oracle_sample(wl, inputs, heads)
+        if i >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = flops * len(times) / total / 1e12
+    sample = f"{len(heads)} of {wl.n_heads} heads of batch 0, all {wl.N} tokens, recurrent form, fp64 numpy"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_of(wl),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="wan13b_layer", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--ref-heads", type=int, default=12, help="heads the oracle sample covers")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel-impl", default="auto", choices=["auto", "simt", "tensor"])
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    wl = synth.CONFIGS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the operator has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    from paper_2601_04342_b200 import binding, build
+    if rank == 0:
+        build.build()
+    if dist:
+        dist.barrier()
+
+    # every rank draws its own layer input (weak scaling over independent problems)
+    wl_rank = wl.with_(seed=wl.seed + 1000 * rank)
+    host = synth.make_inputs(wl_rank)
+    dev = {n: host[n].cuda() for n in ("q", "k", "v")}
+    phi_q = {n: t.cuda() for n, t in host["phi_q"].items()}
+    phi_k = {n: t.cuda() for n, t in host["phi_k"].items()}
+    out = torch.empty_like(dev["q"])
+    op = binding.for_workload(wl, impl=args.kernel_impl, device=local_rank)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        op.forward(dev["q"], dev["k"], dev["v"], phi_q, phi_k, wl.T, wl.H, wl.W, wl.Tc, wl.To, out=out, stream=stream)
+
+    def barrier():
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert op.status() == 0, "device status word set during warm-up"
+    launches_per_step = op.last_launches
+    kernel_family = op.last_impl
+
+    flops = geometry.flop_model(wl.B, wl.n_heads, wl.head_dim, wl.T, wl.HW, wl.Tc, wl.To, wl.D_h, wl.D_out)
+    sampler = ClockSampler(local_rank)
+    op.profile_enable(True)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    prof = op.profile_read()
+    op.profile_enable(False)
+    assert op.status() == 0, "device status word set during the timed region"
+    if dist:
+        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * flops["total"] / (ms_step * 1e-3) / 1e12
+
+    # end to end through the host-buffer entry point (pinned host tensors, copies timed)
+    pinned = {n: host[n].pin_memory() for n in ("q", "k", "v")}
+    out_host = torch.empty_like(host["q"]).pin_memory()
+    nbytes = host["q"].numel() * host["q"].element_size()
+
+    def e2e_step():
+        op.forward_host(pinned["q"], pinned["k"], pinned["v"], out_host, phi_q, phi_k, wl.T, wl.H, wl.W, wl.Tc, wl.To,
+                        stream=stream)
+
+    e2e_step()
+    barrier()
+    e0.record(stream)
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
+    if dist:
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * flops["total"] / (e2e_ms * 1e-3) / 1e12
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    timed_s = ms_total * 1e-3
+    peak_kind = "sustained" if timed_s >= 2.0 else "burst"
+    peak = peaks["bf16_sustained"] if peak_kind == "sustained" else peaks["bf16_burst"]
+    win_ms, win_n = prof["window"]
+    win_flops_per_launch = flops["window"] * args.steps / max(win_n, 1)
+    achieved = win_flops_per_launch / (win_ms / max(win_n, 1) * 1e-3) / 1e12 if win_ms > 0 else None
+    kernel_name = "window_tc" if kernel_family == "tensor" else "window_simt"
+    roofline = {"bound": "tensor", "kernel": kernel_name, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak if achieved else None, "traffic": NCU_TRAFFIC_BYTES.get(kernel_name),
+                "peak_source": f"{peaks['source']} bf16 {peak_kind} (MEASURED_PEAKS.json)" if peaks["source"] == "measured"
+                else "fallback",
+                "frac_of_nominal_2250": achieved / 2250.0 if achieved else None,
+                "launches": win_n, "avg_launch_ms": win_ms / max(win_n, 1),
+                "algorithmic_flop_per_launch": win_flops_per_launch,
+                "hbm_gbs_whole_step": geometry.io_bytes(wl.B, wl.n_heads, wl.head_dim, wl.N, 2) / (ms_step * 1e-3) / 1e9,
+                "hbm_peak_gbs": peaks["hbm_gbs"]}
+    kernel_ms = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps} for k, v in prof.items()}
+
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        heads = list(range(args.ref_heads))
+        dt, fl = oracle_sample(wl, host, heads)
+        cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+               "sample": f"{len(heads)} of {wl.n_heads} heads of batch 0, all {wl.N} tokens, recurrent form, "
+                         f"fp64 numpy, {dt:.1f} s"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": config_of(wl, {"kernels": kernel_family, "parallelism": f"dp{world} over (batch, head) problems"}),
+            "tokens_per_s": world * wl.B * wl.N / (ms_step * 1e-3),
+            "frac_of_bf16_peak": {"measured_burst": value / world / peaks["bf16_burst"],
+                                  "measured_sustained": value / world / peaks["bf16_sustained"],
+                                  "nominal_2250": value / world / 2250.0},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes,
+                    "ms_per_step": e2e_ms},
+            "gpu_launches": launches_per_step * args.steps,
+            "kernel_ms": kernel_ms, "workspace_bytes": op.workspace_bytes,
+            "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    op.close()
+    if dist:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -144,6 +144,19 @@ int rehyat_last_launches(const rehyat_ctx* ctx);
 /* 1 if the last forward ran the tensor-core kernels, 0 for the SIMT kernels. */
 int rehyat_last_impl(const rehyat_ctx* ctx);
 
+/* Per-kernel timing for measurement.  While enabled, every kernel launch of rehyat_forward is
+ * bracketed by CUDA events recorded on the launching stream (a few microseconds of overhead per
+ * launch).  rehyat_profile_read waits for the recorded events, writes the summed milliseconds and
+ * the launch counts of each kernel kind into ms[REHYAT_PROF_KINDS] / launches[REHYAT_PROF_KINDS]
+ * (host arrays) and clears the record.  Read at least once per few hundred forwards. */
+#define REHYAT_PROF_STATE   0   /* phi_k + chunk-state increments (Eq. 17-18)    */
+#define REHYAT_PROF_SCAN    1   /* running sum along the chunk axis (Eq. 14-15) */
+#define REHYAT_PROF_READOUT 2   /* phi_q + linear read-out (Eq. 7, 9)            */
+#define REHYAT_PROF_WINDOW  3   /* softmax window + joint normaliser (Eq. 5-8)   */
+#define REHYAT_PROF_KINDS   4
+int rehyat_profile_enable(rehyat_ctx* ctx, int on);
+int rehyat_profile_read(rehyat_ctx* ctx, double* ms, int32_t* launches);
+
 const char* rehyat_strerror(int code);
 int rehyat_version(void);
 

@@ -18,7 +18,8 @@ IMPL = {"auto": 0, "simt": 1, "tensor": 2}
 
 EXPORTS = ["rehyat_create", "rehyat_forward", "rehyat_forward_host", "rehyat_destroy",
            "rehyat_workspace_bytes", "rehyat_status", "rehyat_last_launches", "rehyat_last_impl",
-           "rehyat_strerror", "rehyat_version"]
+           "rehyat_profile_enable", "rehyat_profile_read", "rehyat_strerror", "rehyat_version"]
+PROF_KINDS = ("state", "scan", "readout", "window")
 
 
 class Config(C.Structure):
@@ -57,6 +58,8 @@ def lib():
         L.rehyat_status.argtypes = [C.c_void_p, C.c_void_p]
         L.rehyat_last_launches.argtypes = [C.c_void_p]
         L.rehyat_last_impl.argtypes = [C.c_void_p]
+        L.rehyat_profile_enable.argtypes = [C.c_void_p, C.c_int]
+        L.rehyat_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int32)]
         L.rehyat_strerror.argtypes = [C.c_int]
         L.rehyat_strerror.restype = C.c_char_p
         for name in EXPORTS:
@@ -153,6 +156,16 @@ class Rehyat:
         _check(lib().rehyat_forward_host(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), C.byref(phi), B, frames, H,
                                          W, chunk, overlap, C.c_void_p(st.cuda_stream)), "rehyat_forward_host")
         return out
+
+    def profile_enable(self, on=True):
+        _check(lib().rehyat_profile_enable(self._h, int(on)), "rehyat_profile_enable")
+
+    def profile_read(self):
+        """{kind: (summed ms, launches)} since the last read; waits for the recorded events."""
+        ms = (C.c_double * len(PROF_KINDS))()
+        n = (C.c_int32 * len(PROF_KINDS))()
+        _check(lib().rehyat_profile_read(self._h, ms, n), "rehyat_profile_read")
+        return {k: (ms[i], n[i]) for i, k in enumerate(PROF_KINDS)}
 
     def status(self, stream=None):
         st = stream if stream is not None else torch.cuda.current_stream(self.cfg.device)

@@ -14,6 +14,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "../../include/rehyat.h"
 #include "rehyat_common.cuh"
@@ -22,8 +23,27 @@
 
 using namespace rehyat;
 
+// Optional per-kernel timing: CUDA events recorded on the launching stream around every launch
+// of each kernel kind, summed when read.
+struct Profiler {
+  bool on = false;
+  std::vector<cudaEvent_t> ev[REHYAT_PROF_KINDS];   // begin/end pairs
+  void begin(int kind, cudaStream_t st) {
+    if (!on) return;
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return;
+    cudaEventRecord(e, st);
+    ev[kind].push_back(e);
+  }
+  void end(int kind, cudaStream_t st) { begin(kind, st); }
+  void clear() {
+    for (auto& v : ev) { for (cudaEvent_t e : v) cudaEventDestroy(e); v.clear(); }
+  }
+};
+
 struct rehyat_ctx {
   rehyat_config cfg;
+  Profiler prof;
   float* state = nullptr;      // [Gmax][BHmax][Dp][d+4]
   float* partial = nullptr;    // [partial_units][BHmax][Dp][d+4]
   float* readout = nullptr;    // [BHmax][rd_rows][d+4]
@@ -93,20 +113,28 @@ int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* ou
     PhiPtrs<T> wk = {(const T*)phi->k_W1, (const T*)phi->k_b1, (const T*)phi->k_W2, (const T*)phi->k_b2};
     PhiPtrs<T> wq = {(const T*)phi->q_W1, (const T*)phi->q_b1, (const T*)phi->q_W2, (const T*)phi->q_b2};
     const size_t smem_state = (size_t)SIMT_TM * (2 * D + pd.Dh + pd.Dp) * sizeof(float);
+    ctx->prof.begin(REHYAT_PROF_STATE, st);
     state_partial_simt<T, D><<<dim3(n_split, g.G, g.BH), SIMT_PHI_THREADS, smem_state, st>>>(
         k, v, wk, pd, g, n_split, ctx->partial);
+    ctx->prof.end(REHYAT_PROF_STATE, st);
     const size_t per_slot = (size_t)g.BH * pd.Dp * SD;
+    ctx->prof.begin(REHYAT_PROF_SCAN, st);
     scan_states<<<(unsigned)((per_slot + 255) / 256), 256, 0, st>>>(ctx->partial, ctx->state, per_slot, g.G,
                                                                      n_split, carry_slot);
+    ctx->prof.end(REHYAT_PROF_SCAN, st);
     const size_t smem_rd = (size_t)SIMT_TM * (D + pd.Dh + pd.Dp) * sizeof(float);
+    ctx->prof.begin(REHYAT_PROF_READOUT, st);
     readout_simt<T, D><<<dim3(tiles, g.G, g.BH), SIMT_PHI_THREADS, smem_rd, st>>>(q, wq, pd, g, ctx->state,
                                                                                  ctx->readout, ctx->rd_rows);
+    ctx->prof.end(REHYAT_PROF_READOUT, st);
     ctx->last_launches += 3;
   }
   const size_t smem_win = (size_t)(WIN_BM * (D + 4) + WIN_BN * (D + 4) + WIN_BN * D + WIN_BM * (WIN_BN + 4)) * sizeof(float);
   const int wtiles = (g.Np + WIN_BM - 1) / WIN_BM;
+  ctx->prof.begin(REHYAT_PROF_WINDOW, st);
   window_simt<T, D><<<dim3(wtiles, g.G, g.BH), WIN_THREADS, smem_win, st>>>(
       q, k, v, out, g, ctx->readout, ctx->rd_rows, 1.0f / sqrtf((float)D), c.c_mode);
+  ctx->prof.end(REHYAT_PROF_WINDOW, st);
   ctx->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
@@ -189,6 +217,7 @@ int rehyat_destroy(rehyat_ctx* ctx) {
   DeviceGuard guard(ctx->cfg.device);
   cudaFree(ctx->state); cudaFree(ctx->partial); cudaFree(ctx->readout); cudaFree(ctx->status_dev);
   tc_workspace_destroy(&ctx->tc);
+  ctx->prof.clear();
   for (void* p : ctx->stage) cudaFree(p);
   delete ctx;
   return REHYAT_OK;
@@ -197,6 +226,32 @@ int rehyat_destroy(rehyat_ctx* ctx) {
 size_t rehyat_workspace_bytes(const rehyat_ctx* ctx) { return ctx ? ctx->ws_bytes : 0; }
 int rehyat_last_launches(const rehyat_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
 int rehyat_last_impl(const rehyat_ctx* ctx) { return ctx ? ctx->last_impl : 0; }
+
+int rehyat_profile_enable(rehyat_ctx* ctx, int on) {
+  if (!ctx) return REHYAT_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->cfg.device);
+  ctx->prof.clear();
+  ctx->prof.on = on != 0;
+  return REHYAT_OK;
+}
+
+int rehyat_profile_read(rehyat_ctx* ctx, double* ms, int32_t* launches) {
+  if (!ctx || !ms || !launches) return REHYAT_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->cfg.device);
+  for (int kind = 0; kind < REHYAT_PROF_KINDS; ++kind) {
+    auto& v = ctx->prof.ev[kind];
+    ms[kind] = 0.0;
+    launches[kind] = (int32_t)(v.size() / 2);
+    for (size_t i = 0; i + 1 < v.size(); i += 2) {
+      float t = 0.f;
+      if (cudaEventSynchronize(v[i + 1]) != cudaSuccess || cudaEventElapsedTime(&t, v[i], v[i + 1]) != cudaSuccess)
+        return REHYAT_ERR_CUDA;
+      ms[kind] += t;
+    }
+  }
+  ctx->prof.clear();
+  return REHYAT_OK;
+}
 
 int rehyat_status(rehyat_ctx* ctx, void* cuda_stream) {
   if (!ctx) return REHYAT_ERR_INVALID_ARG;
