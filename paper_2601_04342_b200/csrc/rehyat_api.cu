@@ -104,7 +104,8 @@ int set_simt_attributes(const rehyat_config& c) {
 
 template <typename T, int D>
 int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* out, const rehyat_phi_params* phi,
-                      const Geo& g, int n_split, int carry_slot, bool any_linear, cudaStream_t st) {
+                      const Geo& g, int n_split, int carry_slot, bool any_linear, cudaStream_t st,
+                      bool with_window = true) {
   const rehyat_config& c = ctx->cfg;
   PhiDims pd = {D, c.phi_hidden, c.phi_dim, c.poly_degree, c.act_hidden, c.act_out};
   constexpr int SD = D + 4;
@@ -129,6 +130,7 @@ int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* ou
     ctx->prof.end(REHYAT_PROF_READOUT, st);
     ctx->last_launches += 3;
   }
+  if (!with_window) return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
   const size_t smem_win = (size_t)(WIN_BM * (D + 4) + WIN_BN * (D + 4) + WIN_BN * D + WIN_BM * (WIN_BN + 4)) * sizeof(float);
   const int wtiles = (g.Np + WIN_BM - 1) / WIN_BM;
   ctx->prof.begin(REHYAT_PROF_WINDOW, st);
@@ -319,11 +321,16 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
     const bool any_linear = geo_lo(g, t0 + g.G - 1) > 0;
     int rc;
     if (ctx->tensor_ok) {
-      int launches = 0;
-      rc = tc_launch_group(&ctx->tc, q, k, v, out, phi, g, c.phi_hidden, c.phi_dim, c.c_mode, n_split, carry_slot,
-                           any_linear, ctx->state, ctx->partial, ctx->readout, ctx->rd_rows, ctx->status_dev, st,
-                           &launches);
-      ctx->last_launches += launches;
+      using B = __nv_bfloat16;
+      rc = launch_group_simt<B, 128>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot,
+                                     any_linear, st, /*with_window=*/false);
+      if (rc == REHYAT_OK) {
+        ctx->prof.begin(REHYAT_PROF_WINDOW, st);
+        rc = tc_launch_window(&ctx->tc, q, k, v, out, g, batch, ctx->readout, ctx->rd_rows, c.c_mode,
+                              ctx->status_dev, st);
+        ctx->prof.end(REHYAT_PROF_WINDOW, st);
+        ctx->last_launches += 1;
+      }
     } else if (c.dtype == REHYAT_DTYPE_FP32) {
       rc = c.head_dim == 64
                ? launch_group_simt<float, 64>(ctx, (const float*)q, (const float*)k, (const float*)v, (float*)out, phi, g, n_split, carry_slot, any_linear, st)

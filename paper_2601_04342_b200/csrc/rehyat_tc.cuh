@@ -1,22 +1,360 @@
-// Tensor-core (tcgen05) path of the operator.  Placeholder until the kernels land: reports that
-// no shape is covered, so every call runs the SIMT kernels.
+// Tensor-core (tcgen05 / TMEM / TMA) path of the operator for bf16, head_dim 128.
+//
+// window_tc: softmax window of Eq. 6 and 8 plus the joint normalisation of Eq. 5.
+//   One CTA owns two 128-row query tiles of one chunk and walks the chunk's key window in tiles of
+//   128 keys.  Roles (384 threads):
+//     warp 0        TMA producer: Q once, then K and V tiles through two-stage rings
+//     warp 1        UMMA issuer: S_i = Q_i K^T into TMEM, O_i += P_i V with P_i read from TMEM
+//     warps 4-7     softmax of query tile 0 (one thread per row), warps 8-11 of query tile 1
+//   TMEM (512 columns): S_0 [0,128) S_1 [128,256) O_0 [256,384) O_1 [384,512); P_i (bf16) overwrites
+//   the first 64 columns of S_i.  While one tile's softmax runs on the ALUs the tensor core works on
+//   the other tile.  The running maximum is applied lazily: O and l are rescaled only when the row
+//   maximum grew by more than 2^8 since the last rescale; the true maximum is tracked separately and
+//   applied once after the last key tile, so that O and l end up relative to c_i = final row maximum
+//   before the un-rescaled linear terms are added (Eq. 5-9).
 #pragma once
+
+#include <cuda.h>
 
 #include "../../include/rehyat.h"
 #include "rehyat_common.cuh"
+#include "rehyat_ptx.cuh"
 
 namespace rehyat {
 
-struct TcWorkspace {};
+constexpr int TC_D = 128;             // head_dim
+constexpr int TC_BM = 128;            // rows per query tile
+constexpr int TC_QT = 2;              // query tiles per CTA
+constexpr int TC_BN = 128;            // keys per tile
+constexpr int TC_STAGES = 2;          // K ring and V ring depth
+constexpr int TC_THREADS = 384;
+constexpr int TC_TILE_BYTES = TC_BN * TC_D * 2;       // 32 KB: two [128 x 64] swizzled sub-tiles
+constexpr int TC_SUB_BYTES = TC_TILE_BYTES / 2;
+constexpr int TC_WIN_SMEM = (TC_QT + 2 * TC_STAGES) * TC_TILE_BYTES + 1024 /*barriers*/ + 1024 /*align*/;
 
-inline bool tc_shape_supported(bool, int, int, int, int, int, int) { return false; }
-inline bool tc_workspace_create(TcWorkspace*, int, int, int, int, size_t* extra) { *extra = 0; return true; }
+enum TcErr : int { TC_ERR_LOAD = 1, TC_ERR_MMA = 2, TC_ERR_SOFTMAX = 4 };
+
+struct WinBars {   // offsets (bytes) inside the barrier block
+  uint64_t q_full;
+  uint64_t k_full[TC_STAGES], k_empty[TC_STAGES], v_full[TC_STAGES], v_empty[TC_STAGES];
+  uint64_t s_ready[TC_QT], p_ready[TC_QT], pv_done[TC_QT];
+  uint64_t drained;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+          const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ out, Geo g,
+          const float* __restrict__ rd, int rd_rows, float scale, int c_mode, int* __restrict__ status) {
+  using namespace ptx;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t sQ = smem_base;                                   // TC_QT tiles
+  const uint32_t sK = sQ + TC_QT * TC_TILE_BYTES;                  // TC_STAGES tiles
+  const uint32_t sV = sK + TC_STAGES * TC_TILE_BYTES;              // TC_STAGES tiles
+  WinBars* bars = reinterpret_cast<WinBars*>(smem + (TC_QT + 2 * TC_STAGES) * TC_TILE_BYTES);
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
+  const int q0 = geo_q0(g, t), q1 = geo_q1(g, t), lo = geo_lo(g, t), hi = q1;
+  const int row_base = q0 + blockIdx.x * (TC_QT * TC_BM);
+  if (row_base >= q1) return;                                      // uniform for the CTA
+  const int ntiles = (row_base + TC_BM < q1) ? 2 : 1;              // query tiles with at least one valid row
+  const int n_kv = (hi - lo + TC_BN - 1) / TC_BN;
+  const int b_idx = bh / g.n_heads, h_idx = bh % g.n_heads;
+
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bars->q_full), 1);
+    for (int s = 0; s < TC_STAGES; ++s) {
+      mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1);
+      mbar_init(smem_u32(&bars->v_full[s]), 1); mbar_init(smem_u32(&bars->v_empty[s]), 1);
+    }
+    for (int i = 0; i < TC_QT; ++i) {
+      mbar_init(smem_u32(&bars->s_ready[i]), 1);
+      mbar_init(smem_u32(&bars->p_ready[i]), TC_BM);
+      mbar_init(smem_u32(&bars->pv_done[i]), 1);
+    }
+    mbar_init(smem_u32(&bars->drained), 1);
+    bars->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bars->tmem_base), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (elect_one()) {
+      prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
+      const uint32_t qf = smem_u32(&bars->q_full);
+      mbar_expect_tx(qf, ntiles * TC_TILE_BYTES);
+      for (int i = 0; i < ntiles; ++i) {
+        tma_load_4d(sQ + i * TC_TILE_BYTES, &tm_q, qf, 0, row_base + i * TC_BM, h_idx, b_idx);
+        tma_load_4d(sQ + i * TC_TILE_BYTES + TC_SUB_BYTES, &tm_q, qf, 64, row_base + i * TC_BM, h_idx, b_idx);
+      }
+      bool alive = true;
+      for (int j = 0; j < n_kv && alive; ++j) {
+        const int s = j % TC_STAGES;
+        const uint32_t ph = (j / TC_STAGES) & 1;
+        const int key0 = lo + j * TC_BN;
+        alive = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1, abort_flag, status, TC_ERR_LOAD);
+        if (!alive) break;
+        const uint32_t kf = smem_u32(&bars->k_full[s]);
+        mbar_expect_tx(kf, TC_TILE_BYTES);
+        tma_load_4d(sK + s * TC_TILE_BYTES, &tm_k, kf, 0, key0, h_idx, b_idx);
+        tma_load_4d(sK + s * TC_TILE_BYTES + TC_SUB_BYTES, &tm_k, kf, 64, key0, h_idx, b_idx);
+        alive = mbar_wait(smem_u32(&bars->v_empty[s]), ph ^ 1, abort_flag, status, TC_ERR_LOAD);
+        if (!alive) break;
+        const uint32_t vf = smem_u32(&bars->v_full[s]);
+        mbar_expect_tx(vf, TC_TILE_BYTES);
+        tma_load_4d(sV + s * TC_TILE_BYTES, &tm_v, vf, 0, key0, h_idx, b_idx);
+        tma_load_4d(sV + s * TC_TILE_BYTES + TC_SUB_BYTES, &tm_v, vf, 64, key0, h_idx, b_idx);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ UMMA issuer
+    if (elect_one()) {
+      constexpr uint32_t idesc_qk = idesc_bf16(TC_BM, TC_BN, 0, 0);   // A = Q (K-major), B = K (K-major)
+      constexpr uint32_t idesc_pv = idesc_bf16(TC_BM, TC_D, 0, 1);    // A = P (TMEM),    B = V (MN-major)
+      auto issue_qk = [&](int i, int s) {
+        const uint32_t a0 = sQ + i * TC_TILE_BYTES, b0 = sK + s * TC_TILE_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < TC_D / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * TC_SUB_BYTES + (kk & 3) * 32;
+          umma_ss(tmem + i * TC_BN, smem_desc_sw128(a0 + off, 16, 1024), smem_desc_sw128(b0 + off, 16, 1024),
+                  idesc_qk, kk > 0);
+        }
+      };
+      auto issue_pv = [&](int i, int s, bool acc) {
+        const uint32_t b0 = sV + s * TC_TILE_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < TC_BN / 16; ++kk)
+          umma_ts(tmem + 256 + i * TC_D, tmem + i * TC_BN + kk * 8,
+                  smem_desc_sw128(b0 + kk * 16 * 128, TC_SUB_BYTES, 1024), idesc_pv, (acc || kk > 0) ? 1u : 0u);
+      };
+      bool alive = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag, status, TC_ERR_MMA);
+      alive = alive && mbar_wait(smem_u32(&bars->k_full[0]), 0, abort_flag, status, TC_ERR_MMA);
+      tc_fence_after();
+      for (int i = 0; i < ntiles; ++i) {
+        issue_qk(i, 0);
+        umma_commit(smem_u32(&bars->s_ready[i]));
+      }
+      umma_commit(smem_u32(&bars->k_empty[0]));
+      for (int j = 0; j < n_kv; ++j) {
+        const int s = j % TC_STAGES;
+        const uint32_t ph = (j / TC_STAGES) & 1;
+        mbar_wait(smem_u32(&bars->v_full[s]), ph, abort_flag, status, TC_ERR_MMA);
+        for (int i = 0; i < ntiles; ++i) {
+          mbar_wait(smem_u32(&bars->p_ready[i]), j & 1, abort_flag, status, TC_ERR_MMA);
+          tc_fence_after();
+          issue_pv(i, s, j > 0);
+          umma_commit(smem_u32(&bars->pv_done[i]));
+          if (i == ntiles - 1) umma_commit(smem_u32(&bars->v_empty[s]));
+          if (j + 1 < n_kv) {
+            const int s1 = (j + 1) % TC_STAGES;
+            if (i == 0) {
+              mbar_wait(smem_u32(&bars->k_full[s1]), ((j + 1) / TC_STAGES) & 1, abort_flag, status, TC_ERR_MMA);
+              tc_fence_after();
+            }
+            issue_qk(i, s1);
+            umma_commit(smem_u32(&bars->s_ready[i]));
+            if (i == ntiles - 1) umma_commit(smem_u32(&bars->k_empty[s1]));
+          }
+        }
+      }
+      // everything this thread issued has completed once `drained` flips
+      umma_commit(smem_u32(&bars->drained));
+      mbar_wait(smem_u32(&bars->drained), 0, abort_flag, status, TC_ERR_MMA);
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ softmax + epilogue
+    const int i = (warp - 4) >> 2;                                   // query tile of this warpgroup
+    if (i < ntiles) {
+      const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+      const uint32_t tS = tmem + lane_off + i * TC_BN, tO = tmem + lane_off + 256 + i * TC_D;
+      const float c = scale * 1.4426950408889634f;                   // logits -> log2 domain
+      float m_true = -INFINITY, m_used = -INFINITY, l = 0.f;
+      for (int j = 0; j < n_kv; ++j) {
+        mbar_wait(smem_u32(&bars->s_ready[i]), j & 1, abort_flag, status, TC_ERR_SOFTMAX);
+        tc_fence_after();
+        uint32_t sr[4][32];
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) tmem_ld32(tS + cc * 32, sr[cc]);
+        tmem_wait_ld();
+        const int n_valid = hi - (lo + j * TC_BN);                   // >= 1
+        if (n_valid < TC_BN) {
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (cc * 32 + e >= n_valid) sr[cc][e] = 0xff800000u;   // -inf
+        }
+        float mx = -INFINITY;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(sr[cc][e]));
+        m_true = fmaxf(m_true, mx);
+        const bool need = (m_true - m_used) * c > 8.f;               // true on the first tile (m_used = -inf)
+        if (j > 0) {
+          mbar_wait(smem_u32(&bars->pv_done[i]), (j - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+          tc_fence_after();
+        }
+        if (__any_sync(0xffffffffu, need)) {
+          const float m_new = need ? m_true : m_used;
+          if (j > 0) {
+            const float f = ex2((m_used - m_new) * c);               // 1 for lanes that keep their reference
+            l *= f;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+              uint32_t o[32];
+              tmem_ld32(tO + cc * 32, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
+              tmem_st32(tO + cc * 32, o);
+            }
+          }
+          m_used = m_new;
+        }
+        const float mc = m_used * c;
+        float psum = 0.f;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float p0 = ex2(fmaf(__uint_as_float(sr[cc][e]), c, -mc));
+            const float p1 = ex2(fmaf(__uint_as_float(sr[cc][e + 1]), c, -mc));
+            psum += p0 + p1;
+            sr[cc >> 1][(cc & 1) * 16 + (e >> 1)] = pack_bf16(p0, p1);
+          }
+          if (cc & 1) tmem_st32(tS + (cc >> 1) * 32, sr[cc >> 1]);
+        }
+        l += psum;
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(smem_u32(&bars->p_ready[i]));
+      }
+      mbar_wait(smem_u32(&bars->pv_done[i]), (n_kv - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+      tc_fence_after();
+
+      // Eq. 5: bring O and l to the final row maximum, add the linear read-out, divide, store.
+      const int row = row_base + i * TC_BM + (warp & 3) * 32 + lane;
+      const bool valid = row < q1;
+      const float fin = ex2((m_used - m_true) * c);
+      float ws = fin, lam = 0.f, nL = 0.f;
+      const float* rrow = nullptr;
+      if (lo > 0) {
+        rrow = rd + ((size_t)bh * rd_rows + (size_t)((valid ? row : q0) - geo_q0(g, g.t0))) * (TC_D + 4);
+        lam = 1.f;
+        if (c_mode == C_ZERO) {
+          const float mm = m_true * scale, r = fmaxf(mm, 0.f);
+          ws = fin * __expf(mm - r);
+          lam = __expf(-r);
+        }
+        nL = rrow[TC_D];
+      }
+      const float inv = 1.f / (l * ws + lam * nL);
+      __nv_bfloat16* orow = out + head_offset(g, bh) + (long long)row * g.stride_n;
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        uint32_t o[32];
+        tmem_ld32(tO + cc * 32, o);
+        tmem_wait_ld();
+        if (valid) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 8) {
+            float a[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) a[u] = 0.f;
+            if (lo > 0) {
+              const float4 x0 = *reinterpret_cast<const float4*>(rrow + cc * 32 + e);
+              const float4 x1 = *reinterpret_cast<const float4*>(rrow + cc * 32 + e + 4);
+              a[0] = x0.x; a[1] = x0.y; a[2] = x0.z; a[3] = x0.w; a[4] = x1.x; a[5] = x1.y; a[6] = x1.z; a[7] = x1.w;
+            }
+            uint4 w;
+            w.x = pack_bf16((__uint_as_float(o[e + 0]) * ws + lam * a[0]) * inv, (__uint_as_float(o[e + 1]) * ws + lam * a[1]) * inv);
+            w.y = pack_bf16((__uint_as_float(o[e + 2]) * ws + lam * a[2]) * inv, (__uint_as_float(o[e + 3]) * ws + lam * a[3]) * inv);
+            w.z = pack_bf16((__uint_as_float(o[e + 4]) * ws + lam * a[4]) * inv, (__uint_as_float(o[e + 5]) * ws + lam * a[5]) * inv);
+            w.w = pack_bf16((__uint_as_float(o[e + 6]) * ws + lam * a[6]) * inv, (__uint_as_float(o[e + 7]) * ws + lam * a[7]) * inv);
+            *reinterpret_cast<uint4*>(orow + cc * 32 + e) = w;
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+
+struct TcWorkspace {
+  void* encode_fn = nullptr;   // cuTensorMapEncodeTiled, resolved through the runtime
+};
+
+inline bool tc_shape_supported(bool bf16, int d, int, int, int, int, int) { return bf16 && d == TC_D; }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline bool tc_workspace_create(TcWorkspace* w, int, int, int, int, size_t* extra) {
+  *extra = 0;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn)
+    return false;
+  w->encode_fn = fn;
+  return true;
+}
 inline void tc_workspace_destroy(TcWorkspace*) {}
-inline int tc_set_attributes() { return REHYAT_OK; }
-inline int tc_launch_group(TcWorkspace*, const void*, const void*, const void*, void*, const rehyat_phi_params*,
-                           const Geo&, int, int, int, int, int, bool, float*, float*, float*, int, int*,
-                           cudaStream_t, int*) {
-  return REHYAT_ERR_UNSUPPORTED;
+
+inline int tc_set_attributes() {
+  return cudaFuncSetAttribute(window_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess
+             ? REHYAT_OK : REHYAT_ERR_CUDA;
+}
+
+// Tensor map over one of q, k, v: dims (d, N, heads, batch), box [64 x 128 rows], 128-byte swizzle,
+// out-of-range rows read as zero.
+inline bool tc_make_tmap(const TcWorkspace* w, CUtensorMap* tm, const void* base, const Geo& g, int batch) {
+  const cuuint64_t dims[4] = {(cuuint64_t)TC_D, (cuuint64_t)g.N, (cuuint64_t)g.n_heads, (cuuint64_t)batch};
+  const cuuint64_t strides[3] = {(cuuint64_t)g.stride_n * 2, (cuuint64_t)g.stride_h * 2, (cuuint64_t)g.stride_b * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)TC_BN, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = ((EncodeTiledFn)w->encode_fn)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
+                                             strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// Launches window_tc for the chunks of one group.  `rd` is the linear read-out of the group's queries.
+inline int tc_launch_window(const TcWorkspace* w, const void* q, const void* k, const void* v, void* out, const Geo& g,
+                            int batch, const float* rd, int rd_rows, int c_mode, int* status, cudaStream_t st) {
+  CUtensorMap tq, tk, tv;
+  if (!tc_make_tmap(w, &tq, q, g, batch) || !tc_make_tmap(w, &tk, k, g, batch) || !tc_make_tmap(w, &tv, v, g, batch))
+    return REHYAT_ERR_CUDA;
+  const int pairs = (g.Np + TC_QT * TC_BM - 1) / (TC_QT * TC_BM);
+  window_tc<<<dim3(pairs, g.G, g.BH), TC_THREADS, TC_WIN_SMEM, st>>>(
+      tq, tk, tv, (__nv_bfloat16*)out, g, rd, rd_rows, 1.0f / sqrtf((float)TC_D), c_mode, status);
+  return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
 }  // namespace rehyat

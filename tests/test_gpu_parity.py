@@ -123,7 +123,8 @@ def test_small_cases_every_element(case, c_mode):
     # phi parameters x1.5: about 0.8 of the normaliser is linear, 13-20 % of phi in the squared part
     x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
     ref, frac = oracle_full(wl, x, c_mode)
-    y, _ = run_gpu(wl, x, c_mode=c_mode)
+    y, used = run_gpu(wl, x, c_mode=c_mode)
+    assert used == ("tensor" if (dtype == "bf16" and d == 128) else "simt")
     check(y, ref, dtype)
     if To < T - Tc and c_mode == "rowmax":
         assert frac.max() > 0.05
