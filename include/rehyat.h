@@ -55,9 +55,12 @@ typedef enum {
 typedef enum { REHYAT_C_ROWMAX = 0, REHYAT_C_ZERO = 1 } rehyat_c_mode;
 
 /* Kernel family.  AUTO: tensor-core (tcgen05) kernels when dtype is bf16 and the shape is one
- * they cover, SIMT fp32 kernels otherwise.  SIMT / TENSOR force one (TENSOR fails with
- * REHYAT_ERR_UNSUPPORTED where it does not apply). */
-typedef enum { REHYAT_IMPL_AUTO = 0, REHYAT_IMPL_SIMT = 1, REHYAT_IMPL_TENSOR = 2 } rehyat_impl;
+ * they cover (head_dim 128 for the softmax window; D_h = D' = 256 as well for the linear branch),
+ * SIMT fp32 kernels otherwise.  SIMT / TENSOR force one (TENSOR fails with REHYAT_ERR_UNSUPPORTED
+ * where it does not apply).  TENSOR_WINDOW: tensor-core window, SIMT linear branch (a cross-check). */
+typedef enum {
+  REHYAT_IMPL_AUTO = 0, REHYAT_IMPL_SIMT = 1, REHYAT_IMPL_TENSOR = 2, REHYAT_IMPL_TENSOR_WINDOW = 3
+} rehyat_impl;
 
 typedef struct rehyat_config {
   int32_t device;               /* CUDA device ordinal                                        */

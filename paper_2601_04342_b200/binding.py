@@ -14,7 +14,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_ARCH, ERR_ALLOC, ERR_DEVICE_
 DTYPE = {"bf16": 0, "fp32": 1}
 ACT = {"relu": 0, "identity": 1, "softplus": 2, "elu1": 3, "gelu": 4}
 C_MODE = {"rowmax": 0, "zero": 1}
-IMPL = {"auto": 0, "simt": 1, "tensor": 2}
+IMPL = {"auto": 0, "simt": 1, "tensor": 2, "tensor_window": 3}
 
 EXPORTS = ["rehyat_create", "rehyat_forward", "rehyat_forward_host", "rehyat_destroy",
            "rehyat_workspace_bytes", "rehyat_status", "rehyat_last_launches", "rehyat_last_impl",

@@ -82,7 +82,7 @@ int check_config(const rehyat_config* c) {
     return REHYAT_ERR_INVALID_ARG;
   if (c->act_hidden < 0 || c->act_hidden > 4 || c->act_out < 0 || c->act_out > 4) return REHYAT_ERR_INVALID_ARG;
   if (c->c_mode != REHYAT_C_ROWMAX && c->c_mode != REHYAT_C_ZERO) return REHYAT_ERR_INVALID_ARG;
-  if (c->impl < REHYAT_IMPL_AUTO || c->impl > REHYAT_IMPL_TENSOR) return REHYAT_ERR_INVALID_ARG;
+  if (c->impl < REHYAT_IMPL_AUTO || c->impl > REHYAT_IMPL_TENSOR_WINDOW) return REHYAT_ERR_INVALID_ARG;
   if (c->max_tokens_per_frame < 1 || c->max_chunk_frames < 1 || c->group_tokens < 0) return REHYAT_ERR_INVALID_ARG;
   if ((long long)c->max_tokens_per_frame * c->max_chunk_frames > (1 << 24)) return REHYAT_ERR_INVALID_ARG;
   if (c->head_dim < 1) return REHYAT_ERR_INVALID_ARG;
@@ -180,8 +180,9 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
   const rehyat_config& c = ctx->cfg;
   ctx->tensor_ok = tc_shape_supported(c.dtype == REHYAT_DTYPE_BF16, c.head_dim, c.phi_hidden, c.phi_dim,
                                       c.poly_degree, c.act_hidden, c.act_out);
-  if (c.impl == REHYAT_IMPL_TENSOR && !ctx->tensor_ok) { delete ctx; return REHYAT_ERR_UNSUPPORTED; }
+  if ((c.impl == REHYAT_IMPL_TENSOR || c.impl == REHYAT_IMPL_TENSOR_WINDOW) && !ctx->tensor_ok) { delete ctx; return REHYAT_ERR_UNSUPPORTED; }
   if (c.impl == REHYAT_IMPL_SIMT) ctx->tensor_ok = false;
+  ctx->tc.phi_ok = ctx->tensor_ok && c.impl != REHYAT_IMPL_TENSOR_WINDOW && tc_phi_supported(c.phi_hidden, c.phi_dim);
 
   const int np_max = c.max_tokens_per_frame * c.max_chunk_frames;
   const int want = c.group_tokens > 0 ? c.group_tokens : 32768;
@@ -322,8 +323,29 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
     int rc;
     if (ctx->tensor_ok) {
       using B = __nv_bfloat16;
-      rc = launch_group_simt<B, 128>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot,
-                                     any_linear, st, /*with_window=*/false);
+      if (!ctx->tc.phi_ok) {
+        rc = launch_group_simt<B, 128>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot,
+                                       any_linear, st, /*with_window=*/false);
+      } else if (any_linear) {
+        ctx->prof.begin(REHYAT_PROF_STATE, st);
+        rc = tc_launch_state(&ctx->tc, k, v, phi, g, batch, c.poly_degree, c.act_hidden, c.act_out, n_split,
+                             ctx->partial, ctx->status_dev, st);
+        ctx->prof.end(REHYAT_PROF_STATE, st);
+        const size_t per_slot = (size_t)g.BH * c.phi_dim * (c.head_dim + 4);
+        ctx->prof.begin(REHYAT_PROF_SCAN, st);
+        scan_states<<<(unsigned)((per_slot + 255) / 256), 256, 0, st>>>(ctx->partial, ctx->state, per_slot, g.G, n_split,
+                                                                         carry_slot, ctx->tc.state_bf16, c.head_dim);
+        ctx->prof.end(REHYAT_PROF_SCAN, st);
+        if (rc == REHYAT_OK) {
+          ctx->prof.begin(REHYAT_PROF_READOUT, st);
+          rc = tc_launch_readout(&ctx->tc, q, phi, g, batch, c.poly_degree, c.act_hidden, c.act_out, ctx->state,
+                                 ctx->readout, ctx->rd_rows, ctx->status_dev, st);
+          ctx->prof.end(REHYAT_PROF_READOUT, st);
+        }
+        ctx->last_launches += 3;
+      } else {
+        rc = REHYAT_OK;
+      }
       if (rc == REHYAT_OK) {
         ctx->prof.begin(REHYAT_PROF_WINDOW, st);
         rc = tc_launch_window(&ctx->tc, q, k, v, out, g, batch, ctx->readout, ctx->rd_rows, c.c_mode,

@@ -1,0 +1,406 @@
+// Tensor-core kernels of the linear branch for bf16, head_dim 128, phi widths D_h = D' = 256.
+//
+// phi_tc<MODE> evaluates the feature map of Section 3.2 ("Characterization of phi") on tiles of
+// 128 tokens with tcgen05.mma and feeds it straight into the contraction that consumes it:
+//   PHI_STATE    phi_k(K tile)^T [V | 1] accumulated in TMEM over the CTA's share of the keys a
+//                chunk newly admits (Eq. 17-18); flushed once as an fp32 partial state.
+//   PHI_READOUT  phi_q(Q tile) s_t on the tensor core and phi_q(Q tile) z_t on the ALUs
+//                (Eq. 7, 9, 16); written as the fp32 linear read-out of the tile.
+//
+// Per tile the chain is  H = act(X W1^T + b1) -> U = act(H W2^T + b2) -> phi = U^(1..P)  with the
+// two GEMMs done as 128x128 halves through one 128-column TMEM scratch accumulator:
+//   warps 0-3  one thread per token (= TMEM lane): bias, activation, power, bf16, swizzled smem tile
+//   warp 4     TMA producer: X (and V), weight / state tiles [128 x 64] through a 3-stage ring
+//   warp 5     UMMA issuer
+// The phi tile is written once in the 128-byte-swizzled [token][feature] image; the state GEMM reads
+// it as an MN-major A operand (features are M), the read-out GEMM as a K-major A operand.
+#pragma once
+
+#include <cuda.h>
+
+#include "rehyat_common.cuh"
+#include "rehyat_ptx.cuh"
+
+namespace rehyat {
+
+enum PhiMode : int { PHI_STATE = 0, PHI_READOUT = 1 };
+
+constexpr int PH_D = 128, PH_DH = 256, PH_DP = 256, PH_SD = PH_D + 4;
+constexpr int PH_THREADS = 192;
+constexpr int PH_RING = 3;
+constexpr int PH_WT_BYTES = 128 * 64 * 2;          // one weight / state tile: 16 KB
+constexpr int PH_TILE_BYTES = 128 * 128 * 2;       // X, V, phi half: 32 KB (two swizzled sub-tiles)
+constexpr int PH_SUB = PH_TILE_BYTES / 2;
+// shared memory map (bytes from the 1024-aligned base)
+constexpr int PH_OFF_X = 0;
+constexpr int PH_OFF_V = PH_OFF_X + PH_TILE_BYTES;
+constexpr int PH_OFF_HB = PH_OFF_V + PH_TILE_BYTES;            // 64 KB; its first half doubles as phi half 1
+constexpr int PH_OFF_PHI0 = PH_OFF_HB + 2 * PH_TILE_BYTES;
+constexpr int PH_OFF_RING = PH_OFF_PHI0 + PH_TILE_BYTES;
+constexpr int PH_OFF_ONES = PH_OFF_RING + PH_RING * PH_WT_BYTES; // [16 x 128] K-major, row 0 = 1
+constexpr int PH_OFF_BIAS = PH_OFF_ONES + 4096;                 // b1[256], b2[256], z[256] fp32
+constexpr int PH_OFF_BARS = PH_OFF_BIAS + 3 * 256 * 4;
+constexpr int PH_SMEM = PH_OFF_BARS + 512 + 1024;
+
+enum PhErr : int { PH_ERR_LOAD = 16, PH_ERR_MMA = 32, PH_ERR_EPI = 64 };
+
+struct PhBars {
+  uint64_t x_full, x_empty, v_full, v_empty;
+  uint64_t ring_full[PH_RING], ring_empty[PH_RING];
+  uint64_t acc_ready, epi_done, out_ready, out_read;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct PhiTcArgs {
+  const __nv_bfloat16* b1;     // [heads][256]
+  const __nv_bfloat16* b2;     // [heads][256]
+  int P, act_hidden, act_out;
+  int n_split;                 // PHI_STATE: splits of a chunk's increment
+  float* partial;              // PHI_STATE: [G][n_split][BH][256][132]
+  const float* state;          // PHI_READOUT: fp32 states (z column is read)
+  float* rd;                   // PHI_READOUT: [BH][rd_rows][132]
+  int rd_rows;
+  int tiles_per_cta;           // PHI_READOUT
+  int* status;
+};
+
+// tm_x: K (state) or Q (read-out), 4-D like the window kernel's maps.  tm_v: V (state only).
+// tm_w1: (128, 256, heads), tm_w2: (256, 256, heads), boxes [64 x 128].  tm_s: bf16 states
+// (128, 256, G*BH), box [64 x 64] (read-out only).
+template <int MODE>
+__global__ void __launch_bounds__(PH_THREADS, 1)
+phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_v,
+       const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2,
+       const __grid_constant__ CUtensorMap tm_s, Geo g, PhiTcArgs a) {
+  using namespace ptx;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t sb = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (sb - smem_u32(smem_raw));
+  PhBars* bars = reinterpret_cast<PhBars*>(smem + PH_OFF_BARS);
+  float* s_b1 = reinterpret_cast<float*>(smem + PH_OFF_BIAS);
+  float* s_b2 = s_b1 + 256;
+  float* s_z = s_b2 + 256;
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
+  const int b_idx = bh / g.n_heads, h_idx = bh % g.n_heads;
+
+  // token range [tok_a, tok_b) of this CTA
+  int tok_a, tok_b;
+  if (MODE == PHI_STATE) {
+    const int lo_prev = t > 0 ? geo_lo(g, t - 1) : 0, lo = geo_lo(g, t);
+    int per = (lo - lo_prev + a.n_split - 1) / a.n_split;
+    per = (per + 127) / 128 * 128;
+    tok_a = min(lo_prev + (int)blockIdx.x * per, lo);
+    tok_b = min(tok_a + per, lo);
+  } else {
+    if (geo_lo(g, t) == 0) return;                                  // empty linear set
+    const int q0 = geo_q0(g, t), q1 = geo_q1(g, t);
+    tok_a = min(q0 + (int)blockIdx.x * a.tiles_per_cta * 128, q1);
+    tok_b = min(tok_a + a.tiles_per_cta * 128, q1);
+    if (tok_a >= tok_b) return;
+  }
+  const int n_tiles = (tok_b - tok_a + 127) / 128;
+
+  if (MODE == PHI_STATE && n_tiles == 0) {                          // nothing admitted: the partial is zero
+    float* dst = a.partial + (((size_t)ci * a.n_split + blockIdx.x) * g.BH + bh) * PH_DP * PH_SD;
+    for (int i = threadIdx.x; i < PH_DP * PH_SD / 4; i += PH_THREADS)
+      reinterpret_cast<float4*>(dst)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    return;
+  }
+
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bars->x_full), 1); mbar_init(smem_u32(&bars->x_empty), 1);
+    mbar_init(smem_u32(&bars->v_full), 1); mbar_init(smem_u32(&bars->v_empty), 1);
+    for (int s = 0; s < PH_RING; ++s) {
+      mbar_init(smem_u32(&bars->ring_full[s]), 1); mbar_init(smem_u32(&bars->ring_empty[s]), 1);
+    }
+    mbar_init(smem_u32(&bars->acc_ready), 1); mbar_init(smem_u32(&bars->epi_done), 128);
+    mbar_init(smem_u32(&bars->out_ready), 1); mbar_init(smem_u32(&bars->out_read), 128);
+    bars->abort_flag = 0;
+    fence_mbar_init();
+  }
+  // biases (and z_t) as fp32; the ones tile: row 0 of both 64-column sub-tiles is 1, the rest 0
+  for (int i = threadIdx.x; i < 256; i += PH_THREADS) {
+    s_b1[i] = __bfloat162float(a.b1[(size_t)h_idx * 256 + i]);
+    s_b2[i] = __bfloat162float(a.b2[(size_t)h_idx * 256 + i]);
+    if (MODE == PHI_READOUT) s_z[i] = a.state[(((size_t)ci * g.BH + bh) * PH_DP + i) * PH_SD + PH_D];
+  }
+  if (MODE == PHI_STATE) {
+    uint32_t* ones = reinterpret_cast<uint32_t*>(smem + PH_OFF_ONES);
+    for (int i = threadIdx.x; i < 1024; i += PH_THREADS) {
+      const int byte = i * 4, sub = byte / 2048, within = byte % 2048;
+      ones[i] = (within < 128 && sub < 2) ? 0x3F803F80u : 0u;       // two bf16 ones
+    }
+    fence_proxy_async_smem();
+  }
+  if (warp == 5) {
+    tmem_alloc(smem_u32(&bars->tmem_base), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+  // TMEM columns: scratch [0,128); STATE: S half0 [128,256) S half1 [256,384) z0 [384,400) z1 [400,416);
+  // READOUT: R [128,256)
+  constexpr uint32_t T_SCR = 0, T_ACC = 128, T_Z = 384;
+
+  const uint32_t sX = sb + PH_OFF_X, sV = sb + PH_OFF_V, sHb = sb + PH_OFF_HB, sPhi0 = sb + PH_OFF_PHI0,
+                 sRing = sb + PH_OFF_RING, sOnes = sb + PH_OFF_ONES;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ TMA producer
+    if (elect_one()) {
+      prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_w1); prefetch_tensormap(&tm_w2);
+      uint32_t ring_i = 0;
+      bool alive = true;
+      auto ring_load = [&](const CUtensorMap* tm, int x, int y, int z, bool state_tile) {
+        const int s = ring_i % PH_RING;
+        const uint32_t ph = (ring_i / PH_RING) & 1;
+        alive = alive && mbar_wait(smem_u32(&bars->ring_empty[s]), ph ^ 1, abort_flag, a.status, PH_ERR_LOAD);
+        if (!alive) return;
+        const uint32_t full = smem_u32(&bars->ring_full[s]);
+        mbar_expect_tx(full, PH_WT_BYTES);
+        if (!state_tile) {
+          tma_load_3d(sRing + s * PH_WT_BYTES, tm, full, x, y, z);
+        } else {                                                     // [64 features x 128 d] as two 64-column boxes
+          tma_load_3d(sRing + s * PH_WT_BYTES, tm, full, 0, y, z);
+          tma_load_3d(sRing + s * PH_WT_BYTES + 8192, tm, full, 64, y, z);
+        }
+        ++ring_i;
+      };
+      for (int j = 0; j < n_tiles && alive; ++j) {
+        const int tok0 = tok_a + j * 128;
+        alive = mbar_wait(smem_u32(&bars->x_empty), (j & 1) ^ 1, abort_flag, a.status, PH_ERR_LOAD);
+        if (!alive) break;
+        const uint32_t xf = smem_u32(&bars->x_full);
+        mbar_expect_tx(xf, PH_TILE_BYTES);
+        tma_load_4d(sX, &tm_x, xf, 0, tok0, h_idx, b_idx);
+        tma_load_4d(sX + PH_SUB, &tm_x, xf, 64, tok0, h_idx, b_idx);
+        for (int nh = 0; nh < 2; ++nh)
+          for (int ks = 0; ks < 2; ++ks) ring_load(&tm_w1, ks * 64, nh * 128, h_idx, false);
+        if (MODE == PHI_STATE) {
+          alive = alive && mbar_wait(smem_u32(&bars->v_empty), (j & 1) ^ 1, abort_flag, a.status, PH_ERR_LOAD);
+          if (!alive) break;
+          const uint32_t vf = smem_u32(&bars->v_full);
+          mbar_expect_tx(vf, PH_TILE_BYTES);
+          tma_load_4d(sV, &tm_v, vf, 0, tok0, h_idx, b_idx);
+          tma_load_4d(sV + PH_SUB, &tm_v, vf, 64, tok0, h_idx, b_idx);
+        }
+        for (int ks = 0; ks < 4; ++ks) ring_load(&tm_w2, ks * 64, 0, h_idx, false);
+        for (int ks = 0; ks < 4; ++ks) ring_load(&tm_w2, ks * 64, 128, h_idx, false);
+        if (MODE == PHI_READOUT)
+          for (int f = 0; f < 4; ++f) ring_load(&tm_s, 0, f * 64, ci * g.BH + bh, true);
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ UMMA issuer
+    if (elect_one()) {
+      constexpr uint32_t id_kk = idesc_bf16(128, 128, 0, 0);       // A K-major, B K-major   (the two MLP GEMMs)
+      constexpr uint32_t id_st = idesc_bf16(128, 128, 1, 1);       // A = phi^T (MN-major), B = V (MN-major)
+      constexpr uint32_t id_z = idesc_bf16(128, 16, 1, 0);         // A = phi^T (MN-major), B = ones (K-major)
+      constexpr uint32_t id_rd = idesc_bf16(128, 128, 0, 1);       // A = phi (K-major),    B = state (MN-major)
+      uint32_t ring_i = 0, n_epi = 0;
+      auto ring_wait = [&]() -> uint32_t {
+        const int s = ring_i % PH_RING;
+        mbar_wait(smem_u32(&bars->ring_full[s]), (ring_i / PH_RING) & 1, abort_flag, a.status, PH_ERR_MMA);
+        tc_fence_after();
+        return sRing + s * PH_WT_BYTES;
+      };
+      auto ring_release = [&]() {
+        umma_commit(smem_u32(&bars->ring_empty[ring_i % PH_RING]));
+        ++ring_i;
+      };
+      auto wait_epi = [&]() {
+        mbar_wait(smem_u32(&bars->epi_done), n_epi & 1, abort_flag, a.status, PH_ERR_MMA);
+        ++n_epi;
+        tc_fence_after();
+      };
+      // one 128x128 half of an MLP GEMM: A tile [128 x 64*nks] K-major at a_base, B tiles from the ring
+      auto mlp_half = [&](uint32_t a_base, int nks) {
+        for (int ks = 0; ks < nks; ++ks) {
+          const uint32_t bt = ring_wait();
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            umma_ss(tmem + T_SCR, smem_desc_sw128(a_base + ks * PH_SUB + kk * 32, 16, 1024),
+                    smem_desc_sw128(bt + kk * 32, 16, 1024), id_kk, (ks | kk) != 0);
+          ring_release();
+        }
+        umma_commit(smem_u32(&bars->acc_ready));
+      };
+      // contraction that consumes phi half `c` (its tile is at phi_base)
+      auto consume_half = [&](int c, uint32_t phi_base, bool first_tile) {
+        if (MODE == PHI_STATE) {
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {                          // 16 tokens per step
+            const uint64_t ad = smem_desc_sw128(phi_base + kk * 2048, PH_SUB, 1024);
+            umma_ss(tmem + T_ACC + c * 128, ad, smem_desc_sw128(sV + kk * 2048, PH_SUB, 1024), id_st,
+                    (!first_tile || kk > 0) ? 1u : 0u);
+            umma_ss(tmem + T_Z + c * 16, ad, smem_desc_sw128(sOnes + (kk >> 2) * 2048 + (kk & 3) * 32, 16, 1024), id_z,
+                    (!first_tile || kk > 0) ? 1u : 0u);
+          }
+        } else {
+          for (int f = 0; f < 2; ++f) {                             // 64 features per state tile
+            const uint32_t bt = ring_wait();
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              umma_ss(tmem + T_ACC, smem_desc_sw128(phi_base + f * PH_SUB + kk * 32, 16, 1024),
+                      smem_desc_sw128(bt + kk * 2048, 8192, 1024), id_rd, (c | f | kk) != 0);
+            ring_release();
+          }
+        }
+      };
+      for (int j = 0; j < n_tiles; ++j) {
+        mbar_wait(smem_u32(&bars->x_full), j & 1, abort_flag, a.status, PH_ERR_MMA);
+        tc_fence_after();
+        if (j > 0) wait_epi();                                      // scratch free: phi half 1 of tile j-1 written
+        if (j > 0) {                                                // ... and consumed
+          if (MODE == PHI_STATE) mbar_wait(smem_u32(&bars->v_full), (j - 1) & 1, abort_flag, a.status, PH_ERR_MMA);
+          tc_fence_after();
+          consume_half(1, sHb, j == 1);
+          if (MODE == PHI_STATE) umma_commit(smem_u32(&bars->v_empty));
+          if (MODE == PHI_READOUT) umma_commit(smem_u32(&bars->out_ready));
+        }
+        mlp_half(sX, 2);                                            // H[:, 0:128]
+        wait_epi();
+        mlp_half(sX, 2);                                            // H[:, 128:256]
+        umma_commit(smem_u32(&bars->x_empty));
+        wait_epi();
+        mlp_half(sHb, 4);                                           // U[:, 0:128]
+        wait_epi();
+        mlp_half(sHb, 4);                                           // U[:, 128:256]
+        if (MODE == PHI_STATE) {
+          mbar_wait(smem_u32(&bars->v_full), j & 1, abort_flag, a.status, PH_ERR_MMA);
+          tc_fence_after();
+        } else if (j > 0) {
+          mbar_wait(smem_u32(&bars->out_read), (j - 1) & 1, abort_flag, a.status, PH_ERR_MMA);
+          tc_fence_after();
+        }
+        consume_half(0, sPhi0, j == 0);
+      }
+      wait_epi();
+      consume_half(1, sHb, n_tiles == 1);
+      umma_commit(smem_u32(&bars->out_ready));
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogues: thread = token = TMEM lane
+    const int r = warp * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    uint32_t n_acc = 0;
+    const int part_w = PH_DP / a.P;
+    for (int j = 0; j < n_tiles; ++j) {
+      const bool tok_valid = tok_a + j * 128 + r < tok_b;
+      float nl = 0.f;
+      for (int step = 0; step < 4; ++step) {                        // H half 0, H half 1, U half 0, U half 1
+        mbar_wait(smem_u32(&bars->acc_ready), n_acc & 1, abort_flag, a.status, PH_ERR_EPI);
+        ++n_acc;
+        tc_fence_after();
+        const int half = step & 1;
+        const bool is_u = step >= 2;
+        const uint32_t dst = !is_u ? sHb : (half == 0 ? sPhi0 : sHb);
+        const int dst_col0 = !is_u ? half * 128 : 0;
+        const float* bias = (is_u ? s_b2 : s_b1) + half * 128;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t x[32];
+          tmem_ld32(tmem + lane_off + T_SCR + cc * 32, x);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; e += 8) {
+            float y[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const int col = cc * 32 + e + u;
+              float val = __uint_as_float(x[e + u]) + bias[col];
+              if (!is_u) {
+                val = apply_act(val, a.act_hidden);
+              } else {
+                val = poly_power(apply_act(val, a.act_out), (half * 128 + col) / part_w);
+                if (!tok_valid) val = 0.f;
+              }
+              y[u] = val;
+            }
+            uint4 w;
+            w.x = pack_bf16(y[0], y[1]); w.y = pack_bf16(y[2], y[3]);
+            w.z = pack_bf16(y[4], y[5]); w.w = pack_bf16(y[6], y[7]);
+            if (MODE == PHI_READOUT && is_u) {
+              // phi_q(q_r) . z_t with the same bf16-rounded features the tensor core sees
+              const float* zz = s_z + half * 128 + cc * 32 + e;
+              const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                nl = fmaf(__uint_as_float(ww[u] << 16), zz[2 * u], nl);
+                nl = fmaf(__uint_as_float(ww[u] & 0xffff0000u), zz[2 * u + 1], nl);
+              }
+            }
+            st_tile_chunk_sw128(dst, PH_SUB, r, dst_col0 + cc * 32 + e, w);
+          }
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        mbar_arrive(smem_u32(&bars->epi_done));
+      }
+      if (MODE == PHI_READOUT) {
+        // read-out of tile j is complete after the consumer of phi half 1, issued at the start of
+        // the next tile (or after the loop)
+        mbar_wait(smem_u32(&bars->out_ready), j & 1, abort_flag, a.status, PH_ERR_EPI);
+        tc_fence_after();
+        const int tok = tok_a + j * 128 + r;
+        float* dst = a.rd + ((size_t)bh * a.rd_rows + (size_t)((tok_valid ? tok : tok_a) - geo_q0(g, g.t0))) * PH_SD;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t x[32];
+          tmem_ld32(tmem + lane_off + T_ACC + cc * 32, x);
+          tmem_wait_ld();
+          if (tok_valid) {
+#pragma unroll
+            for (int e = 0; e < 32; e += 4)
+              *reinterpret_cast<float4*>(dst + cc * 32 + e) =
+                  make_float4(__uint_as_float(x[e]), __uint_as_float(x[e + 1]), __uint_as_float(x[e + 2]),
+                              __uint_as_float(x[e + 3]));
+          }
+        }
+        if (tok_valid) dst[PH_D] = nl;
+        tc_fence_before();
+        mbar_arrive(smem_u32(&bars->out_read));
+      }
+    }
+    if (MODE == PHI_STATE) {
+      // flush: lane r holds feature c*128 + r of half c
+      mbar_wait(smem_u32(&bars->out_ready), 0, abort_flag, a.status, PH_ERR_EPI);
+      tc_fence_after();
+      float* base = a.partial + (((size_t)ci * a.n_split + blockIdx.x) * g.BH + bh) * PH_DP * PH_SD;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        float* dst = base + (size_t)(c * 128 + r) * PH_SD;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t x[32];
+          tmem_ld32(tmem + lane_off + T_ACC + c * 128 + cc * 32, x);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; e += 4)
+            *reinterpret_cast<float4*>(dst + cc * 32 + e) =
+                make_float4(__uint_as_float(x[e]), __uint_as_float(x[e + 1]), __uint_as_float(x[e + 2]),
+                            __uint_as_float(x[e + 3]));
+        }
+        uint32_t zc[16];
+        tmem_ld16(tmem + lane_off + T_Z + c * 16, zc);
+        tmem_wait_ld();
+        *reinterpret_cast<float4*>(dst + PH_D) = make_float4(__uint_as_float(zc[0]), 0.f, 0.f, 0.f);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+}  // namespace rehyat

@@ -51,18 +51,33 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  `abort_flag` (shared memory) is set by whichever thread of the CTA first runs out
 // of patience; once set, every wait of the CTA returns at once so that all roles drain and the
 // kernel ends.  Returns false if the wait was given up.
-constexpr uint32_t kWaitPolls = 1u << 22;   // try_wait itself suspends for a while per poll
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status_word, int code) {
-  if (mbar_try_wait(bar, parity)) return true;
-  for (uint32_t i = 0; i < kWaitPolls; ++i) {
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // one second of wall time per wait
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            int* status_word, int code) {
+  const unsigned long long t0 = global_timer_ns();
+  for (uint32_t i = 0;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (i > 64) __nanosleep(32);
+    if ((i & 63u) == 63u) {
+      // another CTA of the grid has already given up: drain at once instead of waiting a second each
+      if (*reinterpret_cast<volatile int*>(status_word) != 0) { *abort_flag = 1; return false; }
+      if (global_timer_ns() - t0 > kWaitLimitNs) break;
+      __nanosleep(64);
+    }
   }
   *abort_flag = 1;
   atomicOr(status_word, code);
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status_word, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status_word, code);
 }
 
 // ----------------------------------------------------------------------------- TMA
@@ -183,6 +198,15 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
 __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int a_mn_major, int b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
          ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// Writes eight bf16 (one 16-byte chunk) of row `r`, columns [col, col+8) of a [rows x 128] bf16 tile
+// kept as two [rows x 64] sub-tiles in the 128-byte-swizzled image described above.  `sub_bytes` is
+// the size of one sub-tile (rows * 128).
+__device__ __forceinline__ void st_tile_chunk_sw128(uint32_t tile, uint32_t sub_bytes, int r, int col, uint4 v) {
+  const uint32_t addr = tile + (uint32_t)(col >> 6) * sub_bytes + (uint32_t)r * 128u +
+                        ((((uint32_t)(col & 63) >> 3) ^ ((uint32_t)r & 7u)) << 4);
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
 __device__ __forceinline__ float ex2(float x) {

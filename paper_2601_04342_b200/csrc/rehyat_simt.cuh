@@ -162,15 +162,20 @@ state_partial_simt(const T* __restrict__ k, const T* __restrict__ v, PhiPtrs<T> 
 // One thread per state element; the chunk axis is walked in order, splits in fixed order, so the
 // result does not depend on scheduling.
 __global__ void scan_states(const float* __restrict__ partial, float* __restrict__ state,
-                            size_t per_slot, int G, int n_split, int carry_slot) {
+                            size_t per_slot, int G, int n_split, int carry_slot,
+                            __nv_bfloat16* __restrict__ state_bf16 = nullptr, int D = 0) {
   const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= per_slot) return;
   float run = carry_slot >= 0 ? state[(size_t)carry_slot * per_slot + e] : 0.f;
+  // optional bf16 copy of the s part, [slot][bh][feature][D], the B operand of the tensor-core read-out
+  const size_t row = e / (D + 4), col = e % (D + 4);
+  const size_t per_slot_b = per_slot / (D + 4) * D;
   for (int i = 0; i < G; ++i) {
     float inc = 0.f;
     for (int s = 0; s < n_split; ++s) inc += partial[((size_t)i * n_split + s) * per_slot + e];
     run += inc;
     state[(size_t)i * per_slot + e] = run;
+    if (state_bf16 != nullptr && col < (size_t)D) state_bf16[(size_t)i * per_slot_b + row * D + col] = __float2bfloat16_rn(run);
   }
 }
 

@@ -19,6 +19,7 @@
 #include "../../include/rehyat.h"
 #include "rehyat_common.cuh"
 #include "rehyat_ptx.cuh"
+#include "rehyat_phi_tc.cuh"
 
 namespace rehyat {
 
@@ -305,16 +306,19 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
 // ---------------------------------------------------------------------------------------------
 
 struct TcWorkspace {
-  void* encode_fn = nullptr;   // cuTensorMapEncodeTiled, resolved through the runtime
+  void* encode_fn = nullptr;            // cuTensorMapEncodeTiled, resolved through the runtime
+  __nv_bfloat16* state_bf16 = nullptr;  // [Gmax][BHmax][256][128]: bf16 copy of s_t for the read-out GEMM
+  bool phi_ok = false;                  // the linear branch runs on the tensor-core kernels too
 };
 
 inline bool tc_shape_supported(bool bf16, int d, int, int, int, int, int) { return bf16 && d == TC_D; }
+inline bool tc_phi_supported(int Dh, int Dp) { return Dh == PH_DH && Dp == PH_DP; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-inline bool tc_workspace_create(TcWorkspace* w, int, int, int, int, size_t* extra) {
+inline bool tc_workspace_create(TcWorkspace* w, int bh_max, int Gmax, int d, int Dp, size_t* extra) {
   *extra = 0;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -322,13 +326,29 @@ inline bool tc_workspace_create(TcWorkspace* w, int, int, int, int, size_t* extr
       qres != cudaDriverEntryPointSuccess || !fn)
     return false;
   w->encode_fn = fn;
+  if (w->phi_ok) {
+    const size_t bytes = (size_t)Gmax * bh_max * Dp * d * sizeof(__nv_bfloat16);
+    if (cudaMalloc(&w->state_bf16, bytes) != cudaSuccess) return false;
+    *extra = bytes;
+  }
   return true;
 }
-inline void tc_workspace_destroy(TcWorkspace*) {}
+inline void tc_workspace_destroy(TcWorkspace* w) { cudaFree(w->state_bf16); w->state_bf16 = nullptr; }
 
 inline int tc_set_attributes() {
-  return cudaFuncSetAttribute(window_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess
-             ? REHYAT_OK : REHYAT_ERR_CUDA;
+  bool ok = cudaFuncSetAttribute(window_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(phi_tc<PHI_STATE>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(phi_tc<PHI_READOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess;
+  return ok ? REHYAT_OK : REHYAT_ERR_CUDA;
+}
+
+inline bool tc_encode(const TcWorkspace* w, CUtensorMap* tm, const void* base, int rank, const cuuint64_t* dims,
+                      const cuuint64_t* strides, const cuuint32_t* box) {
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return ((EncodeTiledFn)w->encode_fn)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims,
+                                       strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+         CUDA_SUCCESS;
 }
 
 // Tensor map over one of q, k, v: dims (d, N, heads, batch), box [64 x 128 rows], 128-byte swizzle,
@@ -337,12 +357,15 @@ inline bool tc_make_tmap(const TcWorkspace* w, CUtensorMap* tm, const void* base
   const cuuint64_t dims[4] = {(cuuint64_t)TC_D, (cuuint64_t)g.N, (cuuint64_t)g.n_heads, (cuuint64_t)batch};
   const cuuint64_t strides[3] = {(cuuint64_t)g.stride_n * 2, (cuuint64_t)g.stride_h * 2, (cuuint64_t)g.stride_b * 2};
   const cuuint32_t box[4] = {64, (cuuint32_t)TC_BN, 1, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  CUresult r = ((EncodeTiledFn)w->encode_fn)(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
-                                             strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  return tc_encode(w, tm, base, 4, dims, strides, box);
+}
+// Row-major [planes][rows][cols] bf16 matrix stack, box [64 cols x box_rows].
+inline bool tc_make_tmap_3d(const TcWorkspace* w, CUtensorMap* tm, const void* base, int cols, int rows, int planes,
+                            int box_rows) {
+  const cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)planes};
+  const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * rows * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  return tc_encode(w, tm, base, 3, dims, strides, box);
 }
 
 // Launches window_tc for the chunks of one group.  `rd` is the linear read-out of the group's queries.
@@ -354,6 +377,43 @@ inline int tc_launch_window(const TcWorkspace* w, const void* q, const void* k, 
   const int pairs = (g.Np + TC_QT * TC_BM - 1) / (TC_QT * TC_BM);
   window_tc<<<dim3(pairs, g.G, g.BH), TC_THREADS, TC_WIN_SMEM, st>>>(
       tq, tk, tv, (__nv_bfloat16*)out, g, rd, rd_rows, 1.0f / sqrtf((float)TC_D), c_mode, status);
+  return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
+}
+
+// phi_k + chunk-state partial sums of one group (Eq. 17-18).
+inline int tc_launch_state(const TcWorkspace* w, const void* k, const void* v, const rehyat_phi_params* phi,
+                           const Geo& g, int batch, int P, int act_hidden, int act_out, int n_split, float* partial,
+                           int* status, cudaStream_t st) {
+  CUtensorMap tk, tv, tw1, tw2;
+  if (!tc_make_tmap(w, &tk, k, g, batch) || !tc_make_tmap(w, &tv, v, g, batch) ||
+      !tc_make_tmap_3d(w, &tw1, phi->k_W1, PH_D, PH_DH, g.n_heads, 128) ||
+      !tc_make_tmap_3d(w, &tw2, phi->k_W2, PH_DH, PH_DP, g.n_heads, 128))
+    return REHYAT_ERR_CUDA;
+  PhiTcArgs a = {};
+  a.b1 = (const __nv_bfloat16*)phi->k_b1; a.b2 = (const __nv_bfloat16*)phi->k_b2;
+  a.P = P; a.act_hidden = act_hidden; a.act_out = act_out;
+  a.n_split = n_split; a.partial = partial; a.status = status;
+  phi_tc<PHI_STATE><<<dim3(n_split, g.G, g.BH), PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, tw2, g, a);
+  return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
+}
+
+// phi_q + linear read-out of one group's queries (Eq. 7, 9, 16).
+inline int tc_launch_readout(const TcWorkspace* w, const void* q, const rehyat_phi_params* phi, const Geo& g, int batch,
+                             int P, int act_hidden, int act_out, const float* state, float* rd, int rd_rows,
+                             int* status, cudaStream_t st) {
+  CUtensorMap tq, tw1, tw2, ts;
+  if (!tc_make_tmap(w, &tq, q, g, batch) || !tc_make_tmap_3d(w, &tw1, phi->q_W1, PH_D, PH_DH, g.n_heads, 128) ||
+      !tc_make_tmap_3d(w, &tw2, phi->q_W2, PH_DH, PH_DP, g.n_heads, 128) ||
+      !tc_make_tmap_3d(w, &ts, w->state_bf16, PH_D, PH_DP, g.G * g.BH, 64))
+    return REHYAT_ERR_CUDA;
+  PhiTcArgs a = {};
+  a.b1 = (const __nv_bfloat16*)phi->q_b1; a.b2 = (const __nv_bfloat16*)phi->q_b2;
+  a.P = P; a.act_hidden = act_hidden; a.act_out = act_out;
+  a.state = state; a.rd = rd; a.rd_rows = rd_rows; a.status = status;
+  a.tiles_per_cta = 4;
+  const int tiles = (g.Np + 127) / 128;
+  const int ctas = (tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
+  phi_tc<PHI_READOUT><<<dim3(ctas, g.G, g.BH), PH_THREADS, PH_SMEM, st>>>(tq, tq, tw1, tw2, ts, g, a);
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
