@@ -182,7 +182,7 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
                                       c.poly_degree, c.act_hidden, c.act_out);
   if ((c.impl == REHYAT_IMPL_TENSOR || c.impl == REHYAT_IMPL_TENSOR_WINDOW) && !ctx->tensor_ok) { delete ctx; return REHYAT_ERR_UNSUPPORTED; }
   if (c.impl == REHYAT_IMPL_SIMT) ctx->tensor_ok = false;
-  ctx->tc.phi_ok = ctx->tensor_ok && c.impl != REHYAT_IMPL_TENSOR_WINDOW && tc_phi_supported(c.phi_hidden, c.phi_dim);
+  ctx->tc.phi_ok = ctx->tensor_ok && c.impl != REHYAT_IMPL_TENSOR_WINDOW && tc_phi_supported(c.phi_hidden, c.phi_dim, c.poly_degree);
 
   const int np_max = c.max_tokens_per_frame * c.max_chunk_frames;
   const int want = c.group_tokens > 0 ? c.group_tokens : 32768;

@@ -9,9 +9,9 @@
 //
 // Per tile the chain is  H = act(X W1^T + b1) -> U = act(H W2^T + b2) -> phi = U^(1..P)  with the
 // two GEMMs done as 128x128 halves through one 128-column TMEM scratch accumulator:
-//   warps 0-3  one thread per token (= TMEM lane): bias, activation, power, bf16, swizzled smem tile
-//   warp 4     TMA producer: X (and V), weight / state tiles [128 x 64] through a 3-stage ring
-//   warp 5     UMMA issuer
+//   warps 0-7  epilogues, two threads per token (= TMEM lane): bias, activation, power, bf16, swizzled smem tile
+//   warp 8     TMA producer: X (and V), weight / state tiles [128 x 64] through a 3-stage ring
+//   warp 9     UMMA issuer
 // The phi tile is written once in the 128-byte-swizzled [token][feature] image; the state GEMM reads
 // it as an MN-major A operand (features are M), the read-out GEMM as a K-major A operand.
 #pragma once
@@ -26,7 +26,7 @@ namespace rehyat {
 enum PhiMode : int { PHI_STATE = 0, PHI_READOUT = 1 };
 
 constexpr int PH_D = 128, PH_DH = 256, PH_DP = 256, PH_SD = PH_D + 4;
-constexpr int PH_THREADS = 192;
+constexpr int PH_THREADS = 320;            // 8 epilogue warps, TMA producer, UMMA issuer
 constexpr int PH_RING = 3;
 constexpr int PH_WT_BYTES = 128 * 64 * 2;          // one weight / state tile: 16 KB
 constexpr int PH_TILE_BYTES = 128 * 128 * 2;       // X, V, phi half: 32 KB (two swizzled sub-tiles)
@@ -39,7 +39,7 @@ constexpr int PH_OFF_PHI0 = PH_OFF_HB + 2 * PH_TILE_BYTES;
 constexpr int PH_OFF_RING = PH_OFF_PHI0 + PH_TILE_BYTES;
 constexpr int PH_OFF_ONES = PH_OFF_RING + PH_RING * PH_WT_BYTES; // [16 x 128] K-major, row 0 = 1
 constexpr int PH_OFF_BIAS = PH_OFF_ONES + 4096;                 // b1[256], b2[256], z[256] fp32
-constexpr int PH_OFF_BARS = PH_OFF_BIAS + 3 * 256 * 4;
+constexpr int PH_OFF_BARS = PH_OFF_BIAS + 4 * 256 * 4;     // ... and the two partial phi.z sums per token
 constexpr int PH_SMEM = PH_OFF_BARS + 512 + 1024;
 
 enum PhErr : int { PH_ERR_LOAD = 16, PH_ERR_MMA = 32, PH_ERR_EPI = 64 };
@@ -68,7 +68,7 @@ struct PhiTcArgs {
 // tm_x: K (state) or Q (read-out), 4-D like the window kernel's maps.  tm_v: V (state only).
 // tm_w1: (128, 256, heads), tm_w2: (256, 256, heads), boxes [64 x 128].  tm_s: bf16 states
 // (128, 256, G*BH), box [64 x 64] (read-out only).
-template <int MODE>
+template <int MODE, bool RELU>
 __global__ void __launch_bounds__(PH_THREADS, 1)
 phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_v,
        const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2,
@@ -81,6 +81,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   float* s_b1 = reinterpret_cast<float*>(smem + PH_OFF_BIAS);
   float* s_b2 = s_b1 + 256;
   float* s_z = s_b2 + 256;
+  float* s_nl = s_z + 256;
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -117,8 +118,8 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     for (int s = 0; s < PH_RING; ++s) {
       mbar_init(smem_u32(&bars->ring_full[s]), 1); mbar_init(smem_u32(&bars->ring_empty[s]), 1);
     }
-    mbar_init(smem_u32(&bars->acc_ready), 1); mbar_init(smem_u32(&bars->epi_done), 128);
-    mbar_init(smem_u32(&bars->out_ready), 1); mbar_init(smem_u32(&bars->out_read), 128);
+    mbar_init(smem_u32(&bars->acc_ready), 1); mbar_init(smem_u32(&bars->epi_done), 256);
+    mbar_init(smem_u32(&bars->out_ready), 1); mbar_init(smem_u32(&bars->out_read), 256);
     bars->abort_flag = 0;
     fence_mbar_init();
   }
@@ -136,7 +137,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     }
     fence_proxy_async_smem();
   }
-  if (warp == 5) {
+  if (warp == 9) {
     tmem_alloc(smem_u32(&bars->tmem_base), 512);
     tmem_relinquish();
   }
@@ -151,7 +152,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   const uint32_t sX = sb + PH_OFF_X, sV = sb + PH_OFF_V, sHb = sb + PH_OFF_HB, sPhi0 = sb + PH_OFF_PHI0,
                  sRing = sb + PH_OFF_RING, sOnes = sb + PH_OFF_ONES;
 
-  if (warp == 4) {
+  if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
     if (elect_one()) {
       prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_w1); prefetch_tensormap(&tm_w2);
@@ -196,7 +197,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
           for (int f = 0; f < 4; ++f) ring_load(&tm_s, 0, f * 64, ci * g.BH + bh, true);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     // ------------------------------------------------------------------ UMMA issuer
     if (elect_one()) {
       constexpr uint32_t id_kk = idesc_bf16(128, 128, 0, 0);       // A K-major, B K-major   (the two MLP GEMMs)
@@ -286,11 +287,14 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       umma_commit(smem_u32(&bars->out_ready));
     }
   } else {
-    // ------------------------------------------------------------------ epilogues: thread = token = TMEM lane
-    const int r = warp * 32 + lane;
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    // ------------------------------------------------------------------ epilogues
+    // Eight warps: warp w serves TMEM lanes 32*(w%4).. (one token per thread) and the column half
+    // w/4 of every 128-column accumulator, so two threads share a token.
+    const int qd = warp & 3, ch = warp >> 2;
+    const int r = qd * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(qd * 32) << 16;
     uint32_t n_acc = 0;
-    const int part_w = PH_DP / a.P;
+    const int part_w = PH_DP / a.P;                                 // a multiple of 32 (P in {1,2,4})
     for (int j = 0; j < n_tiles; ++j) {
       const bool tok_valid = tok_a + j * 128 + r < tok_b;
       float nl = 0.f;
@@ -303,32 +307,49 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
         const uint32_t dst = !is_u ? sHb : (half == 0 ? sPhi0 : sHb);
         const int dst_col0 = !is_u ? half * 128 : 0;
         const float* bias = (is_u ? s_b2 : s_b1) + half * 128;
+        uint32_t x[2][32];
+        tmem_ld32(tmem + lane_off + T_SCR + ch * 64, x[0]);
+        tmem_ld32(tmem + lane_off + T_SCR + ch * 64 + 32, x[1]);
+        tmem_wait_ld();
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          uint32_t x[32];
-          tmem_ld32(tmem + lane_off + T_SCR + cc * 32, x);
-          tmem_wait_ld();
+        for (int cb = 0; cb < 2; ++cb) {
+          const int col0 = ch * 64 + cb * 32;
+          float y[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[cb][e]) + bias[col0 + e];
+          if (RELU) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) y[e] = fmaxf(y[e], 0.f);
+          } else {
+            const int act = is_u ? a.act_out : a.act_hidden;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) y[e] = apply_act(y[e], act);
+          }
+          if (is_u) {
+            const int part = (half * 128 + col0) / part_w;          // uniform over the 32 columns
+            if (part == 1) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) y[e] *= y[e];
+            } else if (part == 2) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) y[e] *= y[e] * y[e];
+            } else if (part == 3) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) { const float s2 = y[e] * y[e]; y[e] = s2 * s2; }
+            }
+            if (!tok_valid) {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) y[e] = 0.f;
+            }
+          }
 #pragma unroll
           for (int e = 0; e < 32; e += 8) {
-            float y[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-              const int col = cc * 32 + e + u;
-              float val = __uint_as_float(x[e + u]) + bias[col];
-              if (!is_u) {
-                val = apply_act(val, a.act_hidden);
-              } else {
-                val = poly_power(apply_act(val, a.act_out), (half * 128 + col) / part_w);
-                if (!tok_valid) val = 0.f;
-              }
-              y[u] = val;
-            }
             uint4 w;
-            w.x = pack_bf16(y[0], y[1]); w.y = pack_bf16(y[2], y[3]);
-            w.z = pack_bf16(y[4], y[5]); w.w = pack_bf16(y[6], y[7]);
+            w.x = pack_bf16(y[e], y[e + 1]); w.y = pack_bf16(y[e + 2], y[e + 3]);
+            w.z = pack_bf16(y[e + 4], y[e + 5]); w.w = pack_bf16(y[e + 6], y[e + 7]);
             if (MODE == PHI_READOUT && is_u) {
               // phi_q(q_r) . z_t with the same bf16-rounded features the tensor core sees
-              const float* zz = s_z + half * 128 + cc * 32 + e;
+              const float* zz = s_z + half * 128 + col0 + e;
               const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
               for (int u = 0; u < 4; ++u) {
@@ -336,9 +357,10 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
                 nl = fmaf(__uint_as_float(ww[u] & 0xffff0000u), zz[2 * u + 1], nl);
               }
             }
-            st_tile_chunk_sw128(dst, PH_SUB, r, dst_col0 + cc * 32 + e, w);
+            st_tile_chunk_sw128(dst, PH_SUB, r, dst_col0 + col0 + e, w);
           }
         }
+        if (MODE == PHI_READOUT && step == 3) s_nl[ch * 128 + r] = nl;
         fence_proxy_async_smem();
         tc_fence_before();
         mbar_arrive(smem_u32(&bars->epi_done));
@@ -348,28 +370,30 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
         // the next tile (or after the loop)
         mbar_wait(smem_u32(&bars->out_ready), j & 1, abort_flag, a.status, PH_ERR_EPI);
         tc_fence_after();
+        asm volatile("bar.sync 1, 256;" ::: "memory");               // both halves of s_nl are written
         const int tok = tok_a + j * 128 + r;
         float* dst = a.rd + ((size_t)bh * a.rd_rows + (size_t)((tok_valid ? tok : tok_a) - geo_q0(g, g.t0))) * PH_SD;
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
+        for (int cb = 0; cb < 2; ++cb) {
           uint32_t x[32];
-          tmem_ld32(tmem + lane_off + T_ACC + cc * 32, x);
+          tmem_ld32(tmem + lane_off + T_ACC + ch * 64 + cb * 32, x);
           tmem_wait_ld();
           if (tok_valid) {
 #pragma unroll
             for (int e = 0; e < 32; e += 4)
-              *reinterpret_cast<float4*>(dst + cc * 32 + e) =
+              *reinterpret_cast<float4*>(dst + ch * 64 + cb * 32 + e) =
                   make_float4(__uint_as_float(x[e]), __uint_as_float(x[e + 1]), __uint_as_float(x[e + 2]),
                               __uint_as_float(x[e + 3]));
           }
         }
-        if (tok_valid) dst[PH_D] = nl;
+        if (tok_valid && ch == 1) dst[PH_D] = s_nl[r] + s_nl[128 + r];
         tc_fence_before();
+        asm volatile("bar.sync 1, 256;" ::: "memory");               // s_nl may be overwritten by the next tile
         mbar_arrive(smem_u32(&bars->out_read));
       }
     }
     if (MODE == PHI_STATE) {
-      // flush: lane r holds feature c*128 + r of half c
+      // flush: lane r holds feature c*128 + r of half c; this thread writes its 64 columns
       mbar_wait(smem_u32(&bars->out_ready), 0, abort_flag, a.status, PH_ERR_EPI);
       tc_fence_after();
       float* base = a.partial + (((size_t)ci * a.n_split + blockIdx.x) * g.BH + bh) * PH_DP * PH_SD;
@@ -377,27 +401,29 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       for (int c = 0; c < 2; ++c) {
         float* dst = base + (size_t)(c * 128 + r) * PH_SD;
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
+        for (int cb = 0; cb < 2; ++cb) {
           uint32_t x[32];
-          tmem_ld32(tmem + lane_off + T_ACC + c * 128 + cc * 32, x);
+          tmem_ld32(tmem + lane_off + T_ACC + c * 128 + ch * 64 + cb * 32, x);
           tmem_wait_ld();
 #pragma unroll
           for (int e = 0; e < 32; e += 4)
-            *reinterpret_cast<float4*>(dst + cc * 32 + e) =
+            *reinterpret_cast<float4*>(dst + ch * 64 + cb * 32 + e) =
                 make_float4(__uint_as_float(x[e]), __uint_as_float(x[e + 1]), __uint_as_float(x[e + 2]),
                             __uint_as_float(x[e + 3]));
         }
-        uint32_t zc[16];
-        tmem_ld16(tmem + lane_off + T_Z + c * 16, zc);
-        tmem_wait_ld();
-        *reinterpret_cast<float4*>(dst + PH_D) = make_float4(__uint_as_float(zc[0]), 0.f, 0.f, 0.f);
+        if (ch == 1) {
+          uint32_t zc[16];
+          tmem_ld16(tmem + lane_off + T_Z + c * 16, zc);
+          tmem_wait_ld();
+          *reinterpret_cast<float4*>(dst + PH_D) = make_float4(__uint_as_float(zc[0]), 0.f, 0.f, 0.f);
+        }
       }
     }
   }
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == 9) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }

@@ -312,7 +312,7 @@ struct TcWorkspace {
 };
 
 inline bool tc_shape_supported(bool bf16, int d, int, int, int, int, int) { return bf16 && d == TC_D; }
-inline bool tc_phi_supported(int Dh, int Dp) { return Dh == PH_DH && Dp == PH_DP; }
+inline bool tc_phi_supported(int Dh, int Dp, int P) { return Dh == PH_DH && Dp == PH_DP && P != 3; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -337,8 +337,10 @@ inline void tc_workspace_destroy(TcWorkspace* w) { cudaFree(w->state_bf16); w->s
 
 inline int tc_set_attributes() {
   bool ok = cudaFuncSetAttribute(window_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(phi_tc<PHI_STATE>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(phi_tc<PHI_READOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess;
+            cudaFuncSetAttribute(phi_tc<PHI_STATE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(phi_tc<PHI_STATE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(phi_tc<PHI_READOUT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(phi_tc<PHI_READOUT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess;
   return ok ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
@@ -393,7 +395,10 @@ inline int tc_launch_state(const TcWorkspace* w, const void* k, const void* v, c
   a.b1 = (const __nv_bfloat16*)phi->k_b1; a.b2 = (const __nv_bfloat16*)phi->k_b2;
   a.P = P; a.act_hidden = act_hidden; a.act_out = act_out;
   a.n_split = n_split; a.partial = partial; a.status = status;
-  phi_tc<PHI_STATE><<<dim3(n_split, g.G, g.BH), PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, tw2, g, a);
+  if (act_hidden == ACT_RELU && act_out == ACT_RELU)
+    phi_tc<PHI_STATE, true><<<dim3(n_split, g.G, g.BH), PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, tw2, g, a);
+  else
+    phi_tc<PHI_STATE, false><<<dim3(n_split, g.G, g.BH), PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, tw2, g, a);
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
@@ -413,7 +418,10 @@ inline int tc_launch_readout(const TcWorkspace* w, const void* q, const rehyat_p
   a.tiles_per_cta = 4;
   const int tiles = (g.Np + 127) / 128;
   const int ctas = (tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
-  phi_tc<PHI_READOUT><<<dim3(ctas, g.G, g.BH), PH_THREADS, PH_SMEM, st>>>(tq, tq, tw1, tw2, ts, g, a);
+  if (act_hidden == ACT_RELU && act_out == ACT_RELU)
+    phi_tc<PHI_READOUT, true><<<dim3(ctas, g.G, g.BH), PH_THREADS, PH_SMEM, st>>>(tq, tq, tw1, tw2, ts, g, a);
+  else
+    phi_tc<PHI_READOUT, false><<<dim3(ctas, g.G, g.BH), PH_THREADS, PH_SMEM, st>>>(tq, tq, tw1, tw2, ts, g, a);
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
