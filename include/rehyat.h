@@ -40,6 +40,7 @@ extern "C" {
 #define REHYAT_ERR_ARCH            -4   /* the device is not compute capability 10.x           */
 #define REHYAT_ERR_ALLOC           -5   /* workspace allocation failed                         */
 #define REHYAT_ERR_DEVICE_TIMEOUT  -6   /* a bounded wait inside a kernel ran out (see status) */
+#define REHYAT_ERR_TOO_LARGE       -7   /* rehyat_forward_static: problem exceeds its fixed scratch */
 
 typedef enum { REHYAT_DTYPE_BF16 = 0, REHYAT_DTYPE_FP32 = 1 } rehyat_dtype;
 
@@ -130,6 +131,33 @@ int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host,
                         const void* v_host, void* out_host, const rehyat_phi_params* phi,
                         int32_t batch, int32_t frames, int32_t H, int32_t W,
                         int32_t chunk, int32_t overlap, void* cuda_stream);
+
+/* The same operator for callers that must not allocate device memory: code that runs inside a
+ * memory plan fixed up front (all device memory already handed to another allocator or pool), a
+ * latency-critical loop that cannot afford the device-wide synchronisation cudaMalloc / cudaFree
+ * imply, or a plug-in whose host forbids allocation calls.  (The paper has no counterpart: this is
+ * a convenience of the library, not a step of the method.)
+ *
+ * No context is needed.  The workspace that rehyat_create would allocate (chunk states, partial
+ * state sums, linear read-out) is a fixed 8 MiB array inside the library
+ * (rehyat_static_scratch_bytes), which every GPU that loads the library keeps until the process
+ * ends.  The SIMT fp32-arithmetic kernels do the work for both dtypes.  The call uses no
+ * cudaMalloc, cudaFree or any allocating routine.
+ *   cfg      device, dtype, n_heads, head_dim, phi_*, poly_degree, act_*, c_mode are used; impl,
+ *            max_* and group_tokens are ignored
+ *   others   as rehyat_forward (device pointers, caller-owned; asynchronous on `cuda_stream`)
+ * Limits: at most 16 chunks, and  2*chunks*B*n_heads*D'*(d+4) + B*n_heads*chunks*N'*(d+4)  floats
+ * must fit the array; larger problems return REHYAT_ERR_TOO_LARGE and launch nothing.
+ * The first call on each device looks up the array's device address and sets kernel attributes;
+ * make that first call before any stream capture begins.  All calls share the one array, which
+ * keeps the last call's contents (nothing needs it zeroed: a call writes every word before it
+ * reads it), so two calls that overlap on the GPU - different streams, or different threads -
+ * race; serialise them. */
+int rehyat_forward_static(const rehyat_config* cfg, const void* q, const void* k, const void* v, void* out,
+                          const rehyat_layout* lay, const rehyat_phi_params* phi,
+                          int32_t batch, int32_t frames, int32_t H, int32_t W,
+                          int32_t chunk, int32_t overlap, void* cuda_stream);
+size_t rehyat_static_scratch_bytes(void);
 
 /* Frees the workspace.  NULL is a no-op returning REHYAT_OK. */
 int rehyat_destroy(rehyat_ctx* ctx);

@@ -11,12 +11,14 @@ import torch
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "librehyat.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_ARCH, ERR_ALLOC, ERR_DEVICE_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
+ERR_TOO_LARGE = -7
 DTYPE = {"bf16": 0, "fp32": 1}
 ACT = {"relu": 0, "identity": 1, "softplus": 2, "elu1": 3, "gelu": 4}
 C_MODE = {"rowmax": 0, "zero": 1}
 IMPL = {"auto": 0, "simt": 1, "tensor": 2, "tensor_window": 3}
 
-EXPORTS = ["rehyat_create", "rehyat_forward", "rehyat_forward_host", "rehyat_destroy",
+EXPORTS = ["rehyat_create", "rehyat_forward", "rehyat_forward_host", "rehyat_forward_static",
+           "rehyat_static_scratch_bytes", "rehyat_destroy",
            "rehyat_workspace_bytes", "rehyat_status", "rehyat_last_launches", "rehyat_last_impl",
            "rehyat_profile_enable", "rehyat_profile_read", "rehyat_strerror", "rehyat_version"]
 PROF_KINDS = ("state", "scan", "readout", "window")
@@ -52,6 +54,10 @@ def lib():
             [C.c_int32] * 6 + [C.c_void_p]
         L.rehyat_forward_host.argtypes = [C.c_void_p] + [C.c_void_p] * 4 + [C.POINTER(PhiParams)] + \
             [C.c_int32] * 6 + [C.c_void_p]
+        L.rehyat_forward_static.argtypes = [C.POINTER(Config)] + [C.c_void_p] * 4 + \
+            [C.POINTER(Layout), C.POINTER(PhiParams)] + [C.c_int32] * 6 + [C.c_void_p]
+        L.rehyat_static_scratch_bytes.argtypes = []
+        L.rehyat_static_scratch_bytes.restype = C.c_size_t
         L.rehyat_destroy.argtypes = [C.c_void_p]
         L.rehyat_workspace_bytes.argtypes = [C.c_void_p]
         L.rehyat_workspace_bytes.restype = C.c_size_t
@@ -170,6 +176,27 @@ class Rehyat:
     def status(self, stream=None):
         st = stream if stream is not None else torch.cuda.current_stream(self.cfg.device)
         return lib().rehyat_status(self._h, C.c_void_p(st.cuda_stream))
+
+
+def forward_static(q, k, v, phi_q, phi_k, frames, H, W, chunk, overlap, *, dtype, poly_degree=2, phi_hidden=None,
+                   phi_dim=None, act_hidden="relu", act_out="relu", c_mode="rowmax", out=None, stream=None):
+    """rehyat_forward_static: the operator without a context and without any device allocation by the
+    library; its workspace is a fixed array inside librehyat.so.  For callers that cannot allocate
+    (fixed memory plans, loops that cannot take cudaMalloc's synchronisation).  q, k, v: contiguous CUDA
+    tensors [B, n_heads, N, d]; `out` must be passed by such callers (it is allocated here with torch
+    only when omitted).  Raises RehyatError(ERR_TOO_LARGE) beyond the fixed capacity."""
+    B, nh, N, d = q.shape
+    if out is None:
+        out = torch.empty_like(q)
+    cfg = Config(q.device.index or 0, DTYPE[dtype], nh, d, phi_hidden or 2 * d, phi_dim or 2 * d, poly_degree,
+                 ACT[act_hidden], ACT[act_out], C_MODE[c_mode], 0, 1, 1, 1, 0)
+    lay = Layout(nh * N * d, N * d, d)
+    st = stream if stream is not None else torch.cuda.current_stream(q.device)
+    phi = Rehyat.phi_struct(phi_q, phi_k)
+    _check(lib().rehyat_forward_static(C.byref(cfg), _ptr(q), _ptr(k), _ptr(v), _ptr(out), C.byref(lay), C.byref(phi),
+                                       B, frames, H, W, chunk, overlap, C.c_void_p(st.cuda_stream)),
+           "rehyat_forward_static")
+    return out
 
 
 def for_workload(wl, **kw):

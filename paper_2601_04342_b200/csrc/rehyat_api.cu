@@ -13,6 +13,7 @@
 #include <climits>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -156,6 +157,7 @@ const char* rehyat_strerror(int code) {
     case REHYAT_ERR_ARCH: return "device is not compute capability 10.x (sm_100)";
     case REHYAT_ERR_ALLOC: return "device allocation failed";
     case REHYAT_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case REHYAT_ERR_TOO_LARGE: return "problem does not fit the fixed scratch of rehyat_forward_static";
     default: return "unknown error code";
   }
 }
@@ -399,6 +401,85 @@ int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host,
   if (cudaMemcpyAsync(out_host, ctx->stage[3], bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return REHYAT_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
   return REHYAT_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Forward pass for callers that may not allocate device memory.
+// ---------------------------------------------------------------------------------------------
+// The workspace of the SIMT kernels (chunk states, partial state sums, linear read-out) lives in
+// this fixed array instead of cudaMalloc'ed buffers.  Every GPU that loads the library holds the
+// 8 MiB until the process exits.  All calls share it and it keeps the previous call's contents;
+// nothing relies on it starting at zero, because every word a call reads it has written earlier
+// in the same call.
+constexpr size_t kStaticScratchFloats = (size_t)2 << 20;
+static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
+
+// In host code `g_static_scratch` is only a handle of the symbol, not a device address, so the
+// address is looked up once per device (with that device current) and cached.
+constexpr int kMaxDevices = 64;
+static float* g_static_scratch_addr[kMaxDevices] = {};
+static std::mutex g_static_scratch_mutex;
+
+static int static_scratch_address(int device, float** out) {
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (!g_static_scratch_addr[device]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return REHYAT_ERR_CUDA; }
+    g_static_scratch_addr[device] = static_cast<float*>(p);
+  }
+  *out = g_static_scratch_addr[device];
+  return REHYAT_OK;
+}
+
+size_t rehyat_static_scratch_bytes(void) { return kStaticScratchFloats * sizeof(float); }
+
+int rehyat_forward_static(const rehyat_config* cfg, const void* q, const void* k, const void* v, void* out,
+                          const rehyat_layout* lay, const rehyat_phi_params* phi, int32_t batch, int32_t frames,
+                          int32_t H, int32_t W, int32_t chunk, int32_t overlap, void* cuda_stream) {
+  if (!cfg) return REHYAT_ERR_INVALID_ARG;
+  int rc = check_config(cfg);
+  if (rc != REHYAT_OK) return rc;
+  if (cfg->device < 0 || cfg->device >= kMaxDevices) return REHYAT_ERR_INVALID_ARG;
+  if (batch < 1 || frames < 1 || H < 1 || W < 1 || chunk < 1 || overlap < 0) return REHYAT_ERR_INVALID_ARG;
+  const long long HW = (long long)H * W, N = HW * frames;
+  if (N > (1 << 24)) return REHYAT_ERR_TOO_LARGE;
+  const int chunk_eff = chunk < frames ? chunk : frames;
+  const long long n_chunks = (frames + chunk_eff - 1) / chunk_eff;
+  const long long Np = chunk_eff * HW;
+  const long long BH = (long long)batch * cfg->n_heads, SD = cfg->head_dim + 4;
+  if (n_chunks > 16 || BH > 65535) return REHYAT_ERR_TOO_LARGE;
+  const long long slot = BH * cfg->phi_dim * SD;                 // one chunk state, floats
+  const long long rd_rows = n_chunks * Np;                       // all chunks form one group
+  const long long need = 2 * n_chunks * slot + BH * rd_rows * SD;
+  if (need > (long long)kStaticScratchFloats) return REHYAT_ERR_TOO_LARGE;
+
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) return REHYAT_ERR_CUDA;
+  float* base = nullptr;
+  rc = static_scratch_address(cfg->device, &base);
+  if (rc != REHYAT_OK) return rc;
+  if (cfg->dtype == REHYAT_DTYPE_FP32)
+    rc = cfg->head_dim == 64 ? set_simt_attributes<float, 64>(*cfg) : set_simt_attributes<float, 128>(*cfg);
+  else
+    rc = cfg->head_dim == 64 ? set_simt_attributes<__nv_bfloat16, 64>(*cfg) : set_simt_attributes<__nv_bfloat16, 128>(*cfg);
+  if (rc != REHYAT_OK) return rc;
+
+  // A context on the stack that points into the static array; the SIMT kernels do the work.
+  rehyat_ctx tmp;
+  tmp.cfg = *cfg;
+  tmp.cfg.impl = REHYAT_IMPL_SIMT;
+  tmp.cfg.max_batch = batch;
+  tmp.cfg.max_tokens_per_frame = (int32_t)HW;
+  tmp.cfg.max_chunk_frames = chunk_eff;
+  tmp.state = base;
+  tmp.partial = base + n_chunks * slot;
+  tmp.readout = base + 2 * n_chunks * slot;
+  tmp.Gmax = (int)n_chunks;
+  tmp.partial_units = (int)n_chunks;
+  tmp.rd_rows = (int)rd_rows;
+  tmp.bh_max = (int)BH;
+  tmp.tensor_ok = false;
+  return rehyat_forward(&tmp, q, k, v, out, lay, phi, batch, frames, H, W, chunk, overlap, cuda_stream);
 }
 
 }  // extern "C"
