@@ -12,6 +12,7 @@
 
 #include <climits>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -199,6 +200,10 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
   bool ok = cudaMalloc(&ctx->state, b_state) == cudaSuccess && cudaMalloc(&ctx->partial, b_partial) == cudaSuccess &&
             cudaMalloc(&ctx->readout, b_rd) == cudaSuccess && cudaMalloc(&ctx->status_dev, 256) == cudaSuccess;
   ctx->ws_bytes = b_state + b_partial + b_rd + 256;
+  if (const char* e = getenv("REHYAT_EXP_POLY")) {
+    const int n = atoi(e);
+    if (n >= 0 && n <= 3) ctx->tc.exp_poly = n;
+  }
   if (ok && ctx->tensor_ok) {
     size_t extra = 0;
     ok = tc_workspace_create(&ctx->tc, ctx->bh_max, ctx->Gmax, c.head_dim, c.phi_dim, &extra);

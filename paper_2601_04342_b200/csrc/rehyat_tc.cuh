@@ -29,6 +29,8 @@ constexpr int TC_QT = 2;              // query tiles per CTA
 constexpr int TC_BN = 128;            // keys per tile
 constexpr int TC_STAGES = 2;          // K ring and V ring depth
 constexpr int TC_THREADS = 384;
+constexpr int TC_REGS_SOFTMAX = 216;   // registers per thread of the softmax warps (setmaxnreg)
+constexpr int TC_REGS_OTHER = 64;      // ... of the producer / issuer warpgroup
 constexpr int TC_TILE_BYTES = TC_BN * TC_D * 2;       // 32 KB: two [128 x 64] swizzled sub-tiles
 constexpr int TC_SUB_BYTES = TC_TILE_BYTES / 2;
 constexpr int TC_WIN_SMEM = (TC_QT + 2 * TC_STAGES) * TC_TILE_BYTES + 1024 /*barriers*/ + 1024 /*align*/;
@@ -38,12 +40,13 @@ enum TcErr : int { TC_ERR_LOAD = 1, TC_ERR_MMA = 2, TC_ERR_SOFTMAX = 4 };
 struct WinBars {   // offsets (bytes) inside the barrier block
   uint64_t q_full;
   uint64_t k_full[TC_STAGES], k_empty[TC_STAGES], v_full[TC_STAGES], v_empty[TC_STAGES];
-  uint64_t s_ready[TC_QT], p_ready[TC_QT], pv_done[TC_QT];
+  uint64_t s_ready[TC_QT], p_half[TC_QT][2], pv_done[TC_QT];
   uint64_t drained;
   uint32_t tmem_base;
   int abort_flag;
 };
 
+template <int EMU>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
           const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ out, Geo g,
@@ -75,7 +78,8 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     }
     for (int i = 0; i < TC_QT; ++i) {
       mbar_init(smem_u32(&bars->s_ready[i]), 1);
-      mbar_init(smem_u32(&bars->p_ready[i]), TC_BM);
+      mbar_init(smem_u32(&bars->p_half[i][0]), TC_BM);
+      mbar_init(smem_u32(&bars->p_half[i][1]), TC_BM);
       mbar_init(smem_u32(&bars->pv_done[i]), 1);
     }
     mbar_init(smem_u32(&bars->drained), 1);
@@ -91,6 +95,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
 
+  if (warp < 4) setmaxnreg_dec<TC_REGS_OTHER>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (elect_one()) {
@@ -134,10 +139,10 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                   idesc_qk, kk > 0);
         }
       };
-      auto issue_pv = [&](int i, int s, bool acc) {
+      auto issue_pv = [&](int i, int s, int half, bool acc) {        // keys [64*half, 64*half+64) of the tile
         const uint32_t b0 = sV + s * TC_TILE_BYTES;
 #pragma unroll
-        for (int kk = 0; kk < TC_BN / 16; ++kk)
+        for (int kk = half * 4; kk < half * 4 + 4; ++kk)
           umma_ts(tmem + 256 + i * TC_D, tmem + i * TC_BN + kk * 8,
                   smem_desc_sw128(b0 + kk * 16 * 128, TC_SUB_BYTES, 1024), idesc_pv, (acc || kk > 0) ? 1u : 0u);
       };
@@ -154,9 +159,12 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         const uint32_t ph = (j / TC_STAGES) & 1;
         mbar_wait(smem_u32(&bars->v_full[s]), ph, abort_flag, status, TC_ERR_MMA);
         for (int i = 0; i < ntiles; ++i) {
-          mbar_wait(smem_u32(&bars->p_ready[i]), j & 1, abort_flag, status, TC_ERR_MMA);
+          mbar_wait(smem_u32(&bars->p_half[i][0]), j & 1, abort_flag, status, TC_ERR_MMA);
           tc_fence_after();
-          issue_pv(i, s, j > 0);
+          issue_pv(i, s, 0, j > 0);
+          mbar_wait(smem_u32(&bars->p_half[i][1]), j & 1, abort_flag, status, TC_ERR_MMA);
+          tc_fence_after();
+          issue_pv(i, s, 1, true);
           umma_commit(smem_u32(&bars->pv_done[i]));
           if (i == ntiles - 1) umma_commit(smem_u32(&bars->v_empty[s]));
           if (j + 1 < n_kv) {
@@ -177,12 +185,14 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ softmax + epilogue
+    setmaxnreg_inc<TC_REGS_SOFTMAX>();
     const int i = (warp - 4) >> 2;                                   // query tile of this warpgroup
     if (i < ntiles) {
       const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
       const uint32_t tS = tmem + lane_off + i * TC_BN, tO = tmem + lane_off + 256 + i * TC_D;
       const float c = scale * 1.4426950408889634f;                   // logits -> log2 domain
-      float m_true = -INFINITY, m_used = -INFINITY, l = 0.f;
+      float m_true = -INFINITY, m_used = -INFINITY;
+      uint64_t l2a = 0ull, l2b = 0ull;                               // four partial row sums as two fp32 pairs
       for (int j = 0; j < n_kv; ++j) {
         mbar_wait(smem_u32(&bars->s_ready[i]), j & 1, abort_flag, status, TC_ERR_SOFTMAX);
         tc_fence_after();
@@ -198,52 +208,66 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             for (int e = 0; e < 32; ++e)
               if (cc * 32 + e >= n_valid) sr[cc][e] = 0xff800000u;   // -inf
         }
-        float mx = -INFINITY;
+        // row maximum: four independent chains of three-input max
+        float mx[4] = {m_true, m_true, m_true, m_true};
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
-          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(sr[cc][e]));
-        m_true = fmaxf(m_true, mx);
+          for (int e = 0; e < 32; e += 2)
+            mx[cc] = fmax3(mx[cc], __uint_as_float(sr[cc][e]), __uint_as_float(sr[cc][e + 1]));
+        m_true = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
         const bool need = (m_true - m_used) * c > 8.f;               // true on the first tile (m_used = -inf)
-        if (j > 0) {
-          mbar_wait(smem_u32(&bars->pv_done[i]), (j - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
-          tc_fence_after();
-        }
         if (__any_sync(0xffffffffu, need)) {
           const float m_new = need ? m_true : m_used;
           if (j > 0) {
+            // s_ready(j) follows the completion of P V of tile j-1, so O may be touched
+            mbar_wait(smem_u32(&bars->pv_done[i]), (j - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+            tc_fence_after();
             const float f = ex2((m_used - m_new) * c);               // 1 for lanes that keep their reference
-            l *= f;
-#pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-              uint32_t o[32];
-              tmem_ld32(tO + cc * 32, o);
+            const uint64_t f2 = pk2(f, f);
+            l2a = mul2(l2a, f2);
+            l2b = mul2(l2b, f2);
+#pragma unroll 1
+            for (int cc = 0; cc < TC_D / 8; ++cc) {                   // rare: small pieces keep the register peak low
+              uint32_t o[8];
+              tmem_ld8(tO + cc * 8, o);
               tmem_wait_ld();
 #pragma unroll
-              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
-              tmem_st32(tO + cc * 32, o);
+              for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
+              tmem_st8(tO + cc * 8, o);
             }
           }
           m_used = m_new;
         }
-        const float mc = m_used * c;
-        float psum = 0.f;
+        const float mc = -m_used * c;
+        const uint64_t c2 = pk2(c, c), mc2 = pk2(mc, mc);
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) {
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
-            const float p0 = ex2(fmaf(__uint_as_float(sr[cc][e]), c, -mc));
-            const float p1 = ex2(fmaf(__uint_as_float(sr[cc][e + 1]), c, -mc));
-            psum += p0 + p1;
+            float t0, t1, p0, p1;
+            upk2(fma2(pk2u(sr[cc][e], sr[cc][e + 1]), c2, mc2), t0, t1);
+            if (((e >> 1) & 3) < EMU) {                              // EMU of every 4 pairs on the FMA pipe
+              ex2_poly2(t0, t1, p0, p1);
+            } else {
+              p0 = ex2(t0);
+              p1 = ex2(t1);
+            }
+            if ((e >> 1) & 1) l2b = add2(l2b, pk2(p0, p1)); else l2a = add2(l2a, pk2(p0, p1));
             sr[cc >> 1][(cc & 1) * 16 + (e >> 1)] = pack_bf16(p0, p1);
           }
-          if (cc & 1) tmem_st32(tS + (cc >> 1) * 32, sr[cc >> 1]);
+          if (cc & 1) {
+            tmem_st32(tS + (cc >> 1) * 32, sr[cc >> 1]);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars->p_half[i][cc >> 1]));       // P of 64 keys is in place
+          }
         }
-        l += psum;
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(smem_u32(&bars->p_ready[i]));
       }
+      float la0, la1, lb0, lb1;
+      upk2(l2a, la0, la1);
+      upk2(l2b, lb0, lb1);
+      const float l = (la0 + la1) + (lb0 + lb1);
       mbar_wait(smem_u32(&bars->pv_done[i]), (n_kv - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
       tc_fence_after();
 
@@ -309,6 +333,7 @@ struct TcWorkspace {
   void* encode_fn = nullptr;            // cuTensorMapEncodeTiled, resolved through the runtime
   __nv_bfloat16* state_bf16 = nullptr;  // [Gmax][BHmax][256][128]: bf16 copy of s_t for the read-out GEMM
   bool phi_ok = false;                  // the linear branch runs on the tensor-core kernels too
+  int exp_poly = 1;                     // of every 4 pairs of exponentials, how many the FMA pipe evaluates
 };
 
 inline bool tc_shape_supported(bool bf16, int d, int, int, int, int, int) { return bf16 && d == TC_D; }
@@ -336,7 +361,10 @@ inline bool tc_workspace_create(TcWorkspace* w, int bh_max, int Gmax, int d, int
 inline void tc_workspace_destroy(TcWorkspace* w) { cudaFree(w->state_bf16); w->state_bf16 = nullptr; }
 
 inline int tc_set_attributes() {
-  bool ok = cudaFuncSetAttribute(window_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
+  bool ok = cudaFuncSetAttribute(window_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(window_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(window_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(window_tc<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(phi_tc<PHI_STATE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(phi_tc<PHI_STATE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(phi_tc<PHI_READOUT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
@@ -377,8 +405,15 @@ inline int tc_launch_window(const TcWorkspace* w, const void* q, const void* k, 
   if (!tc_make_tmap(w, &tq, q, g, batch) || !tc_make_tmap(w, &tk, k, g, batch) || !tc_make_tmap(w, &tv, v, g, batch))
     return REHYAT_ERR_CUDA;
   const int pairs = (g.Np + TC_QT * TC_BM - 1) / (TC_QT * TC_BM);
-  window_tc<<<dim3(pairs, g.G, g.BH), TC_THREADS, TC_WIN_SMEM, st>>>(
-      tq, tk, tv, (__nv_bfloat16*)out, g, rd, rd_rows, 1.0f / sqrtf((float)TC_D), c_mode, status);
+  const dim3 grid(pairs, g.G, g.BH);
+  const float scale = 1.0f / sqrtf((float)TC_D);
+  __nv_bfloat16* o = (__nv_bfloat16*)out;
+  switch (w->exp_poly) {
+    case 0: window_tc<0><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status); break;
+    default: window_tc<1><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status); break;
+    case 3: window_tc<3><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status); break;
+    case 2: window_tc<2><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status); break;
+  }
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
