@@ -130,21 +130,25 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     if (elect_one()) {
       constexpr uint32_t idesc_qk = idesc_bf16(TC_BM, TC_BN, 0, 0);   // A = Q (K-major), B = K (K-major)
       constexpr uint32_t idesc_pv = idesc_bf16(TC_BM, TC_D, 0, 1);    // A = P (TMEM),    B = V (MN-major)
+      // Descriptors differ only in the start-address field (low word): build them once and add offsets.
+      uint32_t q_lo, q_hi, k_lo, k_hi, v_lo, v_hi;
+      upk2u(smem_desc_sw128(sQ, 16, 1024), q_lo, q_hi);
+      upk2u(smem_desc_sw128(sK, 16, 1024), k_lo, k_hi);
+      upk2u(smem_desc_sw128(sV, TC_SUB_BYTES, 1024), v_lo, v_hi);
       auto issue_qk = [&](int i, int s) {
-        const uint32_t a0 = sQ + i * TC_TILE_BYTES, b0 = sK + s * TC_TILE_BYTES;
+        const uint32_t a0 = q_lo + i * (TC_TILE_BYTES >> 4), b0 = k_lo + s * (TC_TILE_BYTES >> 4);
 #pragma unroll
         for (int kk = 0; kk < TC_D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * TC_SUB_BYTES + (kk & 3) * 32;
-          umma_ss(tmem + i * TC_BN, smem_desc_sw128(a0 + off, 16, 1024), smem_desc_sw128(b0 + off, 16, 1024),
-                  idesc_qk, kk > 0);
+          const uint32_t off = ((kk >> 2) * TC_SUB_BYTES + (kk & 3) * 32) >> 4;
+          umma_ss(tmem + i * TC_BN, pk2u(a0 + off, q_hi), pk2u(b0 + off, k_hi), idesc_qk, kk > 0);
         }
       };
       auto issue_pv = [&](int i, int s, int half, bool acc) {        // keys [64*half, 64*half+64) of the tile
-        const uint32_t b0 = sV + s * TC_TILE_BYTES;
+        const uint32_t b0 = v_lo + s * (TC_TILE_BYTES >> 4);
 #pragma unroll
         for (int kk = half * 4; kk < half * 4 + 4; ++kk)
-          umma_ts(tmem + 256 + i * TC_D, tmem + i * TC_BN + kk * 8,
-                  smem_desc_sw128(b0 + kk * 16 * 128, TC_SUB_BYTES, 1024), idesc_pv, (acc || kk > 0) ? 1u : 0u);
+          umma_ts(tmem + 256 + i * TC_D, tmem + i * TC_BN + kk * 8, pk2u(b0 + kk * (16 * 128 >> 4), v_hi), idesc_pv,
+                  (acc || kk > half * 4) ? 1u : 0u);
       };
       bool alive = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag, status, TC_ERR_MMA);
       alive = alive && mbar_wait(smem_u32(&bars->k_full[0]), 0, abort_flag, status, TC_ERR_MMA);
