@@ -319,6 +319,22 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   if (G > ctx->Gmax) G = ctx->Gmax;
   int n_split = ctx->partial_units / G;
   if (n_split > 8) n_split = 8;
+  if (ctx->tensor_ok && ctx->tc.phi_ok) {
+    // One CTA per (split, chunk, head) and one CTA per SM: pick the split that needs the fewest
+    // token tiles per SM over all waves.
+    int n_sm = 148;
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, c.device);
+    int busy = 0;                                   // chunks of the first group that admit keys into the state
+    for (int t = 1; t < (G < n_chunks ? G : n_chunks); ++t) busy += geo_lo(g, t) > geo_lo(g, t - 1);
+    const long long units = (long long)(busy > 0 ? busy : 1) * g.BH, tiles = (g.Np + 127) / 128;
+    long long best = -1;
+    int best_s = 1;
+    for (int s = 1; s <= n_split; ++s) {
+      const long long cost = ((units * s + n_sm - 1) / n_sm) * ((tiles + s - 1) / s);
+      if (best < 0 || cost < best) { best = cost; best_s = s; }
+    }
+    n_split = best_s;
+  }
 
   ctx->last_launches = 0;
   ctx->last_impl = ctx->tensor_ok ? 1 : 0;

@@ -27,7 +27,8 @@ enum PhiMode : int { PHI_STATE = 0, PHI_READOUT = 1 };
 
 constexpr int PH_D = 128, PH_DH = 256, PH_DP = 256, PH_SD = PH_D + 4;
 constexpr int PH_THREADS = 320;            // 8 epilogue warps, TMA producer, UMMA issuer
-constexpr int PH_RING = 3;
+constexpr int PH_RING = 3;                // weight tiles in flight (PHI_STATE)
+constexpr int PH_RING_MAX = 5;            // PHI_READOUT has no V tile and uses its 32 KB for two more stages
 constexpr int PH_WT_BYTES = 128 * 64 * 2;          // one weight / state tile: 16 KB
 constexpr int PH_TILE_BYTES = 128 * 128 * 2;       // X, V, phi half: 32 KB (two swizzled sub-tiles)
 constexpr int PH_SUB = PH_TILE_BYTES / 2;
@@ -46,7 +47,7 @@ enum PhErr : int { PH_ERR_LOAD = 16, PH_ERR_MMA = 32, PH_ERR_EPI = 64 };
 
 struct PhBars {
   uint64_t x_full, x_empty, v_full, v_empty;
-  uint64_t ring_full[PH_RING], ring_empty[PH_RING];
+  uint64_t ring_full[PH_RING_MAX], ring_empty[PH_RING_MAX];
   uint64_t acc_ready, epi_done, out_ready, out_read;
   uint32_t tmem_base;
   int abort_flag;
@@ -68,7 +69,8 @@ struct PhiTcArgs {
 // tm_x: K (state) or Q (read-out), 4-D like the window kernel's maps.  tm_v: V (state only).
 // tm_w1: (128, 256, heads), tm_w2: (256, 256, heads), boxes [64 x 128].  tm_s: bf16 states
 // (128, 256, G*BH), box [64 x 64] (read-out only).
-template <int MODE, bool RELU>
+// PC: polynomial degree known at compile time (0: read it from the arguments).
+template <int MODE, bool RELU, int PC>
 __global__ void __launch_bounds__(PH_THREADS, 1)
 phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_v,
        const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2,
@@ -115,7 +117,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   if (threadIdx.x == 0) {
     mbar_init(smem_u32(&bars->x_full), 1); mbar_init(smem_u32(&bars->x_empty), 1);
     mbar_init(smem_u32(&bars->v_full), 1); mbar_init(smem_u32(&bars->v_empty), 1);
-    for (int s = 0; s < PH_RING; ++s) {
+    for (int s = 0; s < PH_RING_MAX; ++s) {
       mbar_init(smem_u32(&bars->ring_full[s]), 1); mbar_init(smem_u32(&bars->ring_empty[s]), 1);
     }
     mbar_init(smem_u32(&bars->acc_ready), 1); mbar_init(smem_u32(&bars->epi_done), 256);
@@ -148,9 +150,11 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   // TMEM columns: scratch [0,128); STATE: S half0 [128,256) S half1 [256,384) z0 [384,400) z1 [400,416);
   // READOUT: R [128,256)
   constexpr uint32_t T_SCR = 0, T_ACC = 128, T_Z = 384;
+  constexpr int RING = MODE == PHI_READOUT ? PH_RING_MAX : PH_RING;
 
   const uint32_t sX = sb + PH_OFF_X, sV = sb + PH_OFF_V, sHb = sb + PH_OFF_HB, sPhi0 = sb + PH_OFF_PHI0,
                  sRing = sb + PH_OFF_RING, sOnes = sb + PH_OFF_ONES;
+  auto ring_addr = [&](int s) -> uint32_t { return s < PH_RING ? sRing + s * PH_WT_BYTES : sV + (s - PH_RING) * PH_WT_BYTES; };
 
   if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
@@ -159,17 +163,17 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       uint32_t ring_i = 0;
       bool alive = true;
       auto ring_load = [&](const CUtensorMap* tm, int x, int y, int z, bool state_tile) {
-        const int s = ring_i % PH_RING;
-        const uint32_t ph = (ring_i / PH_RING) & 1;
+        const int s = ring_i % RING;
+        const uint32_t ph = (ring_i / RING) & 1;
         alive = alive && mbar_wait(smem_u32(&bars->ring_empty[s]), ph ^ 1, abort_flag, a.status, PH_ERR_LOAD);
         if (!alive) return;
         const uint32_t full = smem_u32(&bars->ring_full[s]);
         mbar_expect_tx(full, PH_WT_BYTES);
         if (!state_tile) {
-          tma_load_3d(sRing + s * PH_WT_BYTES, tm, full, x, y, z);
+          tma_load_3d(ring_addr(s), tm, full, x, y, z);
         } else {                                                     // [64 features x 128 d] as two 64-column boxes
-          tma_load_3d(sRing + s * PH_WT_BYTES, tm, full, 0, y, z);
-          tma_load_3d(sRing + s * PH_WT_BYTES + 8192, tm, full, 64, y, z);
+          tma_load_3d(ring_addr(s), tm, full, 0, y, z);
+          tma_load_3d(ring_addr(s) + 8192, tm, full, 64, y, z);
         }
         ++ring_i;
       };
@@ -206,13 +210,13 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       constexpr uint32_t id_rd = idesc_bf16(128, 128, 0, 1);       // A = phi (K-major),    B = state (MN-major)
       uint32_t ring_i = 0, n_epi = 0;
       auto ring_wait = [&]() -> uint32_t {
-        const int s = ring_i % PH_RING;
-        mbar_wait(smem_u32(&bars->ring_full[s]), (ring_i / PH_RING) & 1, abort_flag, a.status, PH_ERR_MMA);
+        const int s = ring_i % RING;
+        mbar_wait(smem_u32(&bars->ring_full[s]), (ring_i / RING) & 1, abort_flag, a.status, PH_ERR_MMA);
         tc_fence_after();
-        return sRing + s * PH_WT_BYTES;
+        return ring_addr(s);
       };
       auto ring_release = [&]() {
-        umma_commit(smem_u32(&bars->ring_empty[ring_i % PH_RING]));
+        umma_commit(smem_u32(&bars->ring_empty[ring_i % RING]));
         ++ring_i;
       };
       auto wait_epi = [&]() {
@@ -294,10 +298,11 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     const int r = qd * 32 + lane;
     const uint32_t lane_off = (uint32_t)(qd * 32) << 16;
     uint32_t n_acc = 0;
-    const int part_w = PH_DP / a.P;                                 // a multiple of 32 (P in {1,2,4})
+    const int part_w = PH_DP / (PC ? PC : a.P);                     // a multiple of 32 (P in {1,2,4})
     for (int j = 0; j < n_tiles; ++j) {
       const bool tok_valid = tok_a + j * 128 + r < tok_b;
       float nl = 0.f;
+#pragma unroll
       for (int step = 0; step < 4; ++step) {                        // H half 0, H half 1, U half 0, U half 1
         mbar_wait(smem_u32(&bars->acc_ready), n_acc & 1, abort_flag, a.status, PH_ERR_EPI);
         ++n_acc;
@@ -314,50 +319,55 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
 #pragma unroll
         for (int cb = 0; cb < 2; ++cb) {
           const int col0 = ch * 64 + cb * 32;
-          float y[32];
-#pragma unroll
-          for (int e = 0; e < 32; ++e) y[e] = __uint_as_float(x[cb][e]) + bias[col0 + e];
+          uint32_t w[16];                                           // 32 features as bf16 pairs
           if (RELU) {
+            const int part = !is_u ? 0 : PC == 1 ? 0 : PC == 2 ? half : (half * 128 + col0) / part_w;   // uniform over the 32 columns
 #pragma unroll
-            for (int e = 0; e < 32; ++e) y[e] = fmaxf(y[e], 0.f);
+            for (int e = 0; e < 32; e += 4) {
+              const float4 b4 = *reinterpret_cast<const float4*>(bias + col0 + e);
+              float y0, y1, y2, y3;
+              upk2(add2(pk2u(x[cb][e], x[cb][e + 1]), pk2(b4.x, b4.y)), y0, y1);
+              upk2(add2(pk2u(x[cb][e + 2], x[cb][e + 3]), pk2(b4.z, b4.w)), y2, y3);
+              if (part == 0) {
+                w[e >> 1] = pack_bf16_relu(y0, y1);
+                w[(e >> 1) + 1] = pack_bf16_relu(y2, y3);
+              } else {
+                y0 = fmaxf(y0, 0.f); y1 = fmaxf(y1, 0.f); y2 = fmaxf(y2, 0.f); y3 = fmaxf(y3, 0.f);
+                float p0 = y0 * y0, p1 = y1 * y1, p2 = y2 * y2, p3 = y3 * y3;
+                if (part == 2) { p0 *= y0; p1 *= y1; p2 *= y2; p3 *= y3; }
+                if (part == 3) { p0 *= p0; p1 *= p1; p2 *= p2; p3 *= p3; }
+                w[e >> 1] = pack_bf16(p0, p1);
+                w[(e >> 1) + 1] = pack_bf16(p2, p3);
+              }
+            }
           } else {
             const int act = is_u ? a.act_out : a.act_hidden;
+            const int part = is_u ? (half * 128 + col0) / part_w : 0;
 #pragma unroll
-            for (int e = 0; e < 32; ++e) y[e] = apply_act(y[e], act);
+            for (int e = 0; e < 32; e += 2) {
+              float y0 = apply_act(__uint_as_float(x[cb][e]) + bias[col0 + e], act);
+              float y1 = apply_act(__uint_as_float(x[cb][e + 1]) + bias[col0 + e + 1], act);
+              w[e >> 1] = pack_bf16(poly_power(y0, part), poly_power(y1, part));
+            }
           }
-          if (is_u) {
-            const int part = (half * 128 + col0) / part_w;          // uniform over the 32 columns
-            if (part == 1) {
+          if (is_u && !tok_valid) {
 #pragma unroll
-              for (int e = 0; e < 32; ++e) y[e] *= y[e];
-            } else if (part == 2) {
-#pragma unroll
-              for (int e = 0; e < 32; ++e) y[e] *= y[e] * y[e];
-            } else if (part == 3) {
-#pragma unroll
-              for (int e = 0; e < 32; ++e) { const float s2 = y[e] * y[e]; y[e] = s2 * s2; }
-            }
-            if (!tok_valid) {
-#pragma unroll
-              for (int e = 0; e < 32; ++e) y[e] = 0.f;
-            }
+            for (int e = 0; e < 16; ++e) w[e] = 0u;
           }
 #pragma unroll
           for (int e = 0; e < 32; e += 8) {
-            uint4 w;
-            w.x = pack_bf16(y[e], y[e + 1]); w.y = pack_bf16(y[e + 2], y[e + 3]);
-            w.z = pack_bf16(y[e + 4], y[e + 5]); w.w = pack_bf16(y[e + 6], y[e + 7]);
+            const uint4 w4 = make_uint4(w[e >> 1], w[(e >> 1) + 1], w[(e >> 1) + 2], w[(e >> 1) + 3]);
             if (MODE == PHI_READOUT && is_u) {
               // phi_q(q_r) . z_t with the same bf16-rounded features the tensor core sees
               const float* zz = s_z + half * 128 + col0 + e;
-              const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+              const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
               for (int u = 0; u < 4; ++u) {
                 nl = fmaf(__uint_as_float(ww[u] << 16), zz[2 * u], nl);
                 nl = fmaf(__uint_as_float(ww[u] & 0xffff0000u), zz[2 * u + 1], nl);
               }
             }
-            st_tile_chunk_sw128(dst, PH_SUB, r, dst_col0 + col0 + e, w);
+            st_tile_chunk_sw128(dst, PH_SUB, r, dst_col0 + col0 + e, w4);
           }
         }
         if (MODE == PHI_READOUT && step == 3) s_nl[ch * 128 + r] = nl;

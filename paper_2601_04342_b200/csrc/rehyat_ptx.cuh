@@ -240,6 +240,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+__device__ __forceinline__ uint32_t pack_bf16_relu(float lo, float hi) {   // max(.,0) then round, one instruction
+  uint32_t r;
+  asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
 // ----------------------------------------------------------------------------- packed fp32 pairs
 // sm_100 executes add/sub/mul/fma on two fp32 values held in one 64-bit register per instruction.
 __device__ __forceinline__ uint64_t pk2(float lo, float hi) {

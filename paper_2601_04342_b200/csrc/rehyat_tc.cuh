@@ -369,10 +369,12 @@ inline int tc_set_attributes() {
             cudaFuncSetAttribute(window_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(window_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(window_tc<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(phi_tc<PHI_STATE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(phi_tc<PHI_STATE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(phi_tc<PHI_READOUT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(phi_tc<PHI_READOUT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess;
+            cudaFuncSetAttribute(phi_tc<PHI_STATE, true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(phi_tc<PHI_STATE, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(phi_tc<PHI_STATE, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(phi_tc<PHI_READOUT, true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(phi_tc<PHI_READOUT, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(phi_tc<PHI_READOUT, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess;
   return ok ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
@@ -434,10 +436,14 @@ inline int tc_launch_state(const TcWorkspace* w, const void* k, const void* v, c
   a.b1 = (const __nv_bfloat16*)phi->k_b1; a.b2 = (const __nv_bfloat16*)phi->k_b2;
   a.P = P; a.act_hidden = act_hidden; a.act_out = act_out;
   a.n_split = n_split; a.partial = partial; a.status = status;
-  if (act_hidden == ACT_RELU && act_out == ACT_RELU)
-    phi_tc<PHI_STATE, true><<<dim3(n_split, g.G, g.BH), PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, tw2, g, a);
+  const bool relu = act_hidden == ACT_RELU && act_out == ACT_RELU;
+  const dim3 grid(n_split, g.G, g.BH);
+  if (relu && P == 2)
+    phi_tc<PHI_STATE, true, 2><<<grid, PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, tw2, g, a);
+  else if (relu)
+    phi_tc<PHI_STATE, true, 0><<<grid, PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, tw2, g, a);
   else
-    phi_tc<PHI_STATE, false><<<dim3(n_split, g.G, g.BH), PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, tw2, g, a);
+    phi_tc<PHI_STATE, false, 0><<<grid, PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, tw2, g, a);
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
@@ -457,10 +463,14 @@ inline int tc_launch_readout(const TcWorkspace* w, const void* q, const rehyat_p
   a.tiles_per_cta = 4;
   const int tiles = (g.Np + 127) / 128;
   const int ctas = (tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
-  if (act_hidden == ACT_RELU && act_out == ACT_RELU)
-    phi_tc<PHI_READOUT, true><<<dim3(ctas, g.G, g.BH), PH_THREADS, PH_SMEM, st>>>(tq, tq, tw1, tw2, ts, g, a);
+  const bool relu = act_hidden == ACT_RELU && act_out == ACT_RELU;
+  const dim3 grid(ctas, g.G, g.BH);
+  if (relu && P == 2)
+    phi_tc<PHI_READOUT, true, 2><<<grid, PH_THREADS, PH_SMEM, st>>>(tq, tq, tw1, tw2, ts, g, a);
+  else if (relu)
+    phi_tc<PHI_READOUT, true, 0><<<grid, PH_THREADS, PH_SMEM, st>>>(tq, tq, tw1, tw2, ts, g, a);
   else
-    phi_tc<PHI_READOUT, false><<<dim3(ctas, g.G, g.BH), PH_THREADS, PH_SMEM, st>>>(tq, tq, tw1, tw2, ts, g, a);
+    phi_tc<PHI_READOUT, false, 0><<<grid, PH_THREADS, PH_SMEM, st>>>(tq, tq, tw1, tw2, ts, g, a);
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
