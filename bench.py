@@ -37,7 +37,7 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the ncu
 # capture summarised under profiles/; None until a capture exists for the kernel in use.
-NCU_TRAFFIC_BYTES = {"window_simt": None, "window_tc": None}
+NCU_TRAFFIC_BYTES = {"window_simt": None, "window_tc": 480027392 + 88080128}   # profiles/window_tc_wan13b_layer.md
 
 
 def measured_peaks():
@@ -135,6 +135,74 @@ def config_of(wl, extra=None):
     return cfg
 
 
+def _time_ms(fn, stream, warmup, steps):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        fn()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def full_softmax_comparison(wl, dev, phi_q, phi_k, stream, hybrid_ms, flops):
+    """Full softmax attention (Eq. 2) at the workload's shape: this operator with one chunk covering
+    every frame (exact by the T_c = T limit) and, as an independent time, the library SDPA kernel."""
+    from paper_2601_04342_b200 import binding
+    op = binding.for_workload(wl, max_chunk_frames=wl.T)
+    out = torch.empty_like(dev["q"])
+    ours = _time_ms(lambda: op.forward(dev["q"], dev["k"], dev["v"], phi_q, phi_k, wl.T, wl.H, wl.W, wl.T, 0,
+                                       out=out, stream=stream), stream, 2, 5)
+    assert op.status() == 0
+    op.close()
+    lib = _time_ms(lambda: torch.nn.functional.scaled_dot_product_attention(dev["q"], dev["k"], dev["v"]), stream, 2, 5)
+    return {"flop": flops["full_softmax"], "this_operator_chunk_eq_frames_ms": ours,
+            "this_operator_tflops": flops["full_softmax"] / (ours * 1e-3) / 1e12,
+            "library_sdpa_ms": lib, "library_sdpa_tflops": flops["full_softmax"] / (lib * 1e-3) / 1e12,
+            "hybrid_ms": hybrid_ms, "hybrid_speedup_vs_this_operator_full": ours / hybrid_ms,
+            "hybrid_speedup_vs_library_sdpa": lib / hybrid_ms}
+
+
+def workspace_by_frames(wl, device):
+    """rehyat_workspace_bytes of contexts made for 21, 41 and 81 latent frames: the workspace is a
+    function of the configuration only, not of the video length (Section 3.3, note 3)."""
+    from paper_2601_04342_b200 import binding
+    out = {}
+    for T in (21, 41, 81):
+        op = binding.for_workload(wl.with_(T=T), device=device)
+        out[str(T)] = op.workspace_bytes
+        op.close()
+    return out
+
+
+def time_config(wl, device, stream):
+    """Kernel-resident timing of another configuration.  Inputs are drawn on the device (seeded torch
+    generator, N(0,1), q and k RMS-normalised) because the host recipe takes tens of seconds at these
+    sizes; the parity tests use the host recipe."""
+    from paper_2601_04342_b200 import binding
+    gen = torch.Generator(device="cuda").manual_seed(wl.seed)
+    shape = (wl.B, wl.n_heads, wl.N, wl.head_dim)
+    q, k, v = (torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32) for _ in range(3))
+    q = (q / q.pow(2).mean(-1, keepdim=True).sqrt()).to(torch.bfloat16)
+    k = (k / k.pow(2).mean(-1, keepdim=True).sqrt()).to(torch.bfloat16)
+    v = v.to(torch.bfloat16)
+    pq = {n: t.cuda() for n, t in synth.make_phi_params(wl, "phi_q").items()}
+    pk = {n: t.cuda() for n, t in synth.make_phi_params(wl, "phi_k").items()}
+    out = torch.empty_like(q)
+    op = binding.for_workload(wl, device=device)
+    ms = _time_ms(lambda: op.forward(q, k, v, pq, pk, wl.T, wl.H, wl.W, wl.Tc, wl.To, out=out, stream=stream), stream, 3, 20)
+    assert op.status() == 0
+    fl = geometry.flop_model(wl.B, wl.n_heads, wl.head_dim, wl.T, wl.HW, wl.Tc, wl.To, wl.D_h, wl.D_out)
+    res = {"workload": wl.name, "batch": wl.B, "tokens": wl.N, "ms_per_step": ms, "tflops": fl["total"] / (ms * 1e-3) / 1e12,
+           "tokens_per_s": wl.B * wl.N / (ms * 1e-3), "workspace_bytes": op.workspace_bytes, "launches_per_step": op.last_launches,
+           "full_softmax_flop_ratio": fl["full_softmax"] / fl["total"]}
+    op.close()
+    return res
+
+
 def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -171,6 +239,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel-impl", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--no-full-softmax", action="store_true", help="skip the full-softmax comparison at the same shape")
+    ap.add_argument("--all-configs", action="store_true",
+                    help="also time the CFG-batch and the long-video configurations (device-drawn inputs)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -301,6 +372,14 @@ def main():
                "sample": f"{len(heads)} of {wl.n_heads} heads of batch 0, all {wl.N} tokens, recurrent form, "
                          f"fp64 numpy, {dt:.1f} s"}
 
+    extras = {}
+    if world == 1 and wl.dtype == "bf16" and not args.no_full_softmax:
+        extras["full_softmax_same_shape"] = full_softmax_comparison(wl, dev, phi_q, phi_k, stream, ms_step, flops)
+    if world == 1:
+        extras["workspace_bytes_by_latent_frames"] = workspace_by_frames(wl, local_rank)
+    if world == 1 and args.all_configs:
+        extras["other_configs"] = [time_config(synth.CONFIGS[n], local_rank, stream) for n in ("cfg_long", "long_constant_memory")]
+
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -315,6 +394,7 @@ def main():
             "gpu_launches": launches_per_step * args.steps,
             "kernel_ms": kernel_ms, "workspace_bytes": op.workspace_bytes,
             "roofline": roofline, "cpu_baseline": cpu}
+    line.update(extras)
     print(json.dumps(line), flush=True)
     op.close()
     if dist:

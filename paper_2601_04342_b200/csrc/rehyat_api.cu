@@ -200,6 +200,7 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
   bool ok = cudaMalloc(&ctx->state, b_state) == cudaSuccess && cudaMalloc(&ctx->partial, b_partial) == cudaSuccess &&
             cudaMalloc(&ctx->readout, b_rd) == cudaSuccess && cudaMalloc(&ctx->status_dev, 256) == cudaSuccess;
   ctx->ws_bytes = b_state + b_partial + b_rd + 256;
+  cudaDeviceGetAttribute(&ctx->tc.n_sm, cudaDevAttrMultiProcessorCount, c.device);
   if (const char* e = getenv("REHYAT_EXP_POLY")) {
     const int n = atoi(e);
     if (n >= 0 && n <= 3) ctx->tc.exp_poly = n;
@@ -322,8 +323,7 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   if (ctx->tensor_ok && ctx->tc.phi_ok) {
     // One CTA per (split, chunk, head) and one CTA per SM: pick the split that needs the fewest
     // token tiles per SM over all waves.
-    int n_sm = 148;
-    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, c.device);
+    const int n_sm = ctx->tc.n_sm;
     int busy = 0;                                   // chunks of the first group that admit keys into the state
     for (int t = 1; t < (G < n_chunks ? G : n_chunks); ++t) busy += geo_lo(g, t) > geo_lo(g, t - 1);
     const long long units = (long long)(busy > 0 ? busy : 1) * g.BH, tiles = (g.Np + 127) / 128;

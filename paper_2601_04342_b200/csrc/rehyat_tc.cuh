@@ -337,6 +337,7 @@ struct TcWorkspace {
   void* encode_fn = nullptr;            // cuTensorMapEncodeTiled, resolved through the runtime
   __nv_bfloat16* state_bf16 = nullptr;  // [Gmax][BHmax][256][128]: bf16 copy of s_t for the read-out GEMM
   bool phi_ok = false;                  // the linear branch runs on the tensor-core kernels too
+  int n_sm = 148;                       // SMs of the device
   int exp_poly = 1;                     // of every 4 pairs of exponentials, how many the FMA pipe evaluates
 };
 
@@ -460,8 +461,18 @@ inline int tc_launch_readout(const TcWorkspace* w, const void* q, const rehyat_p
   a.b1 = (const __nv_bfloat16*)phi->q_b1; a.b2 = (const __nv_bfloat16*)phi->q_b2;
   a.P = P; a.act_hidden = act_hidden; a.act_out = act_out;
   a.state = state; a.rd = rd; a.rd_rows = rd_rows; a.status = status;
-  a.tiles_per_cta = 4;
+  // One CTA per SM: split a chunk's query tiles over as many CTAs as costs the fewest tile-times over all waves.
   const int tiles = (g.Np + 127) / 128;
+  int busy = 0;
+  for (int t = g.t0; t < g.t0 + g.G; ++t) busy += geo_lo(g, t) > 0;
+  const long long units = (long long)(busy > 0 ? busy : 1) * g.BH;
+  long long best = -1;
+  int best_s = 1;
+  for (int s = 1; s <= 16; ++s) {
+    const long long cost = ((units * s + w->n_sm - 1) / w->n_sm) * ((tiles + s - 1) / s);
+    if (best < 0 || cost < best) { best = cost; best_s = s; }
+  }
+  a.tiles_per_cta = (tiles + best_s - 1) / best_s;
   const int ctas = (tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
   const bool relu = act_hidden == ACT_RELU && act_out == ACT_RELU;
   const dim3 grid(ctas, g.G, g.BH);
