@@ -29,8 +29,8 @@ constexpr int TC_QT = 2;              // query tiles per CTA
 constexpr int TC_BN = 128;            // keys per tile
 constexpr int TC_STAGES = 2;          // K ring and V ring depth
 constexpr int TC_THREADS = 384;
-constexpr int TC_REGS_SOFTMAX = 216;   // registers per thread of the softmax warps (setmaxnreg)
-constexpr int TC_REGS_OTHER = 64;      // ... of the producer / issuer warpgroup
+constexpr int TC_REGS_SOFTMAX = 200;   // registers per thread of the softmax warps (setmaxnreg)
+constexpr int TC_REGS_OTHER = 96;       // ... of the producer / issuer warpgroup
 constexpr int TC_TILE_BYTES = TC_BN * TC_D * 2;       // 32 KB: two [128 x 64] swizzled sub-tiles
 constexpr int TC_SUB_BYTES = TC_TILE_BYTES / 2;
 constexpr int TC_WIN_SMEM = (TC_QT + 2 * TC_STAGES) * TC_TILE_BYTES + 1024 /*barriers*/ + 1024 /*align*/;
@@ -38,19 +38,44 @@ constexpr int TC_WIN_SMEM = (TC_QT + 2 * TC_STAGES) * TC_TILE_BYTES + 1024 /*bar
 enum TcErr : int { TC_ERR_LOAD = 1, TC_ERR_MMA = 2, TC_ERR_SOFTMAX = 4 };
 
 struct WinBars {   // offsets (bytes) inside the barrier block
-  uint64_t q_full;
+  uint64_t q_full, q_empty;
   uint64_t k_full[TC_STAGES], k_empty[TC_STAGES], v_full[TC_STAGES], v_empty[TC_STAGES];
-  uint64_t s_ready[TC_QT], p_half[TC_QT][2], pv_done[TC_QT];
+  uint64_t s_ready[TC_QT], p_half[TC_QT][2], pv_done[TC_QT], o_free[TC_QT];
   uint64_t drained;
   uint32_t tmem_base;
   int abort_flag;
 };
 
+// One work item of window_tc: two query tiles of one (chunk, batch*head).
+struct WinItem {
+  int bh, b_idx, h_idx;
+  int q0, q1, lo, hi;      // chunk queries [q0, q1), softmax window [lo, hi)
+  int row_base, ntiles, n_kv;
+};
+// Items are numbered (batch*head, chunk, tile pair), tile pair fastest, so that the CTAs running at one
+// time share few K/V windows in L2.  Returns false for pairs beyond the end of a short last chunk.
+__device__ __forceinline__ bool win_item(const Geo& g, int item, int pairs, WinItem& w) {
+  const int pair = item % pairs, rest = item / pairs, ci = rest % g.G;
+  w.bh = rest / g.G;
+  const int t = g.t0 + ci;
+  w.q0 = geo_q0(g, t); w.q1 = geo_q1(g, t); w.lo = geo_lo(g, t); w.hi = w.q1;
+  w.row_base = w.q0 + pair * (TC_QT * TC_BM);
+  if (w.row_base >= w.q1) return false;
+  w.ntiles = (w.row_base + TC_BM < w.q1) ? 2 : 1;                  // query tiles with at least one valid row
+  w.n_kv = (w.hi - w.lo + TC_BN - 1) / TC_BN;
+  w.b_idx = w.bh / g.n_heads; w.h_idx = w.bh % g.n_heads;
+  return true;
+}
+
+// Persistent: gridDim.x CTAs (one per SM) walk the items blockIdx.x, blockIdx.x + gridDim.x, ...  Barriers,
+// TMEM and the K/V rings live across items; every role keeps running counts of the phases it has used.
+// EMU: of every four pairs of exponentials, how many are evaluated on the FMA pipe.
 template <int EMU>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
           const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ out, Geo g,
-          const float* __restrict__ rd, int rd_rows, float scale, int c_mode, int* __restrict__ status) {
+          const float* __restrict__ rd, int rd_rows, float scale, int c_mode, int* __restrict__ status,
+          int n_items, int pairs) {
   using namespace ptx;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -62,16 +87,9 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
-  const int q0 = geo_q0(g, t), q1 = geo_q1(g, t), lo = geo_lo(g, t), hi = q1;
-  const int row_base = q0 + blockIdx.x * (TC_QT * TC_BM);
-  if (row_base >= q1) return;                                      // uniform for the CTA
-  const int ntiles = (row_base + TC_BM < q1) ? 2 : 1;              // query tiles with at least one valid row
-  const int n_kv = (hi - lo + TC_BN - 1) / TC_BN;
-  const int b_idx = bh / g.n_heads, h_idx = bh % g.n_heads;
 
   if (threadIdx.x == 0) {
-    mbar_init(smem_u32(&bars->q_full), 1);
+    mbar_init(smem_u32(&bars->q_full), 1); mbar_init(smem_u32(&bars->q_empty), 1);
     for (int s = 0; s < TC_STAGES; ++s) {
       mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1);
       mbar_init(smem_u32(&bars->v_full[s]), 1); mbar_init(smem_u32(&bars->v_empty[s]), 1);
@@ -81,6 +99,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       mbar_init(smem_u32(&bars->p_half[i][0]), TC_BM);
       mbar_init(smem_u32(&bars->p_half[i][1]), TC_BM);
       mbar_init(smem_u32(&bars->pv_done[i]), 1);
+      mbar_init(smem_u32(&bars->o_free[i]), TC_BM);
     }
     mbar_init(smem_u32(&bars->drained), 1);
     bars->abort_flag = 0;
@@ -100,29 +119,38 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     // ------------------------------------------------------------------ TMA producer
     if (elect_one()) {
       prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
-      const uint32_t qf = smem_u32(&bars->q_full);
-      mbar_expect_tx(qf, ntiles * TC_TILE_BYTES);
-      for (int i = 0; i < ntiles; ++i) {
-        tma_load_4d(sQ + i * TC_TILE_BYTES, &tm_q, qf, 0, row_base + i * TC_BM, h_idx, b_idx);
-        tma_load_4d(sQ + i * TC_TILE_BYTES + TC_SUB_BYTES, &tm_q, qf, 64, row_base + i * TC_BM, h_idx, b_idx);
-      }
+      uint32_t kv_it = 0, n_done = 0;                              // K/V tiles loaded, items loaded
       bool alive = true;
-      for (int j = 0; j < n_kv && alive; ++j) {
-        const int s = j % TC_STAGES;
-        const uint32_t ph = (j / TC_STAGES) & 1;
-        const int key0 = lo + j * TC_BN;
-        alive = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1, abort_flag, status, TC_ERR_LOAD);
+      for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+        WinItem w;
+        if (!win_item(g, item, pairs, w)) continue;
+        // Q of the previous item has been read by its last Q K^T
+        if (n_done > 0) alive = mbar_wait(smem_u32(&bars->q_empty), (n_done - 1) & 1, abort_flag, status, TC_ERR_LOAD);
         if (!alive) break;
-        const uint32_t kf = smem_u32(&bars->k_full[s]);
-        mbar_expect_tx(kf, TC_TILE_BYTES);
-        tma_load_4d(sK + s * TC_TILE_BYTES, &tm_k, kf, 0, key0, h_idx, b_idx);
-        tma_load_4d(sK + s * TC_TILE_BYTES + TC_SUB_BYTES, &tm_k, kf, 64, key0, h_idx, b_idx);
-        alive = mbar_wait(smem_u32(&bars->v_empty[s]), ph ^ 1, abort_flag, status, TC_ERR_LOAD);
-        if (!alive) break;
-        const uint32_t vf = smem_u32(&bars->v_full[s]);
-        mbar_expect_tx(vf, TC_TILE_BYTES);
-        tma_load_4d(sV + s * TC_TILE_BYTES, &tm_v, vf, 0, key0, h_idx, b_idx);
-        tma_load_4d(sV + s * TC_TILE_BYTES + TC_SUB_BYTES, &tm_v, vf, 64, key0, h_idx, b_idx);
+        const uint32_t qf = smem_u32(&bars->q_full);
+        mbar_expect_tx(qf, w.ntiles * TC_TILE_BYTES);
+        for (int i = 0; i < w.ntiles; ++i) {
+          tma_load_4d(sQ + i * TC_TILE_BYTES, &tm_q, qf, 0, w.row_base + i * TC_BM, w.h_idx, w.b_idx);
+          tma_load_4d(sQ + i * TC_TILE_BYTES + TC_SUB_BYTES, &tm_q, qf, 64, w.row_base + i * TC_BM, w.h_idx, w.b_idx);
+        }
+        for (int j = 0; j < w.n_kv && alive; ++j, ++kv_it) {
+          const int s = kv_it % TC_STAGES;
+          const uint32_t ph = (kv_it / TC_STAGES) & 1;
+          const int key0 = w.lo + j * TC_BN;
+          alive = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1, abort_flag, status, TC_ERR_LOAD);
+          if (!alive) break;
+          const uint32_t kf = smem_u32(&bars->k_full[s]);
+          mbar_expect_tx(kf, TC_TILE_BYTES);
+          tma_load_4d(sK + s * TC_TILE_BYTES, &tm_k, kf, 0, key0, w.h_idx, w.b_idx);
+          tma_load_4d(sK + s * TC_TILE_BYTES + TC_SUB_BYTES, &tm_k, kf, 64, key0, w.h_idx, w.b_idx);
+          alive = mbar_wait(smem_u32(&bars->v_empty[s]), ph ^ 1, abort_flag, status, TC_ERR_LOAD);
+          if (!alive) break;
+          const uint32_t vf = smem_u32(&bars->v_full[s]);
+          mbar_expect_tx(vf, TC_TILE_BYTES);
+          tma_load_4d(sV + s * TC_TILE_BYTES, &tm_v, vf, 0, key0, w.h_idx, w.b_idx);
+          tma_load_4d(sV + s * TC_TILE_BYTES + TC_SUB_BYTES, &tm_v, vf, 64, key0, w.h_idx, w.b_idx);
+        }
+        ++n_done;
       }
     }
   } else if (warp == 1) {
@@ -150,38 +178,53 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           umma_ts(tmem + 256 + i * TC_D, tmem + i * TC_BN + kk * 8, pk2u(b0 + kk * (16 * 128 >> 4), v_hi), idesc_pv,
                   (acc || kk > half * 4) ? 1u : 0u);
       };
-      bool alive = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag, status, TC_ERR_MMA);
-      alive = alive && mbar_wait(smem_u32(&bars->k_full[0]), 0, abort_flag, status, TC_ERR_MMA);
-      tc_fence_after();
-      for (int i = 0; i < ntiles; ++i) {
-        issue_qk(i, 0);
-        umma_commit(smem_u32(&bars->s_ready[i]));
-      }
-      umma_commit(smem_u32(&bars->k_empty[0]));
-      for (int j = 0; j < n_kv; ++j) {
-        const int s = j % TC_STAGES;
-        const uint32_t ph = (j / TC_STAGES) & 1;
-        mbar_wait(smem_u32(&bars->v_full[s]), ph, abort_flag, status, TC_ERR_MMA);
-        for (int i = 0; i < ntiles; ++i) {
-          mbar_wait(smem_u32(&bars->p_half[i][0]), j & 1, abort_flag, status, TC_ERR_MMA);
-          tc_fence_after();
-          issue_pv(i, s, 0, j > 0);
-          mbar_wait(smem_u32(&bars->p_half[i][1]), j & 1, abort_flag, status, TC_ERR_MMA);
-          tc_fence_after();
-          issue_pv(i, s, 1, true);
-          umma_commit(smem_u32(&bars->pv_done[i]));
-          if (i == ntiles - 1) umma_commit(smem_u32(&bars->v_empty[s]));
-          if (j + 1 < n_kv) {
-            const int s1 = (j + 1) % TC_STAGES;
-            if (i == 0) {
-              mbar_wait(smem_u32(&bars->k_full[s1]), ((j + 1) / TC_STAGES) & 1, abort_flag, status, TC_ERR_MMA);
-              tc_fence_after();
+      uint32_t kv_it = 0, n_done = 0;                                // K/V tiles consumed, items done
+      uint32_t n_p[TC_QT] = {0, 0}, n_o[TC_QT] = {0, 0};             // P hand-overs and items per query tile
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        WinItem w;
+        if (!win_item(g, item, pairs, w)) continue;
+        mbar_wait(smem_u32(&bars->q_full), n_done & 1, abort_flag, status, TC_ERR_MMA);
+        mbar_wait(smem_u32(&bars->k_full[kv_it % TC_STAGES]), (kv_it / TC_STAGES) & 1, abort_flag, status, TC_ERR_MMA);
+        tc_fence_after();
+        for (int i = 0; i < w.ntiles; ++i) {
+          issue_qk(i, kv_it % TC_STAGES);
+          umma_commit(smem_u32(&bars->s_ready[i]));
+        }
+        umma_commit(smem_u32(&bars->k_empty[kv_it % TC_STAGES]));
+        if (w.n_kv == 1) umma_commit(smem_u32(&bars->q_empty));
+        for (int j = 0; j < w.n_kv; ++j, ++kv_it) {
+          const int s = kv_it % TC_STAGES;
+          mbar_wait(smem_u32(&bars->v_full[s]), (kv_it / TC_STAGES) & 1, abort_flag, status, TC_ERR_MMA);
+          for (int i = 0; i < w.ntiles; ++i) {
+            // the first P V of an item overwrites O: the epilogue of the tile's previous item must have read it
+            if (j == 0 && n_o[i] > 0)
+              mbar_wait(smem_u32(&bars->o_free[i]), (n_o[i] - 1) & 1, abort_flag, status, TC_ERR_MMA);
+            mbar_wait(smem_u32(&bars->p_half[i][0]), n_p[i] & 1, abort_flag, status, TC_ERR_MMA);
+            tc_fence_after();
+            issue_pv(i, s, 0, j > 0);
+            mbar_wait(smem_u32(&bars->p_half[i][1]), n_p[i] & 1, abort_flag, status, TC_ERR_MMA);
+            tc_fence_after();
+            issue_pv(i, s, 1, true);
+            ++n_p[i];
+            umma_commit(smem_u32(&bars->pv_done[i]));
+            if (i == w.ntiles - 1) umma_commit(smem_u32(&bars->v_empty[s]));
+            if (j + 1 < w.n_kv) {
+              const int s1 = (kv_it + 1) % TC_STAGES;
+              if (i == 0) {
+                mbar_wait(smem_u32(&bars->k_full[s1]), ((kv_it + 1) / TC_STAGES) & 1, abort_flag, status, TC_ERR_MMA);
+                tc_fence_after();
+              }
+              issue_qk(i, s1);
+              umma_commit(smem_u32(&bars->s_ready[i]));
+              if (i == w.ntiles - 1) {
+                umma_commit(smem_u32(&bars->k_empty[s1]));
+                if (j + 2 == w.n_kv) umma_commit(smem_u32(&bars->q_empty));   // the item's last Q K^T
+              }
             }
-            issue_qk(i, s1);
-            umma_commit(smem_u32(&bars->s_ready[i]));
-            if (i == ntiles - 1) umma_commit(smem_u32(&bars->k_empty[s1]));
           }
         }
+        ++n_done;
+        for (int i = 0; i < w.ntiles; ++i) ++n_o[i];
       }
       // everything this thread issued has completed once `drained` flips
       umma_commit(smem_u32(&bars->drained));
@@ -191,14 +234,18 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     // ------------------------------------------------------------------ softmax + epilogue
     setmaxnreg_inc<TC_REGS_SOFTMAX>();
     const int i = (warp - 4) >> 2;                                   // query tile of this warpgroup
-    if (i < ntiles) {
-      const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-      const uint32_t tS = tmem + lane_off + i * TC_BN, tO = tmem + lane_off + 256 + i * TC_D;
-      const float c = scale * 1.4426950408889634f;                   // logits -> log2 domain
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + lane_off + i * TC_BN, tO = tmem + lane_off + 256 + i * TC_D;
+    const float c = scale * 1.4426950408889634f;                     // logits -> log2 domain
+    uint32_t n_s = 0;                                                // key tiles this query tile has been through
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+      WinItem w;
+      if (!win_item(g, item, pairs, w) || i >= w.ntiles) continue;
+      const int n_kv = w.n_kv, lo = w.lo, hi = w.hi;
       float m_true = -INFINITY, m_used = -INFINITY;
       uint64_t l2a = 0ull, l2b = 0ull;                               // four partial row sums as two fp32 pairs
       for (int j = 0; j < n_kv; ++j) {
-        mbar_wait(smem_u32(&bars->s_ready[i]), j & 1, abort_flag, status, TC_ERR_SOFTMAX);
+        mbar_wait(smem_u32(&bars->s_ready[i]), (n_s + j) & 1, abort_flag, status, TC_ERR_SOFTMAX);
         tc_fence_after();
         uint32_t sr[4][32];
 #pragma unroll
@@ -225,7 +272,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           const float m_new = need ? m_true : m_used;
           if (j > 0) {
             // s_ready(j) follows the completion of P V of tile j-1, so O may be touched
-            mbar_wait(smem_u32(&bars->pv_done[i]), (j - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+            mbar_wait(smem_u32(&bars->pv_done[i]), (n_s + j - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
             tc_fence_after();
             const float f = ex2((m_used - m_new) * c);               // 1 for lanes that keep their reference
             const uint64_t f2 = pk2(f, f);
@@ -272,49 +319,57 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       upk2(l2a, la0, la1);
       upk2(l2b, lb0, lb1);
       const float l = (la0 + la1) + (lb0 + lb1);
-      mbar_wait(smem_u32(&bars->pv_done[i]), (n_kv - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
-      tc_fence_after();
 
       // Eq. 5: bring O and l to the final row maximum, add the linear read-out, divide, store.
-      const int row = row_base + i * TC_BM + (warp & 3) * 32 + lane;
-      const bool valid = row < q1;
-      const float fin = ex2((m_used - m_true) * c);
-      float ws = fin, lam = 0.f, nL = 0.f;
-      const float* rrow = nullptr;
+      const int row = w.row_base + i * TC_BM + (warp & 3) * 32 + lane;
+      const bool valid = row < w.q1;
+      // the whole read-out row is requested before the wait for the last P V, which hides its latency
+      float4 rdv[TC_D / 4];
+      float nL = 0.f;
       if (lo > 0) {
-        rrow = rd + ((size_t)bh * rd_rows + (size_t)((valid ? row : q0) - geo_q0(g, g.t0))) * (TC_D + 4);
+        const float* rrow = rd + ((size_t)w.bh * rd_rows + (size_t)((valid ? row : w.q0) - geo_q0(g, g.t0))) * (TC_D + 4);
+#pragma unroll
+        for (int u = 0; u < TC_D / 4; ++u) rdv[u] = __ldg(reinterpret_cast<const float4*>(rrow) + u);
+        nL = __ldg(rrow + TC_D);
+      } else {
+#pragma unroll
+        for (int u = 0; u < TC_D / 4; ++u) rdv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      const float fin = ex2((m_used - m_true) * c);
+      float ws = fin, lam = 0.f;
+      if (lo > 0) {
         lam = 1.f;
         if (c_mode == C_ZERO) {
           const float mm = m_true * scale, r = fmaxf(mm, 0.f);
           ws = fin * __expf(mm - r);
           lam = __expf(-r);
         }
-        nL = rrow[TC_D];
       }
+      __nv_bfloat16* orow = out + head_offset(g, w.bh) + (long long)row * g.stride_n;
+      mbar_wait(smem_u32(&bars->pv_done[i]), (n_s + n_kv - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+      tc_fence_after();
+      n_s += n_kv;
       const float inv = 1.f / (l * ws + lam * nL);
-      __nv_bfloat16* orow = out + head_offset(g, bh) + (long long)row * g.stride_n;
+      const float wsi = ws * inv, lami = lam * inv;
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
+      for (int hh = 0; hh < 4; ++hh) {                               // 32 columns of O at a time
         uint32_t o[32];
-        tmem_ld32(tO + cc * 32, o);
+        tmem_ld32(tO + hh * 32, o);
         tmem_wait_ld();
+        if (hh == 3) {                                               // O has been read: TMEM is free for the next item
+          tc_fence_before();
+          mbar_arrive(smem_u32(&bars->o_free[i]));
+        }
         if (valid) {
 #pragma unroll
           for (int e = 0; e < 32; e += 8) {
-            float a[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) a[u] = 0.f;
-            if (lo > 0) {
-              const float4 x0 = *reinterpret_cast<const float4*>(rrow + cc * 32 + e);
-              const float4 x1 = *reinterpret_cast<const float4*>(rrow + cc * 32 + e + 4);
-              a[0] = x0.x; a[1] = x0.y; a[2] = x0.z; a[3] = x0.w; a[4] = x1.x; a[5] = x1.y; a[6] = x1.z; a[7] = x1.w;
-            }
-            uint4 w;
-            w.x = pack_bf16((__uint_as_float(o[e + 0]) * ws + lam * a[0]) * inv, (__uint_as_float(o[e + 1]) * ws + lam * a[1]) * inv);
-            w.y = pack_bf16((__uint_as_float(o[e + 2]) * ws + lam * a[2]) * inv, (__uint_as_float(o[e + 3]) * ws + lam * a[3]) * inv);
-            w.z = pack_bf16((__uint_as_float(o[e + 4]) * ws + lam * a[4]) * inv, (__uint_as_float(o[e + 5]) * ws + lam * a[5]) * inv);
-            w.w = pack_bf16((__uint_as_float(o[e + 6]) * ws + lam * a[6]) * inv, (__uint_as_float(o[e + 7]) * ws + lam * a[7]) * inv);
-            *reinterpret_cast<uint4*>(orow + cc * 32 + e) = w;
+            const float4 x0 = rdv[hh * 8 + (e >> 2)], x1 = rdv[hh * 8 + (e >> 2) + 1];
+            uint4 v4;
+            v4.x = pack_bf16(__uint_as_float(o[e + 0]) * wsi + lami * x0.x, __uint_as_float(o[e + 1]) * wsi + lami * x0.y);
+            v4.y = pack_bf16(__uint_as_float(o[e + 2]) * wsi + lami * x0.z, __uint_as_float(o[e + 3]) * wsi + lami * x0.w);
+            v4.z = pack_bf16(__uint_as_float(o[e + 4]) * wsi + lami * x1.x, __uint_as_float(o[e + 5]) * wsi + lami * x1.y);
+            v4.w = pack_bf16(__uint_as_float(o[e + 6]) * wsi + lami * x1.z, __uint_as_float(o[e + 7]) * wsi + lami * x1.w);
+            *reinterpret_cast<uint4*>(orow + hh * 32 + e) = v4;
           }
         }
       }
@@ -412,15 +467,19 @@ inline int tc_launch_window(const TcWorkspace* w, const void* q, const void* k, 
   if (!tc_make_tmap(w, &tq, q, g, batch) || !tc_make_tmap(w, &tk, k, g, batch) || !tc_make_tmap(w, &tv, v, g, batch))
     return REHYAT_ERR_CUDA;
   const int pairs = (g.Np + TC_QT * TC_BM - 1) / (TC_QT * TC_BM);
-  const dim3 grid(pairs, g.G, g.BH);
+  const int n_items = pairs * g.G * g.BH;
+  const dim3 grid(n_items < w->n_sm ? n_items : w->n_sm);
   const float scale = 1.0f / sqrtf((float)TC_D);
   __nv_bfloat16* o = (__nv_bfloat16*)out;
+#define REHYAT_LAUNCH_WINDOW(E) \
+  window_tc<E><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status, n_items, pairs)
   switch (w->exp_poly) {
-    case 0: window_tc<0><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status); break;
-    default: window_tc<1><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status); break;
-    case 3: window_tc<3><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status); break;
-    case 2: window_tc<2><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status); break;
+    case 0: REHYAT_LAUNCH_WINDOW(0); break;
+    case 2: REHYAT_LAUNCH_WINDOW(2); break;
+    case 3: REHYAT_LAUNCH_WINDOW(3); break;
+    default: REHYAT_LAUNCH_WINDOW(1); break;
   }
+#undef REHYAT_LAUNCH_WINDOW
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
