@@ -132,6 +132,36 @@ int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host,
                         int32_t batch, int32_t frames, int32_t H, int32_t W,
                         int32_t chunk, int32_t overlap, void* cuda_stream);
 
+/* Chunk-by-chunk processing: the recurrent form of Section 3.3 (Eq. 14-18) with the state kept by the
+ * context, for callers that produce or hold one chunk of the video at a time.  Device memory then scales
+ * with one chunk plus the overlap, not with the video (Section 3.3, note 3).
+ *
+ * rehyat_stream_begin starts a sequence (s_0 = 0, z_0 = 0, Eq. 14-15) for chunks of at most `chunk` frames
+ * with `overlap` frames of overlap, and sizes six staging buffers of (overlap + chunk)*H*W tokens per
+ * (batch, head): the only allocation of this API, repeated only when a later sequence needs more.
+ * rehyat_stream_step takes the next chunk,
+ *   q_chunk, k_chunk, v_chunk, out_chunk   device, [batch, n_heads, frames_in_chunk*H*W, head_dim] through `lay`
+ *   frames_in_chunk                        1..chunk; only the last chunk of a video may be shorter than `chunk`
+ * computes its output from the softmax window (the overlap frames kept from earlier chunks plus the chunk,
+ * Eq. 12-13) and the running state (Eq. 16), then folds the tokens that leave the window into the state
+ * (Eq. 17-18, new tokens only).  Asynchronous on `cuda_stream`; the same stream must be used for all steps
+ * of a sequence.  rehyat_forward on the same context ends the sequence (both use the context's workspace).
+ *
+ * rehyat_stream_export writes the sequence's state (a small header, s and z in fp32, the overlap frames of
+ * k and v) to HOST memory after synchronising the stream; rehyat_stream_state_bytes is its size right now.
+ * rehyat_stream_import starts a sequence from such a blob on any context with the same dtype, head count,
+ * head_dim and phi_dim: a checkpoint.  A resumed sequence continues bit-for-bit.
+ * Errors: INVALID_ARG (no active sequence, sizes beyond the context's max_* fields, a blob that does not
+ * match), ALLOC, CUDA. */
+int rehyat_stream_begin(rehyat_ctx* ctx, int32_t batch, int32_t H, int32_t W, int32_t chunk, int32_t overlap,
+                        void* cuda_stream);
+int rehyat_stream_step(rehyat_ctx* ctx, const void* q_chunk, const void* k_chunk, const void* v_chunk,
+                       void* out_chunk, const rehyat_layout* lay, const rehyat_phi_params* phi,
+                       int32_t frames_in_chunk, void* cuda_stream);
+size_t rehyat_stream_state_bytes(const rehyat_ctx* ctx);
+int rehyat_stream_export(rehyat_ctx* ctx, void* host_buf, size_t capacity, void* cuda_stream);
+int rehyat_stream_import(rehyat_ctx* ctx, const void* host_buf, size_t bytes, void* cuda_stream);
+
 /* The same operator for callers that must not allocate device memory: code that runs inside a
  * memory plan fixed up front (all device memory already handed to another allocator or pool), a
  * latency-critical loop that cannot afford the device-wide synchronisation cudaMalloc / cudaFree

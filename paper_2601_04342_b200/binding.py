@@ -19,6 +19,8 @@ IMPL = {"auto": 0, "simt": 1, "tensor": 2, "tensor_window": 3}
 
 EXPORTS = ["rehyat_create", "rehyat_forward", "rehyat_forward_host", "rehyat_forward_static",
            "rehyat_static_scratch_bytes", "rehyat_destroy",
+           "rehyat_stream_begin", "rehyat_stream_step", "rehyat_stream_state_bytes", "rehyat_stream_export",
+           "rehyat_stream_import",
            "rehyat_workspace_bytes", "rehyat_status", "rehyat_last_launches", "rehyat_last_impl",
            "rehyat_profile_enable", "rehyat_profile_read", "rehyat_strerror", "rehyat_version"]
 PROF_KINDS = ("state", "scan", "readout", "window")
@@ -59,6 +61,13 @@ def lib():
         L.rehyat_static_scratch_bytes.argtypes = []
         L.rehyat_static_scratch_bytes.restype = C.c_size_t
         L.rehyat_destroy.argtypes = [C.c_void_p]
+        L.rehyat_stream_begin.argtypes = [C.c_void_p] + [C.c_int32] * 5 + [C.c_void_p]
+        L.rehyat_stream_step.argtypes = [C.c_void_p] + [C.c_void_p] * 4 + [C.POINTER(Layout), C.POINTER(PhiParams),
+                                                                          C.c_int32, C.c_void_p]
+        L.rehyat_stream_state_bytes.argtypes = [C.c_void_p]
+        L.rehyat_stream_state_bytes.restype = C.c_size_t
+        L.rehyat_stream_export.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.rehyat_stream_import.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.rehyat_workspace_bytes.argtypes = [C.c_void_p]
         L.rehyat_workspace_bytes.restype = C.c_size_t
         L.rehyat_status.argtypes = [C.c_void_p, C.c_void_p]
@@ -162,6 +171,37 @@ class Rehyat:
         _check(lib().rehyat_forward_host(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), C.byref(phi), B, frames, H,
                                          W, chunk, overlap, C.c_void_p(st.cuda_stream)), "rehyat_forward_host")
         return out
+
+    # ---- chunk-by-chunk processing (rehyat_stream_*)
+    def stream_begin(self, batch, H, W, chunk, overlap, stream=None):
+        st = stream if stream is not None else torch.cuda.current_stream(self.cfg.device)
+        _check(lib().rehyat_stream_begin(self._h, batch, H, W, chunk, overlap, C.c_void_p(st.cuda_stream)),
+               "rehyat_stream_begin")
+
+    def stream_step(self, q, k, v, phi_q, phi_k, frames_in_chunk, out=None, stream=None):
+        """q, k, v: contiguous CUDA tensors [B, n_heads, frames_in_chunk*H*W, d] of the next chunk."""
+        if out is None:
+            out = torch.empty_like(q)
+        B, nh, N, d = q.shape
+        lay = Layout(nh * N * d, N * d, d)
+        st = stream if stream is not None else torch.cuda.current_stream(q.device)
+        phi = self.phi_struct(phi_q, phi_k)
+        _check(lib().rehyat_stream_step(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), C.byref(lay), C.byref(phi),
+                                        frames_in_chunk, C.c_void_p(st.cuda_stream)), "rehyat_stream_step")
+        return out
+
+    def stream_export(self, stream=None):
+        """The sequence's state as bytes (header, s and z, the overlap frames of k and v)."""
+        st = stream if stream is not None else torch.cuda.current_stream(self.cfg.device)
+        n = lib().rehyat_stream_state_bytes(self._h)
+        buf = (C.c_uint8 * n)()
+        _check(lib().rehyat_stream_export(self._h, buf, n, C.c_void_p(st.cuda_stream)), "rehyat_stream_export")
+        return bytes(buf)
+
+    def stream_import(self, blob, stream=None):
+        st = stream if stream is not None else torch.cuda.current_stream(self.cfg.device)
+        buf = (C.c_uint8 * len(blob)).from_buffer_copy(blob)
+        _check(lib().rehyat_stream_import(self._h, buf, len(blob), C.c_void_p(st.cuda_stream)), "rehyat_stream_import")
 
     def profile_enable(self, on=True):
         _check(lib().rehyat_profile_enable(self._h, int(on)), "rehyat_profile_enable")

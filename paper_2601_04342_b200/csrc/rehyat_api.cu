@@ -57,6 +57,22 @@ struct rehyat_ctx {
   size_t stage_bytes = 0;
   int last_launches = 0, last_impl = 0;
   bool tensor_ok = false;
+  // chunk-by-chunk processing (rehyat_stream_*): the running state lives in slot 0 of `state`, the last
+  // `overlap` frames of k and v and the chunk being processed in staging buffers [BH][cap_tokens][d]
+  struct Stream {
+    bool active = false;
+    int batch = 0, H = 0, W = 0, chunk = 0, overlap = 0;
+    int halo = 0;                 // tokens of earlier chunks still inside the softmax window
+    int has_state = 0;            // the running state covers at least one token
+    long long chunks_done = 0;
+    int cap_tokens = 0;           // tokens per (batch, head) each staging buffer holds
+    int cur = 0;                  // which of the two k / v buffers holds the halo
+    void* kbuf[2] = {nullptr, nullptr};
+    void* vbuf[2] = {nullptr, nullptr};
+    void* qbuf = nullptr;
+    void* obuf = nullptr;
+    size_t bytes = 0;
+  } stream;
 };
 
 namespace {
@@ -104,17 +120,18 @@ int set_simt_attributes(const rehyat_config& c) {
   return REHYAT_OK;
 }
 
+// Which steps of a chunk group to enqueue.
+enum Parts : int { PART_STATE = 1 /* increments + scan */, PART_READOUT = 2, PART_WINDOW = 4 };
+
 template <typename T, int D>
 int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* out, const rehyat_phi_params* phi,
-                      const Geo& g, int n_split, int carry_slot, bool any_linear, cudaStream_t st,
-                      bool with_window = true) {
+                      const Geo& g, int n_split, int carry_slot, int parts, cudaStream_t st) {
   const rehyat_config& c = ctx->cfg;
   PhiDims pd = {D, c.phi_hidden, c.phi_dim, c.poly_degree, c.act_hidden, c.act_out};
   constexpr int SD = D + 4;
   const int tiles = (g.Np + SIMT_TM - 1) / SIMT_TM;
-  if (any_linear) {
+  if (parts & PART_STATE) {
     PhiPtrs<T> wk = {(const T*)phi->k_W1, (const T*)phi->k_b1, (const T*)phi->k_W2, (const T*)phi->k_b2};
-    PhiPtrs<T> wq = {(const T*)phi->q_W1, (const T*)phi->q_b1, (const T*)phi->q_W2, (const T*)phi->q_b2};
     const size_t smem_state = (size_t)SIMT_TM * (2 * D + pd.Dh + pd.Dp) * sizeof(float);
     ctx->prof.begin(REHYAT_PROF_STATE, st);
     state_partial_simt<T, D><<<dim3(n_split, g.G, g.BH), SIMT_PHI_THREADS, smem_state, st>>>(
@@ -125,22 +142,114 @@ int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* ou
     scan_states<<<(unsigned)((per_slot + 255) / 256), 256, 0, st>>>(ctx->partial, ctx->state, per_slot, g.G,
                                                                      n_split, carry_slot);
     ctx->prof.end(REHYAT_PROF_SCAN, st);
+    ctx->last_launches += 2;
+  }
+  if (parts & PART_READOUT) {
+    PhiPtrs<T> wq = {(const T*)phi->q_W1, (const T*)phi->q_b1, (const T*)phi->q_W2, (const T*)phi->q_b2};
     const size_t smem_rd = (size_t)SIMT_TM * (D + pd.Dh + pd.Dp) * sizeof(float);
     ctx->prof.begin(REHYAT_PROF_READOUT, st);
     readout_simt<T, D><<<dim3(tiles, g.G, g.BH), SIMT_PHI_THREADS, smem_rd, st>>>(q, wq, pd, g, ctx->state,
                                                                                  ctx->readout, ctx->rd_rows);
     ctx->prof.end(REHYAT_PROF_READOUT, st);
-    ctx->last_launches += 3;
+    ctx->last_launches += 1;
   }
-  if (!with_window) return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
-  const size_t smem_win = (size_t)(WIN_BM * (D + 4) + WIN_BN * (D + 4) + WIN_BN * D + WIN_BM * (WIN_BN + 4)) * sizeof(float);
-  const int wtiles = (g.Np + WIN_BM - 1) / WIN_BM;
-  ctx->prof.begin(REHYAT_PROF_WINDOW, st);
-  window_simt<T, D><<<dim3(wtiles, g.G, g.BH), WIN_THREADS, smem_win, st>>>(
-      q, k, v, out, g, ctx->readout, ctx->rd_rows, 1.0f / sqrtf((float)D), c.c_mode);
-  ctx->prof.end(REHYAT_PROF_WINDOW, st);
-  ctx->last_launches += 1;
+  if (parts & PART_WINDOW) {
+    const size_t smem_win = (size_t)(WIN_BM * (D + 4) + WIN_BN * (D + 4) + WIN_BN * D + WIN_BM * (WIN_BN + 4)) * sizeof(float);
+    const int wtiles = (g.Np + WIN_BM - 1) / WIN_BM;
+    ctx->prof.begin(REHYAT_PROF_WINDOW, st);
+    window_simt<T, D><<<dim3(wtiles, g.G, g.BH), WIN_THREADS, smem_win, st>>>(
+        q, k, v, out, g, ctx->readout, ctx->rd_rows, 1.0f / sqrtf((float)D), c.c_mode);
+    ctx->prof.end(REHYAT_PROF_WINDOW, st);
+    ctx->last_launches += 1;
+  }
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
+}
+
+// Split of a chunk's state increment over CTAs.  Tensor-core kernels: one CTA per (split, chunk, head)
+// and one CTA per SM, so pick the split that needs the fewest token tiles per SM over all waves.
+int pick_state_split(const rehyat_ctx* ctx, const Geo& g, int n_chunks_in_group, int tokens_per_increment) {
+  int n_split = ctx->partial_units / (n_chunks_in_group > 0 ? n_chunks_in_group : 1);
+  if (n_split > 8) n_split = 8;
+  if (n_split < 1) n_split = 1;
+  if (ctx->tensor_ok && ctx->tc.phi_ok) {
+    const int n_sm = ctx->tc.n_sm;
+    int busy = 0;                                   // chunks of the group that admit keys into the state
+    for (int t = g.t0 > 1 ? g.t0 : 1; t < g.t0 + n_chunks_in_group; ++t) busy += geo_lo(g, t) > geo_lo(g, t - 1);
+    const long long units = (long long)(busy > 0 ? busy : 1) * g.BH, tiles = (tokens_per_increment + 127) / 128;
+    long long best = -1;
+    int best_s = 1;
+    for (int s = 1; s <= n_split; ++s) {
+      const long long cost = ((units * s + n_sm - 1) / n_sm) * ((tiles + s - 1) / s);
+      if (best < 0 || cost < best) { best = cost; best_s = s; }
+    }
+    n_split = best_s;
+  }
+  return n_split;
+}
+
+// Enqueues the requested steps for the chunks [g.t0, g.t0 + g.G) with whichever kernel family the context uses.
+int run_parts(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void* out, const rehyat_phi_params* phi,
+              const Geo& g, int batch, int n_split, int carry_slot, int parts, cudaStream_t st) {
+  const rehyat_config& c = ctx->cfg;
+  int rc = REHYAT_OK;
+  if (ctx->tensor_ok) {
+    using B = __nv_bfloat16;
+    if (!ctx->tc.phi_ok) {
+      rc = launch_group_simt<B, 128>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot,
+                                     parts & (PART_STATE | PART_READOUT), st);
+    } else {
+      if (parts & PART_STATE) {
+        ctx->prof.begin(REHYAT_PROF_STATE, st);
+        rc = tc_launch_state(&ctx->tc, k, v, phi, g, batch, c.poly_degree, c.act_hidden, c.act_out, n_split,
+                             ctx->partial, ctx->status_dev, st);
+        ctx->prof.end(REHYAT_PROF_STATE, st);
+        const size_t per_slot = (size_t)g.BH * c.phi_dim * (c.head_dim + 4);
+        ctx->prof.begin(REHYAT_PROF_SCAN, st);
+        scan_states<<<(unsigned)((per_slot + 255) / 256), 256, 0, st>>>(ctx->partial, ctx->state, per_slot, g.G, n_split,
+                                                                         carry_slot, ctx->tc.state_bf16, c.head_dim);
+        ctx->prof.end(REHYAT_PROF_SCAN, st);
+        ctx->last_launches += 2;
+      }
+      if (rc == REHYAT_OK && (parts & PART_READOUT)) {
+        ctx->prof.begin(REHYAT_PROF_READOUT, st);
+        rc = tc_launch_readout(&ctx->tc, q, phi, g, batch, c.poly_degree, c.act_hidden, c.act_out, ctx->state,
+                               ctx->readout, ctx->rd_rows, ctx->status_dev, st);
+        ctx->prof.end(REHYAT_PROF_READOUT, st);
+        ctx->last_launches += 1;
+      }
+    }
+    if (rc == REHYAT_OK && (parts & PART_WINDOW)) {
+      ctx->prof.begin(REHYAT_PROF_WINDOW, st);
+      rc = tc_launch_window(&ctx->tc, q, k, v, out, g, batch, ctx->readout, ctx->rd_rows, c.c_mode, ctx->status_dev, st);
+      ctx->prof.end(REHYAT_PROF_WINDOW, st);
+      ctx->last_launches += 1;
+    }
+  } else if (c.dtype == REHYAT_DTYPE_FP32) {
+    rc = c.head_dim == 64
+             ? launch_group_simt<float, 64>(ctx, (const float*)q, (const float*)k, (const float*)v, (float*)out, phi, g, n_split, carry_slot, parts, st)
+             : launch_group_simt<float, 128>(ctx, (const float*)q, (const float*)k, (const float*)v, (float*)out, phi, g, n_split, carry_slot, parts, st);
+  } else {
+    using B = __nv_bfloat16;
+    rc = c.head_dim == 64
+             ? launch_group_simt<B, 64>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot, parts, st)
+             : launch_group_simt<B, 128>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot, parts, st);
+  }
+  return rc;
+}
+
+// Copies `rows` token rows of `row_bytes` bytes for each of BH (batch, head) problems between two strided
+// layouts (byte strides; rows are contiguous and 16-byte aligned).  grid (row tiles, BH), 256 threads.
+__global__ void copy_rows(uint8_t* __restrict__ dst, long long dst_b, long long dst_h, long long dst_n,
+                          const uint8_t* __restrict__ src, long long src_b, long long src_h, long long src_n,
+                          int rows, int row_bytes, int n_heads) {
+  const int bh = blockIdx.y, b = bh / n_heads, h = bh % n_heads;
+  const int per_row = row_bytes / 16;
+  const long long total = (long long)rows * per_row;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / per_row, c = (i % per_row) * 16;
+    *reinterpret_cast<uint4*>(dst + b * dst_b + h * dst_h + r * dst_n + c) =
+        *reinterpret_cast<const uint4*>(src + b * src_b + h * src_h + r * src_n + c);
+  }
 }
 
 }  // namespace
@@ -230,6 +339,8 @@ int rehyat_destroy(rehyat_ctx* ctx) {
   tc_workspace_destroy(&ctx->tc);
   ctx->prof.clear();
   for (void* p : ctx->stage) cudaFree(p);
+  for (int i = 0; i < 2; ++i) { cudaFree(ctx->stream.kbuf[i]); cudaFree(ctx->stream.vbuf[i]); }
+  cudaFree(ctx->stream.qbuf); cudaFree(ctx->stream.obuf);
   delete ctx;
   return REHYAT_OK;
 }
@@ -315,77 +426,24 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   g.BH = batch * c.n_heads;
   g.stride_b = lay->stride_batch; g.stride_h = lay->stride_head; g.stride_n = lay->stride_token;
   const int n_chunks = (frames + chunk_eff - 1) / chunk_eff;
+  g.q_shift = 0;
+  g.prefix = 0;
   int G = ctx->rd_rows / g.Np;
   if (G < 1) return REHYAT_ERR_INVALID_ARG;   // cannot happen: rd_rows >= max chunk size
   if (G > ctx->Gmax) G = ctx->Gmax;
-  int n_split = ctx->partial_units / G;
-  if (n_split > 8) n_split = 8;
-  if (ctx->tensor_ok && ctx->tc.phi_ok) {
-    // One CTA per (split, chunk, head) and one CTA per SM: pick the split that needs the fewest
-    // token tiles per SM over all waves.
-    const int n_sm = ctx->tc.n_sm;
-    int busy = 0;                                   // chunks of the first group that admit keys into the state
-    for (int t = 1; t < (G < n_chunks ? G : n_chunks); ++t) busy += geo_lo(g, t) > geo_lo(g, t - 1);
-    const long long units = (long long)(busy > 0 ? busy : 1) * g.BH, tiles = (g.Np + 127) / 128;
-    long long best = -1;
-    int best_s = 1;
-    for (int s = 1; s <= n_split; ++s) {
-      const long long cost = ((units * s + n_sm - 1) / n_sm) * ((tiles + s - 1) / s);
-      if (best < 0 || cost < best) { best = cost; best_s = s; }
-    }
-    n_split = best_s;
-  }
+  g.t0 = 0;
+  const int n_split = pick_state_split(ctx, g, G < n_chunks ? G : n_chunks, g.Np);
 
   ctx->last_launches = 0;
   ctx->last_impl = ctx->tensor_ok ? 1 : 0;
+  ctx->stream.active = false;                 // the workspace is about to be overwritten
   int carry_slot = -1;
   for (int t0 = 0; t0 < n_chunks; t0 += G) {
     g.t0 = t0;
     g.G = (n_chunks - t0) < G ? (n_chunks - t0) : G;
     const bool any_linear = geo_lo(g, t0 + g.G - 1) > 0;
-    int rc;
-    if (ctx->tensor_ok) {
-      using B = __nv_bfloat16;
-      if (!ctx->tc.phi_ok) {
-        rc = launch_group_simt<B, 128>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot,
-                                       any_linear, st, /*with_window=*/false);
-      } else if (any_linear) {
-        ctx->prof.begin(REHYAT_PROF_STATE, st);
-        rc = tc_launch_state(&ctx->tc, k, v, phi, g, batch, c.poly_degree, c.act_hidden, c.act_out, n_split,
-                             ctx->partial, ctx->status_dev, st);
-        ctx->prof.end(REHYAT_PROF_STATE, st);
-        const size_t per_slot = (size_t)g.BH * c.phi_dim * (c.head_dim + 4);
-        ctx->prof.begin(REHYAT_PROF_SCAN, st);
-        scan_states<<<(unsigned)((per_slot + 255) / 256), 256, 0, st>>>(ctx->partial, ctx->state, per_slot, g.G, n_split,
-                                                                         carry_slot, ctx->tc.state_bf16, c.head_dim);
-        ctx->prof.end(REHYAT_PROF_SCAN, st);
-        if (rc == REHYAT_OK) {
-          ctx->prof.begin(REHYAT_PROF_READOUT, st);
-          rc = tc_launch_readout(&ctx->tc, q, phi, g, batch, c.poly_degree, c.act_hidden, c.act_out, ctx->state,
-                                 ctx->readout, ctx->rd_rows, ctx->status_dev, st);
-          ctx->prof.end(REHYAT_PROF_READOUT, st);
-        }
-        ctx->last_launches += 3;
-      } else {
-        rc = REHYAT_OK;
-      }
-      if (rc == REHYAT_OK) {
-        ctx->prof.begin(REHYAT_PROF_WINDOW, st);
-        rc = tc_launch_window(&ctx->tc, q, k, v, out, g, batch, ctx->readout, ctx->rd_rows, c.c_mode,
-                              ctx->status_dev, st);
-        ctx->prof.end(REHYAT_PROF_WINDOW, st);
-        ctx->last_launches += 1;
-      }
-    } else if (c.dtype == REHYAT_DTYPE_FP32) {
-      rc = c.head_dim == 64
-               ? launch_group_simt<float, 64>(ctx, (const float*)q, (const float*)k, (const float*)v, (float*)out, phi, g, n_split, carry_slot, any_linear, st)
-               : launch_group_simt<float, 128>(ctx, (const float*)q, (const float*)k, (const float*)v, (float*)out, phi, g, n_split, carry_slot, any_linear, st);
-    } else {
-      using B = __nv_bfloat16;
-      rc = c.head_dim == 64
-               ? launch_group_simt<B, 64>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot, any_linear, st)
-               : launch_group_simt<B, 128>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot, any_linear, st);
-    }
+    const int rc = run_parts(ctx, q, k, v, out, phi, g, batch, n_split, carry_slot,
+                             (any_linear ? PART_STATE | PART_READOUT : 0) | PART_WINDOW, st);
     if (rc != REHYAT_OK) return rc;
     if (any_linear) carry_slot = g.G - 1;
   }
@@ -422,6 +480,206 @@ int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host,
   if (cudaMemcpyAsync(out_host, ctx->stage[3], bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return REHYAT_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
   return REHYAT_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Chunk-by-chunk processing: the recurrence of Eq. 14-18 with the state held by the context.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+struct StreamHeader {          // first bytes of an exported state
+  uint32_t magic, version;
+  int32_t dtype, n_heads, head_dim, phi_dim, batch, H, W, chunk, overlap, halo, has_state, reserved;
+  int64_t chunks_done;
+};
+constexpr uint32_t kStreamMagic = 0x52485953u;   // "RHYS"
+
+size_t stream_state_floats(const rehyat_ctx* ctx) {
+  return (size_t)ctx->stream.batch * ctx->cfg.n_heads * ctx->cfg.phi_dim * (ctx->cfg.head_dim + 4);
+}
+size_t stream_halo_bytes(const rehyat_ctx* ctx) {      // of k (and as much again of v)
+  return (size_t)ctx->stream.batch * ctx->cfg.n_heads * ctx->stream.halo * ctx->cfg.head_dim * elem_size(ctx->cfg.dtype);
+}
+
+void launch_copy_rows(void* dst, long long dst_b, long long dst_h, long long dst_n, const void* src, long long src_b,
+                      long long src_h, long long src_n, int rows, int row_bytes, int BH, int n_heads, cudaStream_t st) {
+  if (rows <= 0) return;
+  const long long total = (long long)rows * (row_bytes / 16);
+  const unsigned blocks = (unsigned)((total + 255) / 256 < 1024 ? (total + 255) / 256 : 1024);
+  copy_rows<<<dim3(blocks, BH), 256, 0, st>>>((uint8_t*)dst, dst_b, dst_h, dst_n, (const uint8_t*)src, src_b, src_h,
+                                              src_n, rows, row_bytes, n_heads);
+}
+
+}  // namespace
+
+int rehyat_stream_begin(rehyat_ctx* ctx, int32_t batch, int32_t H, int32_t W, int32_t chunk, int32_t overlap,
+                        void* cuda_stream) {
+  if (!ctx) return REHYAT_ERR_INVALID_ARG;
+  const rehyat_config& c = ctx->cfg;
+  if (batch < 1 || batch > c.max_batch || H < 1 || W < 1 || chunk < 1 || overlap < 0) return REHYAT_ERR_INVALID_ARG;
+  const long long HW = (long long)H * W;
+  if (HW > c.max_tokens_per_frame || chunk > c.max_chunk_frames) return REHYAT_ERR_INVALID_ARG;
+  const long long cap = (long long)(overlap + chunk) * HW;
+  if (cap > (1 << 24)) return REHYAT_ERR_INVALID_ARG;
+  DeviceGuard guard(c.device);
+  if (!guard.ok) return REHYAT_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  rehyat_ctx::Stream& s = ctx->stream;
+  const size_t one = (size_t)batch * c.n_heads * cap * c.head_dim * elem_size(c.dtype);
+  if (one * 6 > s.bytes) {                          // grow the six staging buffers (the only allocation of this API)
+    if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
+    void** all[6] = {&s.kbuf[0], &s.kbuf[1], &s.vbuf[0], &s.vbuf[1], &s.qbuf, &s.obuf};
+    for (void** p : all) { cudaFree(*p); *p = nullptr; }
+    s.bytes = 0;
+    for (void** p : all)
+      if (cudaMalloc(p, one) != cudaSuccess) { cudaGetLastError(); return REHYAT_ERR_ALLOC; }
+    s.bytes = one * 6;
+  }
+  s.active = true;
+  s.batch = batch; s.H = H; s.W = W; s.chunk = chunk; s.overlap = overlap;
+  s.cap_tokens = (int)cap;
+  s.halo = 0; s.has_state = 0; s.chunks_done = 0; s.cur = 0;
+  return REHYAT_OK;
+}
+
+int rehyat_stream_step(rehyat_ctx* ctx, const void* q_chunk, const void* k_chunk, const void* v_chunk, void* out_chunk,
+                       const rehyat_layout* lay, const rehyat_phi_params* phi, int32_t frames_in_chunk,
+                       void* cuda_stream) {
+  if (!ctx || !q_chunk || !k_chunk || !v_chunk || !out_chunk || !lay || !phi) return REHYAT_ERR_INVALID_ARG;
+  rehyat_ctx::Stream& s = ctx->stream;
+  if (!s.active || frames_in_chunk < 1 || frames_in_chunk > s.chunk) return REHYAT_ERR_INVALID_ARG;
+  const rehyat_config& c = ctx->cfg;
+  const void* ptrs[] = {q_chunk, k_chunk, v_chunk, out_chunk, phi->q_W1, phi->q_b1, phi->q_W2, phi->q_b2,
+                        phi->k_W1, phi->k_b1, phi->k_W2, phi->k_b2};
+  for (const void* p : ptrs)
+    if (!p || !aligned16(p)) return REHYAT_ERR_INVALID_ARG;
+  const long long es = (long long)elem_size(c.dtype);
+  const long long strides[] = {lay->stride_batch, lay->stride_head, lay->stride_token};
+  for (long long x : strides)
+    if (x < 0 || (x * es) % 16 != 0) return REHYAT_ERR_INVALID_ARG;
+  if (lay->stride_token < c.head_dim) return REHYAT_ERR_INVALID_ARG;
+  DeviceGuard guard(c.device);
+  if (!guard.ok) return REHYAT_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+
+  const int HW = s.H * s.W, Np = frames_in_chunk * HW, h = s.halo, BH = s.batch * c.n_heads;
+  const int row_bytes = c.head_dim * (int)es;
+  // staging layout [batch][head][cap_tokens][d]
+  const long long sn = c.head_dim, sh = (long long)s.cap_tokens * c.head_dim, sb = sh * c.n_heads;
+  uint8_t* kcur = (uint8_t*)s.kbuf[s.cur];
+  uint8_t* vcur = (uint8_t*)s.vbuf[s.cur];
+  // 1. the chunk goes behind the halo
+  const void* src[3] = {q_chunk, k_chunk, v_chunk};
+  uint8_t* dst[3] = {(uint8_t*)s.qbuf, kcur, vcur};
+  for (int i = 0; i < 3; ++i)
+    launch_copy_rows(dst[i] + (long long)h * sn * es, sb * es, sh * es, sn * es, src[i], lay->stride_batch * es,
+                     lay->stride_head * es, lay->stride_token * es, Np, row_bytes, BH, c.n_heads, st);
+  // 2. Eq. 16 for this chunk: one chunk whose queries start at buffer index h and whose window is the whole buffer
+  Geo g;
+  g.N = h + Np; g.Np = Np; g.ToHW = h; g.t0 = 0; g.G = 1; g.n_heads = c.n_heads; g.BH = BH;
+  g.stride_b = sb; g.stride_h = sh; g.stride_n = sn;
+  g.q_shift = h; g.prefix = s.has_state;
+  ctx->last_launches = 0;
+  ctx->last_impl = ctx->tensor_ok ? 1 : 0;
+  int rc = run_parts(ctx, s.qbuf, kcur, vcur, s.obuf, phi, g, s.batch, 1, -1, (s.has_state ? PART_READOUT : 0) | PART_WINDOW, st);
+  if (rc != REHYAT_OK) return rc;
+  launch_copy_rows(out_chunk, lay->stride_batch * es, lay->stride_head * es, lay->stride_token * es,
+                   (uint8_t*)s.obuf + (long long)h * sn * es, sb * es, sh * es, sn * es, Np, row_bytes, BH, c.n_heads, st);
+  // 3. Eq. 17-18: the tokens that leave the window before the next chunk enter the running state
+  const int keep = (long long)s.overlap * HW < (long long)h + Np ? s.overlap * HW : h + Np;
+  const int leave = h + Np - keep;
+  if (leave > 0) {
+    Geo gs = g;
+    gs.Np = leave; gs.ToHW = 0; gs.q_shift = 0; gs.prefix = 0; gs.t0 = 1; gs.G = 1;   // increment of "chunk 1" = [0, leave)
+    const int n_split = pick_state_split(ctx, gs, 1, leave);
+    rc = run_parts(ctx, nullptr, kcur, vcur, nullptr, phi, gs, s.batch, n_split, s.has_state ? 0 : -1, PART_STATE, st);
+    if (rc != REHYAT_OK) return rc;
+    s.has_state = 1;
+  }
+  // 4. the frames that stay in the window move to the front of the other pair of buffers
+  const int nxt = s.cur ^ 1;
+  launch_copy_rows(s.kbuf[nxt], sb * es, sh * es, sn * es, kcur + (long long)leave * sn * es, sb * es, sh * es, sn * es,
+                   keep, row_bytes, BH, c.n_heads, st);
+  launch_copy_rows(s.vbuf[nxt], sb * es, sh * es, sn * es, vcur + (long long)leave * sn * es, sb * es, sh * es, sn * es,
+                   keep, row_bytes, BH, c.n_heads, st);
+  s.cur = nxt;
+  s.halo = keep;
+  ++s.chunks_done;
+  return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
+}
+
+size_t rehyat_stream_state_bytes(const rehyat_ctx* ctx) {
+  if (!ctx || !ctx->stream.active) return 0;
+  return sizeof(StreamHeader) + stream_state_floats(ctx) * sizeof(float) + 2 * stream_halo_bytes(ctx);
+}
+
+int rehyat_stream_export(rehyat_ctx* ctx, void* host_buf, size_t capacity, void* cuda_stream) {
+  if (!ctx || !host_buf || !ctx->stream.active) return REHYAT_ERR_INVALID_ARG;
+  if (capacity < rehyat_stream_state_bytes(ctx)) return REHYAT_ERR_INVALID_ARG;
+  const rehyat_config& c = ctx->cfg;
+  const rehyat_ctx::Stream& s = ctx->stream;
+  DeviceGuard guard(c.device);
+  if (!guard.ok) return REHYAT_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
+  StreamHeader hd = {kStreamMagic, 1, c.dtype, c.n_heads, c.head_dim, c.phi_dim, s.batch, s.H, s.W, s.chunk, s.overlap,
+                     s.halo, s.has_state, 0, s.chunks_done};
+  uint8_t* p = (uint8_t*)host_buf;
+  memcpy(p, &hd, sizeof(hd));
+  p += sizeof(hd);
+  const size_t sbytes = stream_state_floats(ctx) * sizeof(float);
+  if (s.has_state) {
+    if (cudaMemcpy(p, ctx->state, sbytes, cudaMemcpyDeviceToHost) != cudaSuccess) return REHYAT_ERR_CUDA;
+  } else {
+    memset(p, 0, sbytes);
+  }
+  p += sbytes;
+  const size_t es = elem_size(c.dtype), width = (size_t)s.halo * c.head_dim * es, pitch = (size_t)s.cap_tokens * c.head_dim * es;
+  const int BH = s.batch * c.n_heads;
+  if (width > 0) {
+    if (cudaMemcpy2D(p, width, s.kbuf[s.cur], pitch, width, BH, cudaMemcpyDeviceToHost) != cudaSuccess) return REHYAT_ERR_CUDA;
+    p += width * BH;
+    if (cudaMemcpy2D(p, width, s.vbuf[s.cur], pitch, width, BH, cudaMemcpyDeviceToHost) != cudaSuccess) return REHYAT_ERR_CUDA;
+  }
+  return REHYAT_OK;
+}
+
+int rehyat_stream_import(rehyat_ctx* ctx, const void* host_buf, size_t bytes, void* cuda_stream) {
+  if (!ctx || !host_buf || bytes < sizeof(StreamHeader)) return REHYAT_ERR_INVALID_ARG;
+  const rehyat_config& c = ctx->cfg;
+  StreamHeader hd;
+  memcpy(&hd, host_buf, sizeof(hd));
+  if (hd.magic != kStreamMagic || hd.version != 1 || hd.dtype != c.dtype || hd.n_heads != c.n_heads ||
+      hd.head_dim != c.head_dim || hd.phi_dim != c.phi_dim)
+    return REHYAT_ERR_INVALID_ARG;
+  if (hd.halo < 0 || (long long)hd.halo > (long long)hd.overlap * hd.H * hd.W) return REHYAT_ERR_INVALID_ARG;
+  int rc = rehyat_stream_begin(ctx, hd.batch, hd.H, hd.W, hd.chunk, hd.overlap, cuda_stream);
+  if (rc != REHYAT_OK) return rc;
+  rehyat_ctx::Stream& s = ctx->stream;
+  s.halo = hd.halo; s.has_state = hd.has_state ? 1 : 0; s.chunks_done = hd.chunks_done;
+  if (bytes < rehyat_stream_state_bytes(ctx)) { s.active = false; return REHYAT_ERR_INVALID_ARG; }
+  DeviceGuard guard(c.device);
+  if (!guard.ok) return REHYAT_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
+  const uint8_t* p = (const uint8_t*)host_buf + sizeof(hd);
+  const size_t sbytes = stream_state_floats(ctx) * sizeof(float);
+  if (cudaMemcpy(ctx->state, p, sbytes, cudaMemcpyHostToDevice) != cudaSuccess) return REHYAT_ERR_CUDA;
+  p += sbytes;
+  if (s.has_state && ctx->tensor_ok && ctx->tc.phi_ok) {
+    // the bf16 copy of the state that the tensor-core read-out multiplies with: a scan over zero increments
+    const size_t per_slot = stream_state_floats(ctx);
+    scan_states<<<(unsigned)((per_slot + 255) / 256), 256, 0, st>>>(ctx->partial, ctx->state, per_slot, 1, 0, 0,
+                                                                     ctx->tc.state_bf16, c.head_dim);
+  }
+  const size_t es = elem_size(c.dtype), width = (size_t)s.halo * c.head_dim * es, pitch = (size_t)s.cap_tokens * c.head_dim * es;
+  const int BH = s.batch * c.n_heads;
+  if (width > 0) {
+    if (cudaMemcpy2D(s.kbuf[s.cur], pitch, p, width, width, BH, cudaMemcpyHostToDevice) != cudaSuccess) return REHYAT_ERR_CUDA;
+    p += width * BH;
+    if (cudaMemcpy2D(s.vbuf[s.cur], pitch, p, width, width, BH, cudaMemcpyHostToDevice) != cudaSuccess) return REHYAT_ERR_CUDA;
+  }
+  return cudaStreamSynchronize(st) == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
 // ---------------------------------------------------------------------------------------------

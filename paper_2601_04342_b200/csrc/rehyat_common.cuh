@@ -13,10 +13,11 @@ enum Act : int { ACT_RELU = 0, ACT_IDENTITY = 1, ACT_SOFTPLUS = 2, ACT_ELU1 = 3,
 enum CMode : int { C_ROWMAX = 0, C_ZERO = 1 };
 
 // Everything a kernel needs to find chunk t = t0 + (chunk index inside the group).
-// Chunk t (Section 3.3, Eq. 13): queries [t*Np, min((t+1)*Np, N)), softmax window [lo_t, hi_t),
-// lo_t = max(t*Np - ToHW, 0), hi_t = end of the queries; linear prefix [0, lo_t).
+// Chunk t (Section 3.3, Eq. 13): queries [q0_t, q1_t) = [t*Np + q_shift, min((t+1)*Np + q_shift, N)), softmax
+// window [lo_t, q1_t), lo_t = max(q0_t - ToHW, 0); linear prefix [0, lo_t) plus, when `prefix` is set, tokens
+// that are no longer in the buffers and live only in the carried state (the chunk-by-chunk entry points).
 struct Geo {
-  int N;        // tokens per (batch, head)
+  int N;        // tokens per (batch, head) in the buffers
   int Np;       // tokens per chunk, chunk*H*W
   int ToHW;     // overlap*H*W (clamped to N by the host so that it cannot overflow)
   int t0;       // first chunk of the group
@@ -24,17 +25,21 @@ struct Geo {
   int n_heads;
   int BH;       // batch * n_heads
   long long stride_b, stride_h, stride_n;   // element strides of q, k, v, out
+  int q_shift;  // buffer index of the first query of chunk 0 (0 for a whole sequence)
+  int prefix;   // 1: the carried state of chunk t0 covers tokens before buffer index 0
 };
 
-__host__ __device__ inline int geo_q0(const Geo& g, int t) { return t * g.Np; }
+__host__ __device__ inline int geo_q0(const Geo& g, int t) { return t * g.Np + g.q_shift; }
 __host__ __device__ inline int geo_q1(const Geo& g, int t) {
-  long long e = (long long)(t + 1) * g.Np;
+  long long e = (long long)(t + 1) * g.Np + g.q_shift;
   return e < g.N ? (int)e : g.N;
 }
 __host__ __device__ inline int geo_lo(const Geo& g, int t) {
-  long long a = (long long)t * g.Np - g.ToHW;
+  long long a = (long long)t * g.Np + g.q_shift - g.ToHW;
   return a > 0 ? (int)a : 0;
 }
+// Does chunk t have a non-empty linear set TL_t?
+__host__ __device__ inline bool geo_linear(const Geo& g, int t) { return geo_lo(g, t) > 0 || g.prefix != 0; }
 
 __device__ __forceinline__ long long head_offset(const Geo& g, int bh) {
   return (long long)(bh / g.n_heads) * g.stride_b + (long long)(bh % g.n_heads) * g.stride_h;

@@ -99,7 +99,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     tok_a = min(lo_prev + (int)blockIdx.x * per, lo);
     tok_b = min(tok_a + per, lo);
   } else {
-    if (geo_lo(g, t) == 0) return;                                  // empty linear set
+    if (!geo_linear(g, t)) return;                                  // empty linear set
     const int q0 = geo_q0(g, t), q1 = geo_q1(g, t);
     tok_a = min(q0 + (int)blockIdx.x * a.tiles_per_cta * 128, q1);
     tok_b = min(tok_a + a.tiles_per_cta * 128, q1);

@@ -192,7 +192,7 @@ readout_simt(const T* __restrict__ q, PhiPtrs<T> wq, PhiDims pd, Geo g, const fl
   float* Fs = Hs + SIMT_TM * pd.Dh;
 
   const int ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
-  if (geo_lo(g, t) == 0) return;                       // empty linear set: nothing to read out
+  if (!geo_linear(g, t)) return;                       // empty linear set: nothing to read out
   const int q0 = geo_q0(g, t), q1 = geo_q1(g, t);
   const int tok0 = q0 + blockIdx.x * SIMT_TM;
   if (tok0 >= q1) return;
@@ -241,6 +241,7 @@ window_simt(const T* __restrict__ q, const T* __restrict__ k, const T* __restric
 
   const int ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
   const int q0 = geo_q0(g, t), q1 = geo_q1(g, t), lo = geo_lo(g, t), hi = q1;
+  const bool linear = geo_linear(g, t);
   const int row0 = q0 + blockIdx.x * WIN_BM;
   if (row0 >= q1) return;
   const long long hoff = head_offset(g, bh);
@@ -346,7 +347,7 @@ window_simt(const T* __restrict__ q, const T* __restrict__ k, const T* __restric
     if (row >= q1) continue;
     float ws = 1.f, lam = 0.f, nL = 0.f;
     const float* rrow = nullptr;
-    if (lo > 0) {
+    if (linear) {
       rrow = rd + ((size_t)bh * rd_rows + (row - geo_q0(g, g.t0))) * SD;
       lam = 1.f;
       if (c_mode == C_ZERO) {
@@ -360,7 +361,7 @@ window_simt(const T* __restrict__ q, const T* __restrict__ k, const T* __restric
     T* orow = out + hoff + (long long)row * g.stride_n + tx * DC;
 #pragma unroll
     for (int c = 0; c < DC; ++c) {
-      const float aL = lo > 0 ? rrow[tx * DC + c] : 0.f;
+      const float aL = linear ? rrow[tx * DC + c] : 0.f;
       stf(orow + c, (acc[i][c] * ws + lam * aL) * inv);
     }
   }

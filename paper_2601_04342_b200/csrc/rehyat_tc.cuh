@@ -51,6 +51,7 @@ struct WinItem {
   int bh, b_idx, h_idx;
   int q0, q1, lo, hi;      // chunk queries [q0, q1), softmax window [lo, hi)
   int row_base, ntiles, n_kv;
+  bool linear;             // the chunk has a non-empty linear set
 };
 // Items are numbered (batch*head, chunk, tile pair), tile pair fastest, so that the CTAs running at one
 // time share few K/V windows in L2.  Returns false for pairs beyond the end of a short last chunk.
@@ -59,6 +60,7 @@ __device__ __forceinline__ bool win_item(const Geo& g, int item, int pairs, WinI
   w.bh = rest / g.G;
   const int t = g.t0 + ci;
   w.q0 = geo_q0(g, t); w.q1 = geo_q1(g, t); w.lo = geo_lo(g, t); w.hi = w.q1;
+  w.linear = geo_linear(g, t);
   w.row_base = w.q0 + pair * (TC_QT * TC_BM);
   if (w.row_base >= w.q1) return false;
   w.ntiles = (w.row_base + TC_BM < w.q1) ? 2 : 1;                  // query tiles with at least one valid row
@@ -326,7 +328,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       // the whole read-out row is requested before the wait for the last P V, which hides its latency
       float4 rdv[TC_D / 4];
       float nL = 0.f;
-      if (lo > 0) {
+      if (w.linear) {
         const float* rrow = rd + ((size_t)w.bh * rd_rows + (size_t)((valid ? row : w.q0) - geo_q0(g, g.t0))) * (TC_D + 4);
 #pragma unroll
         for (int u = 0; u < TC_D / 4; ++u) rdv[u] = __ldg(reinterpret_cast<const float4*>(rrow) + u);
@@ -337,7 +339,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       }
       const float fin = ex2((m_used - m_true) * c);
       float ws = fin, lam = 0.f;
-      if (lo > 0) {
+      if (w.linear) {
         lam = 1.f;
         if (c_mode == C_ZERO) {
           const float mm = m_true * scale, r = fmaxf(mm, 0.f);
@@ -523,7 +525,7 @@ inline int tc_launch_readout(const TcWorkspace* w, const void* q, const rehyat_p
   // One CTA per SM: split a chunk's query tiles over as many CTAs as costs the fewest tile-times over all waves.
   const int tiles = (g.Np + 127) / 128;
   int busy = 0;
-  for (int t = g.t0; t < g.t0 + g.G; ++t) busy += geo_lo(g, t) > 0;
+  for (int t = g.t0; t < g.t0 + g.G; ++t) busy += geo_linear(g, t);
   const long long units = (long long)(busy > 0 ? busy : 1) * g.BH;
   long long best = -1;
   int best_s = 1;
