@@ -178,6 +178,36 @@ def workspace_by_frames(wl, device):
     return out
 
 
+def stream_timing(wl, dev, phi_q, phi_k, stream, flops):
+    """The same layer fed chunk by chunk through rehyat_stream_step (state held by the context)."""
+    from paper_2601_04342_b200 import binding
+    op = binding.for_workload(wl)
+    HW = wl.HW
+    n_chunks = -(-wl.T // wl.Tc)
+    chunks = []
+    for t in range(n_chunks):
+        sl = slice(t * wl.Tc * HW, min((t + 1) * wl.Tc, wl.T) * HW)
+        chunks.append(tuple(dev[n][:, :, sl].contiguous() for n in ("q", "k", "v")) + (min((t + 1) * wl.Tc, wl.T) - t * wl.Tc,))
+    outs = [torch.empty_like(c[0]) for c in chunks]
+
+    def run():
+        op.stream_begin(wl.B, wl.H, wl.W, wl.Tc, wl.To, stream=stream)
+        for (q, k, v, f), o in zip(chunks, outs):
+            op.stream_step(q, k, v, phi_q, phi_k, f, out=o, stream=stream)
+
+    ms = _time_ms(run, stream, 2, 10)
+    assert op.status() == 0
+    res = {"ms_per_layer": ms, "tflops": flops["total"] / (ms * 1e-3) / 1e12, "steps_per_layer": n_chunks,
+           "state_bytes_after_last_step": lib_state_bytes(op)}
+    op.close()
+    return res
+
+
+def lib_state_bytes(op):
+    from paper_2601_04342_b200 import binding
+    return binding.lib().rehyat_stream_state_bytes(op._h)
+
+
 def time_config(wl, device, stream):
     """Kernel-resident timing of another configuration.  Inputs are drawn on the device (seeded torch
     generator, N(0,1), q and k RMS-normalised) because the host recipe takes tens of seconds at these
@@ -377,6 +407,7 @@ def main():
         extras["full_softmax_same_shape"] = full_softmax_comparison(wl, dev, phi_q, phi_k, stream, ms_step, flops)
     if world == 1:
         extras["workspace_bytes_by_latent_frames"] = workspace_by_frames(wl, local_rank)
+        extras["chunk_by_chunk"] = stream_timing(wl, dev, phi_q, phi_k, stream, flops)
     if world == 1 and args.all_configs:
         extras["other_configs"] = [time_config(synth.CONFIGS[n], local_rank, stream) for n in ("cfg_long", "long_constant_memory")]
 
