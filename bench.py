@@ -203,6 +203,19 @@ def stream_timing(wl, dev, phi_q, phi_k, stream, flops):
     return res
 
 
+def bidirectional_timing(wl, dev, phi_q, phi_k, stream, causal_ms):
+    """The variant of Eq. 10-12 (linear branch over every token outside the window) at the same shape."""
+    from paper_2601_04342_b200 import binding
+    op = binding.for_workload(wl, bidirectional=True)
+    out = torch.empty_like(dev["q"])
+    ms = _time_ms(lambda: op.forward(dev["q"], dev["k"], dev["v"], phi_q, phi_k, wl.T, wl.H, wl.W, wl.Tc, wl.To,
+                                     out=out, stream=stream), stream, 3, 20)
+    assert op.status() == 0
+    res = {"ms_per_step": ms, "causal_ms_per_step": causal_ms, "launches_per_step": op.last_launches}
+    op.close()
+    return res
+
+
 def lib_state_bytes(op):
     from paper_2601_04342_b200 import binding
     return binding.lib().rehyat_stream_state_bytes(op._h)
@@ -410,6 +423,7 @@ def main():
         extras["chunk_by_chunk"] = stream_timing(wl, dev, phi_q, phi_k, stream, flops)
     if world == 1 and args.all_configs:
         extras["other_configs"] = [time_config(synth.CONFIGS[n], local_rank, stream) for n in ("cfg_long", "long_constant_memory")]
+        extras["bidirectional_same_shape"] = bidirectional_timing(wl, dev, phi_q, phi_k, stream, ms_step)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",

@@ -82,6 +82,14 @@ typedef struct rehyat_config {
                                    a group of chunks handles; the workspace grows with it and
                                    with max_chunk_frames*max_tokens_per_frame, never with
                                    `frames`.                                                  */
+  int32_t bidirectional;        /* 0 (default): causal linear branch, TL_t = tokens before the
+                                   window (Eq. 13), the recurrent form.  1: TL_t = every token
+                                   outside the window, earlier AND later (Eq. 10-12), the form
+                                   the paper distils first.  Not a recurrence: rehyat_forward
+                                   then keeps one state per latent frame ((frames+1) x 132 KB per
+                                   (batch, head) at d=128, D'=256), allocated by the first call
+                                   that needs them and kept; rehyat_stream_* and
+                                   rehyat_forward_static refuse it (REHYAT_ERR_UNSUPPORTED).    */
 } rehyat_config;
 
 /* Element strides of q, k, v and out (all four share them); the head_dim axis is contiguous.

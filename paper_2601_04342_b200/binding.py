@@ -29,7 +29,8 @@ PROF_KINDS = ("state", "scan", "readout", "window")
 class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "device", "dtype", "n_heads", "head_dim", "phi_hidden", "phi_dim", "poly_degree", "act_hidden",
-        "act_out", "c_mode", "impl", "max_batch", "max_tokens_per_frame", "max_chunk_frames", "group_tokens")]
+        "act_out", "c_mode", "impl", "max_batch", "max_tokens_per_frame", "max_chunk_frames", "group_tokens",
+        "bidirectional")]
 
 
 class Layout(C.Structure):
@@ -104,10 +105,11 @@ class Rehyat:
 
     def __init__(self, *, n_heads, head_dim, dtype="bf16", phi_hidden=None, phi_dim=None, poly_degree=2,
                  act_hidden="relu", act_out="relu", c_mode="rowmax", impl="auto", max_batch=1,
-                 max_tokens_per_frame=1560, max_chunk_frames=3, group_tokens=0, device=0):
+                 max_tokens_per_frame=1560, max_chunk_frames=3, group_tokens=0, device=0, bidirectional=False):
         self.cfg = Config(device, DTYPE[dtype], n_heads, head_dim, phi_hidden or 2 * head_dim,
                           phi_dim or 2 * head_dim, poly_degree, ACT[act_hidden], ACT[act_out], C_MODE[c_mode],
-                          IMPL[impl], max_batch, max_tokens_per_frame, max_chunk_frames, group_tokens)
+                          IMPL[impl], max_batch, max_tokens_per_frame, max_chunk_frames, group_tokens,
+                          int(bool(bidirectional)))
         self.dtype = dtype
         self._h = C.c_void_p(None)
         _check(lib().rehyat_create(C.byref(self._h), C.byref(self.cfg)), "rehyat_create")

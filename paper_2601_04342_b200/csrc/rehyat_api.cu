@@ -50,6 +50,8 @@ struct rehyat_ctx {
   float* partial = nullptr;    // [partial_units][BHmax][Dp][d+4]
   float* readout = nullptr;    // [BHmax][rd_rows][d+4]
   int* status_dev = nullptr;
+  float* cum = nullptr;        // bidirectional mode: [frames + 1][BHmax][Dp][d+4] states summed over whole frames
+  int cum_frames = 0;
   TcWorkspace tc;              // extra buffers of the tensor-core path
   size_t ws_bytes = 0;
   int Gmax = 0, partial_units = 0, rd_rows = 0, bh_max = 0;
@@ -104,6 +106,7 @@ int check_config(const rehyat_config* c) {
   if (c->max_tokens_per_frame < 1 || c->max_chunk_frames < 1 || c->group_tokens < 0) return REHYAT_ERR_INVALID_ARG;
   if ((long long)c->max_tokens_per_frame * c->max_chunk_frames > (1 << 24)) return REHYAT_ERR_INVALID_ARG;
   if (c->head_dim < 1) return REHYAT_ERR_INVALID_ARG;
+  if (c->bidirectional != 0 && c->bidirectional != 1) return REHYAT_ERR_INVALID_ARG;
   if (c->head_dim != 64 && c->head_dim != 128) return REHYAT_ERR_UNSUPPORTED;
   return REHYAT_OK;
 }
@@ -335,7 +338,7 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
 int rehyat_destroy(rehyat_ctx* ctx) {
   if (!ctx) return REHYAT_OK;
   DeviceGuard guard(ctx->cfg.device);
-  cudaFree(ctx->state); cudaFree(ctx->partial); cudaFree(ctx->readout); cudaFree(ctx->status_dev);
+  cudaFree(ctx->state); cudaFree(ctx->partial); cudaFree(ctx->readout); cudaFree(ctx->status_dev); cudaFree(ctx->cum);
   tc_workspace_destroy(&ctx->tc);
   ctx->prof.clear();
   for (void* p : ctx->stage) cudaFree(p);
@@ -437,6 +440,46 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   ctx->last_launches = 0;
   ctx->last_impl = ctx->tensor_ok ? 1 : 0;
   ctx->stream.active = false;                 // the workspace is about to be overwritten
+  if (c.bidirectional && n_chunks > 1) {
+    // Eq. 10-12: the linear set of a chunk is everything outside its window.  Pass 1 sums the state frame by
+    // frame (running sums cum[0..frames]); pass 2 forms each chunk's state from three of those sums.
+    const size_t per_slot = (size_t)g.BH * c.phi_dim * (c.head_dim + 4), slot_bytes = per_slot * sizeof(float);
+    if (frames + 1 > ctx->cum_frames) {
+      if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
+      cudaFree(ctx->cum);
+      ctx->cum = nullptr; ctx->cum_frames = 0;
+      const size_t full_slot = (size_t)ctx->bh_max * c.phi_dim * (c.head_dim + 4) * sizeof(float);
+      if (cudaMalloc(&ctx->cum, full_slot * (frames + 1)) != cudaSuccess) { cudaGetLastError(); return REHYAT_ERR_ALLOC; }
+      ctx->cum_frames = frames + 1;
+    }
+    if (cudaMemsetAsync(ctx->cum, 0, slot_bytes, st) != cudaSuccess) return REHYAT_ERR_CUDA;
+    Geo gs = g;
+    gs.Np = (int)HW; gs.ToHW = 0;
+    int carry = -1;
+    for (int f0 = 1; f0 <= frames; f0 += ctx->Gmax) {
+      gs.t0 = f0;                                // "chunk" f admits frame f-1: [lo_{f-1}, lo_f) = [(f-1) HW, f HW)
+      gs.G = frames + 1 - f0 < ctx->Gmax ? frames + 1 - f0 : ctx->Gmax;
+      const int ns = pick_state_split(ctx, gs, gs.G, (int)HW);
+      const int rc = run_parts(ctx, nullptr, k, v, nullptr, phi, gs, batch, ns, carry, PART_STATE, st);
+      if (rc != REHYAT_OK) return rc;
+      if (cudaMemcpyAsync((uint8_t*)ctx->cum + (size_t)f0 * slot_bytes, ctx->state, (size_t)gs.G * slot_bytes,
+                          cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return REHYAT_ERR_CUDA;
+      carry = gs.G - 1;
+    }
+    g.prefix = 1;                                // every chunk reads its state, whatever lo_t is
+    for (int t0 = 0; t0 < n_chunks; t0 += G) {
+      g.t0 = t0;
+      g.G = (n_chunks - t0) < G ? (n_chunks - t0) : G;
+      combine_bidirectional<<<(unsigned)((per_slot + 255) / 256), 256, 0, st>>>(
+          ctx->cum, ctx->state, per_slot, g, (int)HW, frames,
+          (ctx->tensor_ok && ctx->tc.phi_ok) ? ctx->tc.state_bf16 : nullptr, c.head_dim);
+      ctx->last_launches += 1;
+      const int rc = run_parts(ctx, q, k, v, out, phi, g, batch, 1, -1, PART_READOUT | PART_WINDOW, st);
+      if (rc != REHYAT_OK) return rc;
+    }
+    return REHYAT_OK;
+  }
   int carry_slot = -1;
   for (int t0 = 0; t0 < n_chunks; t0 += G) {
     g.t0 = t0;
@@ -516,6 +559,7 @@ int rehyat_stream_begin(rehyat_ctx* ctx, int32_t batch, int32_t H, int32_t W, in
                         void* cuda_stream) {
   if (!ctx) return REHYAT_ERR_INVALID_ARG;
   const rehyat_config& c = ctx->cfg;
+  if (c.bidirectional) return REHYAT_ERR_UNSUPPORTED;     // later tokens are not known chunk by chunk
   if (batch < 1 || batch > c.max_batch || H < 1 || W < 1 || chunk < 1 || overlap < 0) return REHYAT_ERR_INVALID_ARG;
   const long long HW = (long long)H * W;
   if (HW > c.max_tokens_per_frame || chunk > c.max_chunk_frames) return REHYAT_ERR_INVALID_ARG;
@@ -719,6 +763,7 @@ int rehyat_forward_static(const rehyat_config* cfg, const void* q, const void* k
   int rc = check_config(cfg);
   if (rc != REHYAT_OK) return rc;
   if (cfg->device < 0 || cfg->device >= kMaxDevices) return REHYAT_ERR_INVALID_ARG;
+  if (cfg->bidirectional) return REHYAT_ERR_UNSUPPORTED;
   if (batch < 1 || frames < 1 || H < 1 || W < 1 || chunk < 1 || overlap < 0) return REHYAT_ERR_INVALID_ARG;
   const long long HW = (long long)H * W, N = HW * frames;
   if (N > (1 << 24)) return REHYAT_ERR_TOO_LARGE;

@@ -179,6 +179,25 @@ __global__ void scan_states(const float* __restrict__ partial, float* __restrict
   }
 }
 
+// Bidirectional linear sets (Eq. 10-12): TL_t = [0, lo_t) + [hi_t, N).  `cum[f]` is the state summed over the
+// frames before frame f (cum[0] = 0, cum[T] = all tokens), so the state of chunk t is
+// cum[lo_t / HW] + (cum[T] - cum[hi_t / HW]).  One thread per state element, written into the slots the
+// read-out uses (plus the bf16 copy of the s part for the tensor-core read-out).
+__global__ void combine_bidirectional(const float* __restrict__ cum, float* __restrict__ state, size_t per_slot, Geo g,
+                                      int HW, int T, __nv_bfloat16* __restrict__ state_bf16 = nullptr, int D = 0) {
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= per_slot) return;
+  const size_t row = e / (D + 4), col = e % (D + 4);
+  const size_t per_slot_b = per_slot / (D + 4) * D;
+  const float total = cum[(size_t)T * per_slot + e];
+  for (int i = 0; i < g.G; ++i) {
+    const int t = g.t0 + i, lo_f = geo_lo(g, t) / HW, hi_f = geo_q1(g, t) / HW;
+    const float sv = cum[(size_t)lo_f * per_slot + e] + (total - cum[(size_t)hi_f * per_slot + e]);
+    state[(size_t)i * per_slot + e] = sv;
+    if (state_bf16 != nullptr && col < (size_t)D) state_bf16[(size_t)i * per_slot_b + row * D + col] = __float2bfloat16_rn(sv);
+  }
+}
+
 // grid (tiles per chunk, G, BH), SIMT_PHI_THREADS threads.  Linear read-out of one tile of
 // SIMT_TM queries of chunk t: rd[bh][row in group][0..d) = phi_q(q_i) s_t, [d] = phi_q(q_i) z_t.
 template <typename T, int D>
