@@ -39,6 +39,8 @@ class Workload:
     rms_norm_qk: bool = False
     P: int = 2
     seed: int = BASE_SEED
+    phi_hidden: int = 0   # 0: the default width 2 * head_dim
+    phi_dim: int = 0      # 0: the default width 2 * head_dim
 
     @property
     def HW(self):
@@ -50,11 +52,11 @@ class Workload:
 
     @property
     def D_h(self):     # phi hidden width: 2 * head_dim (gives the paper's ~2.4 M parameters)
-        return 2 * self.head_dim
+        return self.phi_hidden or 2 * self.head_dim
 
     @property
     def D_out(self):   # phi output width D'
-        return 2 * self.head_dim
+        return self.phi_dim or 2 * self.head_dim
 
     def with_(self, **kw):
         return replace(self, **kw)

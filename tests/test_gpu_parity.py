@@ -225,3 +225,40 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     op.forward_host(pinned["q"], pinned["k"], pinned["v"], out, d["phi_q"], d["phi_k"], wl.T, wl.H, wl.W, wl.Tc, wl.To)
     assert np.array_equal(out.double().numpy(), y_dev)
     op.close()
+
+
+# ------------------------------------------------------------------ other feature maps (activations, degree, widths)
+PHI_VARIANTS = [
+    # id, P, act_hidden, act_out, phi_hidden, phi_dim, kernels expected for bf16 d=128
+    ("degree1_relu", 1, "relu", "relu", 0, 0, "tensor"),
+    ("degree4_relu", 4, "relu", "relu", 0, 0, "tensor"),
+    ("degree2_gelu_softplus", 2, "gelu", "softplus", 0, 0, "tensor"),
+    ("degree2_identity_elu1", 2, "identity", "elu1", 0, 0, "tensor"),
+    ("degree3_width192", 3, "relu", "relu", 128, 192, "tensor"),      # phi on the SIMT kernels, window on the tensor cores
+    ("degree2_narrow", 2, "relu", "softplus", 64, 96, "tensor"),
+]
+
+
+@pytest.mark.parametrize("variant", PHI_VARIANTS, ids=[v[0] for v in PHI_VARIANTS])
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_other_feature_maps(variant, dtype):
+    _, P, ah, ao, Dh, Dp, expect = variant
+    wl = synth.Workload("phi", 1, 2, 128, 5, 10, 20, 2, 1, dtype, dtype == "bf16", P=P, seed=synth.BASE_SEED + 85,
+                        phi_hidden=Dh, phi_dim=Dp)
+    # softplus / elu1 outputs are O(1) per feature, so the linear branch dominates without scaling phi
+    x = synth.make_inputs(wl, phi_scale=1.5 if ao == "relu" else 1.0, v_frame_offsets=True)
+    f = synth.to_f64(x)
+    ref = orc.hybrid_direct(f["q"], f["k"], f["v"], f["phi_q"], f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To, P=P,
+                            act_hidden=ah, act_out=ao)
+    y, used = run_gpu(wl, x, act_hidden=ah, act_out=ao)
+    assert used == (expect if dtype == "bf16" else "simt")
+    check(y, ref, dtype)
+
+
+def test_tensor_window_with_simt_linear_branch_matches_the_all_tensor_path():
+    wl = synth.Workload("tw", 1, 2, 128, 6, 10, 20, 2, 1, "bf16", True, seed=synth.BASE_SEED + 86)
+    x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
+    ref, _ = oracle_full(wl, x)
+    y, used = run_gpu(wl, x, impl="tensor_window")
+    assert used == "tensor"
+    check(y, ref, "bf16")
