@@ -184,8 +184,8 @@ int rehyat_stream_import(rehyat_ctx* ctx, const void* host_buf, size_t bytes, vo
  *   cfg      device, dtype, n_heads, head_dim, phi_*, poly_degree, act_*, c_mode are used; impl,
  *            max_* and group_tokens are ignored
  *   others   as rehyat_forward (device pointers, caller-owned; asynchronous on `cuda_stream`)
- * Limits: at most 16 chunks, and  2*chunks*B*n_heads*D'*(d+4) + B*n_heads*chunks*N'*(d+4)  floats
- * must fit the array; larger problems return REHYAT_ERR_TOO_LARGE and launch nothing.
+ * Limits: at most 16 chunks, and  2*chunks*B*n_heads*D'*(d+4) + B*n_heads*chunks*ceil(N'/128)*128*(d+4)
+ * floats must fit the array; larger problems return REHYAT_ERR_TOO_LARGE and launch nothing.
  * The first call on each device looks up the array's device address and sets kernel attributes;
  * make that first call before any stream capture begins.  All calls share the one array, which
  * keeps the last call's contents (nothing needs it zeroed: a call writes every word before it

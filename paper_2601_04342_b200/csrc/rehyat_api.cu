@@ -48,13 +48,13 @@ struct rehyat_ctx {
   Profiler prof;
   float* state = nullptr;      // [Gmax][BHmax][Dp][d+4]
   float* partial = nullptr;    // [partial_units][BHmax][Dp][d+4]
-  float* readout = nullptr;    // [BHmax][rd_rows][d+4]
+  float* readout = nullptr;    // linear read-out of one chunk group, rd_cap rows per (batch, head), laid out by rd_index
   int* status_dev = nullptr;
   float* cum = nullptr;        // bidirectional mode: [frames + 1][BHmax][Dp][d+4] states summed over whole frames
   int cum_frames = 0;
   TcWorkspace tc;              // extra buffers of the tensor-core path
   size_t ws_bytes = 0;
-  int Gmax = 0, partial_units = 0, rd_rows = 0, bh_max = 0;
+  int Gmax = 0, partial_units = 0, rd_rows = 0, rd_cap = 0, bh_max = 0;
   void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
   size_t stage_bytes = 0;
   int last_launches = 0, last_impl = 0;
@@ -152,7 +152,7 @@ int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* ou
     const size_t smem_rd = (size_t)SIMT_TM * (D + pd.Dh + pd.Dp) * sizeof(float);
     ctx->prof.begin(REHYAT_PROF_READOUT, st);
     readout_simt<T, D><<<dim3(tiles, g.G, g.BH), SIMT_PHI_THREADS, smem_rd, st>>>(q, wq, pd, g, ctx->state,
-                                                                                 ctx->readout, ctx->rd_rows);
+                                                                                 ctx->readout, ctx->rd_cap);
     ctx->prof.end(REHYAT_PROF_READOUT, st);
     ctx->last_launches += 1;
   }
@@ -161,7 +161,7 @@ int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* ou
     const int wtiles = (g.Np + WIN_BM - 1) / WIN_BM;
     ctx->prof.begin(REHYAT_PROF_WINDOW, st);
     window_simt<T, D><<<dim3(wtiles, g.G, g.BH), WIN_THREADS, smem_win, st>>>(
-        q, k, v, out, g, ctx->readout, ctx->rd_rows, 1.0f / sqrtf((float)D), c.c_mode);
+        q, k, v, out, g, ctx->readout, ctx->rd_cap, 1.0f / sqrtf((float)D), c.c_mode);
     ctx->prof.end(REHYAT_PROF_WINDOW, st);
     ctx->last_launches += 1;
   }
@@ -216,14 +216,14 @@ int run_parts(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void
       if (rc == REHYAT_OK && (parts & PART_READOUT)) {
         ctx->prof.begin(REHYAT_PROF_READOUT, st);
         rc = tc_launch_readout(&ctx->tc, q, phi, g, batch, c.poly_degree, c.act_hidden, c.act_out, ctx->state,
-                               ctx->readout, ctx->rd_rows, ctx->status_dev, st);
+                               ctx->readout, ctx->rd_cap, ctx->status_dev, st);
         ctx->prof.end(REHYAT_PROF_READOUT, st);
         ctx->last_launches += 1;
       }
     }
     if (rc == REHYAT_OK && (parts & PART_WINDOW)) {
       ctx->prof.begin(REHYAT_PROF_WINDOW, st);
-      rc = tc_launch_window(&ctx->tc, q, k, v, out, g, batch, ctx->readout, ctx->rd_rows, c.c_mode, ctx->status_dev, st);
+      rc = tc_launch_window(&ctx->tc, q, k, v, out, g, batch, ctx->readout, ctx->rd_cap, c.c_mode, ctx->status_dev, st);
       ctx->prof.end(REHYAT_PROF_WINDOW, st);
       ctx->last_launches += 1;
     }
@@ -303,12 +303,13 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
   const int want = c.group_tokens > 0 ? c.group_tokens : 32768;
   ctx->rd_rows = ((want > np_max ? want : np_max) + 127) / 128 * 128 + 128;
   ctx->Gmax = 16;
+  ctx->rd_cap = ctx->rd_rows + ctx->Gmax * 128;          // every chunk's last 128-row tile may be partly empty
   ctx->partial_units = 32;
   ctx->bh_max = c.max_batch * c.n_heads;
   const size_t SD = c.head_dim + 4;
   const size_t slot = (size_t)ctx->bh_max * c.phi_dim * SD * sizeof(float);
   const size_t b_state = slot * ctx->Gmax, b_partial = slot * ctx->partial_units;
-  const size_t b_rd = (size_t)ctx->bh_max * ctx->rd_rows * SD * sizeof(float);
+  const size_t b_rd = (size_t)ctx->bh_max * ctx->rd_cap * SD * sizeof(float);
   bool ok = cudaMalloc(&ctx->state, b_state) == cudaSuccess && cudaMalloc(&ctx->partial, b_partial) == cudaSuccess &&
             cudaMalloc(&ctx->readout, b_rd) == cudaSuccess && cudaMalloc(&ctx->status_dev, 256) == cudaSuccess;
   ctx->ws_bytes = b_state + b_partial + b_rd + 256;
@@ -774,7 +775,8 @@ int rehyat_forward_static(const rehyat_config* cfg, const void* q, const void* k
   if (n_chunks > 16 || BH > 65535) return REHYAT_ERR_TOO_LARGE;
   const long long slot = BH * cfg->phi_dim * SD;                 // one chunk state, floats
   const long long rd_rows = n_chunks * Np;                       // all chunks form one group
-  const long long need = 2 * n_chunks * slot + BH * rd_rows * SD;
+  const long long rd_cap = n_chunks * ((Np + 127) / 128 * 128);  // whole 128-row tiles per chunk
+  const long long need = 2 * n_chunks * slot + BH * rd_cap * SD;
   if (need > (long long)kStaticScratchFloats) return REHYAT_ERR_TOO_LARGE;
 
   DeviceGuard guard(cfg->device);
@@ -801,6 +803,7 @@ int rehyat_forward_static(const rehyat_config* cfg, const void* q, const void* k
   tmp.Gmax = (int)n_chunks;
   tmp.partial_units = (int)n_chunks;
   tmp.rd_rows = (int)rd_rows;
+  tmp.rd_cap = (int)rd_cap;
   tmp.bh_max = (int)BH;
   tmp.tensor_ok = false;
   return rehyat_forward(&tmp, q, k, v, out, lay, phi, batch, frames, H, W, chunk, overlap, cuda_stream);

@@ -41,6 +41,17 @@ __host__ __device__ inline int geo_lo(const Geo& g, int t) {
 // Does chunk t have a non-empty linear set TL_t?
 __host__ __device__ inline bool geo_linear(const Geo& g, int t) { return geo_lo(g, t) > 0 || g.prefix != 0; }
 
+// Linear read-out workspace (phi_q(q_i) s_t in columns [0, d), phi_q(q_i) z_t in column d).  Per (batch*head)
+// it is cut into tiles of 128 query rows - tile k of chunk ci of the group has index ci*ceil(Np/128) + k - and a
+// tile into d/4 + 1 pieces of four columns, each piece holding the tile's 128 rows contiguously (16 bytes per row).
+// Threads that own consecutive rows therefore read and write consecutive 16-byte pieces.  `rd_rows` is the row
+// capacity per (batch*head), a multiple of 128.  Returns the float index of piece `c4` of the row.
+__host__ __device__ inline size_t rd_index(const Geo& g, int rd_rows, int d, int bh, int ci, int row_in_chunk, int c4) {
+  const int tiles = (g.Np + 127) >> 7;
+  const size_t tile = (size_t)bh * (size_t)(rd_rows >> 7) + (size_t)ci * tiles + (size_t)(row_in_chunk >> 7);
+  return ((tile * (size_t)(d / 4 + 1) + (size_t)c4) * 128 + (size_t)(row_in_chunk & 127)) * 4;
+}
+
 __device__ __forceinline__ long long head_offset(const Geo& g, int bh) {
   return (long long)(bh / g.n_heads) * g.stride_b + (long long)(bh % g.n_heads) * g.stride_h;
 }

@@ -60,7 +60,7 @@ struct PhiTcArgs {
   int n_split;                 // PHI_STATE: splits of a chunk's increment
   float* partial;              // PHI_STATE: [G][n_split][BH][256][132]
   const float* state;          // PHI_READOUT: fp32 states (z column is read)
-  float* rd;                   // PHI_READOUT: [BH][rd_rows][132]
+  float* rd;                   // PHI_READOUT: the read-out workspace (see rd_index)
   int rd_rows;
   int tiles_per_cta;           // PHI_READOUT
   int* status;
@@ -381,8 +381,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
         mbar_wait(smem_u32(&bars->out_ready), j & 1, abort_flag, a.status, PH_ERR_EPI);
         tc_fence_after();
         asm volatile("bar.sync 1, 256;" ::: "memory");               // both halves of s_nl are written
-        const int tok = tok_a + j * 128 + r;
-        float* dst = a.rd + ((size_t)bh * a.rd_rows + (size_t)((tok_valid ? tok : tok_a) - geo_q0(g, g.t0))) * PH_SD;
+        const int ric = tok_a + j * 128 + r - geo_q0(g, t);           // row inside the chunk; its tile is 128-aligned
 #pragma unroll
         for (int cb = 0; cb < 2; ++cb) {
           uint32_t x[32];
@@ -391,12 +390,12 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
           if (tok_valid) {
 #pragma unroll
             for (int e = 0; e < 32; e += 4)
-              *reinterpret_cast<float4*>(dst + ch * 64 + cb * 32 + e) =
+              *reinterpret_cast<float4*>(a.rd + rd_index(g, a.rd_rows, PH_D, bh, ci, ric, (ch * 64 + cb * 32 + e) >> 2)) =
                   make_float4(__uint_as_float(x[e]), __uint_as_float(x[e + 1]), __uint_as_float(x[e + 2]),
                               __uint_as_float(x[e + 3]));
           }
         }
-        if (tok_valid && ch == 1) dst[PH_D] = s_nl[r] + s_nl[128 + r];
+        if (tok_valid && ch == 1) a.rd[rd_index(g, a.rd_rows, PH_D, bh, ci, ric, PH_D / 4)] = s_nl[r] + s_nl[128 + r];
         tc_fence_before();
         asm volatile("bar.sync 1, 256;" ::: "memory");               // s_nl may be overwritten by the next tile
         mbar_arrive(smem_u32(&bars->out_read));

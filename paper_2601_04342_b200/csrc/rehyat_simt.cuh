@@ -237,7 +237,7 @@ readout_simt(const T* __restrict__ q, PhiPtrs<T> wq, PhiDims pd, Geo g, const fl
 #pragma unroll
     for (int r = 0; r < RPG; ++r) {
       const int tok = tok0 + r0 + r;
-      if (tok < q1) rd[((size_t)bh * rd_rows + (tok - geo_q0(g, g.t0))) * SD + c] = acc[r];
+      if (tok < q1) rd[rd_index(g, rd_rows, D, bh, ci, tok - q0, c >> 2) + (c & 3)] = acc[r];
     }
   }
 }
@@ -365,22 +365,20 @@ window_simt(const T* __restrict__ q, const T* __restrict__ k, const T* __restric
     const int row = row0 + ty * 4 + i;
     if (row >= q1) continue;
     float ws = 1.f, lam = 0.f, nL = 0.f;
-    const float* rrow = nullptr;
     if (linear) {
-      rrow = rd + ((size_t)bh * rd_rows + (row - geo_q0(g, g.t0))) * SD;
       lam = 1.f;
       if (c_mode == C_ZERO) {
         const float r = fmaxf(m[i], 0.f);
         ws = expf(m[i] - r);
         lam = expf(-r);
       }
-      nL = rrow[D];
+      nL = rd[rd_index(g, rd_rows, D, bh, ci, row - q0, D / 4)];
     }
     const float inv = 1.f / (l[i] * ws + lam * nL);
     T* orow = out + hoff + (long long)row * g.stride_n + tx * DC;
 #pragma unroll
     for (int c = 0; c < DC; ++c) {
-      const float aL = linear ? rrow[tx * DC + c] : 0.f;
+      const float aL = linear ? rd[rd_index(g, rd_rows, D, bh, ci, row - q0, (tx * DC + c) >> 2) + ((tx * DC + c) & 3)] : 0.f;
       stf(orow + c, (acc[i][c] * ws + lam * aL) * inv);
     }
   }

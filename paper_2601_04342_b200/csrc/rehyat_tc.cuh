@@ -48,7 +48,7 @@ struct WinBars {   // offsets (bytes) inside the barrier block
 
 // One work item of window_tc: two query tiles of one (chunk, batch*head).
 struct WinItem {
-  int bh, b_idx, h_idx;
+  int bh, b_idx, h_idx, ci;
   int q0, q1, lo, hi;      // chunk queries [q0, q1), softmax window [lo, hi)
   int row_base, ntiles, n_kv;
   bool linear;             // the chunk has a non-empty linear set
@@ -58,6 +58,7 @@ struct WinItem {
 __device__ __forceinline__ bool win_item(const Geo& g, int item, int pairs, WinItem& w) {
   const int pair = item % pairs, rest = item / pairs, ci = rest % g.G;
   w.bh = rest / g.G;
+  w.ci = ci;
   const int t = g.t0 + ci;
   w.q0 = geo_q0(g, t); w.q1 = geo_q1(g, t); w.lo = geo_lo(g, t); w.hi = w.q1;
   w.linear = geo_linear(g, t);
@@ -329,10 +330,11 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       float4 rdv[TC_D / 4];
       float nL = 0.f;
       if (w.linear) {
-        const float* rrow = rd + ((size_t)w.bh * rd_rows + (size_t)((valid ? row : w.q0) - geo_q0(g, g.t0))) * (TC_D + 4);
+        const int ric = (valid ? row : w.q0) - w.q0, ci = w.ci;      // row inside the chunk: consecutive threads, consecutive pieces
 #pragma unroll
-        for (int u = 0; u < TC_D / 4; ++u) rdv[u] = __ldg(reinterpret_cast<const float4*>(rrow) + u);
-        nL = __ldg(rrow + TC_D);
+        for (int u = 0; u < TC_D / 4; ++u)
+          rdv[u] = __ldg(reinterpret_cast<const float4*>(rd + rd_index(g, rd_rows, TC_D, w.bh, ci, ric, u)));
+        nL = __ldg(rd + rd_index(g, rd_rows, TC_D, w.bh, ci, ric, TC_D / 4));
       } else {
 #pragma unroll
         for (int u = 0; u < TC_D / 4; ++u) rdv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
