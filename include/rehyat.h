@@ -133,8 +133,10 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
 /* Same operator with q, k, v, out in HOST memory as contiguous [batch, n_heads, N, head_dim]
  * (pinned memory makes the copies asynchronous).  Copies the inputs to device staging buffers
  * owned by the context (grown on demand: the one allocation whose size follows N, because it
- * holds the tensors themselves), runs rehyat_forward, copies `out` back and synchronises the
- * stream.  `phi` stays device-resident. */
+ * holds the tensors themselves), runs the operator, copies `out` back and synchronises the
+ * stream.  The (batch, head) problems are independent, so the call is pipelined over groups of heads
+ * on two extra streams of the context: one group is copied in and another copied out while a third
+ * is computed.  `phi` stays device-resident. */
 int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host,
                         const void* v_host, void* out_host, const rehyat_phi_params* phi,
                         int32_t batch, int32_t frames, int32_t H, int32_t W,

@@ -57,6 +57,9 @@ struct rehyat_ctx {
   int Gmax = 0, partial_units = 0, rd_rows = 0, rd_cap = 0, bh_max = 0;
   void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
   size_t stage_bytes = 0;
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;   // rehyat_forward_host: copies overlap the kernels
+  std::vector<cudaEvent_t> host_events;
+  int head_count = 0;          // > 0: rehyat_forward works on this many heads (pointers already offset to the first)
   int last_launches = 0, last_impl = 0;
   bool tensor_ok = false;
   // chunk-by-chunk processing (rehyat_stream_*): the running state lives in slot 0 of `state`, the last
@@ -343,6 +346,9 @@ int rehyat_destroy(rehyat_ctx* ctx) {
   tc_workspace_destroy(&ctx->tc);
   ctx->prof.clear();
   for (void* p : ctx->stage) cudaFree(p);
+  if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+  if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
+  for (cudaEvent_t e : ctx->host_events) cudaEventDestroy(e);
   for (int i = 0; i < 2; ++i) { cudaFree(ctx->stream.kbuf[i]); cudaFree(ctx->stream.vbuf[i]); }
   cudaFree(ctx->stream.qbuf); cudaFree(ctx->stream.obuf);
   delete ctx;
@@ -426,8 +432,8 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   g.N = (int)N;
   g.Np = (int)(chunk_eff * HW);
   g.ToHW = (int)(overlap_eff * HW);
-  g.n_heads = c.n_heads;
-  g.BH = batch * c.n_heads;
+  g.n_heads = ctx->head_count > 0 ? ctx->head_count : c.n_heads;
+  g.BH = batch * g.n_heads;
   g.stride_b = lay->stride_batch; g.stride_h = lay->stride_head; g.stride_n = lay->stride_token;
   const int n_chunks = (frames + chunk_eff - 1) / chunk_eff;
   g.q_shift = 0;
@@ -514,16 +520,62 @@ int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host,
       if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return REHYAT_ERR_ALLOC; }
     ctx->stage_bytes = bytes;
   }
-  const void* src[3] = {q_host, k_host, v_host};
-  for (int i = 0; i < 3; ++i)
-    if (cudaMemcpyAsync(ctx->stage[i], src[i], bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return REHYAT_ERR_CUDA;
+  // The (batch, head) problems are independent, so the call is pipelined over groups of heads: while group g
+  // is computed on `cuda_stream`, group g+1 is copied in and group g-1 copied out on two streams of the context.
+  if (!ctx->copy_in && cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking) != cudaSuccess) return REHYAT_ERR_CUDA;
+  if (!ctx->copy_out && cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking) != cudaSuccess) return REHYAT_ERR_CUDA;
+  const int per_group = (c.n_heads + 15) / 16, n_groups = (c.n_heads + per_group - 1) / per_group;
+  while ((int)ctx->host_events.size() < 2 * n_groups + 1) {
+    cudaEvent_t e;
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return REHYAT_ERR_CUDA;
+    ctx->host_events.push_back(e);
+  }
+  const size_t es = elem_size(c.dtype), head_bytes = (size_t)N * c.head_dim * es;
   rehyat_layout lay = {(int64_t)c.n_heads * N * c.head_dim, (int64_t)N * c.head_dim, (int64_t)c.head_dim};
-  int rc = rehyat_forward(ctx, ctx->stage[0], ctx->stage[1], ctx->stage[2], ctx->stage[3], &lay, phi, batch, frames,
-                          H, W, chunk, overlap, cuda_stream);
+  // earlier work on the caller's stream may still read the staging buffers
+  cudaEvent_t e_start = ctx->host_events[2 * n_groups];
+  if (cudaEventRecord(e_start, st) != cudaSuccess || cudaStreamWaitEvent(ctx->copy_in, e_start, 0) != cudaSuccess) return REHYAT_ERR_CUDA;
+  const void* src[3] = {q_host, k_host, v_host};
+  int rc = REHYAT_OK;
+  for (int gi = 0; gi < n_groups && rc == REHYAT_OK; ++gi) {
+    const int h0 = gi * per_group, cnt = (c.n_heads - h0) < per_group ? (c.n_heads - h0) : per_group;
+    const size_t off0 = (size_t)h0 * head_bytes, gbytes = (size_t)cnt * head_bytes;
+    for (int b = 0; b < batch; ++b) {
+      const size_t off = (size_t)b * c.n_heads * head_bytes + off0;
+      for (int i = 0; i < 3; ++i)
+        if (cudaMemcpyAsync((uint8_t*)ctx->stage[i] + off, (const uint8_t*)src[i] + off, gbytes, cudaMemcpyHostToDevice,
+                            ctx->copy_in) != cudaSuccess)
+          return REHYAT_ERR_CUDA;
+    }
+    cudaEvent_t e_in = ctx->host_events[2 * gi], e_done = ctx->host_events[2 * gi + 1];
+    if (cudaEventRecord(e_in, ctx->copy_in) != cudaSuccess || cudaStreamWaitEvent(st, e_in, 0) != cudaSuccess) return REHYAT_ERR_CUDA;
+    rehyat_phi_params ph = *phi;                           // parameters of the group's first head
+    const size_t w1 = (size_t)h0 * c.phi_hidden * c.head_dim * es, b1 = (size_t)h0 * c.phi_hidden * es;
+    const size_t w2 = (size_t)h0 * c.phi_dim * c.phi_hidden * es, b2 = (size_t)h0 * c.phi_dim * es;
+    ph.q_W1 = (const uint8_t*)phi->q_W1 + w1; ph.q_b1 = (const uint8_t*)phi->q_b1 + b1;
+    ph.q_W2 = (const uint8_t*)phi->q_W2 + w2; ph.q_b2 = (const uint8_t*)phi->q_b2 + b2;
+    ph.k_W1 = (const uint8_t*)phi->k_W1 + w1; ph.k_b1 = (const uint8_t*)phi->k_b1 + b1;
+    ph.k_W2 = (const uint8_t*)phi->k_W2 + w2; ph.k_b2 = (const uint8_t*)phi->k_b2 + b2;
+    ctx->head_count = cnt;
+    const int launches_before = gi == 0 ? 0 : ctx->last_launches;
+    rc = rehyat_forward(ctx, (uint8_t*)ctx->stage[0] + off0, (uint8_t*)ctx->stage[1] + off0, (uint8_t*)ctx->stage[2] + off0,
+                        (uint8_t*)ctx->stage[3] + off0, &lay, &ph, batch, frames, H, W, chunk, overlap, cuda_stream);
+    ctx->head_count = 0;
+    ctx->last_launches += launches_before;
+    if (rc != REHYAT_OK) break;
+    if (cudaEventRecord(e_done, st) != cudaSuccess || cudaStreamWaitEvent(ctx->copy_out, e_done, 0) != cudaSuccess) return REHYAT_ERR_CUDA;
+    for (int b = 0; b < batch; ++b) {
+      const size_t off = (size_t)b * c.n_heads * head_bytes + off0;
+      if (cudaMemcpyAsync((uint8_t*)out_host + off, (uint8_t*)ctx->stage[3] + off, gbytes, cudaMemcpyDeviceToHost,
+                          ctx->copy_out) != cudaSuccess)
+        return REHYAT_ERR_CUDA;
+    }
+  }
+  // the call returns with `out_host` filled, also after an error in the middle
+  const bool ok = cudaStreamSynchronize(ctx->copy_in) == cudaSuccess && cudaStreamSynchronize(st) == cudaSuccess &&
+                  cudaStreamSynchronize(ctx->copy_out) == cudaSuccess;
   if (rc != REHYAT_OK) return rc;
-  if (cudaMemcpyAsync(out_host, ctx->stage[3], bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return REHYAT_ERR_CUDA;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
-  return REHYAT_OK;
+  return ok ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
 // ---------------------------------------------------------------------------------------------
