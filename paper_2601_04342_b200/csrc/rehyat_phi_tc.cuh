@@ -1,19 +1,18 @@
-// Tensor-core kernels of the linear branch for bf16, head_dim 128, phi widths D_h = D' = 256.
+// Tensor-core kernel of the chunk-state increments for bf16, head_dim 128, phi widths D_h = D' = 256.
 //
-// phi_tc<MODE> evaluates the feature map of Section 3.2 ("Characterization of phi") on tiles of
-// 128 tokens with tcgen05.mma and feeds it straight into the contraction that consumes it:
-//   PHI_STATE    phi_k(K tile)^T [V | 1] accumulated in TMEM over the CTA's share of the keys a
-//                chunk newly admits (Eq. 17-18); flushed once as an fp32 partial state.
-//   PHI_READOUT  phi_q(Q tile) s_t on the tensor core and phi_q(Q tile) z_t on the ALUs
-//                (Eq. 7, 9, 16); written as the fp32 linear read-out of the tile.
+// phi_tc evaluates the feature map phi_k of Section 3.2 ("Characterization of phi") on tiles of 128 keys with
+// tcgen05.mma and feeds it straight into the contraction that consumes it: phi_k(K tile)^T [V | 1] accumulated
+// in TMEM over the CTA's share of the keys a chunk newly admits (Eq. 17-18), flushed once as an fp32 partial
+// state.  (The read-out kernel, readout_tc, has a file of its own; it shares the constants and PhiTcArgs.)
 //
 // Per tile the chain is  H = act(X W1^T + b1) -> U = act(H W2^T + b2) -> phi = U^(1..P)  with the
-// two GEMMs done as 128x128 halves through one 128-column TMEM scratch accumulator:
+// two GEMMs done as 128x128 halves through one 128-column TMEM scratch accumulator (the state accumulators
+// take 288 of the 512 columns):
 //   warps 0-7  epilogues, two threads per token (= TMEM lane): bias, activation, power, bf16, swizzled smem tile
-//   warp 8     TMA producer: X (and V), weight / state tiles [128 x 64] through a 3-stage ring
+//   warp 8     TMA producer: X and V, weight tiles [128 x 64] through a 3-stage ring
 //   warp 9     UMMA issuer
 // The phi tile is written once in the 128-byte-swizzled [token][feature] image; the state GEMM reads
-// it as an MN-major A operand (features are M), the read-out GEMM as a K-major A operand.
+// it as an MN-major A operand (features are M).
 #pragma once
 
 #include <cuda.h>
@@ -23,12 +22,9 @@
 
 namespace rehyat {
 
-enum PhiMode : int { PHI_STATE = 0, PHI_READOUT = 1 };
-
 constexpr int PH_D = 128, PH_DH = 256, PH_DP = 256, PH_SD = PH_D + 4;
 constexpr int PH_THREADS = 320;            // 8 epilogue warps, TMA producer, UMMA issuer
-constexpr int PH_RING = 3;                // weight tiles in flight (PHI_STATE)
-constexpr int PH_RING_MAX = 5;            // PHI_READOUT has no V tile and uses its 32 KB for two more stages
+constexpr int PH_RING = 3;                // weight tiles in flight
 constexpr int PH_WT_BYTES = 128 * 64 * 2;          // one weight / state tile: 16 KB
 constexpr int PH_TILE_BYTES = 128 * 128 * 2;       // X, V, phi half: 32 KB (two swizzled sub-tiles)
 constexpr int PH_SUB = PH_TILE_BYTES / 2;
@@ -39,16 +35,16 @@ constexpr int PH_OFF_HB = PH_OFF_V + PH_TILE_BYTES;            // 64 KB; its fir
 constexpr int PH_OFF_PHI0 = PH_OFF_HB + 2 * PH_TILE_BYTES;
 constexpr int PH_OFF_RING = PH_OFF_PHI0 + PH_TILE_BYTES;
 constexpr int PH_OFF_ONES = PH_OFF_RING + PH_RING * PH_WT_BYTES; // [16 x 128] K-major, row 0 = 1
-constexpr int PH_OFF_BIAS = PH_OFF_ONES + 4096;                 // b1[256], b2[256], z[256] fp32
-constexpr int PH_OFF_BARS = PH_OFF_BIAS + 4 * 256 * 4;     // ... and the two partial phi.z sums per token
+constexpr int PH_OFF_BIAS = PH_OFF_ONES + 4096;                 // b1[256], b2[256] fp32
+constexpr int PH_OFF_BARS = PH_OFF_BIAS + 2 * 256 * 4;
 constexpr int PH_SMEM = PH_OFF_BARS + 512 + 1024;
 
 enum PhErr : int { PH_ERR_LOAD = 16, PH_ERR_MMA = 32, PH_ERR_EPI = 64 };
 
 struct PhBars {
   uint64_t x_full, x_empty, v_full, v_empty;
-  uint64_t ring_full[PH_RING_MAX], ring_empty[PH_RING_MAX];
-  uint64_t acc_ready, epi_done, out_ready, out_read;
+  uint64_t ring_full[PH_RING], ring_empty[PH_RING];
+  uint64_t acc_ready, epi_done, out_ready;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -57,24 +53,21 @@ struct PhiTcArgs {
   const __nv_bfloat16* b1;     // [heads][256]
   const __nv_bfloat16* b2;     // [heads][256]
   int P, act_hidden, act_out;
-  int n_split;                 // PHI_STATE: splits of a chunk's increment
-  float* partial;              // PHI_STATE: [G][n_split][BH][256][132]
-  const float* state;          // PHI_READOUT: fp32 states (z column is read)
-  float* rd;                   // PHI_READOUT: the read-out workspace (see rd_index)
+  int n_split;                 // state kernel: splits of a chunk's increment
+  float* partial;              // state kernel: [G][n_split][BH][256][132]
+  const float* state;          // read-out kernel: fp32 states (z column is read)
+  float* rd;                   // read-out kernel: the read-out workspace (see rd_index)
   int rd_rows;
-  int tiles_per_cta;           // PHI_READOUT
+  int tiles_per_cta;           // read-out kernel
   int* status;
 };
 
-// tm_x: K (state) or Q (read-out), 4-D like the window kernel's maps.  tm_v: V (state only).
-// tm_w1: (128, 256, heads), tm_w2: (256, 256, heads), boxes [64 x 128].  tm_s: bf16 states
-// (128, 256, G*BH), box [64 x 64] (read-out only).
-// PC: polynomial degree known at compile time (0: read it from the arguments).
-template <int MODE, bool RELU, int PC>
+// tm_x: K, tm_v: V, 4-D like the window kernel's maps.  tm_w1: (128, 256, heads), tm_w2: (256, 256, heads),
+// boxes [64 x 128].  PC: polynomial degree known at compile time (0: read it from the arguments).
+template <bool RELU, int PC>
 __global__ void __launch_bounds__(PH_THREADS, 1)
 phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_v,
-       const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2,
-       const __grid_constant__ CUtensorMap tm_s, Geo g, PhiTcArgs a) {
+       const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2, Geo g, PhiTcArgs a) {
   using namespace ptx;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sb = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -82,8 +75,6 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   PhBars* bars = reinterpret_cast<PhBars*>(smem + PH_OFF_BARS);
   float* s_b1 = reinterpret_cast<float*>(smem + PH_OFF_BIAS);
   float* s_b2 = s_b1 + 256;
-  float* s_z = s_b2 + 256;
-  float* s_nl = s_z + 256;
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -91,23 +82,14 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   const int b_idx = bh / g.n_heads, h_idx = bh % g.n_heads;
 
   // token range [tok_a, tok_b) of this CTA
-  int tok_a, tok_b;
-  if (MODE == PHI_STATE) {
-    const int lo_prev = t > 0 ? geo_lo(g, t - 1) : 0, lo = geo_lo(g, t);
-    int per = (lo - lo_prev + a.n_split - 1) / a.n_split;
-    per = (per + 127) / 128 * 128;
-    tok_a = min(lo_prev + (int)blockIdx.x * per, lo);
-    tok_b = min(tok_a + per, lo);
-  } else {
-    if (!geo_linear(g, t)) return;                                  // empty linear set
-    const int q0 = geo_q0(g, t), q1 = geo_q1(g, t);
-    tok_a = min(q0 + (int)blockIdx.x * a.tiles_per_cta * 128, q1);
-    tok_b = min(tok_a + a.tiles_per_cta * 128, q1);
-    if (tok_a >= tok_b) return;
-  }
+  const int lo_prev = t > 0 ? geo_lo(g, t - 1) : 0, lo = geo_lo(g, t);
+  int per = (lo - lo_prev + a.n_split - 1) / a.n_split;
+  per = (per + 127) / 128 * 128;
+  const int tok_a = min(lo_prev + (int)blockIdx.x * per, lo);
+  const int tok_b = min(tok_a + per, lo);
   const int n_tiles = (tok_b - tok_a + 127) / 128;
 
-  if (MODE == PHI_STATE && n_tiles == 0) {                          // nothing admitted: the partial is zero
+  if (n_tiles == 0) {                          // nothing admitted: the partial is zero
     float* dst = a.partial + (((size_t)ci * a.n_split + blockIdx.x) * g.BH + bh) * PH_DP * PH_SD;
     for (int i = threadIdx.x; i < PH_DP * PH_SD / 4; i += PH_THREADS)
       reinterpret_cast<float4*>(dst)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -117,21 +99,20 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   if (threadIdx.x == 0) {
     mbar_init(smem_u32(&bars->x_full), 1); mbar_init(smem_u32(&bars->x_empty), 1);
     mbar_init(smem_u32(&bars->v_full), 1); mbar_init(smem_u32(&bars->v_empty), 1);
-    for (int s = 0; s < PH_RING_MAX; ++s) {
+    for (int s = 0; s < PH_RING; ++s) {
       mbar_init(smem_u32(&bars->ring_full[s]), 1); mbar_init(smem_u32(&bars->ring_empty[s]), 1);
     }
     mbar_init(smem_u32(&bars->acc_ready), 1); mbar_init(smem_u32(&bars->epi_done), 256);
-    mbar_init(smem_u32(&bars->out_ready), 1); mbar_init(smem_u32(&bars->out_read), 256);
+    mbar_init(smem_u32(&bars->out_ready), 1);
     bars->abort_flag = 0;
     fence_mbar_init();
   }
-  // biases (and z_t) as fp32; the ones tile: row 0 of both 64-column sub-tiles is 1, the rest 0
+  // biases as fp32; the ones tile: row 0 of both 64-column sub-tiles is 1, the rest 0
   for (int i = threadIdx.x; i < 256; i += PH_THREADS) {
     s_b1[i] = __bfloat162float(a.b1[(size_t)h_idx * 256 + i]);
     s_b2[i] = __bfloat162float(a.b2[(size_t)h_idx * 256 + i]);
-    if (MODE == PHI_READOUT) s_z[i] = a.state[(((size_t)ci * g.BH + bh) * PH_DP + i) * PH_SD + PH_D];
   }
-  if (MODE == PHI_STATE) {
+  {
     uint32_t* ones = reinterpret_cast<uint32_t*>(smem + PH_OFF_ONES);
     for (int i = threadIdx.x; i < 1024; i += PH_THREADS) {
       const int byte = i * 4, sub = byte / 2048, within = byte % 2048;
@@ -147,14 +128,13 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
-  // TMEM columns: scratch [0,128); STATE: S half0 [128,256) S half1 [256,384) z0 [384,400) z1 [400,416);
-  // READOUT: R [128,256)
+  // TMEM columns: scratch [0,128), S half 0 [128,256), S half 1 [256,384), z half 0 [384,400), z half 1 [400,416)
   constexpr uint32_t T_SCR = 0, T_ACC = 128, T_Z = 384;
-  constexpr int RING = MODE == PHI_READOUT ? PH_RING_MAX : PH_RING;
+  constexpr int RING = PH_RING;
 
   const uint32_t sX = sb + PH_OFF_X, sV = sb + PH_OFF_V, sHb = sb + PH_OFF_HB, sPhi0 = sb + PH_OFF_PHI0,
                  sRing = sb + PH_OFF_RING, sOnes = sb + PH_OFF_ONES;
-  auto ring_addr = [&](int s) -> uint32_t { return s < PH_RING ? sRing + s * PH_WT_BYTES : sV + (s - PH_RING) * PH_WT_BYTES; };
+  auto ring_addr = [&](int s) -> uint32_t { return sRing + s * PH_WT_BYTES; };
 
   if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
@@ -162,19 +142,14 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_w1); prefetch_tensormap(&tm_w2);
       uint32_t ring_i = 0;
       bool alive = true;
-      auto ring_load = [&](const CUtensorMap* tm, int x, int y, int z, bool state_tile) {
+      auto ring_load = [&](const CUtensorMap* tm, int x, int y, int z) {
         const int s = ring_i % RING;
         const uint32_t ph = (ring_i / RING) & 1;
         alive = alive && mbar_wait(smem_u32(&bars->ring_empty[s]), ph ^ 1, abort_flag, a.status, PH_ERR_LOAD);
         if (!alive) return;
         const uint32_t full = smem_u32(&bars->ring_full[s]);
         mbar_expect_tx(full, PH_WT_BYTES);
-        if (!state_tile) {
-          tma_load_3d(ring_addr(s), tm, full, x, y, z);
-        } else {                                                     // [64 features x 128 d] as two 64-column boxes
-          tma_load_3d(ring_addr(s), tm, full, 0, y, z);
-          tma_load_3d(ring_addr(s) + 8192, tm, full, 64, y, z);
-        }
+        tma_load_3d(ring_addr(s), tm, full, x, y, z);
         ++ring_i;
       };
       for (int j = 0; j < n_tiles && alive; ++j) {
@@ -186,8 +161,8 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
         tma_load_4d(sX, &tm_x, xf, 0, tok0, h_idx, b_idx);
         tma_load_4d(sX + PH_SUB, &tm_x, xf, 64, tok0, h_idx, b_idx);
         for (int nh = 0; nh < 2; ++nh)
-          for (int ks = 0; ks < 2; ++ks) ring_load(&tm_w1, ks * 64, nh * 128, h_idx, false);
-        if (MODE == PHI_STATE) {
+          for (int ks = 0; ks < 2; ++ks) ring_load(&tm_w1, ks * 64, nh * 128, h_idx);
+        {
           alive = alive && mbar_wait(smem_u32(&bars->v_empty), (j & 1) ^ 1, abort_flag, a.status, PH_ERR_LOAD);
           if (!alive) break;
           const uint32_t vf = smem_u32(&bars->v_full);
@@ -195,10 +170,8 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
           tma_load_4d(sV, &tm_v, vf, 0, tok0, h_idx, b_idx);
           tma_load_4d(sV + PH_SUB, &tm_v, vf, 64, tok0, h_idx, b_idx);
         }
-        for (int ks = 0; ks < 4; ++ks) ring_load(&tm_w2, ks * 64, 0, h_idx, false);
-        for (int ks = 0; ks < 4; ++ks) ring_load(&tm_w2, ks * 64, 128, h_idx, false);
-        if (MODE == PHI_READOUT)
-          for (int f = 0; f < 4; ++f) ring_load(&tm_s, 0, f * 64, ci * g.BH + bh, true);
+        for (int ks = 0; ks < 4; ++ks) ring_load(&tm_w2, ks * 64, 0, h_idx);
+        for (int ks = 0; ks < 4; ++ks) ring_load(&tm_w2, ks * 64, 128, h_idx);
       }
     }
   } else if (warp == 9) {
@@ -207,7 +180,6 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       constexpr uint32_t id_kk = idesc_bf16(128, 128, 0, 0);       // A K-major, B K-major   (the two MLP GEMMs)
       constexpr uint32_t id_st = idesc_bf16(128, 128, 1, 1);       // A = phi^T (MN-major), B = V (MN-major)
       constexpr uint32_t id_z = idesc_bf16(128, 16, 1, 0);         // A = phi^T (MN-major), B = ones (K-major)
-      constexpr uint32_t id_rd = idesc_bf16(128, 128, 0, 1);       // A = phi (K-major),    B = state (MN-major)
       uint32_t ring_i = 0, n_epi = 0;
       auto ring_wait = [&]() -> uint32_t {
         const int s = ring_i % RING;
@@ -238,24 +210,13 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       };
       // contraction that consumes phi half `c` (its tile is at phi_base)
       auto consume_half = [&](int c, uint32_t phi_base, bool first_tile) {
-        if (MODE == PHI_STATE) {
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {                          // 16 tokens per step
-            const uint64_t ad = smem_desc_sw128(phi_base + kk * 2048, PH_SUB, 1024);
-            umma_ss(tmem + T_ACC + c * 128, ad, smem_desc_sw128(sV + kk * 2048, PH_SUB, 1024), id_st,
-                    (!first_tile || kk > 0) ? 1u : 0u);
-            umma_ss(tmem + T_Z + c * 16, ad, smem_desc_sw128(sOnes + (kk >> 2) * 2048 + (kk & 3) * 32, 16, 1024), id_z,
-                    (!first_tile || kk > 0) ? 1u : 0u);
-          }
-        } else {
-          for (int f = 0; f < 2; ++f) {                             // 64 features per state tile
-            const uint32_t bt = ring_wait();
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              umma_ss(tmem + T_ACC, smem_desc_sw128(phi_base + f * PH_SUB + kk * 32, 16, 1024),
-                      smem_desc_sw128(bt + kk * 2048, 8192, 1024), id_rd, (c | f | kk) != 0);
-            ring_release();
-          }
+        for (int kk = 0; kk < 8; ++kk) {                            // 16 tokens per step
+          const uint64_t ad = smem_desc_sw128(phi_base + kk * 2048, PH_SUB, 1024);
+          umma_ss(tmem + T_ACC + c * 128, ad, smem_desc_sw128(sV + kk * 2048, PH_SUB, 1024), id_st,
+                  (!first_tile || kk > 0) ? 1u : 0u);
+          umma_ss(tmem + T_Z + c * 16, ad, smem_desc_sw128(sOnes + (kk >> 2) * 2048 + (kk & 3) * 32, 16, 1024), id_z,
+                  (!first_tile || kk > 0) ? 1u : 0u);
         }
       };
       for (int j = 0; j < n_tiles; ++j) {
@@ -263,11 +224,10 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
         tc_fence_after();
         if (j > 0) wait_epi();                                      // scratch free: phi half 1 of tile j-1 written
         if (j > 0) {                                                // ... and consumed
-          if (MODE == PHI_STATE) mbar_wait(smem_u32(&bars->v_full), (j - 1) & 1, abort_flag, a.status, PH_ERR_MMA);
+          mbar_wait(smem_u32(&bars->v_full), (j - 1) & 1, abort_flag, a.status, PH_ERR_MMA);
           tc_fence_after();
           consume_half(1, sHb, j == 1);
-          if (MODE == PHI_STATE) umma_commit(smem_u32(&bars->v_empty));
-          if (MODE == PHI_READOUT) umma_commit(smem_u32(&bars->out_ready));
+          umma_commit(smem_u32(&bars->v_empty));
         }
         mlp_half(sX, 2);                                            // H[:, 0:128]
         wait_epi();
@@ -277,13 +237,8 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
         mlp_half(sHb, 4);                                           // U[:, 0:128]
         wait_epi();
         mlp_half(sHb, 4);                                           // U[:, 128:256]
-        if (MODE == PHI_STATE) {
-          mbar_wait(smem_u32(&bars->v_full), j & 1, abort_flag, a.status, PH_ERR_MMA);
-          tc_fence_after();
-        } else if (j > 0) {
-          mbar_wait(smem_u32(&bars->out_read), (j - 1) & 1, abort_flag, a.status, PH_ERR_MMA);
-          tc_fence_after();
-        }
+        mbar_wait(smem_u32(&bars->v_full), j & 1, abort_flag, a.status, PH_ERR_MMA);
+        tc_fence_after();
         consume_half(0, sPhi0, j == 0);
       }
       wait_epi();
@@ -301,7 +256,6 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     const int part_w = PH_DP / (PC ? PC : a.P);                     // a multiple of 32 (P in {1,2,4})
     for (int j = 0; j < n_tiles; ++j) {
       const bool tok_valid = tok_a + j * 128 + r < tok_b;
-      float nl = 0.f;
 #pragma unroll
       for (int step = 0; step < 4; ++step) {                        // H half 0, H half 1, U half 0, U half 1
         mbar_wait(smem_u32(&bars->acc_ready), n_acc & 1, abort_flag, a.status, PH_ERR_EPI);
@@ -357,51 +311,15 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
 #pragma unroll
           for (int e = 0; e < 32; e += 8) {
             const uint4 w4 = make_uint4(w[e >> 1], w[(e >> 1) + 1], w[(e >> 1) + 2], w[(e >> 1) + 3]);
-            if (MODE == PHI_READOUT && is_u) {
-              // phi_q(q_r) . z_t with the same bf16-rounded features the tensor core sees
-              const float* zz = s_z + half * 128 + col0 + e;
-              const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
-#pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                nl = fmaf(__uint_as_float(ww[u] << 16), zz[2 * u], nl);
-                nl = fmaf(__uint_as_float(ww[u] & 0xffff0000u), zz[2 * u + 1], nl);
-              }
-            }
             st_tile_chunk_sw128(dst, PH_SUB, r, dst_col0 + col0 + e, w4);
           }
         }
-        if (MODE == PHI_READOUT && step == 3) s_nl[ch * 128 + r] = nl;
         fence_proxy_async_smem();
         tc_fence_before();
         mbar_arrive(smem_u32(&bars->epi_done));
       }
-      if (MODE == PHI_READOUT) {
-        // read-out of tile j is complete after the consumer of phi half 1, issued at the start of
-        // the next tile (or after the loop)
-        mbar_wait(smem_u32(&bars->out_ready), j & 1, abort_flag, a.status, PH_ERR_EPI);
-        tc_fence_after();
-        asm volatile("bar.sync 1, 256;" ::: "memory");               // both halves of s_nl are written
-        const int ric = tok_a + j * 128 + r - geo_q0(g, t);           // row inside the chunk; its tile is 128-aligned
-#pragma unroll
-        for (int cb = 0; cb < 2; ++cb) {
-          uint32_t x[32];
-          tmem_ld32(tmem + lane_off + T_ACC + ch * 64 + cb * 32, x);
-          tmem_wait_ld();
-          if (tok_valid) {
-#pragma unroll
-            for (int e = 0; e < 32; e += 4)
-              *reinterpret_cast<float4*>(a.rd + rd_index(g, a.rd_rows, PH_D, bh, ci, ric, (ch * 64 + cb * 32 + e) >> 2)) =
-                  make_float4(__uint_as_float(x[e]), __uint_as_float(x[e + 1]), __uint_as_float(x[e + 2]),
-                              __uint_as_float(x[e + 3]));
-          }
-        }
-        if (tok_valid && ch == 1) a.rd[rd_index(g, a.rd_rows, PH_D, bh, ci, ric, PH_D / 4)] = s_nl[r] + s_nl[128 + r];
-        tc_fence_before();
-        asm volatile("bar.sync 1, 256;" ::: "memory");               // s_nl may be overwritten by the next tile
-        mbar_arrive(smem_u32(&bars->out_read));
-      }
     }
-    if (MODE == PHI_STATE) {
+    {
       // flush: lane r holds feature c*128 + r of half c; this thread writes its 64 columns
       mbar_wait(smem_u32(&bars->out_ready), 0, abort_flag, a.status, PH_ERR_EPI);
       tc_fence_after();

@@ -1,0 +1,368 @@
+// Tensor-core kernel of the linear read-out for bf16, head_dim 128, phi widths D_h = D' = 256:
+//   phi_q on tiles of 128 queries (Section 3.2 "Characterization of phi"), then phi_q(Q tile) s_t on the
+//   tensor core and phi_q(Q tile) z_t on the ALUs (Eq. 7, 9, 16), written as the fp32 read-out of the tile.
+//
+// Per tile  H = act(X W1^T + b1) -> U = act(H W2^T + b2) -> phi = U^(1..P) -> R = phi [s_t]  as 128x128 halves.
+// Unlike the state kernel this one has TMEM to spare, which it uses twice:
+//   * two scratch accumulators, so that the epilogue of one half runs while the tensor core works on the next;
+//   * H (bf16) goes back to TMEM and is the A operand of the second GEMM from there, which frees 64 KB of shared
+//     memory for a seven-stage ring of weight / state tiles - a TMA round trip from L2 costs about 1800 cycles
+//     under load, so the bytes in flight are what bounds the weight stream.
+// Roles (320 threads): warps 0-7 epilogues (two threads per token), warp 8 TMA producer, warp 9 UMMA issuer.
+// TMEM columns: scratch A [0,128), scratch B [128,256), H [256,384) (256 hidden units as bf16 pairs), R [384,512).
+#pragma once
+
+#include <cuda.h>
+
+#include "rehyat_common.cuh"
+#include "rehyat_ptx.cuh"
+#include "rehyat_phi_tc.cuh"
+
+namespace rehyat {
+
+constexpr int RD_RING = 7;
+constexpr int RD_WT_BYTES = 128 * 64 * 2;                        // one weight / state tile: 16 KB
+constexpr int RD_OFF_X = 0;
+constexpr int RD_OFF_PHI0 = RD_OFF_X + PH_TILE_BYTES;
+constexpr int RD_OFF_PHI1 = RD_OFF_PHI0 + PH_TILE_BYTES;
+constexpr int RD_OFF_RING = RD_OFF_PHI1 + PH_TILE_BYTES;
+constexpr int RD_OFF_BIAS = RD_OFF_RING + RD_RING * RD_WT_BYTES;  // b1[256], b2[256], z[256], two partial phi.z sums per token
+constexpr int RD_OFF_BARS = RD_OFF_BIAS + 4 * 256 * 4;
+constexpr int RD_SMEM = RD_OFF_BARS + 512 + 1024;
+
+struct RdBars {
+  uint64_t x_full, x_empty;
+  uint64_t ring_full[RD_RING], ring_empty[RD_RING];
+  uint64_t acc_ready[2], epi_done[2], out_ready, out_read;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// tm_x: Q, 4-D like the window kernel's maps.  tm_w1: (128, 256, heads), tm_w2: (256, 256, heads), boxes
+// [64 x 128].  tm_s: bf16 states (128, 256, G*BH), box [64 x 64].  PC: polynomial degree known at compile time
+// (0: read it from the arguments).
+template <bool RELU, int PC>
+__global__ void __launch_bounds__(PH_THREADS, 1)
+readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w1,
+           const __grid_constant__ CUtensorMap tm_w2, const __grid_constant__ CUtensorMap tm_s, Geo g, PhiTcArgs a) {
+  using namespace ptx;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t sb = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (sb - smem_u32(smem_raw));
+  RdBars* bars = reinterpret_cast<RdBars*>(smem + RD_OFF_BARS);
+  float* s_b1 = reinterpret_cast<float*>(smem + RD_OFF_BIAS);
+  float* s_b2 = s_b1 + 256;
+  float* s_z = s_b2 + 256;
+  float* s_nl = s_z + 256;
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
+  const int b_idx = bh / g.n_heads, h_idx = bh % g.n_heads;
+  if (!geo_linear(g, t)) return;                                    // empty linear set
+  const int q0 = geo_q0(g, t), q1 = geo_q1(g, t);
+  const int tok_a = min(q0 + (int)blockIdx.x * a.tiles_per_cta * 128, q1);
+  const int tok_b = min(tok_a + a.tiles_per_cta * 128, q1);
+  if (tok_a >= tok_b) return;
+  const int n_tiles = (tok_b - tok_a + 127) / 128;
+
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bars->x_full), 1); mbar_init(smem_u32(&bars->x_empty), 1);
+    for (int s = 0; s < RD_RING; ++s) {
+      mbar_init(smem_u32(&bars->ring_full[s]), 1); mbar_init(smem_u32(&bars->ring_empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&bars->acc_ready[b]), 1); mbar_init(smem_u32(&bars->epi_done[b]), 256); }
+    mbar_init(smem_u32(&bars->out_ready), 1); mbar_init(smem_u32(&bars->out_read), 256);
+    bars->abort_flag = 0;
+    fence_mbar_init();
+  }
+  for (int i = threadIdx.x; i < 256; i += PH_THREADS) {             // biases and z_t as fp32
+    s_b1[i] = __bfloat162float(a.b1[(size_t)h_idx * 256 + i]);
+    s_b2[i] = __bfloat162float(a.b2[(size_t)h_idx * 256 + i]);
+    s_z[i] = a.state[(((size_t)ci * g.BH + bh) * PH_DP + i) * PH_SD + PH_D];
+  }
+  if (warp == 9) {
+    tmem_alloc(smem_u32(&bars->tmem_base), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+  constexpr uint32_t T_SCR = 0, T_H = 256, T_R = 384;
+  const uint32_t sX = sb + RD_OFF_X, sPhi0 = sb + RD_OFF_PHI0, sPhi1 = sb + RD_OFF_PHI1, sRing = sb + RD_OFF_RING;
+
+  if (warp == 8) {
+    // ------------------------------------------------------------------ TMA producer
+    if (elect_one()) {
+      prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_w1); prefetch_tensormap(&tm_w2); prefetch_tensormap(&tm_s);
+      uint32_t ring_i = 0;
+      bool alive = true;
+      auto ring_slot = [&]() -> uint32_t {                          // waits for the next stage to be free; 0 on abort
+        const int s = ring_i % RD_RING;
+        alive = alive && mbar_wait(smem_u32(&bars->ring_empty[s]), ((ring_i / RD_RING) & 1) ^ 1, abort_flag, a.status, PH_ERR_LOAD);
+        if (!alive) return 0u;
+        mbar_expect_tx(smem_u32(&bars->ring_full[s]), RD_WT_BYTES);
+        ++ring_i;
+        return sRing + s * RD_WT_BYTES;
+      };
+      auto weight_load = [&](const CUtensorMap* tm, int x, int y) {
+        const uint32_t full = smem_u32(&bars->ring_full[ring_i % RD_RING]);
+        const uint32_t dst = ring_slot();
+        if (dst) tma_load_3d(dst, tm, full, x, y, h_idx);
+      };
+      auto state_load = [&](int f) {                                // [64 features x 128 d] as two 64-column boxes
+        const uint32_t full = smem_u32(&bars->ring_full[ring_i % RD_RING]);
+        const uint32_t dst = ring_slot();
+        if (dst) {
+          tma_load_3d(dst, &tm_s, full, 0, f * 64, ci * g.BH + bh);
+          tma_load_3d(dst + 8192, &tm_s, full, 64, f * 64, ci * g.BH + bh);
+        }
+      };
+      for (int j = 0; j < n_tiles && alive; ++j) {
+        alive = mbar_wait(smem_u32(&bars->x_empty), (j & 1) ^ 1, abort_flag, a.status, PH_ERR_LOAD);
+        if (!alive) break;
+        const uint32_t xf = smem_u32(&bars->x_full);
+        mbar_expect_tx(xf, PH_TILE_BYTES);
+        tma_load_4d(sX, &tm_x, xf, 0, tok_a + j * 128, h_idx, b_idx);
+        tma_load_4d(sX + PH_SUB, &tm_x, xf, 64, tok_a + j * 128, h_idx, b_idx);
+        // the ring follows the issue order of the MMAs: read-out of the previous tile between this tile's H halves
+        for (int ks = 0; ks < 2; ++ks) weight_load(&tm_w1, ks * 64, 0);
+        if (j > 0) { state_load(0); state_load(1); }
+        for (int ks = 0; ks < 2; ++ks) weight_load(&tm_w1, ks * 64, 128);
+        if (j > 0) { state_load(2); state_load(3); }
+        for (int ks = 0; ks < 4; ++ks) weight_load(&tm_w2, ks * 64, 0);
+        for (int ks = 0; ks < 4; ++ks) weight_load(&tm_w2, ks * 64, 128);
+      }
+      for (int f = 0; f < 4 && alive; ++f) state_load(f);
+    }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------------ UMMA issuer
+    if (elect_one()) {
+      constexpr uint32_t id_kk = idesc_bf16(128, 128, 0, 0);       // A K-major (smem or TMEM), B K-major: the MLP GEMMs
+      constexpr uint32_t id_rd = idesc_bf16(128, 128, 0, 1);       // A = phi (K-major), B = state (MN-major)
+      uint32_t ring_i = 0, n_epi[2] = {0, 0};
+      auto ring_wait = [&]() -> uint32_t {
+        const int s = ring_i % RD_RING;
+        mbar_wait(smem_u32(&bars->ring_full[s]), (ring_i / RD_RING) & 1, abort_flag, a.status, PH_ERR_MMA);
+        tc_fence_after();
+        return sRing + s * RD_WT_BYTES;
+      };
+      auto ring_release = [&]() {
+        umma_commit(smem_u32(&bars->ring_empty[ring_i % RD_RING]));
+        ++ring_i;
+      };
+      auto wait_epi = [&](int b) {                                  // the next epilogue that used scratch b is done
+        mbar_wait(smem_u32(&bars->epi_done[b]), n_epi[b] & 1, abort_flag, a.status, PH_ERR_MMA);
+        ++n_epi[b];
+        tc_fence_after();
+      };
+      auto h_half = [&](int b) {                                    // H[:, 128 b : 128 b + 128] = X W1[...]^T into scratch b
+        for (int ks = 0; ks < 2; ++ks) {
+          const uint32_t bt = ring_wait();
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            umma_ss(tmem + T_SCR + b * 128, smem_desc_sw128(sX + ks * PH_SUB + kk * 32, 16, 1024),
+                    smem_desc_sw128(bt + kk * 32, 16, 1024), id_kk, (ks | kk) != 0);
+          ring_release();
+        }
+        umma_commit(smem_u32(&bars->acc_ready[b]));
+      };
+      auto u_half = [&](int b) {                                    // U[:, 128 b : ...] = H W2[...]^T with H read from TMEM
+        for (int ks = 0; ks < 4; ++ks) {
+          const uint32_t bt = ring_wait();
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            umma_ts(tmem + T_SCR + b * 128, tmem + T_H + (ks * 4 + kk) * 8, smem_desc_sw128(bt + kk * 32, 16, 1024), id_kk,
+                    (ks | kk) != 0);
+          ring_release();
+        }
+        umma_commit(smem_u32(&bars->acc_ready[b]));
+      };
+      auto readout_half = [&](int c, uint32_t phi_base) {           // R (+)= phi[:, 128 c : ...] s_t[128 c : ..., :]
+        for (int f = 0; f < 2; ++f) {
+          const uint32_t bt = ring_wait();
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            umma_ss(tmem + T_R, smem_desc_sw128(phi_base + f * PH_SUB + kk * 32, 16, 1024),
+                    smem_desc_sw128(bt + kk * 2048, 8192, 1024), id_rd, (c | f | kk) != 0);
+          ring_release();
+        }
+      };
+      for (int j = 0; j < n_tiles; ++j) {
+        mbar_wait(smem_u32(&bars->x_full), j & 1, abort_flag, a.status, PH_ERR_MMA);
+        tc_fence_after();
+        if (j > 0) wait_epi(0);                                     // U half 0 of tile j-1: scratch A free, phi half 0 written
+        h_half(0);
+        if (j > 0) {
+          if (j > 1) {                                              // the read-out of tile j-2 has left TMEM
+            mbar_wait(smem_u32(&bars->out_read), (j - 2) & 1, abort_flag, a.status, PH_ERR_MMA);
+            tc_fence_after();
+          }
+          readout_half(0, sPhi0);
+          wait_epi(1);                                              // U half 1 of tile j-1
+        }
+        h_half(1);
+        umma_commit(smem_u32(&bars->x_empty));
+        if (j > 0) {
+          readout_half(1, sPhi1);
+          umma_commit(smem_u32(&bars->out_ready));
+        }
+        wait_epi(0);
+        wait_epi(1);                                                // all of H is in TMEM
+        u_half(0);
+        u_half(1);
+      }
+      wait_epi(0);
+      if (n_tiles > 1) {
+        mbar_wait(smem_u32(&bars->out_read), (n_tiles - 2) & 1, abort_flag, a.status, PH_ERR_MMA);
+        tc_fence_after();
+      }
+      readout_half(0, sPhi0);
+      wait_epi(1);
+      readout_half(1, sPhi1);
+      umma_commit(smem_u32(&bars->out_ready));
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogues
+    // Eight warps: warp w serves TMEM lanes 32*(w%4).. (one token per thread) and the column half w/4 of every
+    // 128-column accumulator, so two threads share a token.
+    const int qd = warp & 3, ch = warp >> 2;
+    const int r = qd * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(qd * 32) << 16;
+    uint32_t n_acc[2] = {0, 0};
+    const int part_w = PH_DP / (PC ? PC : a.P);                     // a multiple of 32 (P in {1,2,4})
+    // bias + activation (+ power) of 32 accumulator columns -> 16 bf16 pairs
+    auto activate = [&](const uint32_t (&x)[32], const float* bias, bool is_u, int col0, uint32_t (&w)[16]) {
+      if (RELU) {
+        const int part = !is_u ? 0 : PC == 1 ? 0 : PC == 2 ? (col0 >> 7) : col0 / part_w;   // uniform over the 32 columns
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          const float4 b4 = *reinterpret_cast<const float4*>(bias + e);
+          float y0, y1, y2, y3;
+          upk2(add2(pk2u(x[e], x[e + 1]), pk2(b4.x, b4.y)), y0, y1);
+          upk2(add2(pk2u(x[e + 2], x[e + 3]), pk2(b4.z, b4.w)), y2, y3);
+          if (part == 0) {
+            w[e >> 1] = pack_bf16_relu(y0, y1);
+            w[(e >> 1) + 1] = pack_bf16_relu(y2, y3);
+          } else {
+            y0 = fmaxf(y0, 0.f); y1 = fmaxf(y1, 0.f); y2 = fmaxf(y2, 0.f); y3 = fmaxf(y3, 0.f);
+            float p0 = y0 * y0, p1 = y1 * y1, p2 = y2 * y2, p3 = y3 * y3;
+            if (part == 2) { p0 *= y0; p1 *= y1; p2 *= y2; p3 *= y3; }
+            if (part == 3) { p0 *= p0; p1 *= p1; p2 *= p2; p3 *= p3; }
+            w[e >> 1] = pack_bf16(p0, p1);
+            w[(e >> 1) + 1] = pack_bf16(p2, p3);
+          }
+        }
+      } else {
+        const int act = is_u ? a.act_out : a.act_hidden;
+        const int part = is_u ? col0 / part_w : 0;
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+          const float y0 = apply_act(__uint_as_float(x[e]) + bias[e], act);
+          const float y1 = apply_act(__uint_as_float(x[e + 1]) + bias[e + 1], act);
+          w[e >> 1] = pack_bf16(poly_power(y0, part), poly_power(y1, part));
+        }
+      }
+    };
+    auto readout_store = [&](int jt) {                              // fp32 read-out of tile jt leaves TMEM
+      mbar_wait(smem_u32(&bars->out_ready), jt & 1, abort_flag, a.status, PH_ERR_EPI);
+      tc_fence_after();
+      asm volatile("bar.sync 1, 256;" ::: "memory");                 // both halves of s_nl are written
+      const bool tok_valid = tok_a + jt * 128 + r < tok_b;
+      const int ric = tok_a + jt * 128 + r - q0;                    // row inside the chunk; its tile is 128-aligned
+#pragma unroll
+      for (int cb = 0; cb < 2; ++cb) {
+        uint32_t x[32];
+        tmem_ld32(tmem + lane_off + T_R + ch * 64 + cb * 32, x);
+        tmem_wait_ld();
+        if (tok_valid) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 4)
+            *reinterpret_cast<float4*>(a.rd + rd_index(g, a.rd_rows, PH_D, bh, ci, ric, (ch * 64 + cb * 32 + e) >> 2)) =
+                make_float4(__uint_as_float(x[e]), __uint_as_float(x[e + 1]), __uint_as_float(x[e + 2]),
+                            __uint_as_float(x[e + 3]));
+        }
+      }
+      if (tok_valid && ch == 1) a.rd[rd_index(g, a.rd_rows, PH_D, bh, ci, ric, PH_D / 4)] = s_nl[r] + s_nl[128 + r];
+      tc_fence_before();
+      asm volatile("bar.sync 1, 256;" ::: "memory");                 // s_nl may be overwritten by the next tile
+      mbar_arrive(smem_u32(&bars->out_read));
+    };
+    for (int j = 0; j < n_tiles; ++j) {
+      const bool tok_valid = tok_a + j * 128 + r < tok_b;
+      // H halves: bias, activation, bf16, back to TMEM as the A operand of the second GEMM
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        mbar_wait(smem_u32(&bars->acc_ready[half]), n_acc[half] & 1, abort_flag, a.status, PH_ERR_EPI);
+        ++n_acc[half];
+        tc_fence_after();
+        uint32_t x[2][32];
+        tmem_ld32(tmem + lane_off + T_SCR + half * 128 + ch * 64, x[0]);
+        tmem_ld32(tmem + lane_off + T_SCR + half * 128 + ch * 64 + 32, x[1]);
+        tmem_wait_ld();
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) {
+          const int col0 = half * 128 + ch * 64 + cb * 32;          // hidden unit of the first column
+          uint32_t w[16];
+          activate(x[cb], s_b1 + col0, false, col0, w);
+          tmem_st16(tmem + lane_off + T_H + (col0 >> 1), w);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(smem_u32(&bars->epi_done[half]));
+      }
+      if (j > 0) readout_store(j - 1);
+      // U halves: bias, activation, power, bf16, to the swizzled phi tiles; phi . z_t on the way
+      float nl = 0.f;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        mbar_wait(smem_u32(&bars->acc_ready[half]), n_acc[half] & 1, abort_flag, a.status, PH_ERR_EPI);
+        ++n_acc[half];
+        tc_fence_after();
+        uint32_t x[2][32];
+        tmem_ld32(tmem + lane_off + T_SCR + half * 128 + ch * 64, x[0]);
+        tmem_ld32(tmem + lane_off + T_SCR + half * 128 + ch * 64 + 32, x[1]);
+        tmem_wait_ld();
+        const uint32_t dst = half == 0 ? sPhi0 : sPhi1;
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) {
+          const int col0 = half * 128 + ch * 64 + cb * 32;          // feature of the first column
+          uint32_t w[16];
+          activate(x[cb], s_b2 + col0, true, col0, w);
+          if (!tok_valid) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) w[e] = 0u;
+          }
+#pragma unroll
+          for (int e = 0; e < 32; e += 8) {
+            const uint4 w4 = make_uint4(w[e >> 1], w[(e >> 1) + 1], w[(e >> 1) + 2], w[(e >> 1) + 3]);
+            // phi_q(q_r) . z_t with the same bf16-rounded features the tensor core sees
+            const float* zz = s_z + col0 + e;
+            const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              nl = fmaf(__uint_as_float(ww[u] << 16), zz[2 * u], nl);
+              nl = fmaf(__uint_as_float(ww[u] & 0xffff0000u), zz[2 * u + 1], nl);
+            }
+            st_tile_chunk_sw128(dst, PH_SUB, r, ch * 64 + cb * 32 + e, w4);
+          }
+        }
+        if (half == 1) s_nl[ch * 128 + r] = nl;
+        fence_proxy_async_smem();
+        tc_fence_before();
+        mbar_arrive(smem_u32(&bars->epi_done[half]));
+      }
+    }
+    readout_store(n_tiles - 1);
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+}  // namespace rehyat

@@ -20,6 +20,7 @@
 #include "rehyat_common.cuh"
 #include "rehyat_ptx.cuh"
 #include "rehyat_phi_tc.cuh"
+#include "rehyat_readout_tc.cuh"
 
 namespace rehyat {
 
@@ -429,12 +430,12 @@ inline int tc_set_attributes() {
             cudaFuncSetAttribute(window_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(window_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(window_tc<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(phi_tc<PHI_STATE, true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(phi_tc<PHI_STATE, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(phi_tc<PHI_STATE, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(phi_tc<PHI_READOUT, true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(phi_tc<PHI_READOUT, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(phi_tc<PHI_READOUT, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess;
+            cudaFuncSetAttribute(phi_tc<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(phi_tc<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(phi_tc<false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(readout_tc<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, RD_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(readout_tc<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, RD_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(readout_tc<false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, RD_SMEM) == cudaSuccess;
   return ok ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
@@ -503,11 +504,11 @@ inline int tc_launch_state(const TcWorkspace* w, const void* k, const void* v, c
   const bool relu = act_hidden == ACT_RELU && act_out == ACT_RELU;
   const dim3 grid(n_split, g.G, g.BH);
   if (relu && P == 2)
-    phi_tc<PHI_STATE, true, 2><<<grid, PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, tw2, g, a);
+    phi_tc<true, 2><<<grid, PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, g, a);
   else if (relu)
-    phi_tc<PHI_STATE, true, 0><<<grid, PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, tw2, g, a);
+    phi_tc<true, 0><<<grid, PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, g, a);
   else
-    phi_tc<PHI_STATE, false, 0><<<grid, PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, tw2, g, a);
+    phi_tc<false, 0><<<grid, PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, g, a);
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
@@ -540,11 +541,11 @@ inline int tc_launch_readout(const TcWorkspace* w, const void* q, const rehyat_p
   const bool relu = act_hidden == ACT_RELU && act_out == ACT_RELU;
   const dim3 grid(ctas, g.G, g.BH);
   if (relu && P == 2)
-    phi_tc<PHI_READOUT, true, 2><<<grid, PH_THREADS, PH_SMEM, st>>>(tq, tq, tw1, tw2, ts, g, a);
+    readout_tc<true, 2><<<grid, PH_THREADS, RD_SMEM, st>>>(tq, tw1, tw2, ts, g, a);
   else if (relu)
-    phi_tc<PHI_READOUT, true, 0><<<grid, PH_THREADS, PH_SMEM, st>>>(tq, tq, tw1, tw2, ts, g, a);
+    readout_tc<true, 0><<<grid, PH_THREADS, RD_SMEM, st>>>(tq, tw1, tw2, ts, g, a);
   else
-    phi_tc<PHI_READOUT, false, 0><<<grid, PH_THREADS, PH_SMEM, st>>>(tq, tq, tw1, tw2, ts, g, a);
+    readout_tc<false, 0><<<grid, PH_THREADS, RD_SMEM, st>>>(tq, tw1, tw2, ts, g, a);
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
