@@ -37,7 +37,7 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the ncu
 # capture summarised under profiles/; None until a capture exists for the kernel in use.
-NCU_TRAFFIC_BYTES = {"window_simt": None, "window_tc": 481437952 + 86796544}   # profiles/window_tc_wan13b_layer.md
+NCU_TRAFFIC_BYTES = {"window_simt": None, "window_tc": 481645824 + 87647232}   # profiles/window_tc_wan13b_layer.md
 
 
 def measured_peaks():
