@@ -108,17 +108,20 @@ def blas_threads():
         return os.cpu_count()
 
 
-def oracle_sample(wl, inputs, heads):
-    """Times the fp64 oracle (recurrent form, as it stands) on `heads` of batch 0 of the workload."""
+def oracle_sample(wl, inputs, heads, frames=None):
+    """Times the fp64 oracle (recurrent form, as it stands) on `heads` of batch 0 of the workload, optionally on
+    its first `frames` latent frames only.  Returns (seconds, algorithmic FLOPs of what was computed)."""
     from oracle import rehyat_oracle as orc
-    sel = lambda t: t[:1, heads].to(torch.float64).numpy()
+    T = wl.T if frames is None else frames
+    n = T * wl.HW
+    sel = lambda t: t[:1, heads, :n].to(torch.float64).numpy()
     q, k, v = sel(inputs["q"]), sel(inputs["k"]), sel(inputs["v"])
-    pq = {n: t[heads].to(torch.float64).numpy() for n, t in inputs["phi_q"].items()}
-    pk = {n: t[heads].to(torch.float64).numpy() for n, t in inputs["phi_k"].items()}
+    pq = {n_: t[heads].to(torch.float64).numpy() for n_, t in inputs["phi_q"].items()}
+    pk = {n_: t[heads].to(torch.float64).numpy() for n_, t in inputs["phi_k"].items()}
     t0 = time.perf_counter()
-    orc.hybrid_rnn(q, k, v, pq, pk, wl.T, wl.HW, wl.Tc, wl.To, P=wl.P)
+    orc.hybrid_rnn(q, k, v, pq, pk, T, wl.HW, wl.Tc, wl.To, P=wl.P)
     dt = time.perf_counter() - t0
-    flops = geometry.flop_model(1, len(heads), wl.head_dim, wl.T, wl.HW, wl.Tc, wl.To, wl.D_h, wl.D_out)["total"]
+    flops = geometry.flop_model(1, len(heads), wl.head_dim, T, wl.HW, wl.Tc, wl.To, wl.D_h, wl.D_out)["total"]
     return dt, flops
 
 
@@ -251,16 +254,28 @@ def run_reference(args, wl):
     if rank != 0:
         return
     inputs = synth.make_inputs(wl)
-    heads = list(range(args.ref_heads))
+    # Every step is a bounded sample of the workload, sized from one calibration pass so that the whole run of
+    # warmup + steps stays within about two and a half minutes: as many heads as fit, else one head on its first frames.
+    t_head, _ = oracle_sample(wl, inputs, [0])
+    per_step = 150.0 / max(args.warmup + args.steps, 1)
+    n_heads = int(min(args.ref_heads, wl.n_heads, max(1, per_step // t_head)))
+    frames = None
+    if t_head > per_step:
+        frames = wl.T
+        while frames > wl.Tc + wl.To + 1 and t_head * (frames / wl.T) ** 1.2 > per_step:
+            frames -= wl.Tc
+    heads = list(range(n_heads))
     times = []
     flops = 0
     for i in range(args.warmup + args.steps):
-        dt, flops = oracle_sample(wl, inputs, heads)
+        dt, flops = oracle_sample(wl, inputs, heads, frames)
         if i >= args.warmup:
             times.append(dt)
     total = sum(times)
     value = flops * len(times) / total / 1e12
-    sample = f"{len(heads)} of {wl.n_heads} heads of batch 0, all {wl.N} tokens, recurrent form, fp64 numpy"
+    sample = (f"{len(heads)} of {wl.n_heads} heads of batch 0, " +
+              (f"all {wl.N} tokens" if frames is None else f"the first {frames} of {wl.T} latent frames ({frames * wl.HW} tokens)") +
+              ", recurrent form, fp64 numpy")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
