@@ -1,11 +1,13 @@
-// Tensor-core (tcgen05 / TMEM / TMA) path of the operator for bf16, head_dim 128.
+// Tensor-core (tcgen05 / TMEM / TMA) path of the operator for bf16, head_dim 128: the softmax-window kernel and
+// the host-side launchers of all three tensor-core kernels.
 //
 // window_tc: softmax window of Eq. 6 and 8 plus the joint normalisation of Eq. 5.
-//   One CTA owns two 128-row query tiles of one chunk and walks the chunk's key window in tiles of
-//   128 keys.  Roles (384 threads):
-//     warp 0        TMA producer: Q once, then K and V tiles through two-stage rings
-//     warp 1        UMMA issuer: S_i = Q_i K^T into TMEM, O_i += P_i V with P_i read from TMEM
-//     warps 4-7     softmax of query tile 0 (one thread per row), warps 8-11 of query tile 1
+//   Persistent: one CTA per SM walks work items (batch*head, chunk, pair of 128-row query tiles); barriers, TMEM
+//   and the K/V rings live across items.  An item walks the chunk's key window in tiles of 128 keys.
+//   Roles (384 threads):
+//     warp 0        TMA producer: Q per item, K and V tiles through two-stage rings
+//     warp 1        UMMA issuer: S_i = Q_i K^T into TMEM, O_i += P_i V with P_i read from TMEM (in two halves)
+//     warps 4-7     softmax and epilogue of query tile 0 (one thread per row), warps 8-11 of query tile 1
 //   TMEM (512 columns): S_0 [0,128) S_1 [128,256) O_0 [256,384) O_1 [384,512); P_i (bf16) overwrites
 //   the first 64 columns of S_i.  While one tile's softmax runs on the ALUs the tensor core works on
 //   the other tile.  The running maximum is applied lazily: O and l are rescaled only when the row
