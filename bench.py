@@ -437,7 +437,8 @@ def main():
         extras["workspace_bytes_by_latent_frames"] = workspace_by_frames(wl, local_rank)
         extras["chunk_by_chunk"] = stream_timing(wl, dev, phi_q, phi_k, stream, flops)
     if world == 1 and args.all_configs:
-        extras["other_configs"] = [time_config(synth.CONFIGS[n], local_rank, stream) for n in ("cfg_long", "long_constant_memory")]
+        extras["other_configs"] = [time_config(synth.CONFIGS[n], local_rank, stream)
+                                   for n in ("cfg_long", "long_constant_memory", "wan13b_320x480")]
         extras["bidirectional_same_shape"] = bidirectional_timing(wl, dev, phi_q, phi_k, stream, ms_step)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

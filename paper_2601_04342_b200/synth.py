@@ -70,6 +70,9 @@ CONFIGS = {
                          seed=BASE_SEED + 3),
     "long_constant_memory": Workload("long_constant_memory", 1, 12, 128, 81, 30, 52, 3, 1, "bf16",
                                      True, seed=BASE_SEED + 4),
+    # the 320x480 resolution of the paper's on-device tables: latent 21 x 20 x 30 (12,600 tokens)
+    "wan13b_320x480": Workload("wan13b_320x480", 1, 12, 128, 21, 20, 30, 3, 1, "bf16", True,
+                               seed=BASE_SEED + 6),
 }
 
 

@@ -123,6 +123,17 @@ def test_wan13b_layer_rows_sum_to_one_everywhere():
     assert float((y.float() - 1.0).abs().max()) <= 2.0 ** -8
 
 
+def test_320x480_layer_every_element():
+    """The resolution of the paper's on-device measurements (latent 21 x 20 x 30): HW = 600 is not a
+    multiple of the 128-row tiles either (N' = 1800 = 14 * 128 + 8)."""
+    wl = synth.CONFIGS["wan13b_320x480"]
+    x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
+    y, _, _ = gpu_forward(wl, x)
+    f = synth.to_f64(x)
+    ref = orc.hybrid_rnn(f["q"], f["k"], f["v"], f["phi_q"], f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To, P=wl.P)
+    gate(y.double().numpy(), ref)
+
+
 # ------------------------------------------------------------------ CFG batch, longer video
 def test_cfg_long_sampled_rows():
     wl = synth.CONFIGS["cfg_long"]                 # B=2, 41 frames: 14 chunks, the last one 2 frames
