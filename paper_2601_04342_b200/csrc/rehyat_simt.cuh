@@ -251,7 +251,7 @@ __global__ void __launch_bounds__(WIN_THREADS)
 window_simt(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, T* __restrict__ out,
             Geo g, const float* __restrict__ rd, int rd_rows, float scale, int c_mode) {
   extern __shared__ __align__(16) float smem[];
-  constexpr int SD = D + 4, LDK = D + 4, LDP = WIN_BN + 4;
+  constexpr int LDK = D + 4, LDP = WIN_BN + 4;
   constexpr int DC = D / 16;                 // output columns per thread
   float* Qs = smem;                          // [BM][LDK]
   float* Ks = Qs + WIN_BM * LDK;             // [BN][LDK]
