@@ -113,7 +113,10 @@ typedef struct rehyat_ctx rehyat_ctx;
 /* Creates a context on cfg->device and allocates its fixed workspace (chunk states, partial
  * state sums, the linear read-out of one chunk group, a status word).  The workspace size is a
  * function of the config only (Section 3.3, note 3: memory constant in the video length).
- * Errors: INVALID_ARG (null, sizes out of range), UNSUPPORTED, ARCH, CUDA, ALLOC. */
+ * Errors: INVALID_ARG (null, sizes out of range), UNSUPPORTED, ARCH, CUDA, ALLOC.
+ * Tuning: the environment variable REHYAT_EXP_POLY = 0..3, read here, sets how many of every four pairs of
+ * softmax exponentials the tensor-core window kernel evaluates as a cubic on the FMA pipe instead of the
+ * special-function unit (default 1, the fastest measured on B200; the results agree within bf16 rounding). */
 int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg);
 
 /* Enqueues the operator of Eq. 5-9 with the causal sets of Eq. 13 on `cuda_stream`
