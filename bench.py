@@ -431,6 +431,15 @@ def main():
                          f"fp64 numpy, {dt:.1f} s"}
 
     extras = {}
+    if world == 1:
+        # The timed loop above runs long enough for the GPU to reach its power cap and lower the SM clock.  For
+        # context (never the headline value): ten steps after the GPU has been idle, at the clocks the measured
+        # burst peak was taken at.
+        time.sleep(1.0)
+        idle_ms = _time_ms(step, stream, 3, 10)
+        extras["ten_steps_after_idle"] = {"ms_per_step": idle_ms, "value": flops["total"] / (idle_ms * 1e-3) / 1e12,
+                                          "unit": UNIT, "frac_of_measured_burst": flops["total"] / (idle_ms * 1e-3) / 1e12 / peaks["bf16_burst"],
+                                          "frac_of_nominal_2250": flops["total"] / (idle_ms * 1e-3) / 1e12 / 2250.0}
     if world == 1 and wl.dtype == "bf16" and not args.no_full_softmax:
         extras["full_softmax_same_shape"] = full_softmax_comparison(wl, dev, phi_q, phi_k, stream, ms_step, flops)
     if world == 1:
