@@ -416,6 +416,7 @@ def main():
                 "peak_source": f"{peaks['source']} bf16 {peak_kind} (MEASURED_PEAKS.json)" if peaks["source"] == "measured"
                 else "fallback",
                 "frac_of_nominal_2250": achieved / 2250.0 if achieved else None,
+                "frac_of_measured_sustained": achieved / peaks["bf16_sustained"] if achieved else None,
                 "launches": win_n, "avg_launch_ms": win_ms / max(win_n, 1),
                 "algorithmic_flop_per_launch": win_flops_per_launch,
                 "hbm_gbs_whole_step": geometry.io_bytes(wl.B, wl.n_heads, wl.head_dim, wl.N, 2) / (ms_step * 1e-3) / 1e9,
