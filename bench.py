@@ -151,17 +151,18 @@ def _time_ms(fn, stream, warmup, steps):
     return e0.elapsed_time(e1) / steps
 
 
-def full_softmax_comparison(wl, dev, phi_q, phi_k, stream, hybrid_ms, flops):
+def full_softmax_comparison(wl, dev, phi_q, phi_k, stream, hybrid_ms, flops, warmup=2, steps=5):
     """Full softmax attention (Eq. 2) at the workload's shape: this operator with one chunk covering
     every frame (exact by the T_c = T limit) and, as an independent time, the library SDPA kernel."""
     from paper_2601_04342_b200 import binding
     op = binding.for_workload(wl, max_chunk_frames=wl.T)
     out = torch.empty_like(dev["q"])
     ours = _time_ms(lambda: op.forward(dev["q"], dev["k"], dev["v"], phi_q, phi_k, wl.T, wl.H, wl.W, wl.T, 0,
-                                       out=out, stream=stream), stream, 2, 5)
+                                       out=out, stream=stream), stream, warmup, steps)
     assert op.status() == 0
     op.close()
-    lib = _time_ms(lambda: torch.nn.functional.scaled_dot_product_attention(dev["q"], dev["k"], dev["v"]), stream, 2, 5)
+    lib = _time_ms(lambda: torch.nn.functional.scaled_dot_product_attention(dev["q"], dev["k"], dev["v"]), stream,
+                   warmup, steps)
     return {"flop": flops["full_softmax"], "this_operator_chunk_eq_frames_ms": ours,
             "this_operator_tflops": flops["full_softmax"] / (ours * 1e-3) / 1e12,
             "library_sdpa_ms": lib, "library_sdpa_tflops": flops["full_softmax"] / (lib * 1e-3) / 1e12,
@@ -224,7 +225,7 @@ def lib_state_bytes(op):
     return binding.lib().rehyat_stream_state_bytes(op._h)
 
 
-def time_config(wl, device, stream):
+def time_config(wl, device, stream, full_softmax=False):
     """Kernel-resident timing of another configuration.  Inputs are drawn on the device (seeded torch
     generator, N(0,1), q and k RMS-normalised) because the host recipe takes tens of seconds at these
     sizes; the parity tests use the host recipe."""
@@ -246,6 +247,9 @@ def time_config(wl, device, stream):
            "tokens_per_s": wl.B * wl.N / (ms * 1e-3), "workspace_bytes": op.workspace_bytes, "launches_per_step": op.last_launches,
            "full_softmax_flop_ratio": fl["full_softmax"] / fl["total"]}
     op.close()
+    if full_softmax:
+        res["full_softmax_same_shape"] = full_softmax_comparison(wl, {"q": q, "k": k, "v": v}, pq, pk, stream, ms, fl,
+                                                                 warmup=1, steps=2)
     return res
 
 
@@ -441,13 +445,27 @@ def main():
         extras["ten_steps_after_idle"] = {"ms_per_step": idle_ms, "value": flops["total"] / (idle_ms * 1e-3) / 1e12,
                                           "unit": UNIT, "frac_of_measured_burst": flops["total"] / (idle_ms * 1e-3) / 1e12 / peaks["bf16_burst"],
                                           "frac_of_nominal_2250": flops["total"] / (idle_ms * 1e-3) / 1e12 / 2250.0}
+    if world == 1:
+        # The timed loop leaves L2 as the previous step left it (the steady state of a layer called again and again;
+        # the tensors exceed L2 anyway).  For comparison, ten steps each started after 256 MB of writes have swept L2.
+        sweep = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        f0 = [torch.cuda.Event(enable_timing=True) for _ in range(10)]
+        f1 = [torch.cuda.Event(enable_timing=True) for _ in range(10)]
+        for a, b in zip(f0, f1):
+            sweep.zero_()
+            a.record(stream)
+            step()
+            b.record(stream)
+        torch.cuda.synchronize()
+        extras["l2_swept_before_each_step"] = {"ms_per_step": sum(a.elapsed_time(b) for a, b in zip(f0, f1)) / 10}
+        del sweep
     if world == 1 and wl.dtype == "bf16" and not args.no_full_softmax:
         extras["full_softmax_same_shape"] = full_softmax_comparison(wl, dev, phi_q, phi_k, stream, ms_step, flops)
     if world == 1:
         extras["workspace_bytes_by_latent_frames"] = workspace_by_frames(wl, local_rank)
         extras["chunk_by_chunk"] = stream_timing(wl, dev, phi_q, phi_k, stream, flops)
     if world == 1 and args.all_configs:
-        extras["other_configs"] = [time_config(synth.CONFIGS[n], local_rank, stream)
+        extras["other_configs"] = [time_config(synth.CONFIGS[n], local_rank, stream, full_softmax=(n == "cfg_long"))
                                    for n in ("cfg_long", "long_constant_memory", "wan13b_320x480")]
         extras["bidirectional_same_shape"] = bidirectional_timing(wl, dev, phi_q, phi_k, stream, ms_step)
 
