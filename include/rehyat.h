@@ -116,7 +116,10 @@ typedef struct rehyat_ctx rehyat_ctx;
  * Errors: INVALID_ARG (null, sizes out of range), UNSUPPORTED, ARCH, CUDA, ALLOC.
  * Tuning: the environment variable REHYAT_EXP_POLY = 0..3, read here, sets how many of every four pairs of
  * softmax exponentials the tensor-core window kernel evaluates as a cubic on the FMA pipe instead of the
- * special-function unit (default 1, the fastest measured on B200; the results agree within bf16 rounding). */
+ * special-function unit (default 1, the fastest measured on B200; the results agree within bf16 rounding).
+ * REHYAT_WINDOW_TILES = 1 or 2, read here, fixes the number of 128-row query tiles per work item of that
+ * kernel (default: chosen per launch from how many items there are for the SMs; same results up to the order
+ * of fp32 sums). */
 int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg);
 
 /* Enqueues the operator of Eq. 5-9 with the causal sets of Eq. 13 on `cuda_stream`

@@ -22,6 +22,7 @@
 #include "rehyat_common.cuh"
 #include "rehyat_simt.cuh"
 #include "rehyat_tc.cuh"
+#include "rehyat_tc_single.cuh"
 
 using namespace rehyat;
 
@@ -320,6 +321,10 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
   if (const char* e = getenv("REHYAT_EXP_POLY")) {
     const int n = atoi(e);
     if (n >= 0 && n <= 3) ctx->tc.exp_poly = n;
+  }
+  if (const char* e = getenv("REHYAT_WINDOW_TILES")) {
+    const int n = atoi(e);
+    if (n == 1 || n == 2) ctx->tc.item_tiles = n;
   }
   if (ok && ctx->tensor_ok) {
     size_t extra = 0;

@@ -401,6 +401,7 @@ struct TcWorkspace {
   bool phi_ok = false;                  // the linear branch runs on the tensor-core kernels too
   int n_sm = 148;                       // SMs of the device
   int exp_poly = 1;                     // of every 4 pairs of exponentials, how many the FMA pipe evaluates
+  int item_tiles = 0;                   // query tiles per window item: 1, 2, or 0 = chosen per launch
 };
 
 inline bool tc_shape_supported(bool bf16, int d, int, int, int, int, int) { return bf16 && d == TC_D; }
@@ -427,8 +428,15 @@ inline bool tc_workspace_create(TcWorkspace* w, int bh_max, int Gmax, int d, int
 }
 inline void tc_workspace_destroy(TcWorkspace* w) { cudaFree(w->state_bf16); w->state_bf16 = nullptr; }
 
+// window_tc1 (one query tile per item) and its launcher live in rehyat_tc_single.cuh
+inline int tc_launch_window1(int exp_poly, int n_sm, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                             __nv_bfloat16* o, const Geo& g, const float* rd, int rd_rows, float scale, int c_mode,
+                             int* status, cudaStream_t st);
+inline bool tc_set_attributes1();
+
 inline int tc_set_attributes() {
-  bool ok = cudaFuncSetAttribute(window_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
+  bool ok = tc_set_attributes1() &&
+            cudaFuncSetAttribute(window_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(window_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(window_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(window_tc<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
@@ -478,6 +486,13 @@ inline int tc_launch_window(const TcWorkspace* w, const void* q, const void* k, 
   const dim3 grid(n_items < w->n_sm ? n_items : w->n_sm);
   const float scale = 1.0f / sqrtf((float)TC_D);
   __nv_bfloat16* o = (__nv_bfloat16*)out;
+  // Items of two query tiles share their K/V tiles in shared memory; items of one tile (window_tc1) take half
+  // as long each and fill the SMs better when there are few of them, as in a chunk-by-chunk step.  Whole waves
+  // of items over the SMs decide; per tile a one-tile item costs about 8 % more.
+  const long long n1 = (long long)((g.Np + TC_BM - 1) / TC_BM) * g.G * g.BH;
+  const double cost2 = 2.0 * (double)((n_items + w->n_sm - 1) / w->n_sm), cost1 = 1.08 * (double)((n1 + w->n_sm - 1) / w->n_sm);
+  if (w->item_tiles == 1 || (w->item_tiles == 0 && cost1 < 0.93 * cost2))
+    return tc_launch_window1(w->exp_poly, w->n_sm, tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status, st);
 #define REHYAT_LAUNCH_WINDOW(E) \
   window_tc<E><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status, n_items, pairs)
   switch (w->exp_poly) {

@@ -1,0 +1,402 @@
+// window_tc1: the softmax-window kernel of rehyat_tc.cuh with ONE 128-row query tile per work item.
+//
+// It computes what window_tc computes (Eq. 5, 6, 8) and exists for launches with few items -- a chunk-by-chunk
+// step has 12 heads x 37 tiles at the Wan2.1-1.3B shape -- where items of two tiles leave SMs idle in the last
+// wave.  The roles, the TMEM map (S_0 S_1 O_0 O_1), the K/V rings and the softmax arithmetic are those of
+// window_tc; the difference is what the two TMEM slots hold: the key tiles of the item's window alternate between
+// them (even tiles in slot 0, odd tiles in slot 1), each slot with its own running maximum, row sum and O, so
+// that the tensor core and the two softmax warpgroups overlap exactly as they do for a tile pair.  The epilogue
+// merges the two partial softmax results: with m = max(m_0, m_1),
+//   O = O_0 2^(m_0 - m) + O_1 2^(m_1 - m),   l = l_0 2^(m_0 - m) + l_1 2^(m_1 - m)
+// (Eq. 6 and 8 with the window split in two), then adds the linear read-out and divides (Eq. 5).  Both
+// warpgroups own the same 128 TMEM lanes, so each finishes 64 of the 128 output columns.
+#pragma once
+
+#include "rehyat_tc.cuh"
+
+namespace rehyat {
+
+struct WinBars1 {
+  uint64_t q_full, q_empty;
+  uint64_t k_full[TC_STAGES], k_empty[TC_STAGES], v_full[TC_STAGES], v_empty[TC_STAGES];
+  uint64_t s_ready[2], p_half[2][2], pv_done[2], o_free[2];
+  uint64_t drained;
+  uint32_t tmem_base;
+  int abort_flag;
+  float mrg[2][3][TC_BM];   // per slot: reference maximum, true maximum and row sum of every row
+};
+constexpr int TC_WIN1_SMEM = (1 + 2 * TC_STAGES) * TC_TILE_BYTES + 4096 /*barriers, merge buffer*/ + 1024 /*align*/;
+static_assert(sizeof(WinBars1) <= 4096, "barrier block");
+
+// Items are numbered (batch*head, chunk, query tile), query tile fastest; `tiles` = tiles of a full chunk.
+// Returns false for tiles beyond the end of a short last chunk.
+__device__ __forceinline__ bool win_item1(const Geo& g, int item, int tiles, WinItem& w) {
+  const int tile = item % tiles, rest = item / tiles, ci = rest % g.G;
+  w.bh = rest / g.G;
+  w.ci = ci;
+  const int t = g.t0 + ci;
+  w.q0 = geo_q0(g, t); w.q1 = geo_q1(g, t); w.lo = geo_lo(g, t); w.hi = w.q1;
+  w.linear = geo_linear(g, t);
+  w.row_base = w.q0 + tile * TC_BM;
+  if (w.row_base >= w.q1) return false;
+  w.ntiles = 1;
+  w.n_kv = (w.hi - w.lo + TC_BN - 1) / TC_BN;
+  w.b_idx = w.bh / g.n_heads; w.h_idx = w.bh % g.n_heads;
+  return true;
+}
+
+// Persistent like window_tc: gridDim.x CTAs walk the items blockIdx.x, blockIdx.x + gridDim.x, ...
+// EMU: of every four pairs of exponentials, how many are evaluated on the FMA pipe.
+template <int EMU>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+           const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ out, Geo g,
+           const float* __restrict__ rd, int rd_rows, float scale, int c_mode, int* __restrict__ status,
+           int n_items, int tiles) {
+  using namespace ptx;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t sQ = smem_base;                                   // one tile
+  const uint32_t sK = sQ + TC_TILE_BYTES;                          // TC_STAGES tiles
+  const uint32_t sV = sK + TC_STAGES * TC_TILE_BYTES;              // TC_STAGES tiles
+  WinBars1* bars = reinterpret_cast<WinBars1*>(smem + (1 + 2 * TC_STAGES) * TC_TILE_BYTES);
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bars->q_full), 1); mbar_init(smem_u32(&bars->q_empty), 1);
+    for (int s = 0; s < TC_STAGES; ++s) {
+      mbar_init(smem_u32(&bars->k_full[s]), 1); mbar_init(smem_u32(&bars->k_empty[s]), 1);
+      mbar_init(smem_u32(&bars->v_full[s]), 1); mbar_init(smem_u32(&bars->v_empty[s]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&bars->s_ready[i]), 1);
+      mbar_init(smem_u32(&bars->p_half[i][0]), TC_BM);
+      mbar_init(smem_u32(&bars->p_half[i][1]), TC_BM);
+      mbar_init(smem_u32(&bars->pv_done[i]), 1);
+      mbar_init(smem_u32(&bars->o_free[i]), TC_BM);
+    }
+    mbar_init(smem_u32(&bars->drained), 1);
+    bars->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bars->tmem_base), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+
+  if (warp < 4) setmaxnreg_dec<TC_REGS_OTHER>();
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (elect_one()) {
+      prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
+      uint32_t kv_it = 0, n_done = 0;                              // K/V tiles loaded, items loaded
+      bool alive = true;
+      for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+        WinItem w;
+        if (!win_item1(g, item, tiles, w)) continue;
+        // Q of the previous item has been read by its last Q K^T
+        if (n_done > 0) alive = mbar_wait(smem_u32(&bars->q_empty), (n_done - 1) & 1, abort_flag, status, TC_ERR_LOAD);
+        if (!alive) break;
+        const uint32_t qf = smem_u32(&bars->q_full);
+        mbar_expect_tx(qf, TC_TILE_BYTES);
+        tma_load_4d(sQ, &tm_q, qf, 0, w.row_base, w.h_idx, w.b_idx);
+        tma_load_4d(sQ + TC_SUB_BYTES, &tm_q, qf, 64, w.row_base, w.h_idx, w.b_idx);
+        auto load_tile = [&](bool is_v, int j) {                     // key tile j of the item into its ring stage
+          const uint32_t it = kv_it + j;
+          const int s = it % TC_STAGES;
+          const uint32_t ph = (it / TC_STAGES) & 1;
+          const int key0 = w.lo + j * TC_BN;
+          if (!mbar_wait(smem_u32(is_v ? &bars->v_empty[s] : &bars->k_empty[s]), ph ^ 1, abort_flag, status, TC_ERR_LOAD))
+            return false;
+          const uint32_t full = smem_u32(is_v ? &bars->v_full[s] : &bars->k_full[s]);
+          const uint32_t dst = (is_v ? sV : sK) + s * TC_TILE_BYTES;
+          const CUtensorMap* tm = is_v ? &tm_v : &tm_k;
+          mbar_expect_tx(full, TC_TILE_BYTES);
+          tma_load_4d(dst, tm, full, 0, key0, w.h_idx, w.b_idx);
+          tma_load_4d(dst + TC_SUB_BYTES, tm, full, 64, key0, w.h_idx, w.b_idx);
+          return true;
+        };
+        // Q K^T runs two key tiles ahead of P V, so K stays one tile ahead of V
+        alive = load_tile(false, 0);
+        for (int j = 0; j < w.n_kv && alive; ++j) {
+          if (j + 1 < w.n_kv) alive = load_tile(false, j + 1);
+          alive = alive && load_tile(true, j);
+        }
+        kv_it += w.n_kv;
+        ++n_done;
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ UMMA issuer
+    if (elect_one()) {
+      constexpr uint32_t idesc_qk = idesc_bf16(TC_BM, TC_BN, 0, 0);   // A = Q (K-major), B = K (K-major)
+      constexpr uint32_t idesc_pv = idesc_bf16(TC_BM, TC_D, 0, 1);    // A = P (TMEM),    B = V (MN-major)
+      uint32_t q_lo, q_hi, k_lo, k_hi, v_lo, v_hi;
+      upk2u(smem_desc_sw128(sQ, 16, 1024), q_lo, q_hi);
+      upk2u(smem_desc_sw128(sK, 16, 1024), k_lo, k_hi);
+      upk2u(smem_desc_sw128(sV, TC_SUB_BYTES, 1024), v_lo, v_hi);
+      auto issue_qk = [&](int i, int s) {                            // Q times K stage s into slot i
+        const uint32_t b0 = k_lo + s * (TC_TILE_BYTES >> 4);
+#pragma unroll
+        for (int kk = 0; kk < TC_D / 16; ++kk) {
+          const uint32_t off = ((kk >> 2) * TC_SUB_BYTES + (kk & 3) * 32) >> 4;
+          umma_ss(tmem + i * TC_BN, pk2u(q_lo + off, q_hi), pk2u(b0 + off, k_hi), idesc_qk, kk > 0);
+        }
+      };
+      auto issue_pv = [&](int i, int s, int half, bool acc) {        // keys [64*half, 64*half+64) of the tile
+        const uint32_t b0 = v_lo + s * (TC_TILE_BYTES >> 4);
+#pragma unroll
+        for (int kk = half * 4; kk < half * 4 + 4; ++kk)
+          umma_ts(tmem + 256 + i * TC_D, tmem + i * TC_BN + kk * 8, pk2u(b0 + kk * (16 * 128 >> 4), v_hi), idesc_pv,
+                  (acc || kk > half * 4) ? 1u : 0u);
+      };
+      uint32_t kv_it = 0, n_done = 0;                                // K/V tiles consumed, items done
+      uint32_t n_p[2] = {0, 0};                                      // P hand-overs per slot
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        WinItem w;
+        if (!win_item1(g, item, tiles, w)) continue;
+        mbar_wait(smem_u32(&bars->q_full), n_done & 1, abort_flag, status, TC_ERR_MMA);
+        const uint32_t base = kv_it;
+        auto qk_of = [&](int jj) {                                   // S of key tile jj into slot jj & 1
+          const uint32_t it = base + jj;
+          const int s = it % TC_STAGES;
+          mbar_wait(smem_u32(&bars->k_full[s]), (it / TC_STAGES) & 1, abort_flag, status, TC_ERR_MMA);
+          tc_fence_after();
+          issue_qk(jj & 1, s);
+          umma_commit(smem_u32(&bars->s_ready[jj & 1]));
+          umma_commit(smem_u32(&bars->k_empty[s]));
+          if (jj == w.n_kv - 1) umma_commit(smem_u32(&bars->q_empty));   // the item's last Q K^T
+        };
+        qk_of(0);
+        if (w.n_kv > 1) qk_of(1);
+        for (int j = 0; j < w.n_kv; ++j, ++kv_it) {
+          const int i = j & 1, s = kv_it % TC_STAGES;
+          mbar_wait(smem_u32(&bars->v_full[s]), (kv_it / TC_STAGES) & 1, abort_flag, status, TC_ERR_MMA);
+          // the first P V of an item overwrites O: both warpgroups read both O slots in the previous epilogue
+          if (j == 0 && n_done > 0) {
+            mbar_wait(smem_u32(&bars->o_free[0]), (n_done - 1) & 1, abort_flag, status, TC_ERR_MMA);
+            mbar_wait(smem_u32(&bars->o_free[1]), (n_done - 1) & 1, abort_flag, status, TC_ERR_MMA);
+          }
+          mbar_wait(smem_u32(&bars->p_half[i][0]), n_p[i] & 1, abort_flag, status, TC_ERR_MMA);
+          tc_fence_after();
+          issue_pv(i, s, 0, j >= 2);
+          mbar_wait(smem_u32(&bars->p_half[i][1]), n_p[i] & 1, abort_flag, status, TC_ERR_MMA);
+          tc_fence_after();
+          issue_pv(i, s, 1, true);
+          ++n_p[i];
+          umma_commit(smem_u32(&bars->pv_done[i]));
+          umma_commit(smem_u32(&bars->v_empty[s]));
+          if (j + 2 < w.n_kv) qk_of(j + 2);                          // into the slot this P V has just read
+        }
+        ++n_done;
+      }
+      // everything this thread issued has completed once `drained` flips
+      umma_commit(smem_u32(&bars->drained));
+      mbar_wait(smem_u32(&bars->drained), 0, abort_flag, status, TC_ERR_MMA);
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ softmax + epilogue
+    setmaxnreg_inc<TC_REGS_SOFTMAX>();
+    const int i = (warp - 4) >> 2;                                   // TMEM slot of this warpgroup
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + lane_off + i * TC_BN, tO = tmem + lane_off + 256 + i * TC_D;
+    const float c = scale * 1.4426950408889634f;                     // logits -> log2 domain
+    const int r = (warp & 3) * 32 + lane;                            // row of the query tile
+    uint32_t n_s[2] = {0, 0};                                        // key tiles each slot has been through
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+      WinItem w;
+      if (!win_item1(g, item, tiles, w)) continue;
+      const int n_kv = w.n_kv, lo = w.lo, hi = w.hi;
+      const int cnt0 = (n_kv + 1) >> 1, cnt1 = n_kv >> 1, cnt = i == 0 ? cnt0 : cnt1;   // this slot: tiles i, i+2, ...
+      float m_true = -INFINITY, m_used = -INFINITY;
+      uint64_t l2a = 0ull, l2b = 0ull;                               // four partial row sums as two fp32 pairs
+      for (int t = 0; t < cnt; ++t) {
+        const int j = i + 2 * t;
+        mbar_wait(smem_u32(&bars->s_ready[i]), (n_s[i] + t) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+        tc_fence_after();
+        uint32_t sr[4][32];
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) tmem_ld32(tS + cc * 32, sr[cc]);
+        tmem_wait_ld();
+        const int n_valid = hi - (lo + j * TC_BN);                   // >= 1
+        if (n_valid < TC_BN) {
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (cc * 32 + e >= n_valid) sr[cc][e] = 0xff800000u;   // -inf
+        }
+        // row maximum: four independent chains of three-input max
+        float mx[4] = {m_true, m_true, m_true, m_true};
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+          for (int e = 0; e < 32; e += 2)
+            mx[cc] = fmax3(mx[cc], __uint_as_float(sr[cc][e]), __uint_as_float(sr[cc][e + 1]));
+        m_true = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        const bool need = (m_true - m_used) * c > 8.f;               // true on the slot's first tile (m_used = -inf)
+        if (__any_sync(0xffffffffu, need)) {
+          const float m_new = need ? m_true : m_used;
+          if (t > 0) {
+            // s_ready follows the completion of P V of this slot's previous tile, so O may be touched
+            mbar_wait(smem_u32(&bars->pv_done[i]), (n_s[i] + t - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+            tc_fence_after();
+            const float f = ex2((m_used - m_new) * c);               // 1 for lanes that keep their reference
+            const uint64_t f2 = pk2(f, f);
+            l2a = mul2(l2a, f2);
+            l2b = mul2(l2b, f2);
+#pragma unroll 1
+            for (int cc = 0; cc < TC_D / 8; ++cc) {                   // rare: small pieces keep the register peak low
+              uint32_t o[8];
+              tmem_ld8(tO + cc * 8, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
+              tmem_st8(tO + cc * 8, o);
+            }
+          }
+          m_used = m_new;
+        }
+        const float mc = -m_used * c;
+        const uint64_t c2 = pk2(c, c), mc2 = pk2(mc, mc);
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            float t0, t1, p0, p1;
+            upk2(fma2(pk2u(sr[cc][e], sr[cc][e + 1]), c2, mc2), t0, t1);
+            if (((e >> 1) & 3) < EMU) {                              // EMU of every 4 pairs on the FMA pipe
+              ex2_poly2(t0, t1, p0, p1);
+            } else {
+              p0 = ex2(t0);
+              p1 = ex2(t1);
+            }
+            if ((e >> 1) & 1) l2b = add2(l2b, pk2(p0, p1)); else l2a = add2(l2a, pk2(p0, p1));
+            sr[cc >> 1][(cc & 1) * 16 + (e >> 1)] = pack_bf16(p0, p1);
+          }
+          if (cc & 1) {
+            tmem_st32(tS + (cc >> 1) * 32, sr[cc >> 1]);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars->p_half[i][cc >> 1]));       // P of 64 keys is in place
+          }
+        }
+      }
+      float la0, la1, lb0, lb1;
+      upk2(l2a, la0, la1);
+      upk2(l2b, lb0, lb1);
+      const float l = (la0 + la1) + (lb0 + lb1);
+
+      // Exchange the slots' maxima and row sums (a slot without key tiles contributes m = -inf, l = 0).
+      bars->mrg[i][0][r] = m_used; bars->mrg[i][1][r] = m_true; bars->mrg[i][2][r] = l;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      const float mu_x = bars->mrg[i ^ 1][0][r], mt_x = bars->mrg[i ^ 1][1][r], l_x = bars->mrg[i ^ 1][2][r];
+      const float m_fin = fmaxf(m_true, mt_x);
+      const float mu0 = i == 0 ? m_used : mu_x, mu1 = i == 0 ? mu_x : m_used;
+      const float l0 = i == 0 ? l : l_x, l1 = i == 0 ? l_x : l;
+      const int row = w.row_base + r;
+      const bool valid = row < w.q1;
+      // this warpgroup's half of the read-out row is requested before the wait for the last P V
+      float4 rdv[TC_D / 8];
+      float nL = 0.f;
+      if (w.linear) {
+        const int ric = (valid ? row : w.q0) - w.q0, ci = w.ci;
+#pragma unroll
+        for (int u = 0; u < TC_D / 8; ++u)
+          rdv[u] = __ldg(reinterpret_cast<const float4*>(rd + rd_index(g, rd_rows, TC_D, w.bh, ci, ric, i * (TC_D / 8) + u)));
+        nL = __ldg(rd + rd_index(g, rd_rows, TC_D, w.bh, ci, ric, TC_D / 4));
+      } else {
+#pragma unroll
+        for (int u = 0; u < TC_D / 8; ++u) rdv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+      float f0 = ex2((mu0 - m_fin) * c), f1 = cnt1 > 0 ? ex2((mu1 - m_fin) * c) : 0.f, lam = 0.f;
+      if (w.linear) {
+        lam = 1.f;
+        if (c_mode == C_ZERO) {
+          const float mm = m_fin * scale, rr = fmaxf(mm, 0.f), e = __expf(mm - rr);
+          f0 *= e; f1 *= e;
+          lam = __expf(-rr);
+        }
+      }
+      __nv_bfloat16* orow = out + head_offset(g, w.bh) + (long long)row * g.stride_n + i * (TC_D / 2);
+      mbar_wait(smem_u32(&bars->pv_done[0]), (n_s[0] + cnt0 - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+      if (cnt1 > 0) mbar_wait(smem_u32(&bars->pv_done[1]), (n_s[1] + cnt1 - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+      tc_fence_after();
+      n_s[0] += cnt0; n_s[1] += cnt1;
+      const float inv = 1.f / (l0 * f0 + l1 * f1 + lam * nL);
+      const float w0 = f0 * inv, w1 = f1 * inv, lami = lam * inv;
+      const uint32_t tO0 = tmem + lane_off + 256 + i * (TC_D / 2);
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {                               // 32 columns at a time
+        uint32_t o0[32], o1[32];
+        tmem_ld32(tO0 + hh * 32, o0);
+        if (cnt1 > 0) {
+          tmem_ld32(tO0 + TC_D + hh * 32, o1);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o1[e] = 0u;                   // slot 1 was not used
+        }
+        tmem_wait_ld();
+        if (hh == 1) {                                               // this warpgroup has read both slots
+          tc_fence_before();
+          mbar_arrive(smem_u32(&bars->o_free[i]));
+        }
+        if (valid) {
+#pragma unroll
+          for (int e = 0; e < 32; e += 8) {
+            const float4 x0 = rdv[hh * 8 + (e >> 2)], x1 = rdv[hh * 8 + (e >> 2) + 1];
+            auto fin = [&](int q, float x) { return __uint_as_float(o0[q]) * w0 + __uint_as_float(o1[q]) * w1 + lami * x; };
+            uint4 v4;
+            v4.x = pack_bf16(fin(e + 0, x0.x), fin(e + 1, x0.y));
+            v4.y = pack_bf16(fin(e + 2, x0.z), fin(e + 3, x0.w));
+            v4.z = pack_bf16(fin(e + 4, x1.x), fin(e + 5, x1.y));
+            v4.w = pack_bf16(fin(e + 6, x1.z), fin(e + 7, x1.w));
+            *reinterpret_cast<uint4*>(orow + hh * 32 + e) = v4;
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// Launches window_tc1 with the tensor maps and arguments tc_launch_window has prepared.
+inline int tc_launch_window1(int exp_poly, int n_sm, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                             __nv_bfloat16* o, const Geo& g, const float* rd, int rd_rows, float scale, int c_mode,
+                             int* status, cudaStream_t st) {
+  const int tiles = (g.Np + TC_BM - 1) / TC_BM;
+  const int n_items = tiles * g.G * g.BH;
+  const dim3 grid(n_items < n_sm ? n_items : n_sm);
+#define REHYAT_LAUNCH_WINDOW1(E) \
+  window_tc1<E><<<grid, TC_THREADS, TC_WIN1_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status, n_items, tiles)
+  switch (exp_poly) {
+    case 0: REHYAT_LAUNCH_WINDOW1(0); break;
+    case 2: REHYAT_LAUNCH_WINDOW1(2); break;
+    case 3: REHYAT_LAUNCH_WINDOW1(3); break;
+    default: REHYAT_LAUNCH_WINDOW1(1); break;
+  }
+#undef REHYAT_LAUNCH_WINDOW1
+  return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
+}
+
+inline bool tc_set_attributes1() {
+  return cudaFuncSetAttribute(window_tc1<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN1_SMEM) == cudaSuccess &&
+         cudaFuncSetAttribute(window_tc1<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN1_SMEM) == cudaSuccess &&
+         cudaFuncSetAttribute(window_tc1<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN1_SMEM) == cudaSuccess &&
+         cudaFuncSetAttribute(window_tc1<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN1_SMEM) == cudaSuccess;
+}
+
+}  // namespace rehyat

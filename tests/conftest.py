@@ -20,3 +20,12 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(params=["1", "2"], ids=["one_tile_items", "two_tile_items"])
+def both_window_kernels(request, monkeypatch):
+    """The softmax window has two kernels, picked per launch from the number of work items: window_tc (two
+    query tiles per item) and window_tc1 (one).  Small test shapes would all land on the second; this fixture
+    runs a test once with each (REHYAT_WINDOW_TILES is read when a context is created)."""
+    monkeypatch.setenv("REHYAT_WINDOW_TILES", request.param)
+    return request.param

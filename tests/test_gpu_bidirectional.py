@@ -7,7 +7,7 @@ import torch
 from oracle import rehyat_oracle as orc
 from paper_2601_04342_b200 import synth
 
-pytestmark = pytest.mark.gpu
+pytestmark = [pytest.mark.gpu, pytest.mark.usefixtures("both_window_kernels")]
 
 
 @pytest.fixture(scope="module", autouse=True)

@@ -13,7 +13,7 @@ import torch
 from oracle import rehyat_oracle as orc
 from paper_2601_04342_b200 import synth
 
-pytestmark = pytest.mark.gpu
+pytestmark = [pytest.mark.gpu, pytest.mark.usefixtures("both_window_kernels")]
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -275,3 +275,17 @@ def test_every_share_of_polynomial_exponentials(n_poly, monkeypatch):
         y, used = run_gpu(wl, x)
         assert used == "tensor"
         check(y, ref, "bf16")
+
+
+def test_window_items_of_one_tile_edge_shapes():
+    """Shapes that matter to window_tc1, where the key tiles of one query tile alternate between the two TMEM
+    slots and the epilogue merges the two partial softmax results (Eq. 5 with the window split in two): windows
+    of one key tile (the second slot stays empty), of an odd and of an even number of tiles, both c modes."""
+    for name, args in (("a", (1, 2, 128, 6, 10, 20, 2, 1)), ("b", (2, 3, 128, 5, 9, 13, 1, 0)), ("c", (1, 2, 128, 3, 5, 7, 3, 2))):
+        wl = synth.Workload("tiles_" + name, *args, "bf16", True, seed=synth.BASE_SEED + 91)
+        for c_mode in ("rowmax", "zero"):
+            x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
+            ref, _ = oracle_full(wl, x, c_mode=c_mode)
+            y, used = run_gpu(wl, x, c_mode=c_mode)
+            assert used == "tensor"
+            check(y, ref, "bf16")
