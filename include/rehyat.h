@@ -20,7 +20,9 @@
  *   - Unless a parameter says "host", tensor pointers are DEVICE pointers owned by the caller,
  *     16-byte aligned, and `out` must not alias an input.
  *   - rehyat_forward only enqueues work on the given stream: no host synchronisation and no
- *     allocation.  A context serves one stream at a time (it owns the workspace).
+ *     allocation, in the causal and in the bidirectional form.  A context serves one stream at a
+ *     time (it owns the workspace).  The library keeps no process-wide state and reads no
+ *     environment variable.
  *   - There is no CPU fallback: on a machine without an sm_100 device rehyat_create fails.
  */
 #ifndef REHYAT_H
@@ -86,10 +88,22 @@ typedef struct rehyat_config {
                                    window (Eq. 13), the recurrent form.  1: TL_t = every token
                                    outside the window, earlier AND later (Eq. 10-12), the form
                                    the paper distils first.  Not a recurrence: rehyat_forward
-                                   then keeps one state per latent frame ((frames+1) x 132 KB per
-                                   (batch, head) at d=128, D'=256), allocated by the first call
-                                   that needs them and kept; rehyat_stream_* and
-                                   rehyat_forward_static refuse it (REHYAT_ERR_UNSUPPORTED).    */
+                                   then keeps one state per latent frame ((max_frames+1) x 132 KB
+                                   per (batch, head) at d=128, D'=256), allocated by
+                                   rehyat_create; rehyat_stream_* and rehyat_forward_static
+                                   refuse it (REHYAT_ERR_UNSUPPORTED).                         */
+  int32_t max_frames;           /* bidirectional = 1 only: largest `frames` a forward call may
+                                   pass (>= 1).  Ignored, and may be 0, in the causal form,
+                                   whose memory does not depend on the video length.          */
+  int32_t exp_poly;             /* tensor-core window kernel: of every four pairs of softmax
+                                   exponentials, how many are evaluated as a cubic on the FMA
+                                   pipe instead of the special-function unit.  0 = the
+                                   library's choice (1, the fastest measured on B200), 1..3 =
+                                   that many, -1 = none.  Results agree within bf16 rounding. */
+  int32_t window_tiles;         /* tensor-core window kernel: 128-row query tiles per work
+                                   item.  0 = chosen per launch from how many items there are
+                                   for the SMs; 1 or 2 fixes it (same results up to the order
+                                   of fp32 sums).                                              */
 } rehyat_config;
 
 /* Element strides of q, k, v and out (all four share them); the head_dim axis is contiguous.
@@ -113,13 +127,9 @@ typedef struct rehyat_ctx rehyat_ctx;
 /* Creates a context on cfg->device and allocates its fixed workspace (chunk states, partial
  * state sums, the linear read-out of one chunk group, a status word).  The workspace size is a
  * function of the config only (Section 3.3, note 3: memory constant in the video length).
- * Errors: INVALID_ARG (null, sizes out of range), UNSUPPORTED, ARCH, CUDA, ALLOC.
- * Tuning: the environment variable REHYAT_EXP_POLY = 0..3, read here, sets how many of every four pairs of
- * softmax exponentials the tensor-core window kernel evaluates as a cubic on the FMA pipe instead of the
- * special-function unit (default 1, the fastest measured on B200; the results agree within bf16 rounding).
- * REHYAT_WINDOW_TILES = 1 or 2, read here, fixes the number of 128-row query tiles per work item of that
- * kernel (default: chosen per launch from how many items there are for the SMs; same results up to the order
- * of fp32 sums). */
+ * In the bidirectional form it also allocates the per-frame states for max_frames frames.
+ * Nothing is read from the environment: every tuning knob is a field of the config.
+ * Errors: INVALID_ARG (null, sizes out of range), UNSUPPORTED, ARCH, CUDA, ALLOC. */
 int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg);
 
 /* Enqueues the operator of Eq. 5-9 with the causal sets of Eq. 13 on `cuda_stream`
@@ -212,8 +222,19 @@ int rehyat_destroy(rehyat_ctx* ctx);
 size_t rehyat_workspace_bytes(const rehyat_ctx* ctx);
 
 /* Synchronises `cuda_stream`, reads the device status word and clears it.  Returns REHYAT_OK,
- * REHYAT_ERR_DEVICE_TIMEOUT or REHYAT_ERR_CUDA. */
+ * REHYAT_ERR_DEVICE_TIMEOUT or REHYAT_ERR_CUDA.
+ * Every wait inside the tensor-core kernels (on an mbarrier: for a TMA load, a tcgen05.mma, another
+ * role of the CTA) is bounded in wall time.  A wait that runs out makes its CTA stop issuing work,
+ * wait for what it has already put in flight, free its TMEM and return; the other CTAs of the same
+ * launch follow at their next wait.  The output of that launch is then undefined, the status word
+ * records the time-out until it is read here, and later launches are not affected. */
 int rehyat_status(rehyat_ctx* ctx, void* cuda_stream);
+
+/* Sets the bound of those waits for the launches that follow: wait_limit_us microseconds
+ * (0 = the default of one second).  withhold_loads is a test hook, 0 in production: non-zero makes
+ * the producers of the tensor-core kernels issue no loads at all, so that every launch runs into
+ * the bound with nothing in flight - the way to exercise the time-out path without a fault. */
+int rehyat_set_wait_limit(rehyat_ctx* ctx, int32_t wait_limit_us, int32_t withhold_loads);
 
 /* Number of kernel launches the last rehyat_forward on this context enqueued. */
 int rehyat_last_launches(const rehyat_ctx* ctx);

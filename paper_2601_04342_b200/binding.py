@@ -21,7 +21,7 @@ EXPORTS = ["rehyat_create", "rehyat_forward", "rehyat_forward_host", "rehyat_for
            "rehyat_static_scratch_bytes", "rehyat_destroy",
            "rehyat_stream_begin", "rehyat_stream_step", "rehyat_stream_state_bytes", "rehyat_stream_export",
            "rehyat_stream_import",
-           "rehyat_workspace_bytes", "rehyat_status", "rehyat_last_launches", "rehyat_last_impl",
+           "rehyat_workspace_bytes", "rehyat_status", "rehyat_set_wait_limit", "rehyat_last_launches", "rehyat_last_impl",
            "rehyat_profile_enable", "rehyat_profile_read", "rehyat_strerror", "rehyat_version"]
 PROF_KINDS = ("state", "scan", "readout", "window")
 
@@ -30,7 +30,11 @@ class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "device", "dtype", "n_heads", "head_dim", "phi_hidden", "phi_dim", "poly_degree", "act_hidden",
         "act_out", "c_mode", "impl", "max_batch", "max_tokens_per_frame", "max_chunk_frames", "group_tokens",
-        "bidirectional")]
+        "bidirectional", "max_frames", "exp_poly", "window_tiles")]
+
+
+# Values of the tuning fields of rehyat_config that a Rehyat(...) call does not name (0 = the library's choice).
+TUNING_DEFAULTS = {"exp_poly": 0, "window_tiles": 0}
 
 
 class Layout(C.Structure):
@@ -72,6 +76,7 @@ def lib():
         L.rehyat_workspace_bytes.argtypes = [C.c_void_p]
         L.rehyat_workspace_bytes.restype = C.c_size_t
         L.rehyat_status.argtypes = [C.c_void_p, C.c_void_p]
+        L.rehyat_set_wait_limit.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
         L.rehyat_last_launches.argtypes = [C.c_void_p]
         L.rehyat_last_impl.argtypes = [C.c_void_p]
         L.rehyat_profile_enable.argtypes = [C.c_void_p, C.c_int]
@@ -105,11 +110,16 @@ class Rehyat:
 
     def __init__(self, *, n_heads, head_dim, dtype="bf16", phi_hidden=None, phi_dim=None, poly_degree=2,
                  act_hidden="relu", act_out="relu", c_mode="rowmax", impl="auto", max_batch=1,
-                 max_tokens_per_frame=1560, max_chunk_frames=3, group_tokens=0, device=0, bidirectional=False):
+                 max_tokens_per_frame=1560, max_chunk_frames=3, group_tokens=0, device=0, bidirectional=False,
+                 max_frames=0, **tuning):
+        unknown = set(tuning) - set(TUNING_DEFAULTS)
+        if unknown:
+            raise TypeError(f"unknown arguments {sorted(unknown)}")
+        tune = {**TUNING_DEFAULTS, **tuning}
         self.cfg = Config(device, DTYPE[dtype], n_heads, head_dim, phi_hidden or 2 * head_dim,
                           phi_dim or 2 * head_dim, poly_degree, ACT[act_hidden], ACT[act_out], C_MODE[c_mode],
                           IMPL[impl], max_batch, max_tokens_per_frame, max_chunk_frames, group_tokens,
-                          int(bool(bidirectional)))
+                          int(bool(bidirectional)), max_frames, int(tune["exp_poly"]), int(tune["window_tiles"]))
         self.dtype = dtype
         self._h = C.c_void_p(None)
         _check(lib().rehyat_create(C.byref(self._h), C.byref(self.cfg)), "rehyat_create")
@@ -215,6 +225,9 @@ class Rehyat:
         _check(lib().rehyat_profile_read(self._h, ms, n), "rehyat_profile_read")
         return {k: (ms[i], n[i]) for i, k in enumerate(PROF_KINDS)}
 
+    def set_wait_limit(self, wait_limit_us=0, withhold_loads=False):
+        _check(lib().rehyat_set_wait_limit(self._h, int(wait_limit_us), int(bool(withhold_loads))), "rehyat_set_wait_limit")
+
     def status(self, stream=None):
         st = stream if stream is not None else torch.cuda.current_stream(self.cfg.device)
         return lib().rehyat_status(self._h, C.c_void_p(st.cuda_stream))
@@ -244,6 +257,7 @@ def forward_static(q, k, v, phi_q, phi_k, frames, H, W, chunk, overlap, *, dtype
 def for_workload(wl, **kw):
     """A context sized for a synth.Workload."""
     args = dict(n_heads=wl.n_heads, head_dim=wl.head_dim, dtype=wl.dtype, phi_hidden=wl.D_h, phi_dim=wl.D_out,
-                poly_degree=wl.P, max_batch=wl.B, max_tokens_per_frame=wl.HW, max_chunk_frames=min(wl.Tc, wl.T))
+                poly_degree=wl.P, max_batch=wl.B, max_tokens_per_frame=wl.HW, max_chunk_frames=min(wl.Tc, wl.T),
+                max_frames=wl.T)
     args.update(kw)
     return Rehyat(**args)

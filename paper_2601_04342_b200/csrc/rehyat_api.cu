@@ -63,6 +63,9 @@ struct rehyat_ctx {
   int head_count = 0;          // > 0: rehyat_forward works on this many heads (pointers already offset to the first)
   int last_launches = 0, last_impl = 0;
   bool tensor_ok = false;
+  int epoch = 0;               // number of the last tensor-core launch, 1, 2, ... (see ptx::WaitCtx)
+  unsigned wait_limit_us = 1000000u;   // bound of every device-side wait
+  int withhold_loads = 0;      // test hook of rehyat_set_wait_limit
   // chunk-by-chunk processing (rehyat_stream_*): the running state lives in slot 0 of `state`, the last
   // `overlap` frames of k and v and the chunk being processed in staging buffers [BH][cap_tokens][d]
   struct Stream {
@@ -111,20 +114,42 @@ int check_config(const rehyat_config* c) {
   if ((long long)c->max_tokens_per_frame * c->max_chunk_frames > (1 << 24)) return REHYAT_ERR_INVALID_ARG;
   if (c->head_dim < 1) return REHYAT_ERR_INVALID_ARG;
   if (c->bidirectional != 0 && c->bidirectional != 1) return REHYAT_ERR_INVALID_ARG;
+  if (c->max_frames < 0 || c->max_frames > (1 << 20) || (c->bidirectional && c->max_frames < 1)) return REHYAT_ERR_INVALID_ARG;
+  if (c->exp_poly < -1 || c->exp_poly > 3) return REHYAT_ERR_INVALID_ARG;
+  if (c->window_tiles < 0 || c->window_tiles > 2) return REHYAT_ERR_INVALID_ARG;
   if (c->head_dim != 64 && c->head_dim != 128) return REHYAT_ERR_UNSUPPORTED;
   return REHYAT_OK;
 }
 
+// The shared-memory limit of a kernel is a property of the function, not of a context, so it is always set to
+// what the widest phi check_config admits (D_h = D' = 256) needs: a later context with narrower widths then
+// cannot lower it under a live one.
 template <typename T, int D>
-int set_simt_attributes(const rehyat_config& c) {
-  const int smem_state = SIMT_TM * (2 * D + c.phi_hidden + c.phi_dim) * (int)sizeof(float);
-  const int smem_rd = SIMT_TM * (D + c.phi_hidden + c.phi_dim) * (int)sizeof(float);
+int set_simt_attributes() {
+  const int smem_state = SIMT_TM * (2 * D + 256 + 256) * (int)sizeof(float);
+  const int smem_rd = SIMT_TM * (D + 256 + 256) * (int)sizeof(float);
   const int smem_win = (WIN_BM * (D + 4) + WIN_BN * (D + 4) + WIN_BN * D + WIN_BM * (WIN_BN + 4)) * (int)sizeof(float);
   if (cudaFuncSetAttribute(state_partial_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_state) != cudaSuccess ||
       cudaFuncSetAttribute(readout_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_rd) != cudaSuccess ||
       cudaFuncSetAttribute(window_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_win) != cudaSuccess)
     return REHYAT_ERR_CUDA;
   return REHYAT_OK;
+}
+
+int set_simt_attributes_for(int dtype, int head_dim) {
+  if (dtype == REHYAT_DTYPE_FP32) return head_dim == 64 ? set_simt_attributes<float, 64>() : set_simt_attributes<float, 128>();
+  return head_dim == 64 ? set_simt_attributes<__nv_bfloat16, 64>() : set_simt_attributes<__nv_bfloat16, 128>();
+}
+
+// What every tensor-core launch is told about waiting: a fresh epoch per launch, the limit of one wait.
+ptx::WaitArgs next_wait(rehyat_ctx* ctx) {
+  ctx->epoch = ctx->epoch == INT_MAX ? 1 : ctx->epoch + 1;
+  ptx::WaitArgs wa;
+  wa.status = ctx->status_dev;
+  wa.epoch = ctx->epoch;
+  wa.limit_us = ctx->wait_limit_us;
+  wa.withhold_loads = ctx->withhold_loads;
+  return wa;
 }
 
 // Which steps of a chunk group to enqueue.
@@ -208,7 +233,7 @@ int run_parts(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void
       if (parts & PART_STATE) {
         ctx->prof.begin(REHYAT_PROF_STATE, st);
         rc = tc_launch_state(&ctx->tc, k, v, phi, g, batch, c.poly_degree, c.act_hidden, c.act_out, n_split,
-                             ctx->partial, ctx->status_dev, st);
+                             ctx->partial, next_wait(ctx), st);
         ctx->prof.end(REHYAT_PROF_STATE, st);
         const size_t per_slot = (size_t)g.BH * c.phi_dim * (c.head_dim + 4);
         ctx->prof.begin(REHYAT_PROF_SCAN, st);
@@ -220,14 +245,14 @@ int run_parts(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void
       if (rc == REHYAT_OK && (parts & PART_READOUT)) {
         ctx->prof.begin(REHYAT_PROF_READOUT, st);
         rc = tc_launch_readout(&ctx->tc, q, phi, g, batch, c.poly_degree, c.act_hidden, c.act_out, ctx->state,
-                               ctx->readout, ctx->rd_cap, ctx->status_dev, st);
+                               ctx->readout, ctx->rd_cap, next_wait(ctx), st);
         ctx->prof.end(REHYAT_PROF_READOUT, st);
         ctx->last_launches += 1;
       }
     }
     if (rc == REHYAT_OK && (parts & PART_WINDOW)) {
       ctx->prof.begin(REHYAT_PROF_WINDOW, st);
-      rc = tc_launch_window(&ctx->tc, q, k, v, out, g, batch, ctx->readout, ctx->rd_cap, c.c_mode, ctx->status_dev, st);
+      rc = tc_launch_window(&ctx->tc, q, k, v, out, g, batch, ctx->readout, ctx->rd_cap, c.c_mode, next_wait(ctx), st);
       ctx->prof.end(REHYAT_PROF_WINDOW, st);
       ctx->last_launches += 1;
     }
@@ -242,6 +267,19 @@ int run_parts(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void
              : launch_group_simt<B, 128>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot, parts, st);
   }
   return rc;
+}
+
+// The size arguments of a forward call against the limits of the context (nothing is enqueued before this passes).
+int check_sizes(const rehyat_ctx* ctx, int batch, int frames, int H, int W, int chunk, int overlap) {
+  const rehyat_config& c = ctx->cfg;
+  if (batch < 1 || batch > c.max_batch || frames < 1 || H < 1 || W < 1 || chunk < 1 || overlap < 0)
+    return REHYAT_ERR_INVALID_ARG;
+  const long long HW = (long long)H * W;
+  if (HW > c.max_tokens_per_frame) return REHYAT_ERR_INVALID_ARG;
+  if (HW * frames > INT_MAX / 2) return REHYAT_ERR_INVALID_ARG;
+  if ((chunk < frames ? chunk : frames) > c.max_chunk_frames) return REHYAT_ERR_INVALID_ARG;   // one chunk covers everything beyond `frames`
+  if (c.bidirectional && frames + 1 > ctx->cum_frames) return REHYAT_ERR_INVALID_ARG;
+  return REHYAT_OK;
 }
 
 // Copies `rows` token rows of `row_bytes` bytes for each of BH (batch, head) problems between two strided
@@ -317,15 +355,16 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
   bool ok = cudaMalloc(&ctx->state, b_state) == cudaSuccess && cudaMalloc(&ctx->partial, b_partial) == cudaSuccess &&
             cudaMalloc(&ctx->readout, b_rd) == cudaSuccess && cudaMalloc(&ctx->status_dev, 256) == cudaSuccess;
   ctx->ws_bytes = b_state + b_partial + b_rd + 256;
+  if (ok && c.bidirectional) {
+    // Eq. 10-12 is not a recurrence: one running state per latent frame, sized here so that forward never allocates
+    const size_t b_cum = slot * ((size_t)c.max_frames + 1);
+    ok = cudaMalloc(&ctx->cum, b_cum) == cudaSuccess;
+    ctx->cum_frames = c.max_frames + 1;
+    ctx->ws_bytes += b_cum;
+  }
   cudaDeviceGetAttribute(&ctx->tc.n_sm, cudaDevAttrMultiProcessorCount, c.device);
-  if (const char* e = getenv("REHYAT_EXP_POLY")) {
-    const int n = atoi(e);
-    if (n >= 0 && n <= 3) ctx->tc.exp_poly = n;
-  }
-  if (const char* e = getenv("REHYAT_WINDOW_TILES")) {
-    const int n = atoi(e);
-    if (n == 1 || n == 2) ctx->tc.item_tiles = n;
-  }
+  ctx->tc.exp_poly = c.exp_poly == 0 ? 1 : (c.exp_poly < 0 ? 0 : c.exp_poly);
+  ctx->tc.item_tiles = c.window_tiles;
   if (ok && ctx->tensor_ok) {
     size_t extra = 0;
     ok = tc_workspace_create(&ctx->tc, ctx->bh_max, ctx->Gmax, c.head_dim, c.phi_dim, &extra);
@@ -334,10 +373,7 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
   if (!ok) { cudaGetLastError(); rehyat_destroy(ctx); return REHYAT_ERR_ALLOC; }
   if (cudaMemset(ctx->status_dev, 0, 256) != cudaSuccess) { rehyat_destroy(ctx); return REHYAT_ERR_CUDA; }
 
-  if (c.dtype == REHYAT_DTYPE_FP32)
-    rc = c.head_dim == 64 ? set_simt_attributes<float, 64>(c) : set_simt_attributes<float, 128>(c);
-  else
-    rc = c.head_dim == 64 ? set_simt_attributes<__nv_bfloat16, 64>(c) : set_simt_attributes<__nv_bfloat16, 128>(c);
+  rc = set_simt_attributes_for(c.dtype, c.head_dim);
   if (rc == REHYAT_OK && ctx->tensor_ok) rc = tc_set_attributes();
   if (rc != REHYAT_OK) { rehyat_destroy(ctx); return rc; }
   *out = ctx;
@@ -398,9 +434,17 @@ int rehyat_status(rehyat_ctx* ctx, void* cuda_stream) {
   if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
   if (cudaMemcpy(&word, ctx->status_dev, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return REHYAT_ERR_CUDA;
   if (word != 0) {
-    cudaMemset(ctx->status_dev, 0, 256);
+    // the sticky bits are cleared; launches after the one that timed out carry another epoch and are not affected
+    if (cudaMemset(ctx->status_dev, 0, 256) != cudaSuccess) return REHYAT_ERR_CUDA;
     return REHYAT_ERR_DEVICE_TIMEOUT;
   }
+  return REHYAT_OK;
+}
+
+int rehyat_set_wait_limit(rehyat_ctx* ctx, int32_t wait_limit_us, int32_t withhold_loads) {
+  if (!ctx || wait_limit_us < 0) return REHYAT_ERR_INVALID_ARG;
+  ctx->wait_limit_us = wait_limit_us > 0 ? (unsigned)wait_limit_us : 1000000u;
+  ctx->withhold_loads = withhold_loads != 0;
   return REHYAT_OK;
 }
 
@@ -409,14 +453,10 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
                    int32_t H, int32_t W, int32_t chunk, int32_t overlap, void* cuda_stream) {
   if (!ctx || !q || !k || !v || !out || !lay || !phi) return REHYAT_ERR_INVALID_ARG;
   const rehyat_config& c = ctx->cfg;
-  if (batch < 1 || batch > c.max_batch || frames < 1 || H < 1 || W < 1 || chunk < 1 || overlap < 0)
-    return REHYAT_ERR_INVALID_ARG;
+  if (const int bad = check_sizes(ctx, batch, frames, H, W, chunk, overlap)) return bad;
   const long long HW = (long long)H * W;
-  if (HW > c.max_tokens_per_frame) return REHYAT_ERR_INVALID_ARG;
   const long long N = HW * frames;
-  if (N > INT_MAX / 2) return REHYAT_ERR_INVALID_ARG;
   const int chunk_eff = chunk < frames ? chunk : frames;      // one chunk covers everything beyond that
-  if (chunk_eff > c.max_chunk_frames) return REHYAT_ERR_INVALID_ARG;
   const int overlap_eff = overlap < frames ? overlap : frames; // the window is clamped at token 0 anyway
   if (out == q || out == k || out == v) return REHYAT_ERR_INVALID_ARG;
   const void* ptrs[] = {q, k, v, out, phi->q_W1, phi->q_b1, phi->q_W2, phi->q_b2,
@@ -428,6 +468,10 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   for (long long s : strides)
     if (s < 0 || (s * (long long)es) % 16 != 0) return REHYAT_ERR_INVALID_ARG;
   if (lay->stride_token < c.head_dim) return REHYAT_ERR_INVALID_ARG;
+  const int heads_here = ctx->head_count > 0 ? ctx->head_count : c.n_heads;
+  // an axis of more than one element needs a stride that keeps its elements apart
+  if ((heads_here > 1 && lay->stride_head < c.head_dim) || (batch > 1 && lay->stride_batch < c.head_dim))
+    return REHYAT_ERR_INVALID_ARG;
 
   DeviceGuard guard(c.device);
   if (!guard.ok) return REHYAT_ERR_CUDA;
@@ -440,6 +484,9 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   g.n_heads = ctx->head_count > 0 ? ctx->head_count : c.n_heads;
   g.BH = batch * g.n_heads;
   g.stride_b = lay->stride_batch; g.stride_h = lay->stride_head; g.stride_n = lay->stride_token;
+  // the stride of a one-element axis is never used for addressing; tensor maps still want it non-zero
+  if (g.stride_h == 0) g.stride_h = g.stride_n * N;
+  if (g.stride_b == 0) g.stride_b = g.stride_h * g.n_heads;
   const int n_chunks = (frames + chunk_eff - 1) / chunk_eff;
   g.q_shift = 0;
   g.prefix = 0;
@@ -456,14 +503,6 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
     // Eq. 10-12: the linear set of a chunk is everything outside its window.  Pass 1 sums the state frame by
     // frame (running sums cum[0..frames]); pass 2 forms each chunk's state from three of those sums.
     const size_t per_slot = (size_t)g.BH * c.phi_dim * (c.head_dim + 4), slot_bytes = per_slot * sizeof(float);
-    if (frames + 1 > ctx->cum_frames) {
-      if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
-      cudaFree(ctx->cum);
-      ctx->cum = nullptr; ctx->cum_frames = 0;
-      const size_t full_slot = (size_t)ctx->bh_max * c.phi_dim * (c.head_dim + 4) * sizeof(float);
-      if (cudaMalloc(&ctx->cum, full_slot * (frames + 1)) != cudaSuccess) { cudaGetLastError(); return REHYAT_ERR_ALLOC; }
-      ctx->cum_frames = frames + 1;
-    }
     if (cudaMemsetAsync(ctx->cum, 0, slot_bytes, st) != cudaSuccess) return REHYAT_ERR_CUDA;
     Geo gs = g;
     gs.Np = (int)HW; gs.ToHW = 0;
@@ -509,10 +548,13 @@ int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host,
                         void* out_host, const rehyat_phi_params* phi, int32_t batch, int32_t frames, int32_t H,
                         int32_t W, int32_t chunk, int32_t overlap, void* cuda_stream) {
   if (!ctx || !q_host || !k_host || !v_host || !out_host || !phi) return REHYAT_ERR_INVALID_ARG;
-  if (batch < 1 || frames < 1 || H < 1 || W < 1) return REHYAT_ERR_INVALID_ARG;
+  // every argument is checked before the first copy is enqueued
+  if (const int bad = check_sizes(ctx, batch, frames, H, W, chunk, overlap)) return bad;
+  const void* pp[] = {phi->q_W1, phi->q_b1, phi->q_W2, phi->q_b2, phi->k_W1, phi->k_b1, phi->k_W2, phi->k_b2};
+  for (const void* p : pp)
+    if (!p || !aligned16(p)) return REHYAT_ERR_INVALID_ARG;
   const rehyat_config& c = ctx->cfg;
   const long long N = (long long)H * W * frames;
-  if (N > INT_MAX / 2 || batch > c.max_batch) return REHYAT_ERR_INVALID_ARG;
   const size_t bytes = (size_t)batch * c.n_heads * N * c.head_dim * elem_size(c.dtype);
   DeviceGuard guard(c.device);
   if (!guard.ok) return REHYAT_ERR_CUDA;
@@ -799,14 +841,26 @@ static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
 // address is looked up once per device (with that device current) and cached.
 constexpr int kMaxDevices = 64;
 static float* g_static_scratch_addr[kMaxDevices] = {};
+static unsigned g_static_attr_done[kMaxDevices] = {};     // bit (2*dtype + (head_dim == 128)): kernel attributes set
 static std::mutex g_static_scratch_mutex;
 
-static int static_scratch_address(int device, float** out) {
+// First call on a device (with that device current): checks that it exists and is an sm_100 part, looks up the
+// array's address and sets the attributes of the kernels this dtype / head_dim uses.  Later calls only read.
+static int static_device_setup(int device, int dtype, int head_dim, float** out) {
   std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
   if (!g_static_scratch_addr[device]) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { cudaGetLastError(); return REHYAT_ERR_CUDA; }
+    if (prop.major != 10) return REHYAT_ERR_ARCH;
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return REHYAT_ERR_CUDA; }
     g_static_scratch_addr[device] = static_cast<float*>(p);
+  }
+  const unsigned bit = 1u << (2 * (dtype == REHYAT_DTYPE_FP32 ? 1 : 0) + (head_dim == 128 ? 1 : 0));
+  if (!(g_static_attr_done[device] & bit)) {
+    const int rc = set_simt_attributes_for(dtype, head_dim);
+    if (rc != REHYAT_OK) { cudaGetLastError(); return rc; }
+    g_static_attr_done[device] |= bit;
   }
   *out = g_static_scratch_addr[device];
   return REHYAT_OK;
@@ -820,7 +874,9 @@ int rehyat_forward_static(const rehyat_config* cfg, const void* q, const void* k
   if (!cfg) return REHYAT_ERR_INVALID_ARG;
   int rc = check_config(cfg);
   if (rc != REHYAT_OK) return rc;
-  if (cfg->device < 0 || cfg->device >= kMaxDevices) return REHYAT_ERR_INVALID_ARG;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess) { cudaGetLastError(); return REHYAT_ERR_CUDA; }
+  if (cfg->device < 0 || cfg->device >= ndev || cfg->device >= kMaxDevices) return REHYAT_ERR_INVALID_ARG;
   if (cfg->bidirectional) return REHYAT_ERR_UNSUPPORTED;
   if (batch < 1 || frames < 1 || H < 1 || W < 1 || chunk < 1 || overlap < 0) return REHYAT_ERR_INVALID_ARG;
   const long long HW = (long long)H * W, N = HW * frames;
@@ -839,12 +895,7 @@ int rehyat_forward_static(const rehyat_config* cfg, const void* q, const void* k
   DeviceGuard guard(cfg->device);
   if (!guard.ok) return REHYAT_ERR_CUDA;
   float* base = nullptr;
-  rc = static_scratch_address(cfg->device, &base);
-  if (rc != REHYAT_OK) return rc;
-  if (cfg->dtype == REHYAT_DTYPE_FP32)
-    rc = cfg->head_dim == 64 ? set_simt_attributes<float, 64>(*cfg) : set_simt_attributes<float, 128>(*cfg);
-  else
-    rc = cfg->head_dim == 64 ? set_simt_attributes<__nv_bfloat16, 64>(*cfg) : set_simt_attributes<__nv_bfloat16, 128>(*cfg);
+  rc = static_device_setup(cfg->device, cfg->dtype, cfg->head_dim, &base);
   if (rc != REHYAT_OK) return rc;
 
   // A context on the stack that points into the static array; the SIMT kernels do the work.

@@ -45,8 +45,9 @@ struct PhBars {
   uint64_t x_full, x_empty, v_full, v_empty;
   uint64_t ring_full[PH_RING], ring_empty[PH_RING];
   uint64_t acc_ready, epi_done, out_ready;
+  uint64_t drained;            // every tcgen05.mma of the issuer has completed
   uint32_t tmem_base;
-  int abort_flag;
+  ptx::WaitCtx wctx;
 };
 
 struct PhiTcArgs {
@@ -59,7 +60,7 @@ struct PhiTcArgs {
   float* rd;                   // read-out kernel: the read-out workspace (see rd_index)
   int rd_rows;
   int tiles_per_cta;           // read-out kernel
-  int* status;
+  ptx::WaitArgs wa;            // status word, launch epoch, wait limit
 };
 
 // tm_x: K, tm_v: V, 4-D like the window kernel's maps.  tm_w1: (128, 256, heads), tm_w2: (256, 256, heads),
@@ -75,7 +76,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   PhBars* bars = reinterpret_cast<PhBars*>(smem + PH_OFF_BARS);
   float* s_b1 = reinterpret_cast<float*>(smem + PH_OFF_BIAS);
   float* s_b2 = s_b1 + 256;
-  volatile int* abort_flag = &bars->abort_flag;
+  const uint32_t wc = smem_u32(&bars->wctx);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
@@ -104,7 +105,8 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     }
     mbar_init(smem_u32(&bars->acc_ready), 1); mbar_init(smem_u32(&bars->epi_done), 256);
     mbar_init(smem_u32(&bars->out_ready), 1);
-    bars->abort_flag = 0;
+    mbar_init(smem_u32(&bars->drained), 1);
+    wait_ctx_init(&bars->wctx, a.wa);
     fence_mbar_init();
   }
   // biases as fp32; the ones tile: row 0 of both 64-column sub-tiles is 1, the rest 0
@@ -138,14 +140,14 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
 
   if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
-    if (elect_one()) {
+    if (elect_one() && !a.wa.withhold_loads) {
       prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_w1); prefetch_tensormap(&tm_w2);
-      uint32_t ring_i = 0;
+      uint32_t ring_i = 0, n_x = 0, n_v = 0;                       // ring tiles, X tiles and V tiles issued so far
       bool alive = true;
       auto ring_load = [&](const CUtensorMap* tm, int x, int y, int z) {
         const int s = ring_i % RING;
         const uint32_t ph = (ring_i / RING) & 1;
-        alive = alive && mbar_wait(smem_u32(&bars->ring_empty[s]), ph ^ 1, abort_flag, a.status, PH_ERR_LOAD);
+        alive = alive && mbar_wait(smem_u32(&bars->ring_empty[s]), ph ^ 1, wc, PH_ERR_LOAD);
         if (!alive) return;
         const uint32_t full = smem_u32(&bars->ring_full[s]);
         mbar_expect_tx(full, PH_WT_BYTES);
@@ -154,24 +156,35 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       };
       for (int j = 0; j < n_tiles && alive; ++j) {
         const int tok0 = tok_a + j * 128;
-        alive = mbar_wait(smem_u32(&bars->x_empty), (j & 1) ^ 1, abort_flag, a.status, PH_ERR_LOAD);
+        alive = mbar_wait(smem_u32(&bars->x_empty), (j & 1) ^ 1, wc, PH_ERR_LOAD);
         if (!alive) break;
         const uint32_t xf = smem_u32(&bars->x_full);
         mbar_expect_tx(xf, PH_TILE_BYTES);
         tma_load_4d(sX, &tm_x, xf, 0, tok0, h_idx, b_idx);
         tma_load_4d(sX + PH_SUB, &tm_x, xf, 64, tok0, h_idx, b_idx);
+        ++n_x;
         for (int nh = 0; nh < 2; ++nh)
           for (int ks = 0; ks < 2; ++ks) ring_load(&tm_w1, ks * 64, nh * 128, h_idx);
         {
-          alive = alive && mbar_wait(smem_u32(&bars->v_empty), (j & 1) ^ 1, abort_flag, a.status, PH_ERR_LOAD);
+          alive = alive && mbar_wait(smem_u32(&bars->v_empty), (j & 1) ^ 1, wc, PH_ERR_LOAD);
           if (!alive) break;
           const uint32_t vf = smem_u32(&bars->v_full);
           mbar_expect_tx(vf, PH_TILE_BYTES);
           tma_load_4d(sV, &tm_v, vf, 0, tok0, h_idx, b_idx);
           tma_load_4d(sV + PH_SUB, &tm_v, vf, 64, tok0, h_idx, b_idx);
+          ++n_v;
         }
         for (int ks = 0; ks < 4; ++ks) ring_load(&tm_w2, ks * 64, 0, h_idx);
         for (int ks = 0; ks < 4; ++ks) ring_load(&tm_w2, ks * 64, 128, h_idx);
+      }
+      if (!alive) {
+        // Given up: wait for the last load issued into every buffer before the CTA exits (the full barriers
+        // complete by byte count, whatever the consumers do).
+        if (n_x > 0) mbar_wait_drain(smem_u32(&bars->x_full), (n_x - 1) & 1, wc);
+        if (n_v > 0) mbar_wait_drain(smem_u32(&bars->v_full), (n_v - 1) & 1, wc);
+        for (uint32_t back = 0; back < (uint32_t)RING; ++back)
+          if (ring_i > back)
+            mbar_wait_drain(smem_u32(&bars->ring_full[(ring_i - 1 - back) % RING]), ((ring_i - 1 - back) / RING) & 1, wc);
       }
     }
   } else if (warp == 9) {
@@ -181,25 +194,24 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       constexpr uint32_t id_st = idesc_bf16(128, 128, 1, 1);       // A = phi^T (MN-major), B = V (MN-major)
       constexpr uint32_t id_z = idesc_bf16(128, 16, 1, 0);         // A = phi^T (MN-major), B = ones (K-major)
       uint32_t ring_i = 0, n_epi = 0;
-      auto ring_wait = [&]() -> uint32_t {
-        const int s = ring_i % RING;
-        mbar_wait(smem_u32(&bars->ring_full[s]), (ring_i / RING) & 1, abort_flag, a.status, PH_ERR_MMA);
-        tc_fence_after();
-        return ring_addr(s);
+      bool alive = true;                                            // false once a wait has been given up: issue nothing more
+      auto wait = [&](uint64_t* bar, uint32_t parity) {
+        alive = alive && mbar_wait(smem_u32(bar), parity, wc, PH_ERR_MMA);
+        if (alive) tc_fence_after();
+        return alive;
       };
       auto ring_release = [&]() {
         umma_commit(smem_u32(&bars->ring_empty[ring_i % RING]));
         ++ring_i;
       };
       auto wait_epi = [&]() {
-        mbar_wait(smem_u32(&bars->epi_done), n_epi & 1, abort_flag, a.status, PH_ERR_MMA);
-        ++n_epi;
-        tc_fence_after();
+        if (wait(&bars->epi_done, n_epi & 1)) ++n_epi;
       };
       // one 128x128 half of an MLP GEMM: A tile [128 x 64*nks] K-major at a_base, B tiles from the ring
       auto mlp_half = [&](uint32_t a_base, int nks) {
         for (int ks = 0; ks < nks; ++ks) {
-          const uint32_t bt = ring_wait();
+          if (!wait(&bars->ring_full[ring_i % RING], (ring_i / RING) & 1)) return;
+          const uint32_t bt = ring_addr(ring_i % RING);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
             umma_ss(tmem + T_SCR, smem_desc_sw128(a_base + ks * PH_SUB + kk * 32, 16, 1024),
@@ -210,6 +222,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       };
       // contraction that consumes phi half `c` (its tile is at phi_base)
       auto consume_half = [&](int c, uint32_t phi_base, bool first_tile) {
+        if (!alive) return;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {                            // 16 tokens per step
           const uint64_t ad = smem_desc_sw128(phi_base + kk * 2048, PH_SUB, 1024);
@@ -219,31 +232,35 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
                   (!first_tile || kk > 0) ? 1u : 0u);
         }
       };
-      for (int j = 0; j < n_tiles; ++j) {
-        mbar_wait(smem_u32(&bars->x_full), j & 1, abort_flag, a.status, PH_ERR_MMA);
-        tc_fence_after();
+      for (int j = 0; j < n_tiles && alive; ++j) {
+        if (!wait(&bars->x_full, j & 1)) break;
         if (j > 0) wait_epi();                                      // scratch free: phi half 1 of tile j-1 written
         if (j > 0) {                                                // ... and consumed
-          mbar_wait(smem_u32(&bars->v_full), (j - 1) & 1, abort_flag, a.status, PH_ERR_MMA);
-          tc_fence_after();
+          if (!wait(&bars->v_full, (j - 1) & 1)) break;
           consume_half(1, sHb, j == 1);
           umma_commit(smem_u32(&bars->v_empty));
         }
         mlp_half(sX, 2);                                            // H[:, 0:128]
         wait_epi();
         mlp_half(sX, 2);                                            // H[:, 128:256]
+        if (!alive) break;
         umma_commit(smem_u32(&bars->x_empty));
         wait_epi();
         mlp_half(sHb, 4);                                           // U[:, 0:128]
         wait_epi();
         mlp_half(sHb, 4);                                           // U[:, 128:256]
-        mbar_wait(smem_u32(&bars->v_full), j & 1, abort_flag, a.status, PH_ERR_MMA);
-        tc_fence_after();
+        if (!wait(&bars->v_full, j & 1)) break;
         consume_half(0, sPhi0, j == 0);
       }
       wait_epi();
-      consume_half(1, sHb, n_tiles == 1);
-      umma_commit(smem_u32(&bars->out_ready));
+      if (alive) {
+        consume_half(1, sHb, n_tiles == 1);
+        umma_commit(smem_u32(&bars->out_ready));
+      }
+      // Everything this thread has issued is complete once `drained` flips; the abort flag does not cut this
+      // wait short, so that TMEM is never freed with a tcgen05.mma still running.
+      umma_commit(smem_u32(&bars->drained));
+      mbar_wait_drain(smem_u32(&bars->drained), 0, wc);
     }
   } else {
     // ------------------------------------------------------------------ epilogues
@@ -254,11 +271,17 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     const uint32_t lane_off = (uint32_t)(qd * 32) << 16;
     uint32_t n_acc = 0;
     const int part_w = PH_DP / (PC ? PC : a.P);                     // a multiple of 32 (P in {1,2,4})
-    for (int j = 0; j < n_tiles; ++j) {
+    // A wait that was given up ends the role; the warp decides together (tcgen05.ld needs all 32 lanes).
+    bool alive = true;
+    auto wait = [&](uint64_t* bar, uint32_t parity) {
+      alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, wc, PH_ERR_EPI));
+      return alive;
+    };
+    for (int j = 0; j < n_tiles && alive; ++j) {
       const bool tok_valid = tok_a + j * 128 + r < tok_b;
 #pragma unroll
       for (int step = 0; step < 4; ++step) {                        // H half 0, H half 1, U half 0, U half 1
-        mbar_wait(smem_u32(&bars->acc_ready), n_acc & 1, abort_flag, a.status, PH_ERR_EPI);
+        if (!wait(&bars->acc_ready, n_acc & 1)) break;
         ++n_acc;
         tc_fence_after();
         const int half = step & 1;
@@ -319,9 +342,8 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
         mbar_arrive(smem_u32(&bars->epi_done));
       }
     }
-    {
+    if (alive && wait(&bars->out_ready, 0)) {
       // flush: lane r holds feature c*128 + r of half c; this thread writes its 64 columns
-      mbar_wait(smem_u32(&bars->out_ready), 0, abort_flag, a.status, PH_ERR_EPI);
       tc_fence_after();
       float* base = a.partial + (((size_t)ci * a.n_split + blockIdx.x) * g.BH + bh) * PH_DP * PH_SD;
 #pragma unroll

@@ -48,36 +48,73 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait.  `abort_flag` (shared memory) is set by whichever thread of the CTA first runs out
-// of patience; once set, every wait of the CTA returns at once so that all roles drain and the
-// kernel ends.  Returns false if the wait was given up.
-constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // one second of wall time per wait
+// Bounded waits.  Every spin on an mbarrier in the tensor-core kernels goes through mbar_wait: it gives up after
+// `limit_ns` of wall time, records `code` in the sticky status word status[0] and publishes the launch's epoch in
+// status[1], so that the other CTAs of the same launch stop at their next slow wait instead of each waiting
+// out the limit.  `abort_flag` makes the other roles of the CTA stop at once.  A role whose wait returns false
+// must not issue anything further (no TMA load, no tcgen05.mma, no barrier arrival it owes): it leaves its loops
+// and goes to the common exit of the kernel.  A later launch carries another epoch, so one timeout does not
+// poison the launches that follow; the sticky bits stay until the host reads them.
+// The context lives in the CTA's shared memory (set up by one thread before the first __syncthreads) and the
+// waits take its shared-memory address, so that it costs the hot loops no registers.
+struct WaitCtx {
+  int abort_flag;                  // set by whichever thread of the CTA first gives up
+  int epoch;                       // of this launch (never 0)
+  unsigned long long limit_ns;     // wall-time limit of one wait
+  int* status;                     // global: [0] sticky error bits, [1] epoch of a launch in which a CTA gave up
+};
+// What a kernel receives from the host about waiting (and, for the one test that makes a wait run out, the
+// switch that makes the TMA producer withhold every load so that nothing is ever in flight).
+struct WaitArgs {
+  int* status;
+  int epoch;
+  unsigned int limit_us;
+  int withhold_loads;
+};
+__device__ __forceinline__ void wait_ctx_init(WaitCtx* w, const WaitArgs& a) {
+  w->abort_flag = 0;
+  w->epoch = a.epoch;
+  w->limit_ns = (unsigned long long)a.limit_us * 1000ull;
+  w->status = a.status;
+}
 __device__ __forceinline__ unsigned long long global_timer_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                            int* status_word, int code) {
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t wctx, int code) {
+  volatile WaitCtx* w = reinterpret_cast<volatile WaitCtx*>(__cvta_shared_to_generic(wctx));
   const unsigned long long t0 = global_timer_ns();
   for (uint32_t i = 0;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
+    if (w->abort_flag) return false;
     if ((i & 63u) == 63u) {
-      // another CTA of the grid has already given up: drain at once instead of waiting a second each
-      if (*reinterpret_cast<volatile int*>(status_word) != 0) { *abort_flag = 1; return false; }
-      if (global_timer_ns() - t0 > kWaitLimitNs) break;
+      if (*reinterpret_cast<volatile int*>(w->status + 1) == w->epoch) { w->abort_flag = 1; return false; }
+      if (global_timer_ns() - t0 > w->limit_ns) break;
       __nanosleep(64);
     }
   }
-  *abort_flag = 1;
-  atomicOr(status_word, code);
+  w->abort_flag = 1;
+  atomicOr(w->status, code);
+  atomicExch(w->status + 1, w->epoch);
   return false;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status_word, int code) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t wctx, int code) {
   if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, status_word, code);
+  return mbar_wait_slow(bar, parity, wctx, code);
+}
+// Wait of a role for what it has itself put in flight (its TMA loads, its tcgen05.mma through a commit) before
+// the CTA may free TMEM and exit.  The abort flag does not cut it short; only the time limit does.
+__device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity, uint32_t wctx) {
+  const unsigned long long limit_ns = reinterpret_cast<volatile WaitCtx*>(__cvta_shared_to_generic(wctx))->limit_ns;
+  const unsigned long long t0 = global_timer_ns();
+  for (uint32_t i = 0;; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 63u) {
+      if (global_timer_ns() - t0 > limit_ns) return false;
+      __nanosleep(64);
+    }
+  }
 }
 
 // ----------------------------------------------------------------------------- TMA

@@ -26,16 +26,18 @@ constexpr int RD_OFF_X = 0;
 constexpr int RD_OFF_PHI0 = RD_OFF_X + PH_TILE_BYTES;
 constexpr int RD_OFF_PHI1 = RD_OFF_PHI0 + PH_TILE_BYTES;
 constexpr int RD_OFF_RING = RD_OFF_PHI1 + PH_TILE_BYTES;
-constexpr int RD_OFF_BIAS = RD_OFF_RING + RD_RING * RD_WT_BYTES;  // b1[256], b2[256], z[256], two partial phi.z sums per token
-constexpr int RD_OFF_BARS = RD_OFF_BIAS + 4 * 256 * 4;
+constexpr int RD_OFF_BIAS = RD_OFF_RING + RD_RING * RD_WT_BYTES;  // b1[256], b2[256], z[256], two partial phi.z sums per token (x2: by tile parity)
+constexpr int RD_OFF_BARS = RD_OFF_BIAS + 5 * 256 * 4;
 constexpr int RD_SMEM = RD_OFF_BARS + 512 + 1024;
 
 struct RdBars {
   uint64_t x_full, x_empty;
   uint64_t ring_full[RD_RING], ring_empty[RD_RING];
   uint64_t acc_ready[2], epi_done[2], out_ready, out_read;
+  uint64_t nl_ready;           // both halves of a tile's phi.z sums are in shared memory
+  uint64_t drained;            // every tcgen05.mma of the issuer has completed
   uint32_t tmem_base;
-  int abort_flag;
+  ptx::WaitCtx wctx;
 };
 
 // tm_x: Q, 4-D like the window kernel's maps.  tm_w1: (128, 256, heads), tm_w2: (256, 256, heads), boxes
@@ -54,7 +56,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
   float* s_b2 = s_b1 + 256;
   float* s_z = s_b2 + 256;
   float* s_nl = s_z + 256;
-  volatile int* abort_flag = &bars->abort_flag;
+  const uint32_t wc = smem_u32(&bars->wctx);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
@@ -73,7 +75,8 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
     }
     for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&bars->acc_ready[b]), 1); mbar_init(smem_u32(&bars->epi_done[b]), 256); }
     mbar_init(smem_u32(&bars->out_ready), 1); mbar_init(smem_u32(&bars->out_read), 256);
-    bars->abort_flag = 0;
+    mbar_init(smem_u32(&bars->nl_ready), 256); mbar_init(smem_u32(&bars->drained), 1);
+    wait_ctx_init(&bars->wctx, a.wa);
     fence_mbar_init();
   }
   for (int i = threadIdx.x; i < 256; i += PH_THREADS) {             // biases and z_t as fp32
@@ -94,38 +97,40 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
 
   if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
-    if (elect_one()) {
+    if (elect_one() && !a.wa.withhold_loads) {
       prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_w1); prefetch_tensormap(&tm_w2); prefetch_tensormap(&tm_s);
-      uint32_t ring_i = 0;
+      uint32_t ring_i = 0, n_x = 0;                                 // ring tiles and X tiles issued so far
       bool alive = true;
-      auto ring_slot = [&]() -> uint32_t {                          // waits for the next stage to be free; 0 on abort
+      auto ring_slot = [&](uint32_t& full) -> uint32_t {            // waits for the next stage to be free; 0 on abort
         const int s = ring_i % RD_RING;
-        alive = alive && mbar_wait(smem_u32(&bars->ring_empty[s]), ((ring_i / RD_RING) & 1) ^ 1, abort_flag, a.status, PH_ERR_LOAD);
+        alive = alive && mbar_wait(smem_u32(&bars->ring_empty[s]), ((ring_i / RD_RING) & 1) ^ 1, wc, PH_ERR_LOAD);
         if (!alive) return 0u;
-        mbar_expect_tx(smem_u32(&bars->ring_full[s]), RD_WT_BYTES);
+        full = smem_u32(&bars->ring_full[s]);
+        mbar_expect_tx(full, RD_WT_BYTES);
         ++ring_i;
         return sRing + s * RD_WT_BYTES;
       };
       auto weight_load = [&](const CUtensorMap* tm, int x, int y) {
-        const uint32_t full = smem_u32(&bars->ring_full[ring_i % RD_RING]);
-        const uint32_t dst = ring_slot();
+        uint32_t full = 0;
+        const uint32_t dst = ring_slot(full);
         if (dst) tma_load_3d(dst, tm, full, x, y, h_idx);
       };
       auto state_load = [&](int f) {                                // [64 features x 128 d] as two 64-column boxes
-        const uint32_t full = smem_u32(&bars->ring_full[ring_i % RD_RING]);
-        const uint32_t dst = ring_slot();
+        uint32_t full = 0;
+        const uint32_t dst = ring_slot(full);
         if (dst) {
           tma_load_3d(dst, &tm_s, full, 0, f * 64, ci * g.BH + bh);
           tma_load_3d(dst + 8192, &tm_s, full, 64, f * 64, ci * g.BH + bh);
         }
       };
       for (int j = 0; j < n_tiles && alive; ++j) {
-        alive = mbar_wait(smem_u32(&bars->x_empty), (j & 1) ^ 1, abort_flag, a.status, PH_ERR_LOAD);
+        alive = mbar_wait(smem_u32(&bars->x_empty), (j & 1) ^ 1, wc, PH_ERR_LOAD);
         if (!alive) break;
         const uint32_t xf = smem_u32(&bars->x_full);
         mbar_expect_tx(xf, PH_TILE_BYTES);
         tma_load_4d(sX, &tm_x, xf, 0, tok_a + j * 128, h_idx, b_idx);
         tma_load_4d(sX + PH_SUB, &tm_x, xf, 64, tok_a + j * 128, h_idx, b_idx);
+        ++n_x;
         // the ring follows the issue order of the MMAs: read-out of the previous tile between this tile's H halves
         for (int ks = 0; ks < 2; ++ks) weight_load(&tm_w1, ks * 64, 0);
         if (j > 0) { state_load(0); state_load(1); }
@@ -135,6 +140,14 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         for (int ks = 0; ks < 4; ++ks) weight_load(&tm_w2, ks * 64, 128);
       }
       for (int f = 0; f < 4 && alive; ++f) state_load(f);
+      if (!alive) {
+        // Given up: wait for the last load issued into every buffer before the CTA exits (the full barriers
+        // complete by byte count, whatever the consumers do).
+        if (n_x > 0) mbar_wait_drain(smem_u32(&bars->x_full), (n_x - 1) & 1, wc);
+        for (uint32_t back = 0; back < (uint32_t)RD_RING; ++back)
+          if (ring_i > back)
+            mbar_wait_drain(smem_u32(&bars->ring_full[(ring_i - 1 - back) % RD_RING]), ((ring_i - 1 - back) / RD_RING) & 1, wc);
+      }
     }
   } else if (warp == 9) {
     // ------------------------------------------------------------------ UMMA issuer
@@ -142,24 +155,27 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       constexpr uint32_t id_kk = idesc_bf16(128, 128, 0, 0);       // A K-major (smem or TMEM), B K-major: the MLP GEMMs
       constexpr uint32_t id_rd = idesc_bf16(128, 128, 0, 1);       // A = phi (K-major), B = state (MN-major)
       uint32_t ring_i = 0, n_epi[2] = {0, 0};
-      auto ring_wait = [&]() -> uint32_t {
+      bool alive = true;                                            // false once a wait has been given up: issue nothing more
+      auto wait = [&](uint64_t* bar, uint32_t parity) {
+        alive = alive && mbar_wait(smem_u32(bar), parity, wc, PH_ERR_MMA);
+        if (alive) tc_fence_after();
+        return alive;
+      };
+      auto ring_wait = [&]() -> uint32_t {                          // 0 on abort
         const int s = ring_i % RD_RING;
-        mbar_wait(smem_u32(&bars->ring_full[s]), (ring_i / RD_RING) & 1, abort_flag, a.status, PH_ERR_MMA);
-        tc_fence_after();
-        return sRing + s * RD_WT_BYTES;
+        return wait(&bars->ring_full[s], (ring_i / RD_RING) & 1) ? sRing + s * RD_WT_BYTES : 0u;
       };
       auto ring_release = [&]() {
         umma_commit(smem_u32(&bars->ring_empty[ring_i % RD_RING]));
         ++ring_i;
       };
       auto wait_epi = [&](int b) {                                  // the next epilogue that used scratch b is done
-        mbar_wait(smem_u32(&bars->epi_done[b]), n_epi[b] & 1, abort_flag, a.status, PH_ERR_MMA);
-        ++n_epi[b];
-        tc_fence_after();
+        if (wait(&bars->epi_done[b], n_epi[b] & 1)) ++n_epi[b];
       };
       auto h_half = [&](int b) {                                    // H[:, 128 b : 128 b + 128] = X W1[...]^T into scratch b
         for (int ks = 0; ks < 2; ++ks) {
           const uint32_t bt = ring_wait();
+          if (!bt) return;
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
             umma_ss(tmem + T_SCR + b * 128, smem_desc_sw128(sX + ks * PH_SUB + kk * 32, 16, 1024),
@@ -171,6 +187,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       auto u_half = [&](int b) {                                    // U[:, 128 b : ...] = H W2[...]^T with H read from TMEM
         for (int ks = 0; ks < 4; ++ks) {
           const uint32_t bt = ring_wait();
+          if (!bt) return;
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
             umma_ts(tmem + T_SCR + b * 128, tmem + T_H + (ks * 4 + kk) * 8, smem_desc_sw128(bt + kk * 32, 16, 1024), id_kk,
@@ -182,6 +199,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       auto readout_half = [&](int c, uint32_t phi_base) {           // R (+)= phi[:, 128 c : ...] s_t[128 c : ..., :]
         for (int f = 0; f < 2; ++f) {
           const uint32_t bt = ring_wait();
+          if (!bt) return;
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
             umma_ss(tmem + T_R, smem_desc_sw128(phi_base + f * PH_SUB + kk * 32, 16, 1024),
@@ -189,23 +207,21 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
           ring_release();
         }
       };
-      for (int j = 0; j < n_tiles; ++j) {
-        mbar_wait(smem_u32(&bars->x_full), j & 1, abort_flag, a.status, PH_ERR_MMA);
-        tc_fence_after();
+      for (int j = 0; j < n_tiles && alive; ++j) {
+        if (!wait(&bars->x_full, j & 1)) break;
         if (j > 0) wait_epi(0);                                     // U half 0 of tile j-1: scratch A free, phi half 0 written
         h_half(0);
         if (j > 0) {
-          if (j > 1) {                                              // the read-out of tile j-2 has left TMEM
-            mbar_wait(smem_u32(&bars->out_read), (j - 2) & 1, abort_flag, a.status, PH_ERR_MMA);
-            tc_fence_after();
-          }
+          if (j > 1 && !wait(&bars->out_read, (j - 2) & 1)) break;  // the read-out of tile j-2 has left TMEM
           readout_half(0, sPhi0);
           wait_epi(1);                                              // U half 1 of tile j-1
         }
         h_half(1);
+        if (!alive) break;
         umma_commit(smem_u32(&bars->x_empty));
         if (j > 0) {
           readout_half(1, sPhi1);
+          if (!alive) break;
           umma_commit(smem_u32(&bars->out_ready));
         }
         wait_epi(0);
@@ -214,14 +230,15 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         u_half(1);
       }
       wait_epi(0);
-      if (n_tiles > 1) {
-        mbar_wait(smem_u32(&bars->out_read), (n_tiles - 2) & 1, abort_flag, a.status, PH_ERR_MMA);
-        tc_fence_after();
-      }
+      if (n_tiles > 1) wait(&bars->out_read, (n_tiles - 2) & 1);
       readout_half(0, sPhi0);
       wait_epi(1);
       readout_half(1, sPhi1);
-      umma_commit(smem_u32(&bars->out_ready));
+      if (alive) umma_commit(smem_u32(&bars->out_ready));
+      // Everything this thread has issued is complete once `drained` flips; the abort flag does not cut this
+      // wait short, so that TMEM is never freed with a tcgen05.mma still running.
+      umma_commit(smem_u32(&bars->drained));
+      mbar_wait_drain(smem_u32(&bars->drained), 0, wc);
     }
   } else {
     // ------------------------------------------------------------------ epilogues
@@ -232,6 +249,12 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
     const uint32_t lane_off = (uint32_t)(qd * 32) << 16;
     uint32_t n_acc[2] = {0, 0};
     const int part_w = PH_DP / (PC ? PC : a.P);                     // a multiple of 32 (P in {1,2,4})
+    // A wait that was given up ends the role; the warp decides together (tcgen05.ld / st need all 32 lanes).
+    bool alive = true;
+    auto wait = [&](uint64_t* bar, uint32_t parity) {
+      alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, wc, PH_ERR_EPI));
+      return alive;
+    };
     // bias + activation (+ power) of 32 accumulator columns -> 16 bf16 pairs
     auto activate = [&](const uint32_t (&x)[32], const float* bias, bool is_u, int col0, uint32_t (&w)[16]) {
       if (RELU) {
@@ -266,9 +289,10 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       }
     };
     auto readout_store = [&](int jt) {                              // fp32 read-out of tile jt leaves TMEM
-      mbar_wait(smem_u32(&bars->out_ready), jt & 1, abort_flag, a.status, PH_ERR_EPI);
+      if (!alive || !wait(&bars->out_ready, jt & 1)) return;
       tc_fence_after();
-      asm volatile("bar.sync 1, 256;" ::: "memory");                 // both halves of s_nl are written
+      if (!wait(&bars->nl_ready, jt & 1)) return;                    // both halves of the tile's phi.z sums are written
+      const float* nlp = s_nl + (jt & 1) * 256;
       const bool tok_valid = tok_a + jt * 128 + r < tok_b;
       const int ric = tok_a + jt * 128 + r - q0;                    // row inside the chunk; its tile is 128-aligned
 #pragma unroll
@@ -284,17 +308,16 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
                             __uint_as_float(x[e + 3]));
         }
       }
-      if (tok_valid && ch == 1) a.rd[rd_index(g, a.rd_rows, PH_D, bh, ci, ric, PH_D / 4)] = s_nl[r] + s_nl[128 + r];
+      if (tok_valid && ch == 1) a.rd[rd_index(g, a.rd_rows, PH_D, bh, ci, ric, PH_D / 4)] = nlp[r] + nlp[128 + r];
       tc_fence_before();
-      asm volatile("bar.sync 1, 256;" ::: "memory");                 // s_nl may be overwritten by the next tile
       mbar_arrive(smem_u32(&bars->out_read));
     };
-    for (int j = 0; j < n_tiles; ++j) {
+    for (int j = 0; j < n_tiles && alive; ++j) {
       const bool tok_valid = tok_a + j * 128 + r < tok_b;
       // H halves: bias, activation, bf16, back to TMEM as the A operand of the second GEMM
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
-        mbar_wait(smem_u32(&bars->acc_ready[half]), n_acc[half] & 1, abort_flag, a.status, PH_ERR_EPI);
+        if (!wait(&bars->acc_ready[half], n_acc[half] & 1)) break;
         ++n_acc[half];
         tc_fence_after();
         uint32_t x[2][32];
@@ -312,12 +335,13 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         tc_fence_before();
         mbar_arrive(smem_u32(&bars->epi_done[half]));
       }
+      if (!alive) break;
       if (j > 0) readout_store(j - 1);
       // U halves: bias, activation, power, bf16, to the swizzled phi tiles; phi . z_t on the way
       float nl = 0.f;
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
-        mbar_wait(smem_u32(&bars->acc_ready[half]), n_acc[half] & 1, abort_flag, a.status, PH_ERR_EPI);
+        if (!wait(&bars->acc_ready[half], n_acc[half] & 1)) break;
         ++n_acc[half];
         tc_fence_after();
         uint32_t x[2][32];
@@ -348,7 +372,13 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
             st_tile_chunk_sw128(dst, PH_SUB, r, ch * 64 + cb * 32 + e, w4);
           }
         }
-        if (half == 1) s_nl[ch * 128 + r] = nl;
+        if (half == 1) {
+          // The buffer alternates with the tile.  It is free: its last reader (read-out store of tile j-2)
+          // precedes, for every thread, that thread's arrival for U half 0 of tile j-1, which the issuer
+          // waited for before the MMAs of this tile could start.
+          s_nl[(j & 1) * 256 + ch * 128 + r] = nl;
+          mbar_arrive(smem_u32(&bars->nl_ready));
+        }
         fence_proxy_async_smem();
         tc_fence_before();
         mbar_arrive(smem_u32(&bars->epi_done[half]));

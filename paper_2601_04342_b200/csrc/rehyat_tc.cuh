@@ -46,7 +46,7 @@ struct WinBars {   // offsets (bytes) inside the barrier block
   uint64_t s_ready[TC_QT], p_half[TC_QT][2], pv_done[TC_QT], o_free[TC_QT];
   uint64_t drained;
   uint32_t tmem_base;
-  int abort_flag;
+  ptx::WaitCtx wctx;
 };
 
 // One work item of window_tc: two query tiles of one (chunk, batch*head).
@@ -80,7 +80,7 @@ template <int EMU>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
           const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ out, Geo g,
-          const float* __restrict__ rd, int rd_rows, float scale, int c_mode, int* __restrict__ status,
+          const float* __restrict__ rd, int rd_rows, float scale, int c_mode, ptx::WaitArgs wa,
           int n_items, int pairs) {
   using namespace ptx;
   extern __shared__ uint8_t smem_raw[];
@@ -90,7 +90,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
   const uint32_t sK = sQ + TC_QT * TC_TILE_BYTES;                  // TC_STAGES tiles
   const uint32_t sV = sK + TC_STAGES * TC_TILE_BYTES;              // TC_STAGES tiles
   WinBars* bars = reinterpret_cast<WinBars*>(smem + (TC_QT + 2 * TC_STAGES) * TC_TILE_BYTES);
-  volatile int* abort_flag = &bars->abort_flag;
+  const uint32_t wc = smem_u32(&bars->wctx);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -108,7 +108,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       mbar_init(smem_u32(&bars->o_free[i]), TC_BM);
     }
     mbar_init(smem_u32(&bars->drained), 1);
-    bars->abort_flag = 0;
+    wait_ctx_init(&bars->wctx, wa);
     fence_mbar_init();
   }
   if (warp == 1) {
@@ -123,15 +123,15 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
   if (warp < 4) setmaxnreg_dec<TC_REGS_OTHER>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (elect_one()) {
+    if (elect_one() && !wa.withhold_loads) {
       prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
-      uint32_t kv_it = 0, n_done = 0;                              // K/V tiles loaded, items loaded
+      uint32_t n_k = 0, n_v = 0, n_q = 0;                          // K tiles, V tiles and Q loads issued so far
       bool alive = true;
       for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
         WinItem w;
         if (!win_item(g, item, pairs, w)) continue;
         // Q of the previous item has been read by its last Q K^T
-        if (n_done > 0) alive = mbar_wait(smem_u32(&bars->q_empty), (n_done - 1) & 1, abort_flag, status, TC_ERR_LOAD);
+        if (n_q > 0) alive = mbar_wait(smem_u32(&bars->q_empty), (n_q - 1) & 1, wc, TC_ERR_LOAD);
         if (!alive) break;
         const uint32_t qf = smem_u32(&bars->q_full);
         mbar_expect_tx(qf, w.ntiles * TC_TILE_BYTES);
@@ -139,24 +139,35 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           tma_load_4d(sQ + i * TC_TILE_BYTES, &tm_q, qf, 0, w.row_base + i * TC_BM, w.h_idx, w.b_idx);
           tma_load_4d(sQ + i * TC_TILE_BYTES + TC_SUB_BYTES, &tm_q, qf, 64, w.row_base + i * TC_BM, w.h_idx, w.b_idx);
         }
-        for (int j = 0; j < w.n_kv && alive; ++j, ++kv_it) {
-          const int s = kv_it % TC_STAGES;
-          const uint32_t ph = (kv_it / TC_STAGES) & 1;
+        ++n_q;
+        for (int j = 0; j < w.n_kv && alive; ++j) {
+          const int s = n_k % TC_STAGES;
+          const uint32_t ph = (n_k / TC_STAGES) & 1;
           const int key0 = w.lo + j * TC_BN;
-          alive = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1, abort_flag, status, TC_ERR_LOAD);
+          alive = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1, wc, TC_ERR_LOAD);
           if (!alive) break;
           const uint32_t kf = smem_u32(&bars->k_full[s]);
           mbar_expect_tx(kf, TC_TILE_BYTES);
           tma_load_4d(sK + s * TC_TILE_BYTES, &tm_k, kf, 0, key0, w.h_idx, w.b_idx);
           tma_load_4d(sK + s * TC_TILE_BYTES + TC_SUB_BYTES, &tm_k, kf, 64, key0, w.h_idx, w.b_idx);
-          alive = mbar_wait(smem_u32(&bars->v_empty[s]), ph ^ 1, abort_flag, status, TC_ERR_LOAD);
+          ++n_k;
+          alive = mbar_wait(smem_u32(&bars->v_empty[s]), ph ^ 1, wc, TC_ERR_LOAD);
           if (!alive) break;
           const uint32_t vf = smem_u32(&bars->v_full[s]);
           mbar_expect_tx(vf, TC_TILE_BYTES);
           tma_load_4d(sV + s * TC_TILE_BYTES, &tm_v, vf, 0, key0, w.h_idx, w.b_idx);
           tma_load_4d(sV + s * TC_TILE_BYTES + TC_SUB_BYTES, &tm_v, vf, 64, key0, w.h_idx, w.b_idx);
+          ++n_v;
         }
-        ++n_done;
+      }
+      if (!alive) {
+        // Given up: the loads already issued still write shared memory.  Wait for the last one into every
+        // buffer (the full barriers complete by byte count, whatever the consumers do) before the CTA exits.
+        if (n_q > 0) mbar_wait_drain(smem_u32(&bars->q_full), (n_q - 1) & 1, wc);
+        for (uint32_t back = 0; back < (uint32_t)TC_STAGES; ++back) {
+          if (n_k > back) mbar_wait_drain(smem_u32(&bars->k_full[(n_k - 1 - back) % TC_STAGES]), ((n_k - 1 - back) / TC_STAGES) & 1, wc);
+          if (n_v > back) mbar_wait_drain(smem_u32(&bars->v_full[(n_v - 1 - back) % TC_STAGES]), ((n_v - 1 - back) / TC_STAGES) & 1, wc);
+        }
       }
     }
   } else if (warp == 1) {
@@ -186,11 +197,16 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       };
       uint32_t kv_it = 0, n_done = 0;                                // K/V tiles consumed, items done
       uint32_t n_p[TC_QT] = {0, 0}, n_o[TC_QT] = {0, 0};             // P hand-overs and items per query tile
-      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+      bool alive = true;                                             // false once a wait has been given up: issue nothing more
+      auto wait = [&](uint64_t* bar, uint32_t parity) {
+        alive = alive && mbar_wait(smem_u32(bar), parity, wc, TC_ERR_MMA);
+        return alive;
+      };
+      for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
         WinItem w;
         if (!win_item(g, item, pairs, w)) continue;
-        mbar_wait(smem_u32(&bars->q_full), n_done & 1, abort_flag, status, TC_ERR_MMA);
-        mbar_wait(smem_u32(&bars->k_full[kv_it % TC_STAGES]), (kv_it / TC_STAGES) & 1, abort_flag, status, TC_ERR_MMA);
+        if (!wait(&bars->q_full, n_done & 1)) break;
+        if (!wait(&bars->k_full[kv_it % TC_STAGES], (kv_it / TC_STAGES) & 1)) break;
         tc_fence_after();
         for (int i = 0; i < w.ntiles; ++i) {
           issue_qk(i, kv_it % TC_STAGES);
@@ -198,17 +214,16 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         }
         umma_commit(smem_u32(&bars->k_empty[kv_it % TC_STAGES]));
         if (w.n_kv == 1) umma_commit(smem_u32(&bars->q_empty));
-        for (int j = 0; j < w.n_kv; ++j, ++kv_it) {
+        for (int j = 0; j < w.n_kv && alive; ++j, ++kv_it) {
           const int s = kv_it % TC_STAGES;
-          mbar_wait(smem_u32(&bars->v_full[s]), (kv_it / TC_STAGES) & 1, abort_flag, status, TC_ERR_MMA);
+          if (!wait(&bars->v_full[s], (kv_it / TC_STAGES) & 1)) break;
           for (int i = 0; i < w.ntiles; ++i) {
             // the first P V of an item overwrites O: the epilogue of the tile's previous item must have read it
-            if (j == 0 && n_o[i] > 0)
-              mbar_wait(smem_u32(&bars->o_free[i]), (n_o[i] - 1) & 1, abort_flag, status, TC_ERR_MMA);
-            mbar_wait(smem_u32(&bars->p_half[i][0]), n_p[i] & 1, abort_flag, status, TC_ERR_MMA);
+            if (j == 0 && n_o[i] > 0 && !wait(&bars->o_free[i], (n_o[i] - 1) & 1)) break;
+            if (!wait(&bars->p_half[i][0], n_p[i] & 1)) break;
             tc_fence_after();
             issue_pv(i, s, 0, j > 0);
-            mbar_wait(smem_u32(&bars->p_half[i][1]), n_p[i] & 1, abort_flag, status, TC_ERR_MMA);
+            if (!wait(&bars->p_half[i][1], n_p[i] & 1)) break;
             tc_fence_after();
             issue_pv(i, s, 1, true);
             ++n_p[i];
@@ -217,7 +232,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             if (j + 1 < w.n_kv) {
               const int s1 = (kv_it + 1) % TC_STAGES;
               if (i == 0) {
-                mbar_wait(smem_u32(&bars->k_full[s1]), ((kv_it + 1) / TC_STAGES) & 1, abort_flag, status, TC_ERR_MMA);
+                if (!wait(&bars->k_full[s1], ((kv_it + 1) / TC_STAGES) & 1)) break;
                 tc_fence_after();
               }
               issue_qk(i, s1);
@@ -232,9 +247,10 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         ++n_done;
         for (int i = 0; i < w.ntiles; ++i) ++n_o[i];
       }
-      // everything this thread issued has completed once `drained` flips
+      // Everything this thread has issued is complete once `drained` flips.  This wait is not cut short by the
+      // abort flag: TMEM must not be freed, nor the CTA exit, with a tcgen05.mma still running.
       umma_commit(smem_u32(&bars->drained));
-      mbar_wait(smem_u32(&bars->drained), 0, abort_flag, status, TC_ERR_MMA);
+      mbar_wait_drain(smem_u32(&bars->drained), 0, wc);
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ softmax + epilogue
@@ -244,14 +260,21 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     const uint32_t tS = tmem + lane_off + i * TC_BN, tO = tmem + lane_off + 256 + i * TC_D;
     const float c = scale * 1.4426950408889634f;                     // logits -> log2 domain
     uint32_t n_s = 0;                                                // key tiles this query tile has been through
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    // A wait that was given up ends the role.  The warp decides together (tcgen05.ld / st and the votes below
+    // need all 32 lanes), so every wait is followed by a vote.
+    bool alive = true;
+    auto wait = [&](uint64_t* bar, uint32_t parity) {
+      alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, wc, TC_ERR_SOFTMAX));
+      return alive;
+    };
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
       WinItem w;
       if (!win_item(g, item, pairs, w) || i >= w.ntiles) continue;
       const int n_kv = w.n_kv, lo = w.lo, hi = w.hi;
       float m_true = -INFINITY, m_used = -INFINITY;
       uint64_t l2a = 0ull, l2b = 0ull;                               // four partial row sums as two fp32 pairs
       for (int j = 0; j < n_kv; ++j) {
-        mbar_wait(smem_u32(&bars->s_ready[i]), (n_s + j) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+        if (!wait(&bars->s_ready[i], (n_s + j) & 1)) break;
         tc_fence_after();
         uint32_t sr[4][32];
 #pragma unroll
@@ -278,7 +301,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           const float m_new = need ? m_true : m_used;
           if (j > 0) {
             // s_ready(j) follows the completion of P V of tile j-1, so O may be touched
-            mbar_wait(smem_u32(&bars->pv_done[i]), (n_s + j - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+            if (!wait(&bars->pv_done[i], (n_s + j - 1) & 1)) break;
             tc_fence_after();
             const float f = ex2((m_used - m_new) * c);               // 1 for lanes that keep their reference
             const uint64_t f2 = pk2(f, f);
@@ -321,6 +344,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           }
         }
       }
+      if (!alive) break;
       float la0, la1, lb0, lb1;
       upk2(l2a, la0, la1);
       upk2(l2b, lb0, lb1);
@@ -353,7 +377,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         }
       }
       __nv_bfloat16* orow = out + head_offset(g, w.bh) + (long long)row * g.stride_n;
-      mbar_wait(smem_u32(&bars->pv_done[i]), (n_s + n_kv - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+      if (!wait(&bars->pv_done[i], (n_s + n_kv - 1) & 1)) break;
       tc_fence_after();
       n_s += n_kv;
       const float inv = 1.f / (l * ws + lam * nL);
@@ -431,7 +455,7 @@ inline void tc_workspace_destroy(TcWorkspace* w) { cudaFree(w->state_bf16); w->s
 // window_tc1 (one query tile per item) and its launcher live in rehyat_tc_single.cuh
 inline int tc_launch_window1(int exp_poly, int n_sm, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                              __nv_bfloat16* o, const Geo& g, const float* rd, int rd_rows, float scale, int c_mode,
-                             int* status, cudaStream_t st);
+                             const ptx::WaitArgs& wa, cudaStream_t st);
 inline bool tc_set_attributes1();
 
 inline int tc_set_attributes() {
@@ -477,7 +501,7 @@ inline bool tc_make_tmap_3d(const TcWorkspace* w, CUtensorMap* tm, const void* b
 
 // Launches window_tc for the chunks of one group.  `rd` is the linear read-out of the group's queries.
 inline int tc_launch_window(const TcWorkspace* w, const void* q, const void* k, const void* v, void* out, const Geo& g,
-                            int batch, const float* rd, int rd_rows, int c_mode, int* status, cudaStream_t st) {
+                            int batch, const float* rd, int rd_rows, int c_mode, const ptx::WaitArgs& wa, cudaStream_t st) {
   CUtensorMap tq, tk, tv;
   if (!tc_make_tmap(w, &tq, q, g, batch) || !tc_make_tmap(w, &tk, k, g, batch) || !tc_make_tmap(w, &tv, v, g, batch))
     return REHYAT_ERR_CUDA;
@@ -492,9 +516,9 @@ inline int tc_launch_window(const TcWorkspace* w, const void* q, const void* k, 
   const long long n1 = (long long)((g.Np + TC_BM - 1) / TC_BM) * g.G * g.BH;
   const double cost2 = 2.0 * (double)((n_items + w->n_sm - 1) / w->n_sm), cost1 = 1.08 * (double)((n1 + w->n_sm - 1) / w->n_sm);
   if (w->item_tiles == 1 || (w->item_tiles == 0 && cost1 < 0.93 * cost2))
-    return tc_launch_window1(w->exp_poly, w->n_sm, tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status, st);
+    return tc_launch_window1(w->exp_poly, w->n_sm, tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, st);
 #define REHYAT_LAUNCH_WINDOW(E) \
-  window_tc<E><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status, n_items, pairs)
+  window_tc<E><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, n_items, pairs)
   switch (w->exp_poly) {
     case 0: REHYAT_LAUNCH_WINDOW(0); break;
     case 2: REHYAT_LAUNCH_WINDOW(2); break;
@@ -508,7 +532,7 @@ inline int tc_launch_window(const TcWorkspace* w, const void* q, const void* k, 
 // phi_k + chunk-state partial sums of one group (Eq. 17-18).
 inline int tc_launch_state(const TcWorkspace* w, const void* k, const void* v, const rehyat_phi_params* phi,
                            const Geo& g, int batch, int P, int act_hidden, int act_out, int n_split, float* partial,
-                           int* status, cudaStream_t st) {
+                           const ptx::WaitArgs& wa, cudaStream_t st) {
   CUtensorMap tk, tv, tw1, tw2;
   if (!tc_make_tmap(w, &tk, k, g, batch) || !tc_make_tmap(w, &tv, v, g, batch) ||
       !tc_make_tmap_3d(w, &tw1, phi->k_W1, PH_D, PH_DH, g.n_heads, 128) ||
@@ -517,7 +541,7 @@ inline int tc_launch_state(const TcWorkspace* w, const void* k, const void* v, c
   PhiTcArgs a = {};
   a.b1 = (const __nv_bfloat16*)phi->k_b1; a.b2 = (const __nv_bfloat16*)phi->k_b2;
   a.P = P; a.act_hidden = act_hidden; a.act_out = act_out;
-  a.n_split = n_split; a.partial = partial; a.status = status;
+  a.n_split = n_split; a.partial = partial; a.wa = wa;
   const bool relu = act_hidden == ACT_RELU && act_out == ACT_RELU;
   const dim3 grid(n_split, g.G, g.BH);
   if (relu && P == 2)
@@ -532,7 +556,7 @@ inline int tc_launch_state(const TcWorkspace* w, const void* k, const void* v, c
 // phi_q + linear read-out of one group's queries (Eq. 7, 9, 16).
 inline int tc_launch_readout(const TcWorkspace* w, const void* q, const rehyat_phi_params* phi, const Geo& g, int batch,
                              int P, int act_hidden, int act_out, const float* state, float* rd, int rd_rows,
-                             int* status, cudaStream_t st) {
+                             const ptx::WaitArgs& wa, cudaStream_t st) {
   CUtensorMap tq, tw1, tw2, ts;
   if (!tc_make_tmap(w, &tq, q, g, batch) || !tc_make_tmap_3d(w, &tw1, phi->q_W1, PH_D, PH_DH, g.n_heads, 128) ||
       !tc_make_tmap_3d(w, &tw2, phi->q_W2, PH_DH, PH_DP, g.n_heads, 128) ||
@@ -541,7 +565,7 @@ inline int tc_launch_readout(const TcWorkspace* w, const void* q, const rehyat_p
   PhiTcArgs a = {};
   a.b1 = (const __nv_bfloat16*)phi->q_b1; a.b2 = (const __nv_bfloat16*)phi->q_b2;
   a.P = P; a.act_hidden = act_hidden; a.act_out = act_out;
-  a.state = state; a.rd = rd; a.rd_rows = rd_rows; a.status = status;
+  a.state = state; a.rd = rd; a.rd_rows = rd_rows; a.wa = wa;
   // One CTA per SM: split a chunk's query tiles over as many CTAs as costs the fewest tile-times over all waves.
   const int tiles = (g.Np + 127) / 128;
   int busy = 0;

@@ -21,12 +21,13 @@ struct WinBars1 {
   uint64_t k_full[TC_STAGES], k_empty[TC_STAGES], v_full[TC_STAGES], v_empty[TC_STAGES];
   uint64_t s_ready[2], p_half[2][2], pv_done[2], o_free[2];
   uint64_t drained;
+  uint64_t mrg_ready;       // all 256 softmax threads have written their part of mrg for the current item
   uint32_t tmem_base;
-  int abort_flag;
-  float mrg[2][3][TC_BM];   // per slot: reference maximum, true maximum and row sum of every row
+  ptx::WaitCtx wctx;
+  float mrg[2][2][3][TC_BM];   // [item parity][slot]: reference maximum, true maximum and row sum of every row
 };
-constexpr int TC_WIN1_SMEM = (1 + 2 * TC_STAGES) * TC_TILE_BYTES + 4096 /*barriers, merge buffer*/ + 1024 /*align*/;
-static_assert(sizeof(WinBars1) <= 4096, "barrier block");
+constexpr int TC_WIN1_SMEM = (1 + 2 * TC_STAGES) * TC_TILE_BYTES + 8192 /*barriers, merge buffer*/ + 1024 /*align*/;
+static_assert(sizeof(WinBars1) <= 8192, "barrier block");
 
 // Items are numbered (batch*head, chunk, query tile), query tile fastest; `tiles` = tiles of a full chunk.
 // Returns false for tiles beyond the end of a short last chunk.
@@ -51,7 +52,7 @@ template <int EMU>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ out, Geo g,
-           const float* __restrict__ rd, int rd_rows, float scale, int c_mode, int* __restrict__ status,
+           const float* __restrict__ rd, int rd_rows, float scale, int c_mode, ptx::WaitArgs wa,
            int n_items, int tiles) {
   using namespace ptx;
   extern __shared__ uint8_t smem_raw[];
@@ -61,7 +62,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   const uint32_t sK = sQ + TC_TILE_BYTES;                          // TC_STAGES tiles
   const uint32_t sV = sK + TC_STAGES * TC_TILE_BYTES;              // TC_STAGES tiles
   WinBars1* bars = reinterpret_cast<WinBars1*>(smem + (1 + 2 * TC_STAGES) * TC_TILE_BYTES);
-  volatile int* abort_flag = &bars->abort_flag;
+  const uint32_t wc = smem_u32(&bars->wctx);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -79,7 +80,8 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       mbar_init(smem_u32(&bars->o_free[i]), TC_BM);
     }
     mbar_init(smem_u32(&bars->drained), 1);
-    bars->abort_flag = 0;
+    mbar_init(smem_u32(&bars->mrg_ready), 2 * TC_BM);
+    wait_ctx_init(&bars->wctx, wa);
     fence_mbar_init();
   }
   if (warp == 1) {
@@ -94,26 +96,28 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   if (warp < 4) setmaxnreg_dec<TC_REGS_OTHER>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (elect_one()) {
+    if (elect_one() && !wa.withhold_loads) {
       prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
-      uint32_t kv_it = 0, n_done = 0;                              // K/V tiles loaded, items loaded
+      uint32_t kv_it = 0, n_q = 0;                                 // K/V tiles of finished items, Q loads issued
+      uint32_t n_k = 0, n_v = 0;                                   // K tiles and V tiles issued so far
       bool alive = true;
       for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
         WinItem w;
         if (!win_item1(g, item, tiles, w)) continue;
         // Q of the previous item has been read by its last Q K^T
-        if (n_done > 0) alive = mbar_wait(smem_u32(&bars->q_empty), (n_done - 1) & 1, abort_flag, status, TC_ERR_LOAD);
+        if (n_q > 0) alive = mbar_wait(smem_u32(&bars->q_empty), (n_q - 1) & 1, wc, TC_ERR_LOAD);
         if (!alive) break;
         const uint32_t qf = smem_u32(&bars->q_full);
         mbar_expect_tx(qf, TC_TILE_BYTES);
         tma_load_4d(sQ, &tm_q, qf, 0, w.row_base, w.h_idx, w.b_idx);
         tma_load_4d(sQ + TC_SUB_BYTES, &tm_q, qf, 64, w.row_base, w.h_idx, w.b_idx);
+        ++n_q;
         auto load_tile = [&](bool is_v, int j) {                     // key tile j of the item into its ring stage
           const uint32_t it = kv_it + j;
           const int s = it % TC_STAGES;
           const uint32_t ph = (it / TC_STAGES) & 1;
           const int key0 = w.lo + j * TC_BN;
-          if (!mbar_wait(smem_u32(is_v ? &bars->v_empty[s] : &bars->k_empty[s]), ph ^ 1, abort_flag, status, TC_ERR_LOAD))
+          if (!mbar_wait(smem_u32(is_v ? &bars->v_empty[s] : &bars->k_empty[s]), ph ^ 1, wc, TC_ERR_LOAD))
             return false;
           const uint32_t full = smem_u32(is_v ? &bars->v_full[s] : &bars->k_full[s]);
           const uint32_t dst = (is_v ? sV : sK) + s * TC_TILE_BYTES;
@@ -121,6 +125,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           mbar_expect_tx(full, TC_TILE_BYTES);
           tma_load_4d(dst, tm, full, 0, key0, w.h_idx, w.b_idx);
           tma_load_4d(dst + TC_SUB_BYTES, tm, full, 64, key0, w.h_idx, w.b_idx);
+          if (is_v) ++n_v; else ++n_k;
           return true;
         };
         // Q K^T runs two key tiles ahead of P V, so K stays one tile ahead of V
@@ -130,7 +135,15 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           alive = alive && load_tile(true, j);
         }
         kv_it += w.n_kv;
-        ++n_done;
+      }
+      if (!alive) {
+        // Given up: wait for the last load issued into every buffer before the CTA exits (the full barriers
+        // complete by byte count, whatever the consumers do).
+        if (n_q > 0) mbar_wait_drain(smem_u32(&bars->q_full), (n_q - 1) & 1, wc);
+        for (uint32_t back = 0; back < (uint32_t)TC_STAGES; ++back) {
+          if (n_k > back) mbar_wait_drain(smem_u32(&bars->k_full[(n_k - 1 - back) % TC_STAGES]), ((n_k - 1 - back) / TC_STAGES) & 1, wc);
+          if (n_v > back) mbar_wait_drain(smem_u32(&bars->v_full[(n_v - 1 - back) % TC_STAGES]), ((n_v - 1 - back) / TC_STAGES) & 1, wc);
+        }
       }
     }
   } else if (warp == 1) {
@@ -159,15 +172,20 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       };
       uint32_t kv_it = 0, n_done = 0;                                // K/V tiles consumed, items done
       uint32_t n_p[2] = {0, 0};                                      // P hand-overs per slot
-      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+      bool alive = true;                                             // false once a wait has been given up: issue nothing more
+      auto wait = [&](uint64_t* bar, uint32_t parity) {
+        alive = alive && mbar_wait(smem_u32(bar), parity, wc, TC_ERR_MMA);
+        return alive;
+      };
+      for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
         WinItem w;
         if (!win_item1(g, item, tiles, w)) continue;
-        mbar_wait(smem_u32(&bars->q_full), n_done & 1, abort_flag, status, TC_ERR_MMA);
+        if (!wait(&bars->q_full, n_done & 1)) break;
         const uint32_t base = kv_it;
         auto qk_of = [&](int jj) {                                   // S of key tile jj into slot jj & 1
           const uint32_t it = base + jj;
           const int s = it % TC_STAGES;
-          mbar_wait(smem_u32(&bars->k_full[s]), (it / TC_STAGES) & 1, abort_flag, status, TC_ERR_MMA);
+          if (!wait(&bars->k_full[s], (it / TC_STAGES) & 1)) return;
           tc_fence_after();
           issue_qk(jj & 1, s);
           umma_commit(smem_u32(&bars->s_ready[jj & 1]));
@@ -176,18 +194,18 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         };
         qk_of(0);
         if (w.n_kv > 1) qk_of(1);
-        for (int j = 0; j < w.n_kv; ++j, ++kv_it) {
+        for (int j = 0; j < w.n_kv && alive; ++j, ++kv_it) {
           const int i = j & 1, s = kv_it % TC_STAGES;
-          mbar_wait(smem_u32(&bars->v_full[s]), (kv_it / TC_STAGES) & 1, abort_flag, status, TC_ERR_MMA);
+          if (!wait(&bars->v_full[s], (kv_it / TC_STAGES) & 1)) break;
           // the first P V of an item overwrites O: both warpgroups read both O slots in the previous epilogue
           if (j == 0 && n_done > 0) {
-            mbar_wait(smem_u32(&bars->o_free[0]), (n_done - 1) & 1, abort_flag, status, TC_ERR_MMA);
-            mbar_wait(smem_u32(&bars->o_free[1]), (n_done - 1) & 1, abort_flag, status, TC_ERR_MMA);
+            if (!wait(&bars->o_free[0], (n_done - 1) & 1)) break;
+            if (!wait(&bars->o_free[1], (n_done - 1) & 1)) break;
           }
-          mbar_wait(smem_u32(&bars->p_half[i][0]), n_p[i] & 1, abort_flag, status, TC_ERR_MMA);
+          if (!wait(&bars->p_half[i][0], n_p[i] & 1)) break;
           tc_fence_after();
           issue_pv(i, s, 0, j >= 2);
-          mbar_wait(smem_u32(&bars->p_half[i][1]), n_p[i] & 1, abort_flag, status, TC_ERR_MMA);
+          if (!wait(&bars->p_half[i][1], n_p[i] & 1)) break;
           tc_fence_after();
           issue_pv(i, s, 1, true);
           ++n_p[i];
@@ -197,9 +215,10 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
         ++n_done;
       }
-      // everything this thread issued has completed once `drained` flips
+      // Everything this thread has issued is complete once `drained` flips.  This wait is not cut short by the
+      // abort flag: TMEM must not be freed, nor the CTA exit, with a tcgen05.mma still running.
       umma_commit(smem_u32(&bars->drained));
-      mbar_wait(smem_u32(&bars->drained), 0, abort_flag, status, TC_ERR_MMA);
+      mbar_wait_drain(smem_u32(&bars->drained), 0, wc);
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ softmax + epilogue
@@ -210,7 +229,14 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const float c = scale * 1.4426950408889634f;                     // logits -> log2 domain
     const int r = (warp & 3) * 32 + lane;                            // row of the query tile
     uint32_t n_s[2] = {0, 0};                                        // key tiles each slot has been through
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    uint32_t n_items_done = 0;
+    // A wait that was given up ends the role; the warp decides together (tcgen05.ld / st need all 32 lanes).
+    bool alive = true;
+    auto wait = [&](uint64_t* bar, uint32_t parity) {
+      alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, wc, TC_ERR_SOFTMAX));
+      return alive;
+    };
+    for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
       WinItem w;
       if (!win_item1(g, item, tiles, w)) continue;
       const int n_kv = w.n_kv, lo = w.lo, hi = w.hi;
@@ -219,7 +245,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       uint64_t l2a = 0ull, l2b = 0ull;                               // four partial row sums as two fp32 pairs
       for (int t = 0; t < cnt; ++t) {
         const int j = i + 2 * t;
-        mbar_wait(smem_u32(&bars->s_ready[i]), (n_s[i] + t) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+        if (!wait(&bars->s_ready[i], (n_s[i] + t) & 1)) break;
         tc_fence_after();
         uint32_t sr[4][32];
 #pragma unroll
@@ -246,7 +272,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           const float m_new = need ? m_true : m_used;
           if (t > 0) {
             // s_ready follows the completion of P V of this slot's previous tile, so O may be touched
-            mbar_wait(smem_u32(&bars->pv_done[i]), (n_s[i] + t - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+            if (!wait(&bars->pv_done[i], (n_s[i] + t - 1) & 1)) break;
             tc_fence_after();
             const float f = ex2((m_used - m_new) * c);               // 1 for lanes that keep their reference
             const uint64_t f2 = pk2(f, f);
@@ -289,15 +315,21 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           }
         }
       }
+      if (!alive) break;
       float la0, la1, lb0, lb1;
       upk2(l2a, la0, la1);
       upk2(l2b, lb0, lb1);
       const float l = (la0 + la1) + (lb0 + lb1);
 
-      // Exchange the slots' maxima and row sums (a slot without key tiles contributes m = -inf, l = 0).
-      bars->mrg[i][0][r] = m_used; bars->mrg[i][1][r] = m_true; bars->mrg[i][2][r] = l;
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      const float mu_x = bars->mrg[i ^ 1][0][r], mt_x = bars->mrg[i ^ 1][1][r], l_x = bars->mrg[i ^ 1][2][r];
+      // Exchange the slots' maxima and row sums (a slot without key tiles contributes m = -inf, l = 0).  The
+      // buffer alternates with the item: a warpgroup can be at most one item ahead of the other, because the
+      // barrier of an item completes only with the arrivals of both.
+      float (*mrg)[3][TC_BM] = bars->mrg[n_items_done & 1];
+      mrg[i][0][r] = m_used; mrg[i][1][r] = m_true; mrg[i][2][r] = l;
+      mbar_arrive(smem_u32(&bars->mrg_ready));
+      if (!wait(&bars->mrg_ready, n_items_done & 1)) break;
+      ++n_items_done;
+      const float mu_x = mrg[i ^ 1][0][r], mt_x = mrg[i ^ 1][1][r], l_x = mrg[i ^ 1][2][r];
       const float m_fin = fmaxf(m_true, mt_x);
       const float mu0 = i == 0 ? m_used : mu_x, mu1 = i == 0 ? mu_x : m_used;
       const float l0 = i == 0 ? l : l_x, l1 = i == 0 ? l_x : l;
@@ -326,8 +358,8 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
       }
       __nv_bfloat16* orow = out + head_offset(g, w.bh) + (long long)row * g.stride_n + i * (TC_D / 2);
-      mbar_wait(smem_u32(&bars->pv_done[0]), (n_s[0] + cnt0 - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
-      if (cnt1 > 0) mbar_wait(smem_u32(&bars->pv_done[1]), (n_s[1] + cnt1 - 1) & 1, abort_flag, status, TC_ERR_SOFTMAX);
+      if (!wait(&bars->pv_done[0], (n_s[0] + cnt0 - 1) & 1)) break;
+      if (cnt1 > 0 && !wait(&bars->pv_done[1], (n_s[1] + cnt1 - 1) & 1)) break;
       tc_fence_after();
       n_s[0] += cnt0; n_s[1] += cnt1;
       const float inv = 1.f / (l0 * f0 + l1 * f1 + lam * nL);
@@ -376,12 +408,12 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 // Launches window_tc1 with the tensor maps and arguments tc_launch_window has prepared.
 inline int tc_launch_window1(int exp_poly, int n_sm, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                              __nv_bfloat16* o, const Geo& g, const float* rd, int rd_rows, float scale, int c_mode,
-                             int* status, cudaStream_t st) {
+                             const ptx::WaitArgs& wa, cudaStream_t st) {
   const int tiles = (g.Np + TC_BM - 1) / TC_BM;
   const int n_items = tiles * g.G * g.BH;
   const dim3 grid(n_items < n_sm ? n_items : n_sm);
 #define REHYAT_LAUNCH_WINDOW1(E) \
-  window_tc1<E><<<grid, TC_THREADS, TC_WIN1_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, status, n_items, tiles)
+  window_tc1<E><<<grid, TC_THREADS, TC_WIN1_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, n_items, tiles)
   switch (exp_poly) {
     case 0: REHYAT_LAUNCH_WINDOW1(0); break;
     case 2: REHYAT_LAUNCH_WINDOW1(2); break;

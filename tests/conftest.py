@@ -22,10 +22,11 @@ def pytest_collection_modifyitems(config, items):
             item.add_marker(skip)
 
 
-@pytest.fixture(params=["1", "2"], ids=["one_tile_items", "two_tile_items"])
+@pytest.fixture(params=[1, 2], ids=["one_tile_items", "two_tile_items"])
 def both_window_kernels(request, monkeypatch):
     """The softmax window has two kernels, picked per launch from the number of work items: window_tc (two
     query tiles per item) and window_tc1 (one).  Small test shapes would all land on the second; this fixture
-    runs a test once with each (REHYAT_WINDOW_TILES is read when a context is created)."""
-    monkeypatch.setenv("REHYAT_WINDOW_TILES", request.param)
+    runs a test once with each by setting rehyat_config.window_tiles for every context the test creates."""
+    from paper_2601_04342_b200 import binding
+    monkeypatch.setitem(binding.TUNING_DEFAULTS, "window_tiles", request.param)
     return request.param

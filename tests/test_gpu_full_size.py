@@ -28,8 +28,9 @@ def _built():
 
 
 def gpu_forward(wl, x, **kw):
-    """One forward call through the C ABI; returns (y on the host as float64 numpy, the context's
-    workspace bytes, peak torch allocation during the call beyond the tensors the caller owns)."""
+    """One forward call through the C ABI; returns (y on the host, the context's workspace bytes, device
+    memory that the call took: the larger of what torch's allocator saw and what the driver reports as no
+    longer free, which also catches an allocation made inside the library)."""
     from paper_2601_04342_b200 import binding
     op = binding.for_workload(wl, **kw)
     q, k, v = (x[n].cuda() for n in ("q", "k", "v"))
@@ -39,10 +40,11 @@ def gpu_forward(wl, x, **kw):
     torch.cuda.synchronize()
     torch.cuda.reset_peak_memory_stats()
     before = torch.cuda.memory_allocated()
+    free_before = torch.cuda.mem_get_info()[0]
     op.forward(q, k, v, pq, pk, wl.T, wl.H, wl.W, wl.Tc, wl.To, out=out)
     assert op.status() == 0
     assert op.last_impl == "tensor" and op.last_launches > 0
-    extra = torch.cuda.max_memory_allocated() - before
+    extra = max(torch.cuda.max_memory_allocated() - before, free_before - torch.cuda.mem_get_info()[0])
     ws = op.workspace_bytes
     op.close()
     y = out.cpu()
@@ -78,15 +80,15 @@ def sample_rows(wl, rng, n_random=192):
     return np.unique(np.array(rows, dtype=np.int64))
 
 
-def check_sampled(wl, x, y, problems, seed, weighted_abs_v=False):
+def check_sampled(wl, x, y, problems, seed, weighted_abs_v=False, c_mode="rowmax"):
     f = synth.to_f64(x)
     rng = np.random.default_rng(seed)
     lin_frac = []
     for (b, h) in problems:
         rows = sample_rows(wl, rng)
         args = (f["phi_q"], f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To, b, h, rows)
-        ref, frac = orc.hybrid_rows(f["q"], f["k"], f["v"], *args, P=wl.P)
-        mag = orc.hybrid_rows(f["q"], f["k"], np.abs(f["v"]), *args, P=wl.P)[0] if weighted_abs_v else None
+        ref, frac = orc.hybrid_rows(f["q"], f["k"], f["v"], *args, P=wl.P, c_mode=c_mode)
+        mag = orc.hybrid_rows(f["q"], f["k"], np.abs(f["v"]), *args, P=wl.P, c_mode=c_mode)[0] if weighted_abs_v else None
         gate(y[b, h, rows].double().numpy(), ref, mag)
         lin_frac.append(frac.max())
     return max(lin_frac)
@@ -114,6 +116,27 @@ def test_wan13b_layer_stress_variants_sampled(variant):
     y, _, _ = gpu_forward(wl, x)
     frac = check_sampled(wl, x, y, [(0, 0), (0, 7), (0, 11)], seed=11, weighted_abs_v=(variant == "peaky_logits"))
     assert frac > 0.05                              # the linear branch carries visible mass
+
+
+@pytest.mark.parametrize("tiles", [1, 2], ids=["one_tile_items", "two_tile_items"])
+def test_wan13b_layer_c_zero_sampled(tiles):
+    """c = 0 (the other reading of the stabilising constant of Eq. 6 and 8) at full size, with each window
+    kernel: the epilogue then weighs the window by exp(m - r) and the linear read-out by exp(-r),
+    r = max(m, 0).  q x2 spreads the row maxima over both signs of m."""
+    wl = synth.CONFIGS["wan13b_layer"]
+    x = synth.make_inputs(wl, q_scale=2.0, phi_scale=1.5, v_frame_offsets=True)
+    y, _, _ = gpu_forward(wl, x, c_mode="zero", window_tiles=tiles)
+    frac = check_sampled(wl, x, y, [(0, 0), (0, 5), (0, 11)], seed=15, c_mode="zero", weighted_abs_v=True)
+    assert frac > 0.05
+
+
+def test_wan13b_layer_one_tile_items_sampled():
+    """window_tc1 (one query tile per item) forced through the one-call forward at full size."""
+    wl = synth.CONFIGS["wan13b_layer"]
+    x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
+    y, _, _ = gpu_forward(wl, x, window_tiles=1)
+    frac = check_sampled(wl, x, y, [(0, 0), (0, 6), (0, 11)], seed=16)
+    assert frac > 0.05
 
 
 def test_wan13b_layer_rows_sum_to_one_everywhere():

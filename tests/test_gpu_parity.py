@@ -264,15 +264,15 @@ def test_tensor_window_with_simt_linear_branch_matches_the_all_tensor_path():
     check(y, ref, "bf16")
 
 
-@pytest.mark.parametrize("n_poly", ["0", "1", "2", "3"])
-def test_every_share_of_polynomial_exponentials(n_poly, monkeypatch):
-    """REHYAT_EXP_POLY picks how many of every four pairs of exponentials run as a cubic on the FMA pipe."""
-    monkeypatch.setenv("REHYAT_EXP_POLY", n_poly)
+@pytest.mark.parametrize("n_poly", [-1, 1, 2, 3])
+def test_every_share_of_polynomial_exponentials(n_poly):
+    """rehyat_config.exp_poly picks how many of every four pairs of exponentials run as a cubic on the FMA pipe
+    (-1: none, 0 would be the library's own choice, which is 1)."""
     wl = synth.Workload("poly", 1, 2, 128, 6, 10, 20, 2, 1, "bf16", True, seed=synth.BASE_SEED + 87)
     for kw in (dict(phi_scale=1.5, v_frame_offsets=True), dict(q_scale=4.0, phi_scale=1.5)):
         x = synth.make_inputs(wl, **kw)
         ref, _ = oracle_full(wl, x)
-        y, used = run_gpu(wl, x)
+        y, used = run_gpu(wl, x, exp_poly=n_poly)
         assert used == "tensor"
         check(y, ref, "bf16")
 
