@@ -35,9 +35,28 @@ from paper_2601_04342_b200 import geometry, synth  # noqa: E402
 METRIC = "hybrid-attention TFLOP/s (algorithmic) per layer at 32,760 tokens"
 UNIT = "TFLOP/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the ncu
-# capture summarised under profiles/; None until a capture exists for the kernel in use.
-NCU_TRAFFIC_BYTES = {"window_simt": None, "window_tc": 481645824 + 87647232}   # profiles/window_tc_wan13b_layer.md
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu capture of that
+# kernel at this workload, together with a digest of the kernel's sources at the time of the capture: the figure
+# is reported only for the kernel it was taken on and only while those sources are unchanged.
+KERNEL_SOURCES = {"window_tc": ("rehyat_tc.cuh", "rehyat_ptx.cuh", "rehyat_common.cuh"),
+                  "window_tc1": ("rehyat_tc_single.cuh", "rehyat_tc.cuh", "rehyat_ptx.cuh", "rehyat_common.cuh")}
+NCU_CAPTURES = {}   # kernel -> {"traffic": bytes per launch, "workload": name, "sources": digest}
+
+
+def kernel_source_digest(kernel):
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES.get(kernel, ()):
+        with open(os.path.join(ROOT, "paper_2601_04342_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(kernel, workload):
+    cap = NCU_CAPTURES.get(kernel)
+    if not cap or cap["workload"] != workload or cap["sources"] != kernel_source_digest(kernel):
+        return None
+    return cap["traffic"]
 
 
 def measured_peaks():
@@ -63,7 +82,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
@@ -225,27 +244,47 @@ def lib_state_bytes(op):
     return binding.lib().rehyat_stream_state_bytes(op._h)
 
 
-def time_config(wl, device, stream, full_softmax=False):
+def linear_share_summary(op, wl, run):
+    """Runs one step with the library's diagnostic output switched on and summarises nL / (nS + nL) (Eq. 8, 9):
+    how much of the joint normaliser the linear branch carries, over the rows that have a linear set."""
+    share = torch.zeros((wl.B, wl.n_heads, wl.N), device="cuda", dtype=torch.float32)
+    op.set_linear_share_output(share)
+    run()
+    torch.cuda.synchronize()
+    op.set_linear_share_output(None)
+    first_linear = next((c.q0 for c in geometry.chunk_plan(wl.T, wl.HW, wl.Tc, wl.To) if c.lo > 0), wl.N)
+    rows = share[:, :, first_linear:]
+    if rows.numel() == 0:
+        return {"rows_with_linear_set": 0.0, "mean": 0.0, "median": 0.0, "max": 0.0}
+    return {"rows_with_linear_set": (wl.N - first_linear) / wl.N, "mean": float(rows.mean()),
+            "median": float(rows.median()), "max": float(rows.max())}
+
+
+def time_config(wl, device, stream, full_softmax=False, steps=20, rms_norm=True):
     """Kernel-resident timing of another configuration.  Inputs are drawn on the device (seeded torch
-    generator, N(0,1), q and k RMS-normalised) because the host recipe takes tens of seconds at these
-    sizes; the parity tests use the host recipe."""
+    generator, N(0,1), q and k RMS-normalised where the configuration says so) because the host recipe takes
+    tens of seconds at these sizes; the parity tests use the host recipe."""
     from paper_2601_04342_b200 import binding
     gen = torch.Generator(device="cuda").manual_seed(wl.seed)
     shape = (wl.B, wl.n_heads, wl.N, wl.head_dim)
     q, k, v = (torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32) for _ in range(3))
-    q = (q / q.pow(2).mean(-1, keepdim=True).sqrt()).to(torch.bfloat16)
-    k = (k / k.pow(2).mean(-1, keepdim=True).sqrt()).to(torch.bfloat16)
-    v = v.to(torch.bfloat16)
+    if rms_norm and wl.rms_norm_qk:
+        q = q / q.pow(2).mean(-1, keepdim=True).sqrt()
+        k = k / k.pow(2).mean(-1, keepdim=True).sqrt()
+    q, k, v = q.to(torch.bfloat16), k.to(torch.bfloat16), v.to(torch.bfloat16)
     pq = {n: t.cuda() for n, t in synth.make_phi_params(wl, "phi_q").items()}
     pk = {n: t.cuda() for n, t in synth.make_phi_params(wl, "phi_k").items()}
     out = torch.empty_like(q)
     op = binding.for_workload(wl, device=device)
-    ms = _time_ms(lambda: op.forward(q, k, v, pq, pk, wl.T, wl.H, wl.W, wl.Tc, wl.To, out=out, stream=stream), stream, 3, 20)
+    run = lambda: op.forward(q, k, v, pq, pk, wl.T, wl.H, wl.W, wl.Tc, wl.To, out=out, stream=stream)
+    ms = _time_ms(run, stream, 3, steps)
     assert op.status() == 0
     fl = geometry.flop_model(wl.B, wl.n_heads, wl.head_dim, wl.T, wl.HW, wl.Tc, wl.To, wl.D_h, wl.D_out)
-    res = {"workload": wl.name, "batch": wl.B, "tokens": wl.N, "ms_per_step": ms, "tflops": fl["total"] / (ms * 1e-3) / 1e12,
+    res = {"workload": wl.name, "batch": wl.B, "tokens": wl.N, "chunk_frames": wl.Tc, "overlap_frames": wl.To,
+           "steps": steps, "ms_per_step": ms, "tflops": fl["total"] / (ms * 1e-3) / 1e12,
            "tokens_per_s": wl.B * wl.N / (ms * 1e-3), "workspace_bytes": op.workspace_bytes, "launches_per_step": op.last_launches,
-           "full_softmax_flop_ratio": fl["full_softmax"] / fl["total"]}
+           "window_tiles_per_item": op.last_window_tiles, "full_softmax_flop_ratio": fl["full_softmax"] / fl["total"],
+           "linear_share_of_normaliser": linear_share_summary(op, wl, run)}
     op.close()
     if full_softmax:
         res["full_softmax_same_shape"] = full_softmax_comparison(wl, {"q": q, "k": k, "v": v}, pq, pk, stream, ms, fl,
@@ -303,7 +342,14 @@ def main():
     ap.add_argument("--kernel-impl", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-full-softmax", action="store_true", help="skip the full-softmax comparison at the same shape")
     ap.add_argument("--all-configs", action="store_true",
-                    help="also time the CFG-batch and the long-video configurations (device-drawn inputs)")
+                    help="also the full-softmax comparison at the CFG-batch shape and the bidirectional variant")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
+                    help="with --gpus N > 1: every rank runs its own layer input (weak scaling, the default), or ONE "
+                         "layer's (batch, head) problems are split over the ranks (strong scaling)")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the CFG-batch, long-video, 320x480 and chunk/overlap-sweep timings")
+    ap.add_argument("--sustained-seconds", type=float, default=3.0,
+                    help="length of the power-capped leg (0 skips it)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -331,8 +377,10 @@ def main():
     if dist:
         dist.barrier()
 
-    # every rank draws its own layer input (weak scaling over independent problems)
-    wl_rank = wl.with_(seed=wl.seed + 1000 * rank)
+    # every rank draws its own layer input (weak scaling over independent problems); when one layer is split
+    # over the ranks, all of them draw the same input and each computes its own (batch, head) problems of it
+    shard_heads = args.shard == "heads" and world > 1
+    wl_rank = wl if shard_heads else wl.with_(seed=wl.seed + 1000 * rank)
     host = synth.make_inputs(wl_rank)
     dev = {n: host[n].cuda() for n in ("q", "k", "v")}
     phi_q = {n: t.cuda() for n, t in host["phi_q"].items()}
@@ -340,9 +388,17 @@ def main():
     out = torch.empty_like(dev["q"])
     op = binding.for_workload(wl, impl=args.kernel_impl, device=local_rank)
     stream = torch.cuda.current_stream()
+    sharded = None
+    if shard_heads:
+        sharded = binding.ShardedRehyat(world, rank, batch=wl.B, n_heads=wl.n_heads, head_dim=wl.head_dim, dtype=wl.dtype,
+                                        phi_hidden=wl.D_h, phi_dim=wl.D_out, poly_degree=wl.P, impl=args.kernel_impl,
+                                        max_tokens_per_frame=wl.HW, max_chunk_frames=min(wl.Tc, wl.T), device=local_rank)
 
     def step():
-        op.forward(dev["q"], dev["k"], dev["v"], phi_q, phi_k, wl.T, wl.H, wl.W, wl.Tc, wl.To, out=out, stream=stream)
+        if sharded is not None:
+            sharded.forward(dev["q"], dev["k"], dev["v"], out, phi_q, phi_k, wl.T, wl.H, wl.W, wl.Tc, wl.To, stream=stream)
+        else:
+            op.forward(dev["q"], dev["k"], dev["v"], phi_q, phi_k, wl.T, wl.H, wl.W, wl.Tc, wl.To, out=out, stream=stream)
 
     def barrier():
         if dist:
@@ -352,9 +408,10 @@ def main():
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
-    assert op.status() == 0, "device status word set during warm-up"
-    launches_per_step = op.last_launches
+    assert op.status() == 0 and (sharded is None or sharded.status() == 0), "device status word set during warm-up"
+    launches_per_step = sharded.last_launches if sharded is not None else op.last_launches
     kernel_family = op.last_impl
+    window_tiles = op.last_window_tiles
 
     flops = geometry.flop_model(wl.B, wl.n_heads, wl.head_dim, wl.T, wl.HW, wl.Tc, wl.To, wl.D_h, wl.D_out)
     sampler = ClockSampler(local_rank)
@@ -377,7 +434,8 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms_total = float(t.item())
     ms_step = ms_total / args.steps
-    value = world * flops["total"] / (ms_step * 1e-3) / 1e12
+    jobs = 1 if shard_heads else world               # layers the whole job computes per step
+    value = jobs * flops["total"] / (ms_step * 1e-3) / 1e12
 
     # end to end through the host-buffer entry point (pinned host tensors, copies timed)
     pinned = {n: host[n].pin_memory() for n in ("q", "k", "v")}
@@ -400,7 +458,7 @@ def main():
         t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_ms = float(t.item())
-    e2e_value = world * flops["total"] / (e2e_ms * 1e-3) / 1e12
+    e2e_value = world * flops["total"] / (e2e_ms * 1e-3) / 1e12       # the host-buffer entry point always runs a whole layer per rank
 
     if rank != 0:
         if dist:
@@ -414,9 +472,10 @@ def main():
     win_ms, win_n = prof["window"]
     win_flops_per_launch = flops["window"] * args.steps / max(win_n, 1)
     achieved = win_flops_per_launch / (win_ms / max(win_n, 1) * 1e-3) / 1e12 if win_ms > 0 else None
-    kernel_name = "window_tc" if kernel_family == "tensor" else "window_simt"
+    kernel_name = ("window_tc" if window_tiles == 2 else "window_tc1") if kernel_family == "tensor" else "window_simt"
     roofline = {"bound": "tensor", "kernel": kernel_name, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak if achieved else None, "traffic": NCU_TRAFFIC_BYTES.get(kernel_name),
+                "frac": achieved / peak if achieved else None, "traffic": ncu_traffic(kernel_name, wl.name),
+                "traffic_captured_on": kernel_name if ncu_traffic(kernel_name, wl.name) is not None else None,
                 "peak_source": f"{peaks['source']} bf16 {peak_kind} (MEASURED_PEAKS.json)" if peaks["source"] == "measured"
                 else "fallback",
                 "frac_of_nominal_2250": achieved / 2250.0 if achieved else None,
@@ -436,10 +495,24 @@ def main():
                          f"fp64 numpy, {dt:.1f} s"}
 
     extras = {}
+    if world == 1 and args.sustained_seconds > 0:
+        # The same step looped for seconds, with the clock sampler running across it: the regime in which the GPU
+        # sits at its power cap.  Reported against the sustained peak (a matmul looped for seconds, same regime).
+        n_sus = max(int(args.sustained_seconds / (ms_step * 1e-3)), 10)
+        sus_sampler = ClockSampler(local_rank)
+        torch.cuda.synchronize()
+        sus_sampler.start()
+        sus_ms = _time_ms(step, stream, 3, n_sus)
+        sus_clocks = sus_sampler.stop()
+        sus_tf = flops["total"] / (sus_ms * 1e-3) / 1e12
+        extras["sustained"] = {"steps": n_sus, "seconds": sus_ms * n_sus * 1e-3, "ms_per_step": sus_ms, "value": sus_tf,
+                               "unit": UNIT, "clocks": sus_clocks,
+                               "ms_x_mhz": sus_ms * sus_clocks["sm_mhz"] if sus_clocks.get("sm_mhz") else None,
+                               "frac_of_measured_sustained": sus_tf / peaks["bf16_sustained"],
+                               "frac_of_measured_burst": sus_tf / peaks["bf16_burst"]}
     if world == 1:
-        # The timed loop above runs long enough for the GPU to reach its power cap and lower the SM clock.  For
-        # context (never the headline value): ten steps after the GPU has been idle, at the clocks the measured
-        # burst peak was taken at.
+        # Whether the timed loop above reached the power cap depends on --steps (its clock record is in "clocks").
+        # For context (never the headline value): ten steps after the GPU has been idle for a second.
         time.sleep(1.0)
         idle_ms = _time_ms(step, stream, 3, 10)
         extras["ten_steps_after_idle"] = {"ms_per_step": idle_ms, "value": flops["total"] / (idle_ms * 1e-3) / 1e12,
@@ -465,19 +538,27 @@ def main():
         extras["workspace_bytes_by_latent_frames"] = workspace_by_frames(wl, local_rank)
         extras["chunk_by_chunk"] = stream_timing(wl, dev, phi_q, phi_k, stream, flops)
     if world == 1 and args.all_configs:
-        extras["other_configs"] = [time_config(synth.CONFIGS[n], local_rank, stream, full_softmax=(n == "cfg_long"))
-                                   for n in ("cfg_long", "long_constant_memory", "wan13b_320x480")]
         extras["bidirectional_same_shape"] = bidirectional_timing(wl, dev, phi_q, phi_k, stream, ms_step)
+    if world == 1:
+        extras["linear_share_of_normaliser"] = linear_share_summary(op, wl, step)
+    if world == 1 and not args.no_other_configs:
+        extras["other_configs"] = [time_config(synth.CONFIGS[n], local_rank, stream, steps=10,
+                                               full_softmax=(args.all_configs and n == "cfg_long"))
+                                   for n in ("cfg_long", "long_constant_memory", "wan13b_320x480")]
+        extras["chunk_overlap_sweep"] = [time_config(w, local_rank, stream, steps=5) for w in synth.sweep_configs()]
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "strong" if shard_heads else "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": config_of(wl, {"kernels": kernel_family, "parallelism": f"dp{world} over (batch, head) problems"}),
-            "tokens_per_s": world * wl.B * wl.N / (ms_step * 1e-3),
+            "config": config_of(wl, {"kernels": kernel_family, "parallelism": (f"one layer's {wl.B * wl.n_heads} (batch, head) problems split over {world} ranks, "
+                                                f"at most {geometry.shard_efficiency(wl.B, wl.n_heads, world):.3f} efficient"
+                                                if shard_heads else f"dp{world} over (batch, head) problems")}),
+            "tokens_per_s": jobs * wl.B * wl.N / (ms_step * 1e-3),
             "frac_of_bf16_peak": {"measured_burst": value / world / peaks["bf16_burst"],
                                   "measured_sustained": value / world / peaks["bf16_sustained"],
                                   "nominal_2250": value / world / 2250.0},
-            "clocks": clocks,
+            "clocks": clocks, "ms_x_mhz": ms_step * clocks["sm_mhz"] if clocks.get("sm_mhz") else None,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 3 * nbytes, "d2h_bytes_per_step": nbytes,
                     "ms_per_step": e2e_ms},
             "gpu_launches": launches_per_step * args.steps,

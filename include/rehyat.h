@@ -242,6 +242,18 @@ int rehyat_last_launches(const rehyat_ctx* ctx);
 /* 1 if the last forward ran the tensor-core kernels, 0 for the SIMT kernels. */
 int rehyat_last_impl(const rehyat_ctx* ctx);
 
+/* Query tiles per work item of the last tensor-core window launch: 2 (window_tc) or 1 (window_tc1);
+ * 0 after a forward on the SIMT kernels. */
+int rehyat_last_window_tiles(const rehyat_ctx* ctx);
+
+/* Diagnostic output for measurement.  `share` is a device buffer of batch*n_heads*frames*H*W floats
+ * (caller-owned, 16-byte aligned), or NULL to switch it off.  While set, every rehyat_forward also
+ * writes, for query i of (batch b, head h) at share[(b*n_heads + h)*N + i], the part of the joint
+ * normaliser of Eq. 5 that comes from the linear branch, nL_i / (nS_i + nL_i) with both terms as the
+ * kernel weighs them (Eq. 8, 9; 0 for chunks with an empty linear set).  Not written by
+ * rehyat_forward_host or rehyat_stream_step. */
+int rehyat_set_linear_share_output(rehyat_ctx* ctx, float* share);
+
 /* Per-kernel timing for measurement.  While enabled, every kernel launch of rehyat_forward is
  * bracketed by CUDA events recorded on the launching stream (a few microseconds of overhead per
  * launch).  rehyat_profile_read waits for the recorded events, writes the summed milliseconds and

@@ -22,6 +22,7 @@ EXPORTS = ["rehyat_create", "rehyat_forward", "rehyat_forward_host", "rehyat_for
            "rehyat_stream_begin", "rehyat_stream_step", "rehyat_stream_state_bytes", "rehyat_stream_export",
            "rehyat_stream_import",
            "rehyat_workspace_bytes", "rehyat_status", "rehyat_set_wait_limit", "rehyat_last_launches", "rehyat_last_impl",
+           "rehyat_last_window_tiles", "rehyat_set_linear_share_output",
            "rehyat_profile_enable", "rehyat_profile_read", "rehyat_strerror", "rehyat_version"]
 PROF_KINDS = ("state", "scan", "readout", "window")
 
@@ -79,6 +80,8 @@ def lib():
         L.rehyat_set_wait_limit.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
         L.rehyat_last_launches.argtypes = [C.c_void_p]
         L.rehyat_last_impl.argtypes = [C.c_void_p]
+        L.rehyat_last_window_tiles.argtypes = [C.c_void_p]
+        L.rehyat_set_linear_share_output.argtypes = [C.c_void_p, C.c_void_p]
         L.rehyat_profile_enable.argtypes = [C.c_void_p, C.c_int]
         L.rehyat_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int32)]
         L.rehyat_strerror.argtypes = [C.c_int]
@@ -146,6 +149,14 @@ class Rehyat:
     @property
     def last_impl(self):
         return "tensor" if lib().rehyat_last_impl(self._h) else "simt"
+
+    @property
+    def last_window_tiles(self):
+        return lib().rehyat_last_window_tiles(self._h)
+
+    def set_linear_share_output(self, share):
+        """share: float32 CUDA tensor [B, n_heads, N] the window kernels fill with nL / (nS + nL), or None."""
+        _check(lib().rehyat_set_linear_share_output(self._h, _ptr(share)), "rehyat_set_linear_share_output")
 
     @staticmethod
     def phi_struct(phi_q, phi_k):
@@ -252,6 +263,54 @@ def forward_static(q, k, v, phi_q, phi_k, frames, H, W, chunk, overlap, *, dtype
                                        B, frames, H, W, chunk, overlap, C.c_void_p(st.cuda_stream)),
            "rehyat_forward_static")
     return out
+
+
+def shard_call_args(q, k, v, out, phi_q, phi_k, rect):
+    """Arguments of the operator call for one rectangle (b0, nb, h0, nh) of geometry.shard_rects: views of the
+    [B, n_heads, N, d] tensors that start at (b0, h0) and keep the parent's strides, the phi parameters of heads
+    [h0, h0 + nh), and the layout of those strides.  Marshalling only: nothing is copied."""
+    b0, nb, h0, nh = rect
+    views = tuple(t.narrow(0, b0, nb).narrow(1, h0, nh) for t in (q, k, v, out))
+    sb, sh, sn, sd = q.stride()
+    if sd != 1 or any(t.stride() != q.stride() for t in (k, v, out)):
+        raise ValueError("q, k, v, out must share their strides, with head_dim contiguous")
+    pq = {n: t.narrow(0, h0, nh) for n, t in phi_q.items()}
+    pk = {n: t.narrow(0, h0, nh) for n, t in phi_k.items()}
+    return views, pq, pk, Layout(sb, sh, sn)
+
+
+class ShardedRehyat:
+    """The (batch, head) problems of one operator call split over `world_size` ranks (geometry.shard_rects):
+    this rank's rectangles, one context per distinct head count.  No exchange between ranks is needed."""
+
+    def __init__(self, world_size, rank, *, batch, n_heads, **ctx_args):
+        from . import geometry
+        self.rects = geometry.shard_rects(batch, n_heads, world_size, rank)
+        self._ops = {}
+        for (_, nb, _, nh) in self.rects:
+            if nh not in self._ops:
+                self._ops[nh] = Rehyat(n_heads=nh, max_batch=max(r[1] for r in self.rects if r[3] == nh), **ctx_args)
+
+    def forward(self, q, k, v, out, phi_q, phi_k, frames, H, W, chunk, overlap, stream=None):
+        """q, k, v, out: the FULL [B, n_heads, N, d] CUDA tensors; only this rank's rectangles of `out` are written."""
+        st = stream if stream is not None else torch.cuda.current_stream(q.device)
+        self.last_launches = 0
+        for rect in self.rects:
+            (vq, vk, vv, vo), pq, pk, lay = shard_call_args(q, k, v, out, phi_q, phi_k, rect)
+            op = self._ops[rect[3]]
+            phi = Rehyat.phi_struct(pq, pk)
+            _check(lib().rehyat_forward(op._h, _ptr(vq), _ptr(vk), _ptr(vv), _ptr(vo), C.byref(lay), C.byref(phi),
+                                        rect[1], frames, H, W, chunk, overlap, C.c_void_p(st.cuda_stream)),
+                   "rehyat_forward")
+            self.last_launches += op.last_launches
+        return out
+
+    def status(self, stream=None):
+        return min((op.status(stream) for op in self._ops.values()), default=OK)
+
+    def close(self):
+        for op in self._ops.values():
+            op.close()
 
 
 def for_workload(wl, **kw):

@@ -66,6 +66,8 @@ struct rehyat_ctx {
   int epoch = 0;               // number of the last tensor-core launch, 1, 2, ... (see ptx::WaitCtx)
   unsigned wait_limit_us = 1000000u;   // bound of every device-side wait
   int withhold_loads = 0;      // test hook of rehyat_set_wait_limit
+  float* share_out = nullptr;  // rehyat_set_linear_share_output
+  float* share_now = nullptr;  // what the window launches of the call in progress write (null in chunk-by-chunk steps)
   // chunk-by-chunk processing (rehyat_stream_*): the running state lives in slot 0 of `state`, the last
   // `overlap` frames of k and v and the chunk being processed in staging buffers [BH][cap_tokens][d]
   struct Stream {
@@ -190,7 +192,7 @@ int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* ou
     const int wtiles = (g.Np + WIN_BM - 1) / WIN_BM;
     ctx->prof.begin(REHYAT_PROF_WINDOW, st);
     window_simt<T, D><<<dim3(wtiles, g.G, g.BH), WIN_THREADS, smem_win, st>>>(
-        q, k, v, out, g, ctx->readout, ctx->rd_cap, 1.0f / sqrtf((float)D), c.c_mode);
+        q, k, v, out, g, ctx->readout, ctx->rd_cap, 1.0f / sqrtf((float)D), c.c_mode, ctx->share_now);
     ctx->prof.end(REHYAT_PROF_WINDOW, st);
     ctx->last_launches += 1;
   }
@@ -252,7 +254,7 @@ int run_parts(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void
     }
     if (rc == REHYAT_OK && (parts & PART_WINDOW)) {
       ctx->prof.begin(REHYAT_PROF_WINDOW, st);
-      rc = tc_launch_window(&ctx->tc, q, k, v, out, g, batch, ctx->readout, ctx->rd_cap, c.c_mode, next_wait(ctx), st);
+      rc = tc_launch_window(&ctx->tc, q, k, v, out, g, batch, ctx->readout, ctx->rd_cap, c.c_mode, next_wait(ctx), ctx->share_now, st);
       ctx->prof.end(REHYAT_PROF_WINDOW, st);
       ctx->last_launches += 1;
     }
@@ -399,6 +401,13 @@ int rehyat_destroy(rehyat_ctx* ctx) {
 size_t rehyat_workspace_bytes(const rehyat_ctx* ctx) { return ctx ? ctx->ws_bytes : 0; }
 int rehyat_last_launches(const rehyat_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
 int rehyat_last_impl(const rehyat_ctx* ctx) { return ctx ? ctx->last_impl : 0; }
+int rehyat_last_window_tiles(const rehyat_ctx* ctx) { return ctx && ctx->last_impl ? ctx->tc.last_item_tiles : 0; }
+
+int rehyat_set_linear_share_output(rehyat_ctx* ctx, float* share) {
+  if (!ctx || (share && !aligned16(share))) return REHYAT_ERR_INVALID_ARG;
+  ctx->share_out = share;
+  return REHYAT_OK;
+}
 
 int rehyat_profile_enable(rehyat_ctx* ctx, int on) {
   if (!ctx) return REHYAT_ERR_INVALID_ARG;
@@ -499,6 +508,7 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   ctx->last_launches = 0;
   ctx->last_impl = ctx->tensor_ok ? 1 : 0;
   ctx->stream.active = false;                 // the workspace is about to be overwritten
+  ctx->share_now = ctx->head_count > 0 ? nullptr : ctx->share_out;   // not through rehyat_forward_host
   if (c.bidirectional && n_chunks > 1) {
     // Eq. 10-12: the linear set of a chunk is everything outside its window.  Pass 1 sums the state frame by
     // frame (running sums cum[0..frames]); pass 2 forms each chunk's state from three of those sums.
@@ -723,6 +733,7 @@ int rehyat_stream_step(rehyat_ctx* ctx, const void* q_chunk, const void* k_chunk
   g.N = h + Np; g.Np = Np; g.ToHW = h; g.t0 = 0; g.G = 1; g.n_heads = c.n_heads; g.BH = BH;
   g.stride_b = sb; g.stride_h = sh; g.stride_n = sn;
   g.q_shift = h; g.prefix = s.has_state;
+  ctx->share_now = nullptr;
   ctx->last_launches = 0;
   ctx->last_impl = ctx->tensor_ok ? 1 : 0;
   int rc = run_parts(ctx, s.qbuf, kcur, vcur, s.obuf, phi, g, s.batch, 1, -1, (s.has_state ? PART_READOUT : 0) | PART_WINDOW, st);

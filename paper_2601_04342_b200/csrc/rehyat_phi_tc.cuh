@@ -103,7 +103,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     for (int s = 0; s < PH_RING; ++s) {
       mbar_init(smem_u32(&bars->ring_full[s]), 1); mbar_init(smem_u32(&bars->ring_empty[s]), 1);
     }
-    mbar_init(smem_u32(&bars->acc_ready), 1); mbar_init(smem_u32(&bars->epi_done), 256);
+    mbar_init(smem_u32(&bars->acc_ready), 1); mbar_init(smem_u32(&bars->epi_done), 8);
     mbar_init(smem_u32(&bars->out_ready), 1);
     mbar_init(smem_u32(&bars->drained), 1);
     wait_ctx_init(&bars->wctx, a.wa);
@@ -194,23 +194,26 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       constexpr uint32_t id_st = idesc_bf16(128, 128, 1, 1);       // A = phi^T (MN-major), B = V (MN-major)
       constexpr uint32_t id_z = idesc_bf16(128, 16, 1, 0);         // A = phi^T (MN-major), B = ones (K-major)
       uint32_t ring_i = 0, n_epi = 0;
-      bool alive = true;                                            // false once a wait has been given up: issue nothing more
-      auto wait = [&](uint64_t* bar, uint32_t parity) {
-        alive = alive && mbar_wait(smem_u32(bar), parity, wc, PH_ERR_MMA);
-        if (alive) tc_fence_after();
-        return alive;
+      // A wait that is given up ends the role at once: the helpers return false and run() returns, so nothing
+      // further is issued.  No flag is carried along; the hot path pays one predicated branch per wait.
+      auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
+        if (!mbar_wait(smem_u32(bar), parity, wc, PH_ERR_MMA)) return false;
+        tc_fence_after();
+        return true;
       };
       auto ring_release = [&]() {
         umma_commit(smem_u32(&bars->ring_empty[ring_i % RING]));
         ++ring_i;
       };
-      auto wait_epi = [&]() {
-        if (wait(&bars->epi_done, n_epi & 1)) ++n_epi;
+      auto wait_epi = [&]() -> bool {
+        if (!wait(&bars->epi_done, n_epi & 1)) return false;
+        ++n_epi;
+        return true;
       };
       // one 128x128 half of an MLP GEMM: A tile [128 x 64*nks] K-major at a_base, B tiles from the ring
-      auto mlp_half = [&](uint32_t a_base, int nks) {
+      auto mlp_half = [&](uint32_t a_base, int nks) -> bool {
         for (int ks = 0; ks < nks; ++ks) {
-          if (!wait(&bars->ring_full[ring_i % RING], (ring_i / RING) & 1)) return;
+          if (!wait(&bars->ring_full[ring_i % RING], (ring_i / RING) & 1)) return false;
           const uint32_t bt = ring_addr(ring_i % RING);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
@@ -219,10 +222,10 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
           ring_release();
         }
         umma_commit(smem_u32(&bars->acc_ready));
+        return true;
       };
       // contraction that consumes phi half `c` (its tile is at phi_base)
       auto consume_half = [&](int c, uint32_t phi_base, bool first_tile) {
-        if (!alive) return;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {                            // 16 tokens per step
           const uint64_t ad = smem_desc_sw128(phi_base + kk * 2048, PH_SUB, 1024);
@@ -232,31 +235,31 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
                   (!first_tile || kk > 0) ? 1u : 0u);
         }
       };
-      for (int j = 0; j < n_tiles && alive; ++j) {
-        if (!wait(&bars->x_full, j & 1)) break;
-        if (j > 0) wait_epi();                                      // scratch free: phi half 1 of tile j-1 written
-        if (j > 0) {                                                // ... and consumed
-          if (!wait(&bars->v_full, (j - 1) & 1)) break;
-          consume_half(1, sHb, j == 1);
-          umma_commit(smem_u32(&bars->v_empty));
+      auto run = [&]() {
+        for (int j = 0; j < n_tiles; ++j) {
+          if (!wait(&bars->x_full, j & 1)) return;
+          if (j > 0) {
+            if (!wait_epi()) return;                                  // scratch free: phi half 1 of tile j-1 written
+            if (!wait(&bars->v_full, (j - 1) & 1)) return;            // ... and consumed
+            consume_half(1, sHb, j == 1);
+            umma_commit(smem_u32(&bars->v_empty));
+          }
+          if (!mlp_half(sX, 2)) return;                               // H[:, 0:128]
+          if (!wait_epi()) return;
+          if (!mlp_half(sX, 2)) return;                               // H[:, 128:256]
+          umma_commit(smem_u32(&bars->x_empty));
+          if (!wait_epi()) return;
+          if (!mlp_half(sHb, 4)) return;                              // U[:, 0:128]
+          if (!wait_epi()) return;
+          if (!mlp_half(sHb, 4)) return;                              // U[:, 128:256]
+          if (!wait(&bars->v_full, j & 1)) return;
+          consume_half(0, sPhi0, j == 0);
         }
-        mlp_half(sX, 2);                                            // H[:, 0:128]
-        wait_epi();
-        mlp_half(sX, 2);                                            // H[:, 128:256]
-        if (!alive) break;
-        umma_commit(smem_u32(&bars->x_empty));
-        wait_epi();
-        mlp_half(sHb, 4);                                           // U[:, 0:128]
-        wait_epi();
-        mlp_half(sHb, 4);                                           // U[:, 128:256]
-        if (!wait(&bars->v_full, j & 1)) break;
-        consume_half(0, sPhi0, j == 0);
-      }
-      wait_epi();
-      if (alive) {
+        if (!wait_epi()) return;
         consume_half(1, sHb, n_tiles == 1);
         umma_commit(smem_u32(&bars->out_ready));
-      }
+      };
+      run();
       // Everything this thread has issued is complete once `drained` flips; the abort flag does not cut this
       // wait short, so that TMEM is never freed with a tcgen05.mma still running.
       umma_commit(smem_u32(&bars->drained));
@@ -271,17 +274,18 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     const uint32_t lane_off = (uint32_t)(qd * 32) << 16;
     uint32_t n_acc = 0;
     const int part_w = PH_DP / (PC ? PC : a.P);                     // a multiple of 32 (P in {1,2,4})
-    // A wait that was given up ends the role; the warp decides together (tcgen05.ld needs all 32 lanes).
-    bool alive = true;
-    auto wait = [&](uint64_t* bar, uint32_t parity) {
-      alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, wc, PH_ERR_EPI));
-      return alive;
-    };
-    for (int j = 0; j < n_tiles && alive; ++j) {
+    // After a wait has been given up anywhere in the CTA every later wait returns at once.  These warps then run
+    // through the rest of the current tile on whatever the accumulators hold (tcgen05.ld needs all 32 lanes, so
+    // nothing is skipped lane by lane; every address stays inside the CTA's TMEM and shared memory) and leave
+    // at the head of the next tile, where the whole warp looks at the flag together.
+    auto aborted = [&]() -> bool { return __any_sync(0xffffffffu, wait_ctx_aborted(wc) != 0); };
+    auto wait = [&](uint64_t* bar, uint32_t parity) { mbar_wait(smem_u32(bar), parity, wc, PH_ERR_EPI); };
+    for (int j = 0; j < n_tiles; ++j) {
+      if (aborted()) break;
       const bool tok_valid = tok_a + j * 128 + r < tok_b;
 #pragma unroll
       for (int step = 0; step < 4; ++step) {                        // H half 0, H half 1, U half 0, U half 1
-        if (!wait(&bars->acc_ready, n_acc & 1)) break;
+        wait(&bars->acc_ready, n_acc & 1);
         ++n_acc;
         tc_fence_after();
         const int half = step & 1;
@@ -339,10 +343,11 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
         }
         fence_proxy_async_smem();
         tc_fence_before();
-        mbar_arrive(smem_u32(&bars->epi_done));
+        mbar_arrive_warp(smem_u32(&bars->epi_done), lane);
       }
     }
-    if (alive && wait(&bars->out_ready, 0)) {
+    wait(&bars->out_ready, 0);
+    if (!aborted()) {
       // flush: lane r holds feature c*128 + r of half c; this thread writes its 64 columns
       tc_fence_after();
       float* base = a.partial + (((size_t)ci * a.n_split + blockIdx.x) * g.BH + bh) * PH_DP * PH_SD;

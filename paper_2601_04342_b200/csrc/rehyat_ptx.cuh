@@ -36,6 +36,13 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// One arrival for the whole warp: every lane has finished (and fenced) its part, the warp synchronises, one lane
+// arrives.  The barrier counts warps, not threads: thirty-two arrivals on one address are thirty-two serialised
+// shared-memory atomics in front of whoever waits for the barrier.
+__device__ __forceinline__ void mbar_arrive_warp(uint32_t bar, int lane) {
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar);
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -82,22 +89,31 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
+__device__ __forceinline__ int wait_ctx_aborted(uint32_t wctx) {     // abort_flag is the first word of the context
+  int f;
+  asm volatile("ld.volatile.shared.b32 %0, [%1];" : "=r"(f) : "r"(wctx));
+  return f;
+}
+// The slow path is on the critical path of the roles that wait often (a try_wait that fails returns within a few
+// hundred cycles), so it polls the barrier and the CTA's abort flag only; the global epoch and the timer are
+// looked at once per 1024 polls (some tens of microseconds).
 __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t wctx, int code) {
-  volatile WaitCtx* w = reinterpret_cast<volatile WaitCtx*>(__cvta_shared_to_generic(wctx));
   const unsigned long long t0 = global_timer_ns();
-  for (uint32_t i = 0;; ++i) {
+  for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (w->abort_flag) return false;
-    if ((i & 63u) == 63u) {
+    if (wait_ctx_aborted(wctx)) return false;
+    if ((i & 1023u) == 0u) {
+      volatile WaitCtx* w = reinterpret_cast<volatile WaitCtx*>(__cvta_shared_to_generic(wctx));
       if (*reinterpret_cast<volatile int*>(w->status + 1) == w->epoch) { w->abort_flag = 1; return false; }
-      if (global_timer_ns() - t0 > w->limit_ns) break;
+      if (global_timer_ns() - t0 > w->limit_ns) {
+        w->abort_flag = 1;
+        atomicOr(w->status, code);
+        atomicExch(w->status + 1, w->epoch);
+        return false;
+      }
       __nanosleep(64);
     }
   }
-  w->abort_flag = 1;
-  atomicOr(w->status, code);
-  atomicExch(w->status + 1, w->epoch);
-  return false;
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t wctx, int code) {
   if (mbar_try_wait(bar, parity)) return true;

@@ -73,9 +73,9 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
     for (int s = 0; s < RD_RING; ++s) {
       mbar_init(smem_u32(&bars->ring_full[s]), 1); mbar_init(smem_u32(&bars->ring_empty[s]), 1);
     }
-    for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&bars->acc_ready[b]), 1); mbar_init(smem_u32(&bars->epi_done[b]), 256); }
-    mbar_init(smem_u32(&bars->out_ready), 1); mbar_init(smem_u32(&bars->out_read), 256);
-    mbar_init(smem_u32(&bars->nl_ready), 256); mbar_init(smem_u32(&bars->drained), 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&bars->acc_ready[b]), 1); mbar_init(smem_u32(&bars->epi_done[b]), 8); }
+    mbar_init(smem_u32(&bars->out_ready), 1); mbar_init(smem_u32(&bars->out_read), 8);
+    mbar_init(smem_u32(&bars->nl_ready), 8); mbar_init(smem_u32(&bars->drained), 1);
     wait_ctx_init(&bars->wctx, a.wa);
     fence_mbar_init();
   }
@@ -155,11 +155,12 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       constexpr uint32_t id_kk = idesc_bf16(128, 128, 0, 0);       // A K-major (smem or TMEM), B K-major: the MLP GEMMs
       constexpr uint32_t id_rd = idesc_bf16(128, 128, 0, 1);       // A = phi (K-major), B = state (MN-major)
       uint32_t ring_i = 0, n_epi[2] = {0, 0};
-      bool alive = true;                                            // false once a wait has been given up: issue nothing more
-      auto wait = [&](uint64_t* bar, uint32_t parity) {
-        alive = alive && mbar_wait(smem_u32(bar), parity, wc, PH_ERR_MMA);
-        if (alive) tc_fence_after();
-        return alive;
+      // A wait that is given up ends the role at once: the helpers return false and run() returns, so nothing
+      // further is issued.  No flag is carried along; the hot path pays one predicated branch per wait.
+      auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
+        if (!mbar_wait(smem_u32(bar), parity, wc, PH_ERR_MMA)) return false;
+        tc_fence_after();
+        return true;
       };
       auto ring_wait = [&]() -> uint32_t {                          // 0 on abort
         const int s = ring_i % RD_RING;
@@ -169,13 +170,15 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         umma_commit(smem_u32(&bars->ring_empty[ring_i % RD_RING]));
         ++ring_i;
       };
-      auto wait_epi = [&](int b) {                                  // the next epilogue that used scratch b is done
-        if (wait(&bars->epi_done[b], n_epi[b] & 1)) ++n_epi[b];
+      auto wait_epi = [&](int b) -> bool {                          // the next epilogue that used scratch b is done
+        if (!wait(&bars->epi_done[b], n_epi[b] & 1)) return false;
+        ++n_epi[b];
+        return true;
       };
-      auto h_half = [&](int b) {                                    // H[:, 128 b : 128 b + 128] = X W1[...]^T into scratch b
+      auto h_half = [&](int b) -> bool {                            // H[:, 128 b : 128 b + 128] = X W1[...]^T into scratch b
         for (int ks = 0; ks < 2; ++ks) {
           const uint32_t bt = ring_wait();
-          if (!bt) return;
+          if (!bt) return false;
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
             umma_ss(tmem + T_SCR + b * 128, smem_desc_sw128(sX + ks * PH_SUB + kk * 32, 16, 1024),
@@ -183,11 +186,12 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
           ring_release();
         }
         umma_commit(smem_u32(&bars->acc_ready[b]));
+        return true;
       };
-      auto u_half = [&](int b) {                                    // U[:, 128 b : ...] = H W2[...]^T with H read from TMEM
+      auto u_half = [&](int b) -> bool {                            // U[:, 128 b : ...] = H W2[...]^T with H read from TMEM
         for (int ks = 0; ks < 4; ++ks) {
           const uint32_t bt = ring_wait();
-          if (!bt) return;
+          if (!bt) return false;
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
             umma_ts(tmem + T_SCR + b * 128, tmem + T_H + (ks * 4 + kk) * 8, smem_desc_sw128(bt + kk * 32, 16, 1024), id_kk,
@@ -195,46 +199,47 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
           ring_release();
         }
         umma_commit(smem_u32(&bars->acc_ready[b]));
+        return true;
       };
-      auto readout_half = [&](int c, uint32_t phi_base) {           // R (+)= phi[:, 128 c : ...] s_t[128 c : ..., :]
+      auto readout_half = [&](int c, uint32_t phi_base) -> bool {   // R (+)= phi[:, 128 c : ...] s_t[128 c : ..., :]
         for (int f = 0; f < 2; ++f) {
           const uint32_t bt = ring_wait();
-          if (!bt) return;
+          if (!bt) return false;
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
             umma_ss(tmem + T_R, smem_desc_sw128(phi_base + f * PH_SUB + kk * 32, 16, 1024),
                     smem_desc_sw128(bt + kk * 2048, 8192, 1024), id_rd, (c | f | kk) != 0);
           ring_release();
         }
+        return true;
       };
-      for (int j = 0; j < n_tiles && alive; ++j) {
-        if (!wait(&bars->x_full, j & 1)) break;
-        if (j > 0) wait_epi(0);                                     // U half 0 of tile j-1: scratch A free, phi half 0 written
-        h_half(0);
-        if (j > 0) {
-          if (j > 1 && !wait(&bars->out_read, (j - 2) & 1)) break;  // the read-out of tile j-2 has left TMEM
-          readout_half(0, sPhi0);
-          wait_epi(1);                                              // U half 1 of tile j-1
+      auto run = [&]() {
+        for (int j = 0; j < n_tiles; ++j) {
+          if (!wait(&bars->x_full, j & 1)) return;
+          if (j > 0 && !wait_epi(0)) return;                          // U half 0 of tile j-1: scratch A free, phi half 0 written
+          if (!h_half(0)) return;
+          if (j > 0) {
+            if (j > 1 && !wait(&bars->out_read, (j - 2) & 1)) return; // the read-out of tile j-2 has left TMEM
+            if (!readout_half(0, sPhi0)) return;
+            if (!wait_epi(1)) return;                                 // U half 1 of tile j-1
+          }
+          if (!h_half(1)) return;
+          umma_commit(smem_u32(&bars->x_empty));
+          if (j > 0) {
+            if (!readout_half(1, sPhi1)) return;
+            umma_commit(smem_u32(&bars->out_ready));
+          }
+          if (!wait_epi(0) || !wait_epi(1)) return;                   // all of H is in TMEM
+          if (!u_half(0) || !u_half(1)) return;
         }
-        h_half(1);
-        if (!alive) break;
-        umma_commit(smem_u32(&bars->x_empty));
-        if (j > 0) {
-          readout_half(1, sPhi1);
-          if (!alive) break;
-          umma_commit(smem_u32(&bars->out_ready));
-        }
-        wait_epi(0);
-        wait_epi(1);                                                // all of H is in TMEM
-        u_half(0);
-        u_half(1);
-      }
-      wait_epi(0);
-      if (n_tiles > 1) wait(&bars->out_read, (n_tiles - 2) & 1);
-      readout_half(0, sPhi0);
-      wait_epi(1);
-      readout_half(1, sPhi1);
-      if (alive) umma_commit(smem_u32(&bars->out_ready));
+        if (!wait_epi(0)) return;
+        if (n_tiles > 1 && !wait(&bars->out_read, (n_tiles - 2) & 1)) return;
+        if (!readout_half(0, sPhi0)) return;
+        if (!wait_epi(1)) return;
+        if (!readout_half(1, sPhi1)) return;
+        umma_commit(smem_u32(&bars->out_ready));
+      };
+      run();
       // Everything this thread has issued is complete once `drained` flips; the abort flag does not cut this
       // wait short, so that TMEM is never freed with a tcgen05.mma still running.
       umma_commit(smem_u32(&bars->drained));
@@ -249,12 +254,12 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
     const uint32_t lane_off = (uint32_t)(qd * 32) << 16;
     uint32_t n_acc[2] = {0, 0};
     const int part_w = PH_DP / (PC ? PC : a.P);                     // a multiple of 32 (P in {1,2,4})
-    // A wait that was given up ends the role; the warp decides together (tcgen05.ld / st need all 32 lanes).
-    bool alive = true;
-    auto wait = [&](uint64_t* bar, uint32_t parity) {
-      alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, wc, PH_ERR_EPI));
-      return alive;
-    };
+    // After a wait has been given up anywhere in the CTA every later wait returns at once.  These warps then run
+    // through the rest of the current tile on whatever the accumulators hold (tcgen05.ld / st need all 32 lanes,
+    // so nothing is skipped lane by lane; every address stays inside the CTA's TMEM and shared memory) and leave
+    // at the head of the next tile, where the whole warp looks at the flag together.
+    auto aborted = [&]() -> bool { return __any_sync(0xffffffffu, wait_ctx_aborted(wc) != 0); };
+    auto wait = [&](uint64_t* bar, uint32_t parity) { mbar_wait(smem_u32(bar), parity, wc, PH_ERR_EPI); };
     // bias + activation (+ power) of 32 accumulator columns -> 16 bf16 pairs
     auto activate = [&](const uint32_t (&x)[32], const float* bias, bool is_u, int col0, uint32_t (&w)[16]) {
       if (RELU) {
@@ -289,9 +294,10 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       }
     };
     auto readout_store = [&](int jt) {                              // fp32 read-out of tile jt leaves TMEM
-      if (!alive || !wait(&bars->out_ready, jt & 1)) return;
+      wait(&bars->out_ready, jt & 1);
       tc_fence_after();
-      if (!wait(&bars->nl_ready, jt & 1)) return;                    // both halves of the tile's phi.z sums are written
+      wait(&bars->nl_ready, jt & 1);                                 // both halves of the tile's phi.z sums are written
+      if (aborted()) return;                                         // nothing of an abandoned launch is stored
       const float* nlp = s_nl + (jt & 1) * 256;
       const bool tok_valid = tok_a + jt * 128 + r < tok_b;
       const int ric = tok_a + jt * 128 + r - q0;                    // row inside the chunk; its tile is 128-aligned
@@ -310,14 +316,15 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       }
       if (tok_valid && ch == 1) a.rd[rd_index(g, a.rd_rows, PH_D, bh, ci, ric, PH_D / 4)] = nlp[r] + nlp[128 + r];
       tc_fence_before();
-      mbar_arrive(smem_u32(&bars->out_read));
+      mbar_arrive_warp(smem_u32(&bars->out_read), lane);
     };
-    for (int j = 0; j < n_tiles && alive; ++j) {
+    for (int j = 0; j < n_tiles; ++j) {
+      if (aborted()) break;
       const bool tok_valid = tok_a + j * 128 + r < tok_b;
       // H halves: bias, activation, bf16, back to TMEM as the A operand of the second GEMM
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
-        if (!wait(&bars->acc_ready[half], n_acc[half] & 1)) break;
+        wait(&bars->acc_ready[half], n_acc[half] & 1);
         ++n_acc[half];
         tc_fence_after();
         uint32_t x[2][32];
@@ -333,15 +340,14 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         }
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(smem_u32(&bars->epi_done[half]));
+        mbar_arrive_warp(smem_u32(&bars->epi_done[half]), lane);
       }
-      if (!alive) break;
       if (j > 0) readout_store(j - 1);
       // U halves: bias, activation, power, bf16, to the swizzled phi tiles; phi . z_t on the way
       float nl = 0.f;
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
-        if (!wait(&bars->acc_ready[half], n_acc[half] & 1)) break;
+        wait(&bars->acc_ready[half], n_acc[half] & 1);
         ++n_acc[half];
         tc_fence_after();
         uint32_t x[2][32];
@@ -377,11 +383,11 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
           // precedes, for every thread, that thread's arrival for U half 0 of tile j-1, which the issuer
           // waited for before the MMAs of this tile could start.
           s_nl[(j & 1) * 256 + ch * 128 + r] = nl;
-          mbar_arrive(smem_u32(&bars->nl_ready));
+          mbar_arrive_warp(smem_u32(&bars->nl_ready), lane);
         }
         fence_proxy_async_smem();
         tc_fence_before();
-        mbar_arrive(smem_u32(&bars->epi_done[half]));
+        mbar_arrive_warp(smem_u32(&bars->epi_done[half]), lane);
       }
     }
     readout_store(n_tiles - 1);

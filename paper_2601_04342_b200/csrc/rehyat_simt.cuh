@@ -249,7 +249,7 @@ constexpr int WIN_BM = 32, WIN_BN = 64, WIN_THREADS = 128;
 template <typename T, int D>
 __global__ void __launch_bounds__(WIN_THREADS)
 window_simt(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, T* __restrict__ out,
-            Geo g, const float* __restrict__ rd, int rd_rows, float scale, int c_mode) {
+            Geo g, const float* __restrict__ rd, int rd_rows, float scale, int c_mode, float* __restrict__ share) {
   extern __shared__ __align__(16) float smem[];
   constexpr int LDK = D + 4, LDP = WIN_BN + 4;
   constexpr int DC = D / 16;                 // output columns per thread
@@ -375,6 +375,7 @@ window_simt(const T* __restrict__ q, const T* __restrict__ k, const T* __restric
       nL = rd[rd_index(g, rd_rows, D, bh, ci, row - q0, D / 4)];
     }
     const float inv = 1.f / (l[i] * ws + lam * nL);
+    if (share != nullptr && tx == 0) share[(size_t)bh * g.N + row] = lam * nL * inv;   // part of the normaliser that is linear
     T* orow = out + hoff + (long long)row * g.stride_n + tx * DC;
 #pragma unroll
     for (int c = 0; c < DC; ++c) {

@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
           const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ out, Geo g,
           const float* __restrict__ rd, int rd_rows, float scale, int c_mode, ptx::WaitArgs wa,
-          int n_items, int pairs) {
+          int n_items, int pairs, float* __restrict__ share) {
   using namespace ptx;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -102,10 +102,10 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     }
     for (int i = 0; i < TC_QT; ++i) {
       mbar_init(smem_u32(&bars->s_ready[i]), 1);
-      mbar_init(smem_u32(&bars->p_half[i][0]), TC_BM);
-      mbar_init(smem_u32(&bars->p_half[i][1]), TC_BM);
+      mbar_init(smem_u32(&bars->p_half[i][0]), TC_BM / 32);
+      mbar_init(smem_u32(&bars->p_half[i][1]), TC_BM / 32);
       mbar_init(smem_u32(&bars->pv_done[i]), 1);
-      mbar_init(smem_u32(&bars->o_free[i]), TC_BM);
+      mbar_init(smem_u32(&bars->o_free[i]), TC_BM / 32);
     }
     mbar_init(smem_u32(&bars->drained), 1);
     wait_ctx_init(&bars->wctx, wa);
@@ -340,7 +340,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             tmem_st32(tS + (cc >> 1) * 32, sr[cc >> 1]);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(smem_u32(&bars->p_half[i][cc >> 1]));       // P of 64 keys is in place
+            mbar_arrive_warp(smem_u32(&bars->p_half[i][cc >> 1]), lane);       // P of 64 keys is in place
           }
         }
       }
@@ -382,6 +382,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       n_s += n_kv;
       const float inv = 1.f / (l * ws + lam * nL);
       const float wsi = ws * inv, lami = lam * inv;
+      if (share != nullptr && valid) share[(size_t)w.bh * g.N + row] = lami * nL;   // part of the normaliser that is linear
 #pragma unroll
       for (int hh = 0; hh < 4; ++hh) {                               // 32 columns of O at a time
         uint32_t o[32];
@@ -389,7 +390,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         tmem_wait_ld();
         if (hh == 3) {                                               // O has been read: TMEM is free for the next item
           tc_fence_before();
-          mbar_arrive(smem_u32(&bars->o_free[i]));
+          mbar_arrive_warp(smem_u32(&bars->o_free[i]), lane);
         }
         if (valid) {
 #pragma unroll
@@ -426,6 +427,7 @@ struct TcWorkspace {
   int n_sm = 148;                       // SMs of the device
   int exp_poly = 1;                     // of every 4 pairs of exponentials, how many the FMA pipe evaluates
   int item_tiles = 0;                   // query tiles per window item: 1, 2, or 0 = chosen per launch
+  int last_item_tiles = 0;              // what the last window launch used
 };
 
 inline bool tc_shape_supported(bool bf16, int d, int, int, int, int, int) { return bf16 && d == TC_D; }
@@ -455,7 +457,7 @@ inline void tc_workspace_destroy(TcWorkspace* w) { cudaFree(w->state_bf16); w->s
 // window_tc1 (one query tile per item) and its launcher live in rehyat_tc_single.cuh
 inline int tc_launch_window1(int exp_poly, int n_sm, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                              __nv_bfloat16* o, const Geo& g, const float* rd, int rd_rows, float scale, int c_mode,
-                             const ptx::WaitArgs& wa, cudaStream_t st);
+                             const ptx::WaitArgs& wa, float* share, cudaStream_t st);
 inline bool tc_set_attributes1();
 
 inline int tc_set_attributes() {
@@ -500,8 +502,9 @@ inline bool tc_make_tmap_3d(const TcWorkspace* w, CUtensorMap* tm, const void* b
 }
 
 // Launches window_tc for the chunks of one group.  `rd` is the linear read-out of the group's queries.
-inline int tc_launch_window(const TcWorkspace* w, const void* q, const void* k, const void* v, void* out, const Geo& g,
-                            int batch, const float* rd, int rd_rows, int c_mode, const ptx::WaitArgs& wa, cudaStream_t st) {
+inline int tc_launch_window(TcWorkspace* w, const void* q, const void* k, const void* v, void* out, const Geo& g,
+                            int batch, const float* rd, int rd_rows, int c_mode, const ptx::WaitArgs& wa, float* share,
+                            cudaStream_t st) {
   CUtensorMap tq, tk, tv;
   if (!tc_make_tmap(w, &tq, q, g, batch) || !tc_make_tmap(w, &tk, k, g, batch) || !tc_make_tmap(w, &tv, v, g, batch))
     return REHYAT_ERR_CUDA;
@@ -515,10 +518,13 @@ inline int tc_launch_window(const TcWorkspace* w, const void* q, const void* k, 
   // of items over the SMs decide; per tile a one-tile item costs about 8 % more.
   const long long n1 = (long long)((g.Np + TC_BM - 1) / TC_BM) * g.G * g.BH;
   const double cost2 = 2.0 * (double)((n_items + w->n_sm - 1) / w->n_sm), cost1 = 1.08 * (double)((n1 + w->n_sm - 1) / w->n_sm);
-  if (w->item_tiles == 1 || (w->item_tiles == 0 && cost1 < 0.93 * cost2))
-    return tc_launch_window1(w->exp_poly, w->n_sm, tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, st);
+  if (w->item_tiles == 1 || (w->item_tiles == 0 && cost1 < 0.93 * cost2)) {
+    w->last_item_tiles = 1;
+    return tc_launch_window1(w->exp_poly, w->n_sm, tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, share, st);
+  }
+  w->last_item_tiles = 2;
 #define REHYAT_LAUNCH_WINDOW(E) \
-  window_tc<E><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, n_items, pairs)
+  window_tc<E><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, n_items, pairs, share)
   switch (w->exp_poly) {
     case 0: REHYAT_LAUNCH_WINDOW(0); break;
     case 2: REHYAT_LAUNCH_WINDOW(2); break;

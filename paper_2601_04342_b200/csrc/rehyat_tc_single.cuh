@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ out, Geo g,
            const float* __restrict__ rd, int rd_rows, float scale, int c_mode, ptx::WaitArgs wa,
-           int n_items, int tiles) {
+           int n_items, int tiles, float* __restrict__ share) {
   using namespace ptx;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -74,13 +74,13 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&bars->s_ready[i]), 1);
-      mbar_init(smem_u32(&bars->p_half[i][0]), TC_BM);
-      mbar_init(smem_u32(&bars->p_half[i][1]), TC_BM);
+      mbar_init(smem_u32(&bars->p_half[i][0]), TC_BM / 32);
+      mbar_init(smem_u32(&bars->p_half[i][1]), TC_BM / 32);
       mbar_init(smem_u32(&bars->pv_done[i]), 1);
-      mbar_init(smem_u32(&bars->o_free[i]), TC_BM);
+      mbar_init(smem_u32(&bars->o_free[i]), TC_BM / 32);
     }
     mbar_init(smem_u32(&bars->drained), 1);
-    mbar_init(smem_u32(&bars->mrg_ready), 2 * TC_BM);
+    mbar_init(smem_u32(&bars->mrg_ready), 2 * TC_BM / 32);
     wait_ctx_init(&bars->wctx, wa);
     fence_mbar_init();
   }
@@ -311,7 +311,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             tmem_st32(tS + (cc >> 1) * 32, sr[cc >> 1]);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(smem_u32(&bars->p_half[i][cc >> 1]));       // P of 64 keys is in place
+            mbar_arrive_warp(smem_u32(&bars->p_half[i][cc >> 1]), lane);       // P of 64 keys is in place
           }
         }
       }
@@ -326,7 +326,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       // barrier of an item completes only with the arrivals of both.
       float (*mrg)[3][TC_BM] = bars->mrg[n_items_done & 1];
       mrg[i][0][r] = m_used; mrg[i][1][r] = m_true; mrg[i][2][r] = l;
-      mbar_arrive(smem_u32(&bars->mrg_ready));
+      mbar_arrive_warp(smem_u32(&bars->mrg_ready), lane);
       if (!wait(&bars->mrg_ready, n_items_done & 1)) break;
       ++n_items_done;
       const float mu_x = mrg[i ^ 1][0][r], mt_x = mrg[i ^ 1][1][r], l_x = mrg[i ^ 1][2][r];
@@ -364,6 +364,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       n_s[0] += cnt0; n_s[1] += cnt1;
       const float inv = 1.f / (l0 * f0 + l1 * f1 + lam * nL);
       const float w0 = f0 * inv, w1 = f1 * inv, lami = lam * inv;
+      if (share != nullptr && valid && i == 0) share[(size_t)w.bh * g.N + row] = lami * nL;   // part of the normaliser that is linear
       const uint32_t tO0 = tmem + lane_off + 256 + i * (TC_D / 2);
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh) {                               // 32 columns at a time
@@ -378,7 +379,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         tmem_wait_ld();
         if (hh == 1) {                                               // this warpgroup has read both slots
           tc_fence_before();
-          mbar_arrive(smem_u32(&bars->o_free[i]));
+          mbar_arrive_warp(smem_u32(&bars->o_free[i]), lane);
         }
         if (valid) {
 #pragma unroll
@@ -408,12 +409,12 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 // Launches window_tc1 with the tensor maps and arguments tc_launch_window has prepared.
 inline int tc_launch_window1(int exp_poly, int n_sm, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                              __nv_bfloat16* o, const Geo& g, const float* rd, int rd_rows, float scale, int c_mode,
-                             const ptx::WaitArgs& wa, cudaStream_t st) {
+                             const ptx::WaitArgs& wa, float* share, cudaStream_t st) {
   const int tiles = (g.Np + TC_BM - 1) / TC_BM;
   const int n_items = tiles * g.G * g.BH;
   const dim3 grid(n_items < n_sm ? n_items : n_sm);
 #define REHYAT_LAUNCH_WINDOW1(E) \
-  window_tc1<E><<<grid, TC_THREADS, TC_WIN1_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, n_items, tiles)
+  window_tc1<E><<<grid, TC_THREADS, TC_WIN1_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, n_items, tiles, share)
   switch (exp_poly) {
     case 0: REHYAT_LAUNCH_WINDOW1(0); break;
     case 2: REHYAT_LAUNCH_WINDOW1(2); break;

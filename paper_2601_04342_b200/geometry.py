@@ -71,3 +71,30 @@ def shard_heads(B: int, n_heads: int, world_size: int, rank: int):
     base, rem = divmod(units, world_size)
     u0 = rank * base + min(rank, rem)
     return u0, u0 + base + (1 if rank < rem else 0)
+
+
+def shard_rects(B: int, n_heads: int, world_size: int, rank: int):
+    """The slice of shard_heads as rectangles (b0, nb, h0, nh) of whole (batch, head) blocks, in unit order:
+    a slice that starts or ends inside a batch item is cut at the batch boundaries.  Each rectangle is one
+    operator call on `nh` heads (a context with that head count, tensor and phi pointers offset to head h0)."""
+    u0, u1 = shard_heads(B, n_heads, world_size, rank)
+    rects = []
+    u = u0
+    while u < u1:
+        b, h = divmod(u, n_heads)
+        if h == 0 and u1 - u >= n_heads:                 # whole batch items
+            nb = (u1 - u) // n_heads
+            rects.append((b, nb, 0, n_heads))
+            u += nb * n_heads
+        else:                                            # the rest of batch item b, or up to the slice's end
+            nh = min(n_heads - h, u1 - u)
+            rects.append((b, 1, h, nh))
+            u += nh
+    return rects
+
+
+def shard_efficiency(B: int, n_heads: int, world_size: int):
+    """Units the busiest rank owns against a perfectly even split: the efficiency a head-sharded layer can
+    reach at most (12 heads over 8 ranks: 12 / (8 * 2) = 0.75)."""
+    most = max(u1 - u0 for u0, u1 in (shard_heads(B, n_heads, world_size, r) for r in range(world_size)))
+    return B * n_heads / (world_size * most) if most else 0.0

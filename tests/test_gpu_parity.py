@@ -152,6 +152,28 @@ def test_groups_smaller_than_the_sequence_carry_the_state():
     assert np.max(np.abs(y_one - y_many) / (1e-3 + np.abs(y_one))) <= 2.0 ** -6
 
 
+@pytest.mark.parametrize("impl,c_mode", [("auto", "rowmax"), ("auto", "zero"), ("simt", "rowmax")])
+def test_linear_share_of_the_normaliser(impl, c_mode):
+    """rehyat_set_linear_share_output: nL / (nS + nL) per query row (Eq. 8, 9) as the window kernels weigh it,
+    against the same ratio from the oracle's explicit sums."""
+    from paper_2601_04342_b200 import binding
+    wl = synth.Workload("share", 2, 2, 128, 5, 10, 20, 2, 1, "bf16", True, seed=synth.BASE_SEED + 88)
+    x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
+    ref, frac = oracle_full(wl, x, c_mode)
+    d = _to_dev(x)
+    op = binding.for_workload(wl, impl=impl, c_mode=c_mode)
+    share = torch.full((wl.B, wl.n_heads, wl.N), -1.0, device="cuda")
+    op.set_linear_share_output(share)
+    y = op.forward(d["q"], d["k"], d["v"], d["phi_q"], d["phi_k"], wl.T, wl.H, wl.W, wl.Tc, wl.To)
+    assert op.status() == 0
+    check(y.double().cpu().numpy(), ref, "bf16")
+    got = share.double().cpu().numpy()
+    assert frac.max() > 0.3 and np.abs(got - frac).max() <= 5e-3
+    assert (got[:, :, :wl.Tc * wl.HW] == 0).all()            # chunk 0 has no linear set
+    op.set_linear_share_output(None)
+    op.close()
+
+
 def test_token_major_layout():
     wl = synth.Workload("l", 2, 2, 128, 4, 10, 20, 2, 1, "bf16", True, seed=synth.BASE_SEED + 80)
     x = synth.make_inputs(wl, phi_scale=1.5)

@@ -58,3 +58,25 @@ def test_synth_is_seeded_and_shaped():
     rms = x["q"].float().pow(2).mean(-1).sqrt()
     assert (rms - 1).abs().max() < 2e-2
     assert len(synth.sweep_configs()) == 18
+
+
+def test_shard_rects_cover_every_unit_once_and_in_order():
+    for B, nh, world in ((1, 12, 8), (2, 12, 8), (2, 12, 5), (3, 5, 4), (1, 3, 8), (4, 2, 3)):
+        seen = []
+        for r in range(world):
+            u0, u1 = geo.shard_heads(B, nh, world, r)
+            mine = []
+            for (b0, nb, h0, n) in geo.shard_rects(B, nh, world, r):
+                assert nb >= 1 and n >= 1 and h0 + n <= nh and b0 + nb <= B
+                assert nb == 1 or (h0 == 0 and n == nh)            # several batch items only as whole items
+                mine += [b * nh + h for b in range(b0, b0 + nb) for h in range(h0, h0 + n)]
+            assert mine == list(range(u0, u1))
+            seen += mine
+        assert seen == list(range(B * nh))
+
+
+def test_shard_efficiency():
+    assert geo.shard_efficiency(1, 12, 8) == 0.75                  # 12 heads over 8 ranks: 2/1 imbalance
+    assert geo.shard_efficiency(1, 12, 4) == 1.0
+    assert geo.shard_efficiency(2, 12, 8) == 1.0
+    assert geo.shard_efficiency(1, 12, 1) == 1.0
