@@ -91,19 +91,33 @@ class ClockSampler:
 
     def _pump(self):
         for line in self.proc.stdout:
-            self.lines.append(line)
+            self.lines.append((time.time(), line))
 
-    def stop(self):
+    def wait_running(self, timeout=5.0):
+        """Blocks until the first sample has arrived (nvidia-smi takes a while to start), so that a short timed
+        region that follows is sampled from its start."""
+        t_end = time.time() + timeout
+        while self.proc is not None and not self.lines and time.time() < t_end:
+            time.sleep(0.005)
+
+    def stop(self, t0=None, t1=None):
+        """Summary of the samples that arrived in the host-time window [t0, t1] (all samples if no window is
+        given; the sample nearest to the window if it was shorter than the sampling period)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.03)                               # one more sampling period: the last sample of the window
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
+        lines = self.lines
+        if t0 is not None and lines:
+            inside = [x for x in lines if t0 <= x[0] <= t1 + 0.03]
+            lines = inside or [min(lines, key=lambda x: abs(x[0] - 0.5 * (t0 + t1)))]
         sm, smax, reasons, power = [], [], set(), []
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in self.lines:
+        for _, line in lines:
             tok = [t.strip() for t in line.split(",")]
             if len(tok) < 9:
                 continue
@@ -416,15 +430,17 @@ def main():
     flops = geometry.flop_model(wl.B, wl.n_heads, wl.head_dim, wl.T, wl.HW, wl.Tc, wl.To, wl.D_h, wl.D_out)
     sampler = ClockSampler(local_rank)
     op.profile_enable(True)
-    barrier()
     sampler.start()
+    sampler.wait_running()
+    barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_host0 = time.time()
     e0.record(stream)
     for _ in range(args.steps):
         step()
     e1.record(stream)
     barrier()
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_host0, time.time())
     ms_total = e0.elapsed_time(e1)
     prof = op.profile_read()
     op.profile_enable(False)
@@ -502,6 +518,7 @@ def main():
         sus_sampler = ClockSampler(local_rank)
         torch.cuda.synchronize()
         sus_sampler.start()
+        sus_sampler.wait_running()
         sus_ms = _time_ms(step, stream, 3, n_sus)
         sus_clocks = sus_sampler.stop()
         sus_tf = flops["total"] / (sus_ms * 1e-3) / 1e12

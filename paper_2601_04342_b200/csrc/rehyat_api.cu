@@ -161,6 +161,7 @@ template <typename T, int D>
 int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* out, const rehyat_phi_params* phi,
                       const Geo& g, int n_split, int carry_slot, int parts, cudaStream_t st) {
   const rehyat_config& c = ctx->cfg;
+  const int rd_half = ctx->tensor_ok ? 1 : 0;     // the tensor-core window kernels read the bf16 form of the read-out
   PhiDims pd = {D, c.phi_hidden, c.phi_dim, c.poly_degree, c.act_hidden, c.act_out};
   constexpr int SD = D + 4;
   const int tiles = (g.Np + SIMT_TM - 1) / SIMT_TM;
@@ -183,7 +184,7 @@ int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* ou
     const size_t smem_rd = (size_t)SIMT_TM * (D + pd.Dh + pd.Dp) * sizeof(float);
     ctx->prof.begin(REHYAT_PROF_READOUT, st);
     readout_simt<T, D><<<dim3(tiles, g.G, g.BH), SIMT_PHI_THREADS, smem_rd, st>>>(q, wq, pd, g, ctx->state,
-                                                                                 ctx->readout, ctx->rd_cap);
+                                                                                 ctx->readout, ctx->rd_cap, rd_half);
     ctx->prof.end(REHYAT_PROF_READOUT, st);
     ctx->last_launches += 1;
   }
@@ -353,7 +354,10 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
   const size_t SD = c.head_dim + 4;
   const size_t slot = (size_t)ctx->bh_max * c.phi_dim * SD * sizeof(float);
   const size_t b_state = slot * ctx->Gmax, b_partial = slot * ctx->partial_units;
-  const size_t b_rd = (size_t)ctx->bh_max * ctx->rd_cap * SD * sizeof(float);
+  // read-out of one chunk group: fp32 rows of d + 4 for the SIMT window kernel, RDH_PIECES 16-byte pieces per row
+  // (bf16) for the tensor-core ones
+  const size_t b_rd = ctx->tensor_ok ? (size_t)ctx->bh_max * ctx->rd_cap * RDH_PIECES * 16
+                                     : (size_t)ctx->bh_max * ctx->rd_cap * SD * sizeof(float);
   bool ok = cudaMalloc(&ctx->state, b_state) == cudaSuccess && cudaMalloc(&ctx->partial, b_partial) == cudaSuccess &&
             cudaMalloc(&ctx->readout, b_rd) == cudaSuccess && cudaMalloc(&ctx->status_dev, 256) == cudaSuccess;
   ctx->ws_bytes = b_state + b_partial + b_rd + 256;

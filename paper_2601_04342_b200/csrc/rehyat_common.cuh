@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -50,6 +51,31 @@ __host__ __device__ inline size_t rd_index(const Geo& g, int rd_rows, int d, int
   const int tiles = (g.Np + 127) >> 7;
   const size_t tile = (size_t)bh * (size_t)(rd_rows >> 7) + (size_t)ci * tiles + (size_t)(row_in_chunk >> 7);
   return ((tile * (size_t)(d / 4 + 1) + (size_t)c4) * 128 + (size_t)(row_in_chunk & 127)) * 4;
+}
+
+// The same workspace as the tensor-core kernels keep it (bf16 operator, head_dim 128): nL_i = phi_q(q_i) z_t in
+// fp32 and the d columns of the RATIO aL_i / nL_i = phi_q(q_i) s_t / nL_i in fp16, eight to a 16-byte piece:
+// RDH_PIECES pieces per 128-row tile (the last one holds nL in its first word), each with the tile's rows
+// contiguous.  For non-negative features the ratio is a weighted mean of the v_j, so it fits fp16 whatever the
+// size of the sums, and its rounding (2^-11 relative) is below the bf16 rounding of the output; a ratio beyond the
+// fp16 range (features of both signs, nL near zero: Eq. 5 is then indefinite anyway) is clamped.  The workspace
+// and the traffic between the read-out and the window kernel are half of the fp32 form.  Returns the index of
+// the 16-byte piece `piece` of the row.
+constexpr int RDH_PIECES = 128 / 8 + 1;
+__host__ __device__ inline size_t rdh_index(const Geo& g, int rd_rows, int bh, int ci, int row_in_chunk, int piece) {
+  const int tiles = (g.Np + 127) >> 7;
+  const size_t tile = (size_t)bh * (size_t)(rd_rows >> 7) + (size_t)ci * tiles + (size_t)(row_in_chunk >> 7);
+  return (tile * (size_t)RDH_PIECES + (size_t)piece) * 128 + (size_t)(row_in_chunk & 127);
+}
+
+// Packs two ratios (see rdh_index) into one fp16 pair, clamped to the finite fp16 range.
+__device__ __forceinline__ uint32_t pack_ratio_f16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float2 unpack_f16(uint32_t pair) {
+  return __half22float2(*reinterpret_cast<const __half2*>(&pair));
 }
 
 __device__ __forceinline__ long long head_offset(const Geo& g, int bh) {

@@ -57,7 +57,7 @@ struct PhiTcArgs {
   int n_split;                 // state kernel: splits of a chunk's increment
   float* partial;              // state kernel: [G][n_split][BH][256][132]
   const float* state;          // read-out kernel: fp32 states (z column is read)
-  float* rd;                   // read-out kernel: the read-out workspace (see rd_index)
+  float* rd;                   // read-out kernel: the read-out workspace (see rdh_index)
   int rd_rows;
   int tiles_per_cta;           // read-out kernel
   ptx::WaitArgs wa;            // status word, launch epoch, wait limit

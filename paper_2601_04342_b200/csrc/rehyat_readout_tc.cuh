@@ -301,6 +301,9 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       const float* nlp = s_nl + (jt & 1) * 256;
       const bool tok_valid = tok_a + jt * 128 + r < tok_b;
       const int ric = tok_a + jt * 128 + r - q0;                    // row inside the chunk; its tile is 128-aligned
+      uint4* rdh = reinterpret_cast<uint4*>(a.rd);
+      const float nl_row = nlp[r] + nlp[128 + r];
+      const float inv_nl = nl_row != 0.f ? 1.f / nl_row : 0.f;       // the read-out is stored as the ratio aL / nL
 #pragma unroll
       for (int cb = 0; cb < 2; ++cb) {
         uint32_t x[32];
@@ -308,13 +311,16 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         tmem_wait_ld();
         if (tok_valid) {
 #pragma unroll
-          for (int e = 0; e < 32; e += 4)
-            *reinterpret_cast<float4*>(a.rd + rd_index(g, a.rd_rows, PH_D, bh, ci, ric, (ch * 64 + cb * 32 + e) >> 2)) =
-                make_float4(__uint_as_float(x[e]), __uint_as_float(x[e + 1]), __uint_as_float(x[e + 2]),
-                            __uint_as_float(x[e + 3]));
+          for (int e = 0; e < 32; e += 8)
+            rdh[rdh_index(g, a.rd_rows, bh, ci, ric, (ch * 64 + cb * 32 + e) >> 3)] =
+                make_uint4(pack_ratio_f16(__uint_as_float(x[e]) * inv_nl, __uint_as_float(x[e + 1]) * inv_nl),
+                           pack_ratio_f16(__uint_as_float(x[e + 2]) * inv_nl, __uint_as_float(x[e + 3]) * inv_nl),
+                           pack_ratio_f16(__uint_as_float(x[e + 4]) * inv_nl, __uint_as_float(x[e + 5]) * inv_nl),
+                           pack_ratio_f16(__uint_as_float(x[e + 6]) * inv_nl, __uint_as_float(x[e + 7]) * inv_nl));
         }
       }
-      if (tok_valid && ch == 1) a.rd[rd_index(g, a.rd_rows, PH_D, bh, ci, ric, PH_D / 4)] = nlp[r] + nlp[128 + r];
+      if (tok_valid && ch == 1)
+        rdh[rdh_index(g, a.rd_rows, bh, ci, ric, RDH_PIECES - 1)] = make_uint4(__float_as_uint(nl_row), 0u, 0u, 0u);
       tc_fence_before();
       mbar_arrive_warp(smem_u32(&bars->out_read), lane);
     };

@@ -199,11 +199,12 @@ __global__ void combine_bidirectional(const float* __restrict__ cum, float* __re
 }
 
 // grid (tiles per chunk, G, BH), SIMT_PHI_THREADS threads.  Linear read-out of one tile of
-// SIMT_TM queries of chunk t: rd[bh][row in group][0..d) = phi_q(q_i) s_t, [d] = phi_q(q_i) z_t.
+// SIMT_TM queries of chunk t: rd[bh][row in group][0..d) = phi_q(q_i) s_t, [d] = phi_q(q_i) z_t, in the fp32
+// layout of rd_index or (rd_half, for the tensor-core window kernels) as fp16 ratios in the layout of rdh_index.
 template <typename T, int D>
 __global__ void __launch_bounds__(SIMT_PHI_THREADS)
 readout_simt(const T* __restrict__ q, PhiPtrs<T> wq, PhiDims pd, Geo g, const float* __restrict__ state,
-             float* __restrict__ rd, int rd_rows) {
+             float* __restrict__ rd, int rd_rows, int rd_half) {
   extern __shared__ __align__(16) float smem[];
   constexpr int SD = D + 4;
   float* Xs = smem;
@@ -224,8 +225,20 @@ readout_simt(const T* __restrict__ q, PhiPtrs<T> wq, PhiDims pd, Geo g, const fl
 
   const float* S = state + ((size_t)ci * g.BH + bh) * pd.Dp * SD;
   constexpr int RG = 4, RPG = SIMT_TM / RG;
-  for (int idx = threadIdx.x; idx < (D + 1) * RG; idx += blockDim.x) {
-    const int c = idx % (D + 1), r0 = (idx / (D + 1)) * RPG;
+  float* nl_s = Xs;                                    // phi_q(q_i) z_t of the tile's rows (Xs is no longer needed)
+  if (rd_half) {
+    // the tensor-core window kernels read the ratio aL / nL (see rdh_index): the denominators come first
+    for (int r = threadIdx.x; r < SIMT_TM; r += blockDim.x) {
+      float acc = 0.f;
+      for (int ff = 0; ff < pd.Dp; ++ff) acc = fmaf(Fs[r * pd.Dp + ff], S[(size_t)ff * SD + D], acc);
+      nl_s[r] = acc;
+      if (tok0 + r < q1) rd[rdh_index(g, rd_rows, bh, ci, tok0 + r - q0, RDH_PIECES - 1) * 4] = acc;
+    }
+    __syncthreads();
+  }
+  const int ncol = rd_half ? D : D + 1;
+  for (int idx = threadIdx.x; idx < ncol * RG; idx += blockDim.x) {
+    const int c = idx % ncol, r0 = (idx / ncol) * RPG;
     float acc[RPG];
 #pragma unroll
     for (int r = 0; r < RPG; ++r) acc[r] = 0.f;
@@ -237,7 +250,14 @@ readout_simt(const T* __restrict__ q, PhiPtrs<T> wq, PhiDims pd, Geo g, const fl
 #pragma unroll
     for (int r = 0; r < RPG; ++r) {
       const int tok = tok0 + r0 + r;
-      if (tok < q1) rd[rd_index(g, rd_rows, D, bh, ci, tok - q0, c >> 2) + (c & 3)] = acc[r];
+      if (tok >= q1) continue;
+      if (!rd_half) {
+        rd[rd_index(g, rd_rows, D, bh, ci, tok - q0, c >> 2) + (c & 3)] = acc[r];
+      } else {
+        const float nl = nl_s[r0 + r], ratio = nl != 0.f ? acc[r] / nl : 0.f;
+        reinterpret_cast<__half*>(rd)[rdh_index(g, rd_rows, bh, ci, tok - q0, c >> 3) * 8 + (c & 7)] =
+            __float2half_rn(fminf(fmaxf(ratio, -65504.f), 65504.f));
+      }
     }
   }
 }

@@ -354,17 +354,17 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       const int row = w.row_base + i * TC_BM + (warp & 3) * 32 + lane;
       const bool valid = row < w.q1;
       // the whole read-out row is requested before the wait for the last P V, which hides its latency
-      float4 rdv[TC_D / 4];
+      uint4 rdv[TC_D / 8];                                           // fp16 pairs of aL / nL
       float nL = 0.f;
       if (w.linear) {
         const int ric = (valid ? row : w.q0) - w.q0, ci = w.ci;      // row inside the chunk: consecutive threads, consecutive pieces
+        const uint4* rdh = reinterpret_cast<const uint4*>(rd);
 #pragma unroll
-        for (int u = 0; u < TC_D / 4; ++u)
-          rdv[u] = __ldg(reinterpret_cast<const float4*>(rd + rd_index(g, rd_rows, TC_D, w.bh, ci, ric, u)));
-        nL = __ldg(rd + rd_index(g, rd_rows, TC_D, w.bh, ci, ric, TC_D / 4));
+        for (int u = 0; u < TC_D / 8; ++u) rdv[u] = __ldg(rdh + rdh_index(g, rd_rows, w.bh, ci, ric, u));
+        nL = __ldg(reinterpret_cast<const float*>(rdh + rdh_index(g, rd_rows, w.bh, ci, ric, RDH_PIECES - 1)));
       } else {
 #pragma unroll
-        for (int u = 0; u < TC_D / 4; ++u) rdv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int u = 0; u < TC_D / 8; ++u) rdv[u] = make_uint4(0u, 0u, 0u, 0u);
       }
       const float fin = ex2((m_used - m_true) * c);
       float ws = fin, lam = 0.f;
@@ -381,8 +381,8 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       tc_fence_after();
       n_s += n_kv;
       const float inv = 1.f / (l * ws + lam * nL);
-      const float wsi = ws * inv, lami = lam * inv;
-      if (share != nullptr && valid) share[(size_t)w.bh * g.N + row] = lami * nL;   // part of the normaliser that is linear
+      const float wsi = ws * inv, lami = lam * inv * nL;               // the read-out comes as the ratio aL / nL
+      if (share != nullptr && valid) share[(size_t)w.bh * g.N + row] = lami;       // part of the normaliser that is linear
 #pragma unroll
       for (int hh = 0; hh < 4; ++hh) {                               // 32 columns of O at a time
         uint32_t o[32];
@@ -395,12 +395,16 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         if (valid) {
 #pragma unroll
           for (int e = 0; e < 32; e += 8) {
-            const float4 x0 = rdv[hh * 8 + (e >> 2)], x1 = rdv[hh * 8 + (e >> 2) + 1];
+            const uint4 x = rdv[hh * 4 + (e >> 3)];                  // eight columns of aL / nL as fp16 pairs
+            auto fin = [&](int q, uint32_t pair) {
+              const float2 rr = unpack_f16(pair);
+              return pack_bf16(__uint_as_float(o[q]) * wsi + lami * rr.x, __uint_as_float(o[q + 1]) * wsi + lami * rr.y);
+            };
             uint4 v4;
-            v4.x = pack_bf16(__uint_as_float(o[e + 0]) * wsi + lami * x0.x, __uint_as_float(o[e + 1]) * wsi + lami * x0.y);
-            v4.y = pack_bf16(__uint_as_float(o[e + 2]) * wsi + lami * x0.z, __uint_as_float(o[e + 3]) * wsi + lami * x0.w);
-            v4.z = pack_bf16(__uint_as_float(o[e + 4]) * wsi + lami * x1.x, __uint_as_float(o[e + 5]) * wsi + lami * x1.y);
-            v4.w = pack_bf16(__uint_as_float(o[e + 6]) * wsi + lami * x1.z, __uint_as_float(o[e + 7]) * wsi + lami * x1.w);
+            v4.x = fin(e + 0, x.x);
+            v4.y = fin(e + 2, x.y);
+            v4.z = fin(e + 4, x.z);
+            v4.w = fin(e + 6, x.w);
             *reinterpret_cast<uint4*>(orow + hh * 32 + e) = v4;
           }
         }

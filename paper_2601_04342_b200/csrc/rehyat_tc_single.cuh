@@ -336,17 +336,17 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const int row = w.row_base + r;
       const bool valid = row < w.q1;
       // this warpgroup's half of the read-out row is requested before the wait for the last P V
-      float4 rdv[TC_D / 8];
+      uint4 rdv[TC_D / 16];                                          // fp16 pairs of aL / nL
       float nL = 0.f;
       if (w.linear) {
         const int ric = (valid ? row : w.q0) - w.q0, ci = w.ci;
+        const uint4* rdh = reinterpret_cast<const uint4*>(rd);
 #pragma unroll
-        for (int u = 0; u < TC_D / 8; ++u)
-          rdv[u] = __ldg(reinterpret_cast<const float4*>(rd + rd_index(g, rd_rows, TC_D, w.bh, ci, ric, i * (TC_D / 8) + u)));
-        nL = __ldg(rd + rd_index(g, rd_rows, TC_D, w.bh, ci, ric, TC_D / 4));
+        for (int u = 0; u < TC_D / 16; ++u) rdv[u] = __ldg(rdh + rdh_index(g, rd_rows, w.bh, ci, ric, i * (TC_D / 16) + u));
+        nL = __ldg(reinterpret_cast<const float*>(rdh + rdh_index(g, rd_rows, w.bh, ci, ric, RDH_PIECES - 1)));
       } else {
 #pragma unroll
-        for (int u = 0; u < TC_D / 8; ++u) rdv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int u = 0; u < TC_D / 16; ++u) rdv[u] = make_uint4(0u, 0u, 0u, 0u);
       }
       float f0 = ex2((mu0 - m_fin) * c), f1 = cnt1 > 0 ? ex2((mu1 - m_fin) * c) : 0.f, lam = 0.f;
       if (w.linear) {
@@ -363,8 +363,8 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       tc_fence_after();
       n_s[0] += cnt0; n_s[1] += cnt1;
       const float inv = 1.f / (l0 * f0 + l1 * f1 + lam * nL);
-      const float w0 = f0 * inv, w1 = f1 * inv, lami = lam * inv;
-      if (share != nullptr && valid && i == 0) share[(size_t)w.bh * g.N + row] = lami * nL;   // part of the normaliser that is linear
+      const float w0 = f0 * inv, w1 = f1 * inv, lami = lam * inv * nL;   // the read-out comes as the ratio aL / nL
+      if (share != nullptr && valid && i == 0) share[(size_t)w.bh * g.N + row] = lami;   // part of the normaliser that is linear
       const uint32_t tO0 = tmem + lane_off + 256 + i * (TC_D / 2);
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh) {                               // 32 columns at a time
@@ -384,13 +384,17 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         if (valid) {
 #pragma unroll
           for (int e = 0; e < 32; e += 8) {
-            const float4 x0 = rdv[hh * 8 + (e >> 2)], x1 = rdv[hh * 8 + (e >> 2) + 1];
-            auto fin = [&](int q, float x) { return __uint_as_float(o0[q]) * w0 + __uint_as_float(o1[q]) * w1 + lami * x; };
+            const uint4 x = rdv[hh * 4 + (e >> 3)];                  // eight columns of aL / nL as fp16 pairs
+            auto fin = [&](int q, uint32_t pair) {
+              const float2 rr = unpack_f16(pair);
+              return pack_bf16(__uint_as_float(o0[q]) * w0 + __uint_as_float(o1[q]) * w1 + lami * rr.x,
+                               __uint_as_float(o0[q + 1]) * w0 + __uint_as_float(o1[q + 1]) * w1 + lami * rr.y);
+            };
             uint4 v4;
-            v4.x = pack_bf16(fin(e + 0, x0.x), fin(e + 1, x0.y));
-            v4.y = pack_bf16(fin(e + 2, x0.z), fin(e + 3, x0.w));
-            v4.z = pack_bf16(fin(e + 4, x1.x), fin(e + 5, x1.y));
-            v4.w = pack_bf16(fin(e + 6, x1.z), fin(e + 7, x1.w));
+            v4.x = fin(e + 0, x.x);
+            v4.y = fin(e + 2, x.y);
+            v4.z = fin(e + 4, x.z);
+            v4.w = fin(e + 6, x.w);
             *reinterpret_cast<uint4*>(orow + hh * 32 + e) = v4;
           }
         }
