@@ -38,6 +38,9 @@ Readings taken where the paper is silent or garbled (each is restated in the des
   * phi (text "Characterization of phi" and appendix "Training Details"): a per-head
     two-layer MLP  u = act_out(W2 act_hidden(W1 x + b1) + b2), u split into P equal
     contiguous parts, part p (1-based) raised element-wise to the power p, concatenated.
+    The text also speaks of varying the "transformation complexity" of phi; the deeper maps
+    taken here put further hidden layers h <- act_hidden(Wm h + bm) of width D_h between the
+    two (the widths and activation of the two-layer map, nothing new to choose).
 
 Parity unpinned (the paper prints no numbers that would decide them): rowmax vs zero,
 the activation functions, which chunk is the short one.
@@ -70,13 +73,18 @@ def _act(x: np.ndarray, name: str) -> np.ndarray:
     raise ValueError(f"unknown activation {name!r}")
 
 
-def phi_map(x, W1, b1, W2, b2, P=2, act_hidden="relu", act_out="relu"):
+def phi_map(x, W1, b1, W2, b2, P=2, act_hidden="relu", act_out="relu", Wmid=None, bmid=None):
     """phi(x) = [psi_1(x)^1, psi_2(x)^2, ..., psi_P(x)^P]  (text "Characterization of phi").
 
     x [n, d]; W1 [D_h, d]; b1 [D_h]; W2 [D', D_h]; b2 [D'] of ONE head.  Returns [n, D'].
+    Wmid [L-2, D_h, D_h], bmid [L-2, D_h]: further hidden layers of an L-layer map, applied in order between
+    the first and the last layer (None or empty: the two-layer map).
     """
     x = np.asarray(x, dtype=np.float64)
     h = _act(x @ np.asarray(W1, np.float64).T + np.asarray(b1, np.float64), act_hidden)
+    if Wmid is not None:
+        for Wm, bm in zip(np.asarray(Wmid, np.float64), np.asarray(bmid, np.float64)):
+            h = _act(h @ Wm.T + bm, act_hidden)
     u = _act(h @ np.asarray(W2, np.float64).T + np.asarray(b2, np.float64), act_out)
     Dp = u.shape[-1]
     if Dp % P != 0:
@@ -131,13 +139,13 @@ def linear_set(t, T, HW, Tc, To, causal=True):
 
 def _phi_pair(phi_q, phi_k, h):
     """Slice head h out of the per-head parameter dictionaries."""
-    pq = {n: np.asarray(phi_q[n][h], np.float64) for n in ("W1", "b1", "W2", "b2")}
-    pk = {n: np.asarray(phi_k[n][h], np.float64) for n in ("W1", "b1", "W2", "b2")}
+    pq = {n: np.asarray(phi_q[n][h], np.float64) for n in ("W1", "b1", "W2", "b2", "Wmid", "bmid") if n in phi_q}
+    pk = {n: np.asarray(phi_k[n][h], np.float64) for n in ("W1", "b1", "W2", "b2", "Wmid", "bmid") if n in phi_k}
     return pq, pk
 
 
 def _phi(x, p, P, act_hidden, act_out):
-    return phi_map(x, p["W1"], p["b1"], p["W2"], p["b2"], P, act_hidden, act_out)
+    return phi_map(x, p["W1"], p["b1"], p["W2"], p["b2"], P, act_hidden, act_out, p.get("Wmid"), p.get("bmid"))
 
 
 def _stabiliser(S, c_mode):

@@ -275,6 +275,46 @@ def test_phi_by_hand_and_polynomial_order():
         orc.phi_map(x, W1, b1, W2, b2, P=4)
 
 
+def test_deeper_phi_by_hand():
+    """Three and four layers, every value worked out by hand: x = (1, -2);
+    layer 1: (1, -1, 1) -> relu (1, 0, 1); hidden layer A: (1, 1.5, 0); hidden layer B after A: (1.5 - 1, 1, 2.5);
+    last layer after A: (1, 1.5, 0.5, -1) -> relu, degree 2: (1, 1.5, 0.25, 0);
+    last layer after A, B: (0.5, 3.5, 0.5, 4) -> degree 2: (0.5, 3.5, 0.25, 16).  The order of A and B matters."""
+    x = np.array([[1.0, -2.0]])
+    W1 = np.array([[1.0, 0.0], [0.0, 1.0], [1.0, 1.0]]); b1 = np.array([0.0, 1.0, 2.0])
+    A = np.array([[1.0, 1.0, 0.0], [0.0, -1.0, 1.0], [2.0, 0.0, -1.0]]); a = np.array([0.0, 0.5, -1.0])
+    B = np.array([[0.0, 1.0, 0.0], [1.0, 0.0, 0.0], [1.0, 1.0, 1.0]]); b = np.array([-1.0, 0.0, 0.0])
+    W2 = np.array([[1.0, 0.0, 0.0], [0.0, 1.0, 1.0], [1.0, -1.0, 0.0], [0.0, 0.0, 2.0]]); b2 = np.array([0.0, 0.0, 1.0, -1.0])
+    three = orc.phi_map(x, W1, b1, W2, b2, P=2, Wmid=A[None], bmid=a[None])
+    assert np.allclose(three, [[1.0, 1.5, 0.25, 0.0]], atol=1e-15)
+    four = orc.phi_map(x, W1, b1, W2, b2, P=2, Wmid=np.stack([A, B]), bmid=np.stack([a, b]))
+    assert np.allclose(four, [[0.5, 3.5, 0.25, 16.0]], atol=1e-15)
+    swapped = orc.phi_map(x, W1, b1, W2, b2, P=2, Wmid=np.stack([B, A]), bmid=np.stack([b, a]))
+    assert np.allclose(swapped, [[1.0, 1.5, 0.25, 0.0]], atol=1e-15) and not np.allclose(swapped, four)
+    # no hidden layers in between: the two-layer map
+    assert np.allclose(orc.phi_map(x, W1, b1, W2, b2, P=2, Wmid=np.zeros((0, 3, 3)), bmid=np.zeros((0, 3))),
+                       orc.phi_map(x, W1, b1, W2, b2, P=2))
+    # an identity hidden layer changes nothing after a relu
+    assert np.allclose(orc.phi_map(x, W1, b1, W2, b2, P=2, Wmid=np.eye(3)[None], bmid=np.zeros((1, 3))),
+                       orc.phi_map(x, W1, b1, W2, b2, P=2))
+
+
+def test_deeper_phi_through_the_operator():
+    """The three evaluations of the operator agree with a three-layer phi as they do with two layers."""
+    rng = np.random.default_rng(5)
+    nh, d, Dh, Dp, T, HW = 2, 4, 6, 4, 4, 3
+    mk = lambda: {"W1": rng.standard_normal((nh, Dh, d)), "b1": rng.standard_normal((nh, Dh)),
+                  "W2": rng.standard_normal((nh, Dp, Dh)), "b2": rng.standard_normal((nh, Dp)),
+                  "Wmid": rng.standard_normal((nh, 1, Dh, Dh)), "bmid": rng.standard_normal((nh, 1, Dh))}
+    pq, pk = mk(), mk()
+    q, k, v = (rng.standard_normal((1, nh, T * HW, d)) for _ in range(3))
+    brute = orc.hybrid_brute(q, k, v, pq, pk, T, HW, 1, 1)
+    assert np.abs(orc.hybrid_direct(q, k, v, pq, pk, T, HW, 1, 1) - brute).max() < 1e-12
+    assert np.abs(orc.hybrid_rnn(q, k, v, pq, pk, T, HW, 1, 1) - brute).max() < 1e-12
+    two = {n: t for n, t in pq.items() if n not in ("Wmid", "bmid")}
+    assert np.abs(orc.hybrid_direct(q, k, v, two, pk, T, HW, 1, 1) - brute).max() > 1e-3   # the hidden layer is not ignored
+
+
 def test_phi_is_nonnegative_with_relu_output():
     rng = np.random.default_rng(0)
     x = rng.standard_normal((50, 8))
