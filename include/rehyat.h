@@ -163,8 +163,11 @@ int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host,
  * with one chunk plus the overlap, not with the video (Section 3.3, note 3).
  *
  * rehyat_stream_begin starts a sequence (s_0 = 0, z_0 = 0, Eq. 14-15) for chunks of at most `chunk` frames
- * with `overlap` frames of overlap, and sizes six staging buffers of (overlap + chunk)*H*W tokens per
- * (batch, head): the only allocation of this API, repeated only when a later sequence needs more.
+ * with `overlap` frames of overlap, and sizes two buffers (k and v) of (overlap + 4*chunk)*H*W tokens per
+ * (batch, head) - more chunks where overlap > 3*chunk: the only allocation of this API, repeated only when a
+ * later sequence needs more.  The softmax window slides through these buffers: a step appends its chunk's k and
+ * v behind the kept overlap frames, the frames that stay are addressed rather than moved, and only at the end
+ * of the buffers (every few steps) are they copied back to the front.  q and out are read and written in place.
  * rehyat_stream_step takes the next chunk,
  *   q_chunk, k_chunk, v_chunk, out_chunk   device, [batch, n_heads, frames_in_chunk*H*W, head_dim] through `lay`
  *   frames_in_chunk                        1..chunk; only the last chunk of a video may be shorter than `chunk`

@@ -68,20 +68,21 @@ struct rehyat_ctx {
   int withhold_loads = 0;      // test hook of rehyat_set_wait_limit
   float* share_out = nullptr;  // rehyat_set_linear_share_output
   float* share_now = nullptr;  // what the window launches of the call in progress write (null in chunk-by-chunk steps)
-  // chunk-by-chunk processing (rehyat_stream_*): the running state lives in slot 0 of `state`, the last
-  // `overlap` frames of k and v and the chunk being processed in staging buffers [BH][cap_tokens][d]
+  // chunk-by-chunk processing (rehyat_stream_*): the running state lives in slot 0 of `state`; k and v of the
+  // softmax window (the kept overlap frames, then the chunk being processed) sit in two buffers
+  // [BH][cap_tokens][d] at token index `start`.  Every step appends its chunk behind the window and moves
+  // `start` past the tokens that leave it; only when the end of the buffers is reached are the kept frames
+  // copied back to the front.  q and out are used in place.
   struct Stream {
     bool active = false;
     int batch = 0, H = 0, W = 0, chunk = 0, overlap = 0;
     int halo = 0;                 // tokens of earlier chunks still inside the softmax window
     int has_state = 0;            // the running state covers at least one token
     long long chunks_done = 0;
-    int cap_tokens = 0;           // tokens per (batch, head) each staging buffer holds
-    int cur = 0;                  // which of the two k / v buffers holds the halo
-    void* kbuf[2] = {nullptr, nullptr};
-    void* vbuf[2] = {nullptr, nullptr};
-    void* qbuf = nullptr;
-    void* obuf = nullptr;
+    int cap_tokens = 0;           // tokens per (batch, head) each buffer holds
+    int start = 0;                // token index of the window's first token
+    void* kbuf = nullptr;
+    void* vbuf = nullptr;
     size_t bytes = 0;
   } stream;
 };
@@ -204,7 +205,8 @@ int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* ou
 // and one CTA per SM, so pick the split that needs the fewest token tiles per SM over all waves.
 int pick_state_split(const rehyat_ctx* ctx, const Geo& g, int n_chunks_in_group, int tokens_per_increment) {
   int n_split = ctx->partial_units / (n_chunks_in_group > 0 ? n_chunks_in_group : 1);
-  if (n_split > 8) n_split = 8;
+  const int most = ctx->tensor_ok && ctx->tc.phi_ok ? 16 : 8;   // a lone chunk (a chunk-by-chunk step) over all SMs
+  if (n_split > most) n_split = most;
   if (n_split < 1) n_split = 1;
   if (ctx->tensor_ok && ctx->tc.phi_ok) {
     const int n_sm = ctx->tc.n_sm;
@@ -287,9 +289,12 @@ int check_sizes(const rehyat_ctx* ctx, int batch, int frames, int H, int W, int 
 
 // Copies `rows` token rows of `row_bytes` bytes for each of BH (batch, head) problems between two strided
 // layouts (byte strides; rows are contiguous and 16-byte aligned).  grid (row tiles, BH), 256 threads.
-__global__ void copy_rows(uint8_t* __restrict__ dst, long long dst_b, long long dst_h, long long dst_n,
-                          const uint8_t* __restrict__ src, long long src_b, long long src_h, long long src_n,
-                          int rows, int row_bytes, int n_heads) {
+__global__ void copy_rows(uint8_t* __restrict__ dst0, uint8_t* __restrict__ dst1, long long dst_b, long long dst_h, long long dst_n,
+                          const uint8_t* __restrict__ src0, const uint8_t* __restrict__ src1, long long src_b, long long src_h,
+                          long long src_n, int rows, int row_bytes, int n_heads) {
+  // blockIdx.z picks one of two tensor pairs that share their layouts (k and v)
+  uint8_t* __restrict__ dst = blockIdx.z ? dst1 : dst0;
+  const uint8_t* __restrict__ src = blockIdx.z ? src1 : src0;
   const int bh = blockIdx.y, b = bh / n_heads, h = bh % n_heads;
   const int per_row = row_bytes / 16;
   const long long total = (long long)rows * per_row;
@@ -396,8 +401,7 @@ int rehyat_destroy(rehyat_ctx* ctx) {
   if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
   if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
   for (cudaEvent_t e : ctx->host_events) cudaEventDestroy(e);
-  for (int i = 0; i < 2; ++i) { cudaFree(ctx->stream.kbuf[i]); cudaFree(ctx->stream.vbuf[i]); }
-  cudaFree(ctx->stream.qbuf); cudaFree(ctx->stream.obuf);
+  cudaFree(ctx->stream.kbuf); cudaFree(ctx->stream.vbuf);
   delete ctx;
   return REHYAT_OK;
 }
@@ -500,6 +504,8 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   // the stride of a one-element axis is never used for addressing; tensor maps still want it non-zero
   if (g.stride_h == 0) g.stride_h = g.stride_n * N;
   if (g.stride_b == 0) g.stride_b = g.stride_h * g.n_heads;
+  g.qstride_b = g.stride_b; g.qstride_h = g.stride_h; g.qstride_n = g.stride_n;   // q and out: laid out like k and v
+  g.q_off = 0; g.Nq = g.N;
   const int n_chunks = (frames + chunk_eff - 1) / chunk_eff;
   g.q_shift = 0;
   g.prefix = 0;
@@ -658,13 +664,15 @@ size_t stream_halo_bytes(const rehyat_ctx* ctx) {      // of k (and as much agai
   return (size_t)ctx->stream.batch * ctx->cfg.n_heads * ctx->stream.halo * ctx->cfg.head_dim * elem_size(ctx->cfg.dtype);
 }
 
-void launch_copy_rows(void* dst, long long dst_b, long long dst_h, long long dst_n, const void* src, long long src_b,
-                      long long src_h, long long src_n, int rows, int row_bytes, int BH, int n_heads, cudaStream_t st) {
+// Copies dst0 <- src0 and dst1 <- src1 (two tensors with the same layouts) in one launch.
+void launch_copy_rows2(void* dst0, void* dst1, long long dst_b, long long dst_h, long long dst_n, const void* src0,
+                       const void* src1, long long src_b, long long src_h, long long src_n, int rows, int row_bytes, int BH,
+                       int n_heads, cudaStream_t st) {
   if (rows <= 0) return;
   const long long total = (long long)rows * (row_bytes / 16);
-  const unsigned blocks = (unsigned)((total + 255) / 256 < 1024 ? (total + 255) / 256 : 1024);
-  copy_rows<<<dim3(blocks, BH), 256, 0, st>>>((uint8_t*)dst, dst_b, dst_h, dst_n, (const uint8_t*)src, src_b, src_h,
-                                              src_n, rows, row_bytes, n_heads);
+  const unsigned blocks = (unsigned)((total + 255) / 256 < 256 ? (total + 255) / 256 : 256);
+  copy_rows<<<dim3(blocks, BH, 2), 256, 0, st>>>((uint8_t*)dst0, (uint8_t*)dst1, dst_b, dst_h, dst_n, (const uint8_t*)src0,
+                                                 (const uint8_t*)src1, src_b, src_h, src_n, rows, row_bytes, n_heads);
 }
 
 }  // namespace
@@ -677,26 +685,29 @@ int rehyat_stream_begin(rehyat_ctx* ctx, int32_t batch, int32_t H, int32_t W, in
   if (batch < 1 || batch > c.max_batch || H < 1 || W < 1 || chunk < 1 || overlap < 0) return REHYAT_ERR_INVALID_ARG;
   const long long HW = (long long)H * W;
   if (HW > c.max_tokens_per_frame || chunk > c.max_chunk_frames) return REHYAT_ERR_INVALID_ARG;
-  const long long cap = (long long)(overlap + chunk) * HW;
+  // room for the kept frames and several chunks behind them, so that the kept frames go back to the front only
+  // every few steps; (rounds - 1) chunks >= overlap keeps that copy from overlapping itself
+  const long long rounds = 4 > (overlap + chunk - 1) / chunk + 1 ? 4 : (overlap + chunk - 1) / chunk + 1;
+  const long long cap = ((long long)overlap + rounds * chunk) * HW;
   if (cap > (1 << 24)) return REHYAT_ERR_INVALID_ARG;
   DeviceGuard guard(c.device);
   if (!guard.ok) return REHYAT_ERR_CUDA;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   rehyat_ctx::Stream& s = ctx->stream;
   const size_t one = (size_t)batch * c.n_heads * cap * c.head_dim * elem_size(c.dtype);
-  if (one * 6 > s.bytes) {                          // grow the six staging buffers (the only allocation of this API)
+  if (one * 2 > s.bytes) {                          // grow the two buffers (the only allocation of this API)
     if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
-    void** all[6] = {&s.kbuf[0], &s.kbuf[1], &s.vbuf[0], &s.vbuf[1], &s.qbuf, &s.obuf};
+    void** all[2] = {&s.kbuf, &s.vbuf};
     for (void** p : all) { cudaFree(*p); *p = nullptr; }
     s.bytes = 0;
     for (void** p : all)
       if (cudaMalloc(p, one) != cudaSuccess) { cudaGetLastError(); return REHYAT_ERR_ALLOC; }
-    s.bytes = one * 6;
+    s.bytes = one * 2;
   }
   s.active = true;
   s.batch = batch; s.H = H; s.W = W; s.chunk = chunk; s.overlap = overlap;
   s.cap_tokens = (int)cap;
-  s.halo = 0; s.has_state = 0; s.chunks_done = 0; s.cur = 0;
+  s.halo = 0; s.has_state = 0; s.chunks_done = 0; s.start = 0;
   return REHYAT_OK;
 }
 
@@ -707,6 +718,7 @@ int rehyat_stream_step(rehyat_ctx* ctx, const void* q_chunk, const void* k_chunk
   rehyat_ctx::Stream& s = ctx->stream;
   if (!s.active || frames_in_chunk < 1 || frames_in_chunk > s.chunk) return REHYAT_ERR_INVALID_ARG;
   const rehyat_config& c = ctx->cfg;
+  if (out_chunk == q_chunk || out_chunk == k_chunk || out_chunk == v_chunk) return REHYAT_ERR_INVALID_ARG;
   const void* ptrs[] = {q_chunk, k_chunk, v_chunk, out_chunk, phi->q_W1, phi->q_b1, phi->q_W2, phi->q_b2,
                         phi->k_W1, phi->k_b1, phi->k_W2, phi->k_b2};
   for (const void* p : ptrs)
@@ -716,34 +728,43 @@ int rehyat_stream_step(rehyat_ctx* ctx, const void* q_chunk, const void* k_chunk
   for (long long x : strides)
     if (x < 0 || (x * es) % 16 != 0) return REHYAT_ERR_INVALID_ARG;
   if (lay->stride_token < c.head_dim) return REHYAT_ERR_INVALID_ARG;
+  if ((c.n_heads > 1 && lay->stride_head < c.head_dim) || (s.batch > 1 && lay->stride_batch < c.head_dim))
+    return REHYAT_ERR_INVALID_ARG;
   DeviceGuard guard(c.device);
   if (!guard.ok) return REHYAT_ERR_CUDA;
   cudaStream_t st = (cudaStream_t)cuda_stream;
 
   const int HW = s.H * s.W, Np = frames_in_chunk * HW, h = s.halo, BH = s.batch * c.n_heads;
   const int row_bytes = c.head_dim * (int)es;
-  // staging layout [batch][head][cap_tokens][d]
+  // buffer layout [batch][head][cap_tokens][d]
   const long long sn = c.head_dim, sh = (long long)s.cap_tokens * c.head_dim, sb = sh * c.n_heads;
-  uint8_t* kcur = (uint8_t*)s.kbuf[s.cur];
-  uint8_t* vcur = (uint8_t*)s.vbuf[s.cur];
-  // 1. the chunk goes behind the halo
-  const void* src[3] = {q_chunk, k_chunk, v_chunk};
-  uint8_t* dst[3] = {(uint8_t*)s.qbuf, kcur, vcur};
-  for (int i = 0; i < 3; ++i)
-    launch_copy_rows(dst[i] + (long long)h * sn * es, sb * es, sh * es, sn * es, src[i], lay->stride_batch * es,
-                     lay->stride_head * es, lay->stride_token * es, Np, row_bytes, BH, c.n_heads, st);
-  // 2. Eq. 16 for this chunk: one chunk whose queries start at buffer index h and whose window is the whole buffer
+  // 0. at the end of the buffers the kept frames go back to the front (every few steps)
+  if (s.start + h + Np > s.cap_tokens) {
+    const long long off = (long long)s.start * sn * es;
+    launch_copy_rows2(s.kbuf, s.vbuf, sb * es, sh * es, sn * es, (uint8_t*)s.kbuf + off, (uint8_t*)s.vbuf + off, sb * es, sh * es,
+                      sn * es, h, row_bytes, BH, c.n_heads, st);
+    s.start = 0;
+  }
+  uint8_t* kwin = (uint8_t*)s.kbuf + (long long)s.start * sn * es;     // first token of the softmax window
+  uint8_t* vwin = (uint8_t*)s.vbuf + (long long)s.start * sn * es;
+  // 1. k and v of the chunk go behind the kept frames (they have to outlive the call); q and out stay where they are
+  launch_copy_rows2(kwin + (long long)h * sn * es, vwin + (long long)h * sn * es, sb * es, sh * es, sn * es, k_chunk, v_chunk,
+                    lay->stride_batch * es, lay->stride_head * es, lay->stride_token * es, Np, row_bytes, BH, c.n_heads, st);
+  // 2. Eq. 16 for this chunk: one chunk whose queries are rows [h, h + Np) of the window and whose softmax set
+  //    is the whole window
   Geo g;
   g.N = h + Np; g.Np = Np; g.ToHW = h; g.t0 = 0; g.G = 1; g.n_heads = c.n_heads; g.BH = BH;
   g.stride_b = sb; g.stride_h = sh; g.stride_n = sn;
   g.q_shift = h; g.prefix = s.has_state;
+  g.qstride_b = lay->stride_batch; g.qstride_h = lay->stride_head; g.qstride_n = lay->stride_token;
+  if (g.qstride_h == 0) g.qstride_h = g.qstride_n * Np;
+  if (g.qstride_b == 0) g.qstride_b = g.qstride_h * c.n_heads;
+  g.q_off = h; g.Nq = Np;
   ctx->share_now = nullptr;
   ctx->last_launches = 0;
   ctx->last_impl = ctx->tensor_ok ? 1 : 0;
-  int rc = run_parts(ctx, s.qbuf, kcur, vcur, s.obuf, phi, g, s.batch, 1, -1, (s.has_state ? PART_READOUT : 0) | PART_WINDOW, st);
+  int rc = run_parts(ctx, q_chunk, kwin, vwin, out_chunk, phi, g, s.batch, 1, -1, (s.has_state ? PART_READOUT : 0) | PART_WINDOW, st);
   if (rc != REHYAT_OK) return rc;
-  launch_copy_rows(out_chunk, lay->stride_batch * es, lay->stride_head * es, lay->stride_token * es,
-                   (uint8_t*)s.obuf + (long long)h * sn * es, sb * es, sh * es, sn * es, Np, row_bytes, BH, c.n_heads, st);
   // 3. Eq. 17-18: the tokens that leave the window before the next chunk enter the running state
   const int keep = (long long)s.overlap * HW < (long long)h + Np ? s.overlap * HW : h + Np;
   const int leave = h + Np - keep;
@@ -751,17 +772,12 @@ int rehyat_stream_step(rehyat_ctx* ctx, const void* q_chunk, const void* k_chunk
     Geo gs = g;
     gs.Np = leave; gs.ToHW = 0; gs.q_shift = 0; gs.prefix = 0; gs.t0 = 1; gs.G = 1;   // increment of "chunk 1" = [0, leave)
     const int n_split = pick_state_split(ctx, gs, 1, leave);
-    rc = run_parts(ctx, nullptr, kcur, vcur, nullptr, phi, gs, s.batch, n_split, s.has_state ? 0 : -1, PART_STATE, st);
+    rc = run_parts(ctx, nullptr, kwin, vwin, nullptr, phi, gs, s.batch, n_split, s.has_state ? 0 : -1, PART_STATE, st);
     if (rc != REHYAT_OK) return rc;
     s.has_state = 1;
   }
-  // 4. the frames that stay in the window move to the front of the other pair of buffers
-  const int nxt = s.cur ^ 1;
-  launch_copy_rows(s.kbuf[nxt], sb * es, sh * es, sn * es, kcur + (long long)leave * sn * es, sb * es, sh * es, sn * es,
-                   keep, row_bytes, BH, c.n_heads, st);
-  launch_copy_rows(s.vbuf[nxt], sb * es, sh * es, sn * es, vcur + (long long)leave * sn * es, sb * es, sh * es, sn * es,
-                   keep, row_bytes, BH, c.n_heads, st);
-  s.cur = nxt;
+  // 4. the window moves on: the frames that stay are addressed, not copied
+  s.start += leave;
   s.halo = keep;
   ++s.chunks_done;
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
@@ -796,9 +812,10 @@ int rehyat_stream_export(rehyat_ctx* ctx, void* host_buf, size_t capacity, void*
   const size_t es = elem_size(c.dtype), width = (size_t)s.halo * c.head_dim * es, pitch = (size_t)s.cap_tokens * c.head_dim * es;
   const int BH = s.batch * c.n_heads;
   if (width > 0) {
-    if (cudaMemcpy2D(p, width, s.kbuf[s.cur], pitch, width, BH, cudaMemcpyDeviceToHost) != cudaSuccess) return REHYAT_ERR_CUDA;
+    const size_t first = (size_t)s.start * c.head_dim * es;          // the kept frames begin at token `start`
+    if (cudaMemcpy2D(p, width, (const uint8_t*)s.kbuf + first, pitch, width, BH, cudaMemcpyDeviceToHost) != cudaSuccess) return REHYAT_ERR_CUDA;
     p += width * BH;
-    if (cudaMemcpy2D(p, width, s.vbuf[s.cur], pitch, width, BH, cudaMemcpyDeviceToHost) != cudaSuccess) return REHYAT_ERR_CUDA;
+    if (cudaMemcpy2D(p, width, (const uint8_t*)s.vbuf + first, pitch, width, BH, cudaMemcpyDeviceToHost) != cudaSuccess) return REHYAT_ERR_CUDA;
   }
   return REHYAT_OK;
 }
@@ -834,9 +851,9 @@ int rehyat_stream_import(rehyat_ctx* ctx, const void* host_buf, size_t bytes, vo
   const size_t es = elem_size(c.dtype), width = (size_t)s.halo * c.head_dim * es, pitch = (size_t)s.cap_tokens * c.head_dim * es;
   const int BH = s.batch * c.n_heads;
   if (width > 0) {
-    if (cudaMemcpy2D(s.kbuf[s.cur], pitch, p, width, width, BH, cudaMemcpyHostToDevice) != cudaSuccess) return REHYAT_ERR_CUDA;
+    if (cudaMemcpy2D(s.kbuf, pitch, p, width, width, BH, cudaMemcpyHostToDevice) != cudaSuccess) return REHYAT_ERR_CUDA;
     p += width * BH;
-    if (cudaMemcpy2D(s.vbuf[s.cur], pitch, p, width, width, BH, cudaMemcpyHostToDevice) != cudaSuccess) return REHYAT_ERR_CUDA;
+    if (cudaMemcpy2D(s.vbuf, pitch, p, width, width, BH, cudaMemcpyHostToDevice) != cudaSuccess) return REHYAT_ERR_CUDA;
   }
   return cudaStreamSynchronize(st) == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }

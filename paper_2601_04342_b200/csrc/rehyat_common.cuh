@@ -25,9 +25,14 @@ struct Geo {
   int G;        // chunks in the group
   int n_heads;
   int BH;       // batch * n_heads
-  long long stride_b, stride_h, stride_n;   // element strides of q, k, v, out
+  long long stride_b, stride_h, stride_n;   // element strides of k and v
   int q_shift;  // buffer index of the first query of chunk 0 (0 for a whole sequence)
   int prefix;   // 1: the carried state of chunk t0 covers tokens before buffer index 0
+  // q and out may live in tensors of their own (a chunk-by-chunk step reads the caller's chunk in place while k
+  // and v sit behind the kept overlap frames): row r of the k / v buffers is row r - q_off of q and out, which
+  // have Nq rows and their own strides.  A whole-sequence call has q_off = 0, Nq = N and the strides of k, v.
+  long long qstride_b, qstride_h, qstride_n;
+  int q_off, Nq;
 };
 
 __host__ __device__ inline int geo_q0(const Geo& g, int t) { return t * g.Np + g.q_shift; }
@@ -80,6 +85,11 @@ __device__ __forceinline__ float2 unpack_f16(uint32_t pair) {
 
 __device__ __forceinline__ long long head_offset(const Geo& g, int bh) {
   return (long long)(bh / g.n_heads) * g.stride_b + (long long)(bh % g.n_heads) * g.stride_h;
+}
+// Element offset of buffer row `row` (a query row) of (batch*head) bh inside q or out.
+__device__ __forceinline__ long long q_row_offset(const Geo& g, int bh, int row) {
+  return (long long)(bh / g.n_heads) * g.qstride_b + (long long)(bh % g.n_heads) * g.qstride_h +
+         (long long)(row - g.q_off) * g.qstride_n;
 }
 
 __device__ __forceinline__ float ldf(const float* p) { return *p; }

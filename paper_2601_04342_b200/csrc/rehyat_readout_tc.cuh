@@ -128,8 +128,8 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         if (!alive) break;
         const uint32_t xf = smem_u32(&bars->x_full);
         mbar_expect_tx(xf, PH_TILE_BYTES);
-        tma_load_4d(sX, &tm_x, xf, 0, tok_a + j * 128, h_idx, b_idx);
-        tma_load_4d(sX + PH_SUB, &tm_x, xf, 64, tok_a + j * 128, h_idx, b_idx);
+        tma_load_4d(sX, &tm_x, xf, 0, tok_a - g.q_off + j * 128, h_idx, b_idx);
+        tma_load_4d(sX + PH_SUB, &tm_x, xf, 64, tok_a - g.q_off + j * 128, h_idx, b_idx);
         ++n_x;
         // the ring follows the issue order of the MMAs: read-out of the previous tile between this tile's H halves
         for (int ks = 0; ks < 2; ++ks) weight_load(&tm_w1, ks * 64, 0);

@@ -219,7 +219,7 @@ readout_simt(const T* __restrict__ q, PhiPtrs<T> wq, PhiDims pd, Geo g, const fl
   const int head = bh % g.n_heads;
   PhiPtrs<T> w = {wq.W1 + (size_t)head * pd.Dh * D, wq.b1 + (size_t)head * pd.Dh,
                   wq.W2 + (size_t)head * pd.Dp * pd.Dh, wq.b2 + (size_t)head * pd.Dp};
-  load_rows_simt(Xs, q + head_offset(g, bh), g.stride_n, tok0, q1, D);
+  load_rows_simt(Xs, q + q_row_offset(g, bh, 0), g.qstride_n, tok0, q1, D);
   __syncthreads();
   phi_tile_simt(Xs, Hs, Fs, w, pd, q1 - tok0);
 
@@ -289,7 +289,7 @@ window_simt(const T* __restrict__ q, const T* __restrict__ k, const T* __restric
   for (int idx = tid; idx < WIN_BM * (D / 4); idx += WIN_THREADS) {
     const int r = idx / (D / 4), c = (idx % (D / 4)) * 4;
     float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (row0 + r < q1) x = ld4(q + hoff + (long long)(row0 + r) * g.stride_n + c);
+    if (row0 + r < q1) x = ld4(q + q_row_offset(g, bh, row0 + r) + c);
     *reinterpret_cast<float4*>(Qs + r * LDK + c) = x;
   }
 
@@ -396,7 +396,7 @@ window_simt(const T* __restrict__ q, const T* __restrict__ k, const T* __restric
     }
     const float inv = 1.f / (l[i] * ws + lam * nL);
     if (share != nullptr && tx == 0) share[(size_t)bh * g.N + row] = lam * nL * inv;   // part of the normaliser that is linear
-    T* orow = out + hoff + (long long)row * g.stride_n + tx * DC;
+    T* orow = out + q_row_offset(g, bh, row) + tx * DC;
 #pragma unroll
     for (int c = 0; c < DC; ++c) {
       const float aL = linear ? rd[rd_index(g, rd_rows, D, bh, ci, row - q0, (tx * DC + c) >> 2) + ((tx * DC + c) & 3)] : 0.f;

@@ -136,8 +136,8 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         const uint32_t qf = smem_u32(&bars->q_full);
         mbar_expect_tx(qf, w.ntiles * TC_TILE_BYTES);
         for (int i = 0; i < w.ntiles; ++i) {
-          tma_load_4d(sQ + i * TC_TILE_BYTES, &tm_q, qf, 0, w.row_base + i * TC_BM, w.h_idx, w.b_idx);
-          tma_load_4d(sQ + i * TC_TILE_BYTES + TC_SUB_BYTES, &tm_q, qf, 64, w.row_base + i * TC_BM, w.h_idx, w.b_idx);
+          tma_load_4d(sQ + i * TC_TILE_BYTES, &tm_q, qf, 0, w.row_base - g.q_off + i * TC_BM, w.h_idx, w.b_idx);
+          tma_load_4d(sQ + i * TC_TILE_BYTES + TC_SUB_BYTES, &tm_q, qf, 64, w.row_base - g.q_off + i * TC_BM, w.h_idx, w.b_idx);
         }
         ++n_q;
         for (int j = 0; j < w.n_kv && alive; ++j) {
@@ -376,7 +376,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           lam = __expf(-r);
         }
       }
-      __nv_bfloat16* orow = out + head_offset(g, w.bh) + (long long)row * g.stride_n;
+      __nv_bfloat16* orow = out + q_row_offset(g, w.bh, row);
       if (!wait(&bars->pv_done[i], (n_s + n_kv - 1) & 1)) break;
       tc_fence_after();
       n_s += n_kv;
@@ -496,6 +496,13 @@ inline bool tc_make_tmap(const TcWorkspace* w, CUtensorMap* tm, const void* base
   const cuuint32_t box[4] = {64, (cuuint32_t)TC_BN, 1, 1};
   return tc_encode(w, tm, base, 4, dims, strides, box);
 }
+// The same over q: its own row count and strides (see Geo).
+inline bool tc_make_tmap_q(const TcWorkspace* w, CUtensorMap* tm, const void* base, const Geo& g, int batch) {
+  const cuuint64_t dims[4] = {(cuuint64_t)TC_D, (cuuint64_t)g.Nq, (cuuint64_t)g.n_heads, (cuuint64_t)batch};
+  const cuuint64_t strides[3] = {(cuuint64_t)g.qstride_n * 2, (cuuint64_t)g.qstride_h * 2, (cuuint64_t)g.qstride_b * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)TC_BN, 1, 1};
+  return tc_encode(w, tm, base, 4, dims, strides, box);
+}
 // Row-major [planes][rows][cols] bf16 matrix stack, box [64 cols x box_rows].
 inline bool tc_make_tmap_3d(const TcWorkspace* w, CUtensorMap* tm, const void* base, int cols, int rows, int planes,
                             int box_rows) {
@@ -510,7 +517,7 @@ inline int tc_launch_window(TcWorkspace* w, const void* q, const void* k, const 
                             int batch, const float* rd, int rd_rows, int c_mode, const ptx::WaitArgs& wa, float* share,
                             cudaStream_t st) {
   CUtensorMap tq, tk, tv;
-  if (!tc_make_tmap(w, &tq, q, g, batch) || !tc_make_tmap(w, &tk, k, g, batch) || !tc_make_tmap(w, &tv, v, g, batch))
+  if (!tc_make_tmap_q(w, &tq, q, g, batch) || !tc_make_tmap(w, &tk, k, g, batch) || !tc_make_tmap(w, &tv, v, g, batch))
     return REHYAT_ERR_CUDA;
   const int pairs = (g.Np + TC_QT * TC_BM - 1) / (TC_QT * TC_BM);
   const int n_items = pairs * g.G * g.BH;
@@ -568,7 +575,7 @@ inline int tc_launch_readout(const TcWorkspace* w, const void* q, const rehyat_p
                              int P, int act_hidden, int act_out, const float* state, float* rd, int rd_rows,
                              const ptx::WaitArgs& wa, cudaStream_t st) {
   CUtensorMap tq, tw1, tw2, ts;
-  if (!tc_make_tmap(w, &tq, q, g, batch) || !tc_make_tmap_3d(w, &tw1, phi->q_W1, PH_D, PH_DH, g.n_heads, 128) ||
+  if (!tc_make_tmap_q(w, &tq, q, g, batch) || !tc_make_tmap_3d(w, &tw1, phi->q_W1, PH_D, PH_DH, g.n_heads, 128) ||
       !tc_make_tmap_3d(w, &tw2, phi->q_W2, PH_DH, PH_DP, g.n_heads, 128) ||
       !tc_make_tmap_3d(w, &ts, w->state_bf16, PH_D, PH_DP, g.G * g.BH, 64))
     return REHYAT_ERR_CUDA;

@@ -109,8 +109,8 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         if (!alive) break;
         const uint32_t qf = smem_u32(&bars->q_full);
         mbar_expect_tx(qf, TC_TILE_BYTES);
-        tma_load_4d(sQ, &tm_q, qf, 0, w.row_base, w.h_idx, w.b_idx);
-        tma_load_4d(sQ + TC_SUB_BYTES, &tm_q, qf, 64, w.row_base, w.h_idx, w.b_idx);
+        tma_load_4d(sQ, &tm_q, qf, 0, w.row_base - g.q_off, w.h_idx, w.b_idx);
+        tma_load_4d(sQ + TC_SUB_BYTES, &tm_q, qf, 64, w.row_base - g.q_off, w.h_idx, w.b_idx);
         ++n_q;
         auto load_tile = [&](bool is_v, int j) {                     // key tile j of the item into its ring stage
           const uint32_t it = kv_it + j;
@@ -357,7 +357,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           lam = __expf(-rr);
         }
       }
-      __nv_bfloat16* orow = out + head_offset(g, w.bh) + (long long)row * g.stride_n + i * (TC_D / 2);
+      __nv_bfloat16* orow = out + q_row_offset(g, w.bh, row) + i * (TC_D / 2);
       if (!wait(&bars->pv_done[0], (n_s[0] + cnt0 - 1) & 1)) break;
       if (cnt1 > 0 && !wait(&bars->pv_done[1], (n_s[1] + cnt1 - 1) & 1)) break;
       tc_fence_after();
