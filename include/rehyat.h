@@ -100,6 +100,12 @@ typedef struct rehyat_config {
                                    pipe instead of the special-function unit.  0 = the
                                    library's choice (1, the fastest measured on B200), 1..3 =
                                    that many, -1 = none.  Results agree within bf16 rounding. */
+  int32_t phi_layers;           /* layers of the phi MLP: 0 or 2 = the two-layer map of the paper's
+                                   experiments; 3 or 4 = one or two further hidden layers
+                                   h <- act_hidden(Wmid h + bmid) of width D_h between the two
+                                   (Section 4.3 varies the "transformation complexity" of phi).
+                                   Deeper maps run on the SIMT kernels (the softmax window stays
+                                   on the tensor cores).                                       */
   int32_t window_tiles;         /* tensor-core window kernel: 128-row query tiles per work
                                    item.  0 = chosen per launch from how many items there are
                                    for the SMs; 1 or 2 fixes it (same results up to the order
@@ -116,10 +122,13 @@ typedef struct rehyat_layout {
 } rehyat_layout;
 
 /* Device pointers to the parameters of phi_q and phi_k in the operator dtype, row-major:
- * W1 [n_heads, D_h, d], b1 [n_heads, D_h], W2 [n_heads, D', D_h], b2 [n_heads, D']. */
+ * W1 [n_heads, D_h, d], b1 [n_heads, D_h], W2 [n_heads, D', D_h], b2 [n_heads, D'] (W2, b2: the LAST layer),
+ * and with phi_layers = L > 2 the hidden layers in between, in the order they are applied:
+ * Wmid [n_heads, L-2, D_h, D_h], bmid [n_heads, L-2, D_h] (ignored, and may be NULL, for two layers). */
 typedef struct rehyat_phi_params {
   const void* q_W1; const void* q_b1; const void* q_W2; const void* q_b2;
   const void* k_W1; const void* k_b1; const void* k_W2; const void* k_b2;
+  const void* q_Wmid; const void* q_bmid; const void* k_Wmid; const void* k_bmid;
 } rehyat_phi_params;
 
 typedef struct rehyat_ctx rehyat_ctx;

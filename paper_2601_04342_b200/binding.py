@@ -31,7 +31,7 @@ class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "device", "dtype", "n_heads", "head_dim", "phi_hidden", "phi_dim", "poly_degree", "act_hidden",
         "act_out", "c_mode", "impl", "max_batch", "max_tokens_per_frame", "max_chunk_frames", "group_tokens",
-        "bidirectional", "max_frames", "exp_poly", "window_tiles")]
+        "bidirectional", "max_frames", "exp_poly", "phi_layers", "window_tiles")]
 
 
 # Values of the tuning fields of rehyat_config that a Rehyat(...) call does not name (0 = the library's choice).
@@ -43,7 +43,8 @@ class Layout(C.Structure):
 
 
 class PhiParams(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("q_W1", "q_b1", "q_W2", "q_b2", "k_W1", "k_b1", "k_W2", "k_b2")]
+    _fields_ = [(n, C.c_void_p) for n in ("q_W1", "q_b1", "q_W2", "q_b2", "k_W1", "k_b1", "k_W2", "k_b2",
+                                          "q_Wmid", "q_bmid", "k_Wmid", "k_bmid")]
 
 
 _lib = None
@@ -114,7 +115,7 @@ class Rehyat:
     def __init__(self, *, n_heads, head_dim, dtype="bf16", phi_hidden=None, phi_dim=None, poly_degree=2,
                  act_hidden="relu", act_out="relu", c_mode="rowmax", impl="auto", max_batch=1,
                  max_tokens_per_frame=1560, max_chunk_frames=3, group_tokens=0, device=0, bidirectional=False,
-                 max_frames=0, **tuning):
+                 max_frames=0, phi_layers=2, **tuning):
         unknown = set(tuning) - set(TUNING_DEFAULTS)
         if unknown:
             raise TypeError(f"unknown arguments {sorted(unknown)}")
@@ -122,7 +123,7 @@ class Rehyat:
         self.cfg = Config(device, DTYPE[dtype], n_heads, head_dim, phi_hidden or 2 * head_dim,
                           phi_dim or 2 * head_dim, poly_degree, ACT[act_hidden], ACT[act_out], C_MODE[c_mode],
                           IMPL[impl], max_batch, max_tokens_per_frame, max_chunk_frames, group_tokens,
-                          int(bool(bidirectional)), max_frames, int(tune["exp_poly"]), int(tune["window_tiles"]))
+                          int(bool(bidirectional)), max_frames, int(tune["exp_poly"]), phi_layers, int(tune["window_tiles"]))
         self.dtype = dtype
         self._h = C.c_void_p(None)
         _check(lib().rehyat_create(C.byref(self._h), C.byref(self.cfg)), "rehyat_create")
@@ -161,7 +162,8 @@ class Rehyat:
     @staticmethod
     def phi_struct(phi_q, phi_k):
         return PhiParams(*[_ptr(phi_q[n]) for n in ("W1", "b1", "W2", "b2")],
-                         *[_ptr(phi_k[n]) for n in ("W1", "b1", "W2", "b2")])
+                         *[_ptr(phi_k[n]) for n in ("W1", "b1", "W2", "b2")],
+                         _ptr(phi_q.get("Wmid")), _ptr(phi_q.get("bmid")), _ptr(phi_k.get("Wmid")), _ptr(phi_k.get("bmid")))
 
     def forward(self, q, k, v, phi_q, phi_k, frames, H, W, chunk, overlap, out=None, layout="bhnd", stream=None):
         """q, k, v: CUDA tensors [B, n_heads, N, d] ("bhnd") or [B, N, n_heads, d] ("bnhd"), contiguous.
@@ -245,7 +247,7 @@ class Rehyat:
 
 
 def forward_static(q, k, v, phi_q, phi_k, frames, H, W, chunk, overlap, *, dtype, poly_degree=2, phi_hidden=None,
-                   phi_dim=None, act_hidden="relu", act_out="relu", c_mode="rowmax", out=None, stream=None):
+                   phi_dim=None, act_hidden="relu", act_out="relu", c_mode="rowmax", phi_layers=2, out=None, stream=None):
     """rehyat_forward_static: the operator without a context and without any device allocation by the
     library; its workspace is a fixed array inside librehyat.so.  For callers that cannot allocate
     (fixed memory plans, loops that cannot take cudaMalloc's synchronisation).  q, k, v: contiguous CUDA
@@ -255,7 +257,7 @@ def forward_static(q, k, v, phi_q, phi_k, frames, H, W, chunk, overlap, *, dtype
     if out is None:
         out = torch.empty_like(q)
     cfg = Config(q.device.index or 0, DTYPE[dtype], nh, d, phi_hidden or 2 * d, phi_dim or 2 * d, poly_degree,
-                 ACT[act_hidden], ACT[act_out], C_MODE[c_mode], 0, 1, 1, 1, 0)
+                 ACT[act_hidden], ACT[act_out], C_MODE[c_mode], 0, 1, 1, 1, 0, 0, 0, 0, phi_layers, 0)
     lay = Layout(nh * N * d, N * d, d)
     st = stream if stream is not None else torch.cuda.current_stream(q.device)
     phi = Rehyat.phi_struct(phi_q, phi_k)
@@ -317,6 +319,6 @@ def for_workload(wl, **kw):
     """A context sized for a synth.Workload."""
     args = dict(n_heads=wl.n_heads, head_dim=wl.head_dim, dtype=wl.dtype, phi_hidden=wl.D_h, phi_dim=wl.D_out,
                 poly_degree=wl.P, max_batch=wl.B, max_tokens_per_frame=wl.HW, max_chunk_frames=min(wl.Tc, wl.T),
-                max_frames=wl.T)
+                max_frames=wl.T, phi_layers=wl.phi_layers)
     args.update(kw)
     return Rehyat(**args)

@@ -119,6 +119,7 @@ int check_config(const rehyat_config* c) {
   if (c->bidirectional != 0 && c->bidirectional != 1) return REHYAT_ERR_INVALID_ARG;
   if (c->max_frames < 0 || c->max_frames > (1 << 20) || (c->bidirectional && c->max_frames < 1)) return REHYAT_ERR_INVALID_ARG;
   if (c->exp_poly < -1 || c->exp_poly > 3) return REHYAT_ERR_INVALID_ARG;
+  if (c->phi_layers != 0 && (c->phi_layers < 2 || c->phi_layers > 4)) return REHYAT_ERR_INVALID_ARG;
   if (c->window_tiles < 0 || c->window_tiles > 2) return REHYAT_ERR_INVALID_ARG;
   if (c->head_dim != 64 && c->head_dim != 128) return REHYAT_ERR_UNSUPPORTED;
   return REHYAT_OK;
@@ -129,8 +130,8 @@ int check_config(const rehyat_config* c) {
 // cannot lower it under a live one.
 template <typename T, int D>
 int set_simt_attributes() {
-  const int smem_state = SIMT_TM * (2 * D + 256 + 256) * (int)sizeof(float);
-  const int smem_rd = SIMT_TM * (D + 256 + 256) * (int)sizeof(float);
+  const int smem_state = (SIMT_TM * (2 * D + 256) + phi_hidden_floats(256, 1)) * (int)sizeof(float);
+  const int smem_rd = (SIMT_TM * (D + 256) + phi_hidden_floats(256, 1)) * (int)sizeof(float);
   const int smem_win = (WIN_BM * (D + 4) + WIN_BN * (D + 4) + WIN_BN * D + WIN_BM * (WIN_BN + 4)) * (int)sizeof(float);
   if (cudaFuncSetAttribute(state_partial_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_state) != cudaSuccess ||
       cudaFuncSetAttribute(readout_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_rd) != cudaSuccess ||
@@ -163,12 +164,13 @@ int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* ou
                       const Geo& g, int n_split, int carry_slot, int parts, cudaStream_t st) {
   const rehyat_config& c = ctx->cfg;
   const int rd_half = ctx->tensor_ok ? 1 : 0;     // the tensor-core window kernels read the bf16 form of the read-out
-  PhiDims pd = {D, c.phi_hidden, c.phi_dim, c.poly_degree, c.act_hidden, c.act_out};
+  PhiDims pd = {D, c.phi_hidden, c.phi_dim, c.poly_degree, c.act_hidden, c.act_out, c.phi_layers > 2 ? c.phi_layers - 2 : 0};
   constexpr int SD = D + 4;
   const int tiles = (g.Np + SIMT_TM - 1) / SIMT_TM;
   if (parts & PART_STATE) {
-    PhiPtrs<T> wk = {(const T*)phi->k_W1, (const T*)phi->k_b1, (const T*)phi->k_W2, (const T*)phi->k_b2};
-    const size_t smem_state = (size_t)SIMT_TM * (2 * D + pd.Dh + pd.Dp) * sizeof(float);
+    PhiPtrs<T> wk = {(const T*)phi->k_W1, (const T*)phi->k_b1, (const T*)phi->k_W2, (const T*)phi->k_b2,
+                     (const T*)phi->k_Wmid, (const T*)phi->k_bmid};
+    const size_t smem_state = ((size_t)SIMT_TM * (2 * D + pd.Dp) + phi_hidden_floats(pd.Dh, pd.n_mid)) * sizeof(float);
     ctx->prof.begin(REHYAT_PROF_STATE, st);
     state_partial_simt<T, D><<<dim3(n_split, g.G, g.BH), SIMT_PHI_THREADS, smem_state, st>>>(
         k, v, wk, pd, g, n_split, ctx->partial);
@@ -181,8 +183,9 @@ int launch_group_simt(rehyat_ctx* ctx, const T* q, const T* k, const T* v, T* ou
     ctx->last_launches += 2;
   }
   if (parts & PART_READOUT) {
-    PhiPtrs<T> wq = {(const T*)phi->q_W1, (const T*)phi->q_b1, (const T*)phi->q_W2, (const T*)phi->q_b2};
-    const size_t smem_rd = (size_t)SIMT_TM * (D + pd.Dh + pd.Dp) * sizeof(float);
+    PhiPtrs<T> wq = {(const T*)phi->q_W1, (const T*)phi->q_b1, (const T*)phi->q_W2, (const T*)phi->q_b2,
+                     (const T*)phi->q_Wmid, (const T*)phi->q_bmid};
+    const size_t smem_rd = ((size_t)SIMT_TM * (D + pd.Dp) + phi_hidden_floats(pd.Dh, pd.n_mid)) * sizeof(float);
     ctx->prof.begin(REHYAT_PROF_READOUT, st);
     readout_simt<T, D><<<dim3(tiles, g.G, g.BH), SIMT_PHI_THREADS, smem_rd, st>>>(q, wq, pd, g, ctx->state,
                                                                                  ctx->readout, ctx->rd_cap, rd_half);
@@ -274,6 +277,19 @@ int run_parts(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void
   return rc;
 }
 
+// The phi parameter pointers: all there and 16-byte aligned (the hidden layers in between only for deeper maps).
+bool phi_pointers_ok(const rehyat_config& c, const rehyat_phi_params* phi) {
+  const void* two[] = {phi->q_W1, phi->q_b1, phi->q_W2, phi->q_b2, phi->k_W1, phi->k_b1, phi->k_W2, phi->k_b2};
+  for (const void* p : two)
+    if (!p || !aligned16(p)) return false;
+  if (c.phi_layers > 2) {
+    const void* mid[] = {phi->q_Wmid, phi->q_bmid, phi->k_Wmid, phi->k_bmid};
+    for (const void* p : mid)
+      if (!p || !aligned16(p)) return false;
+  }
+  return true;
+}
+
 // The size arguments of a forward call against the limits of the context (nothing is enqueued before this passes).
 int check_sizes(const rehyat_ctx* ctx, int batch, int frames, int H, int W, int chunk, int overlap) {
   const rehyat_config& c = ctx->cfg;
@@ -347,7 +363,8 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
                                       c.poly_degree, c.act_hidden, c.act_out);
   if ((c.impl == REHYAT_IMPL_TENSOR || c.impl == REHYAT_IMPL_TENSOR_WINDOW) && !ctx->tensor_ok) { delete ctx; return REHYAT_ERR_UNSUPPORTED; }
   if (c.impl == REHYAT_IMPL_SIMT) ctx->tensor_ok = false;
-  ctx->tc.phi_ok = ctx->tensor_ok && c.impl != REHYAT_IMPL_TENSOR_WINDOW && tc_phi_supported(c.phi_hidden, c.phi_dim, c.poly_degree);
+  ctx->tc.phi_ok = ctx->tensor_ok && c.impl != REHYAT_IMPL_TENSOR_WINDOW && c.phi_layers <= 2 &&
+                   tc_phi_supported(c.phi_hidden, c.phi_dim, c.poly_degree);
 
   const int np_max = c.max_tokens_per_frame * c.max_chunk_frames;
   const int want = c.group_tokens > 0 ? c.group_tokens : 32768;
@@ -476,10 +493,10 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   const int chunk_eff = chunk < frames ? chunk : frames;      // one chunk covers everything beyond that
   const int overlap_eff = overlap < frames ? overlap : frames; // the window is clamped at token 0 anyway
   if (out == q || out == k || out == v) return REHYAT_ERR_INVALID_ARG;
-  const void* ptrs[] = {q, k, v, out, phi->q_W1, phi->q_b1, phi->q_W2, phi->q_b2,
-                        phi->k_W1, phi->k_b1, phi->k_W2, phi->k_b2};
+  const void* ptrs[] = {q, k, v, out};
   for (const void* p : ptrs)
-    if (!p || !aligned16(p)) return REHYAT_ERR_INVALID_ARG;
+    if (!aligned16(p)) return REHYAT_ERR_INVALID_ARG;
+  if (!phi_pointers_ok(c, phi)) return REHYAT_ERR_INVALID_ARG;
   const size_t es = elem_size(c.dtype);
   const long long strides[] = {lay->stride_batch, lay->stride_head, lay->stride_token};
   for (long long s : strides)
@@ -570,10 +587,8 @@ int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host,
   if (!ctx || !q_host || !k_host || !v_host || !out_host || !phi) return REHYAT_ERR_INVALID_ARG;
   // every argument is checked before the first copy is enqueued
   if (const int bad = check_sizes(ctx, batch, frames, H, W, chunk, overlap)) return bad;
-  const void* pp[] = {phi->q_W1, phi->q_b1, phi->q_W2, phi->q_b2, phi->k_W1, phi->k_b1, phi->k_W2, phi->k_b2};
-  for (const void* p : pp)
-    if (!p || !aligned16(p)) return REHYAT_ERR_INVALID_ARG;
   const rehyat_config& c = ctx->cfg;
+  if (!phi_pointers_ok(c, phi)) return REHYAT_ERR_INVALID_ARG;
   const long long N = (long long)H * W * frames;
   const size_t bytes = (size_t)batch * c.n_heads * N * c.head_dim * elem_size(c.dtype);
   DeviceGuard guard(c.device);
@@ -623,6 +638,11 @@ int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host,
     ph.q_W2 = (const uint8_t*)phi->q_W2 + w2; ph.q_b2 = (const uint8_t*)phi->q_b2 + b2;
     ph.k_W1 = (const uint8_t*)phi->k_W1 + w1; ph.k_b1 = (const uint8_t*)phi->k_b1 + b1;
     ph.k_W2 = (const uint8_t*)phi->k_W2 + w2; ph.k_b2 = (const uint8_t*)phi->k_b2 + b2;
+    if (c.phi_layers > 2) {
+      const size_t wm = (size_t)h0 * (c.phi_layers - 2) * c.phi_hidden * c.phi_hidden * es, bm = (size_t)h0 * (c.phi_layers - 2) * c.phi_hidden * es;
+      ph.q_Wmid = (const uint8_t*)phi->q_Wmid + wm; ph.q_bmid = (const uint8_t*)phi->q_bmid + bm;
+      ph.k_Wmid = (const uint8_t*)phi->k_Wmid + wm; ph.k_bmid = (const uint8_t*)phi->k_bmid + bm;
+    }
     ctx->head_count = cnt;
     const int launches_before = gi == 0 ? 0 : ctx->last_launches;
     rc = rehyat_forward(ctx, (uint8_t*)ctx->stage[0] + off0, (uint8_t*)ctx->stage[1] + off0, (uint8_t*)ctx->stage[2] + off0,
@@ -719,10 +739,10 @@ int rehyat_stream_step(rehyat_ctx* ctx, const void* q_chunk, const void* k_chunk
   if (!s.active || frames_in_chunk < 1 || frames_in_chunk > s.chunk) return REHYAT_ERR_INVALID_ARG;
   const rehyat_config& c = ctx->cfg;
   if (out_chunk == q_chunk || out_chunk == k_chunk || out_chunk == v_chunk) return REHYAT_ERR_INVALID_ARG;
-  const void* ptrs[] = {q_chunk, k_chunk, v_chunk, out_chunk, phi->q_W1, phi->q_b1, phi->q_W2, phi->q_b2,
-                        phi->k_W1, phi->k_b1, phi->k_W2, phi->k_b2};
+  const void* ptrs[] = {q_chunk, k_chunk, v_chunk, out_chunk};
   for (const void* p : ptrs)
-    if (!p || !aligned16(p)) return REHYAT_ERR_INVALID_ARG;
+    if (!aligned16(p)) return REHYAT_ERR_INVALID_ARG;
+  if (!phi_pointers_ok(c, phi)) return REHYAT_ERR_INVALID_ARG;
   const long long es = (long long)elem_size(c.dtype);
   const long long strides[] = {lay->stride_batch, lay->stride_head, lay->stride_token};
   for (long long x : strides)

@@ -16,14 +16,20 @@ constexpr int SIMT_PHI_THREADS = 512;
 
 struct PhiDims {
   int d, Dh, Dp, P, act_hidden, act_out;
+  int n_mid;     // hidden layers between the first and the last (0 for the two-layer map)
 };
 
 template <typename T>
 struct PhiPtrs {
   const T* W1; const T* b1; const T* W2; const T* b2;   // already offset to the head
+  const T* Wm; const T* bm;                             // [n_mid][Dh][Dh], [n_mid][Dh] of the head (n_mid > 0)
 };
 
-// phi of SIMT_TM tokens held in Xs [TM][d] -> Fs [TM][Dp].  Hs [TM][Dh] is scratch.
+// Shared memory (floats) of the hidden activations: one [TM][Dh] buffer, two when there are hidden layers in
+// between (they alternate as input and output).
+__host__ __device__ inline int phi_hidden_floats(int Dh, int n_mid) { return SIMT_TM * Dh * (n_mid > 0 ? 2 : 1); }
+
+// phi of SIMT_TM tokens held in Xs [TM][d] -> Fs [TM][Dp].  Hs (phi_hidden_floats) is scratch.
 // `valid` rows carry tokens; the rest of Fs is forced to zero.
 template <typename T>
 __device__ void phi_tile_simt(const float* Xs, float* Hs, float* Fs, const PhiPtrs<T>& w,
@@ -51,7 +57,33 @@ __device__ void phi_tile_simt(const float* Xs, float* Hs, float* Fs, const PhiPt
     for (int r = 0; r < RPG; ++r) Hs[(r0 + r) * pd.Dh + j] = apply_act(acc[r] + b, pd.act_hidden);
   }
   __syncthreads();
-  // layer 2 + polynomial expansion
+  // hidden layers in between: h <- act_hidden(Wm h + bm), the two buffers alternating
+  for (int m = 0; m < pd.n_mid; ++m) {
+    float* Hn = Hs + ((m & 1) ? 0 : SIMT_TM * pd.Dh);
+    const float* Hp = Hs + ((m & 1) ? SIMT_TM * pd.Dh : 0);
+    for (int idx = tid; idx < pd.Dh * RG; idx += NT) {
+      const int j = idx % pd.Dh, r0 = (idx / pd.Dh) * RPG;
+      float acc[RPG];
+#pragma unroll
+      for (int r = 0; r < RPG; ++r) acc[r] = 0.f;
+      const T* wrow = w.Wm + ((size_t)m * pd.Dh + j) * pd.Dh;
+      for (int k = 0; k < pd.Dh; k += 4) {
+        float4 wv = ld4(wrow + k);
+#pragma unroll
+        for (int r = 0; r < RPG; ++r) {
+          float4 x = *reinterpret_cast<const float4*>(Hp + (r0 + r) * pd.Dh + k);
+          acc[r] = fmaf(x.x, wv.x, acc[r]); acc[r] = fmaf(x.y, wv.y, acc[r]);
+          acc[r] = fmaf(x.z, wv.z, acc[r]); acc[r] = fmaf(x.w, wv.w, acc[r]);
+        }
+      }
+      const float b = ldf(w.bm + (size_t)m * pd.Dh + j);
+#pragma unroll
+      for (int r = 0; r < RPG; ++r) Hn[(r0 + r) * pd.Dh + j] = apply_act(acc[r] + b, pd.act_hidden);
+    }
+    __syncthreads();
+  }
+  Hs += (pd.n_mid & 1) ? SIMT_TM * pd.Dh : 0;          // where the last hidden activations are
+  // last layer + polynomial expansion
   const int part_w = pd.Dp / pd.P;
   for (int idx = tid; idx < pd.Dp * RG; idx += NT) {
     const int j = idx % pd.Dp, r0 = (idx / pd.Dp) * RPG;
@@ -92,7 +124,7 @@ __device__ void load_rows_simt(float* dst, const T* base, long long stride_n, in
   }
 }
 
-// grid (n_split, G, BH), SIMT_PHI_THREADS threads, dynamic smem (TM*(2d + Dh + Dp)) floats.
+// grid (n_split, G, BH), SIMT_PHI_THREADS threads, dynamic smem TM*(2d + Dp) + phi_hidden_floats floats.
 // Chunk t = t0 + blockIdx.y admits the keys [lo_{t-1}, lo_t) into the state (Eq. 17-18: only the
 // newly admitted tokens).  Split s takes a contiguous share of them and writes
 // partial[blockIdx.y][s][bh] = sum_j phi_k(k_j) [v_j | 1]  as [Dp][SD] floats, SD = d + 4,
@@ -106,7 +138,7 @@ state_partial_simt(const T* __restrict__ k, const T* __restrict__ v, PhiPtrs<T> 
   float* Xs = smem;
   float* Vs = Xs + SIMT_TM * D;
   float* Hs = Vs + SIMT_TM * D;
-  float* Fs = Hs + SIMT_TM * pd.Dh;
+  float* Fs = Hs + phi_hidden_floats(pd.Dh, pd.n_mid);
 
   const int s = blockIdx.x, ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
   const int head = bh % g.n_heads;
@@ -117,7 +149,9 @@ state_partial_simt(const T* __restrict__ k, const T* __restrict__ v, PhiPtrs<T> 
   const int a = min(lo_prev + s * per, lo), b = min(a + per, lo);
 
   PhiPtrs<T> w = {wk.W1 + (size_t)head * pd.Dh * D, wk.b1 + (size_t)head * pd.Dh,
-                  wk.W2 + (size_t)head * pd.Dp * pd.Dh, wk.b2 + (size_t)head * pd.Dp};
+                  wk.W2 + (size_t)head * pd.Dp * pd.Dh, wk.b2 + (size_t)head * pd.Dp,
+                  pd.n_mid ? wk.Wm + (size_t)head * pd.n_mid * pd.Dh * pd.Dh : nullptr,
+                  pd.n_mid ? wk.bm + (size_t)head * pd.n_mid * pd.Dh : nullptr};
   const long long hoff = head_offset(g, bh);
 
   // thread -> (feature f, half of the value columns)
@@ -209,7 +243,7 @@ readout_simt(const T* __restrict__ q, PhiPtrs<T> wq, PhiDims pd, Geo g, const fl
   constexpr int SD = D + 4;
   float* Xs = smem;
   float* Hs = Xs + SIMT_TM * D;
-  float* Fs = Hs + SIMT_TM * pd.Dh;
+  float* Fs = Hs + phi_hidden_floats(pd.Dh, pd.n_mid);
 
   const int ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
   if (!geo_linear(g, t)) return;                       // empty linear set: nothing to read out
@@ -218,7 +252,9 @@ readout_simt(const T* __restrict__ q, PhiPtrs<T> wq, PhiDims pd, Geo g, const fl
   if (tok0 >= q1) return;
   const int head = bh % g.n_heads;
   PhiPtrs<T> w = {wq.W1 + (size_t)head * pd.Dh * D, wq.b1 + (size_t)head * pd.Dh,
-                  wq.W2 + (size_t)head * pd.Dp * pd.Dh, wq.b2 + (size_t)head * pd.Dp};
+                  wq.W2 + (size_t)head * pd.Dp * pd.Dh, wq.b2 + (size_t)head * pd.Dp,
+                  pd.n_mid ? wq.Wm + (size_t)head * pd.n_mid * pd.Dh * pd.Dh : nullptr,
+                  pd.n_mid ? wq.bm + (size_t)head * pd.n_mid * pd.Dh : nullptr};
   load_rows_simt(Xs, q + q_row_offset(g, bh, 0), g.qstride_n, tok0, q1, D);
   __syncthreads();
   phi_tile_simt(Xs, Hs, Fs, w, pd, q1 - tok0);

@@ -41,6 +41,7 @@ class Workload:
     seed: int = BASE_SEED
     phi_hidden: int = 0   # 0: the default width 2 * head_dim
     phi_dim: int = 0      # 0: the default width 2 * head_dim
+    phi_layers: int = 2   # layers of the phi MLP; beyond two, hidden layers [D_h, D_h] sit between the first and the last
 
     @property
     def HW(self):
@@ -98,9 +99,12 @@ def _torch_dtype(name):
 
 def make_phi_params(wl: Workload, which: str, scale: float = 1.0, std: float = 0.02):
     """Parameters of phi_q ("phi_q") or phi_k ("phi_k"): W1 [n_h, D_h, d], b1 [n_h, D_h],
-    W2 [n_h, D', D_h], b2 [n_h, D'], in the workload's dtype."""
+    W2 [n_h, D', D_h], b2 [n_h, D'] (and Wmid, bmid of a deeper map), in the workload's dtype."""
     nh, d, Dh, Do = wl.n_heads, wl.head_dim, wl.D_h, wl.D_out
     sizes = {"W1": (nh, Dh, d), "b1": (nh, Dh), "W2": (nh, Do, Dh), "b2": (nh, Do)}
+    if wl.phi_layers > 2:       # drawn after the others, so that the two-layer tensors do not depend on the depth
+        sizes["Wmid"] = (nh, wl.phi_layers - 2, Dh, Dh)
+        sizes["bmid"] = (nh, wl.phi_layers - 2, Dh)
     flat = _normal(wl.seed, _STREAMS[which], (sum(int(np.prod(s)) for s in sizes.values()),))
     out, off = {}, 0
     for name, shp in sizes.items():

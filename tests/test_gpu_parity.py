@@ -277,6 +277,27 @@ def test_other_feature_maps(variant, dtype):
     check(y, ref, dtype)
 
 
+@pytest.mark.parametrize("layers", [3, 4])
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_deeper_feature_maps(layers, dtype):
+    """phi with one or two further hidden layers (rehyat_config.phi_layers): the linear branch runs on the SIMT
+    kernels, the softmax window of the bf16 case on the tensor cores."""
+    wl = synth.Workload("deep", 1, 2, 128, 5, 10, 20, 2, 1, dtype, dtype == "bf16", seed=synth.BASE_SEED + 89,
+                        phi_layers=layers)
+    # every further layer of std-0.02 parameters shrinks the features: scaled so that about half of the normaliser is linear
+    x = synth.make_inputs(wl, phi_scale={3: 2.0, 4: 2.5}[layers], v_frame_offsets=True)
+    assert x["phi_q"]["Wmid"].shape == (2, layers - 2, 256, 256)
+    f = synth.to_f64(x)
+    ref, frac = orc.hybrid_direct(f["q"], f["k"], f["v"], f["phi_q"], f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To,
+                                  return_parts=True)
+    assert 0.3 < frac[:, :, 2 * wl.HW * wl.Tc:].mean() < 0.9   # neither branch drowns the other
+    two = {n: t for n, t in f["phi_q"].items() if n not in ("Wmid", "bmid")}
+    assert np.abs(orc.hybrid_direct(f["q"], f["k"], f["v"], two, f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To) - ref).max() > 1e-2
+    y, used = run_gpu(wl, x)
+    assert used == ("tensor" if dtype == "bf16" else "simt")
+    check(y, ref, dtype)
+
+
 def test_tensor_window_with_simt_linear_branch_matches_the_all_tensor_path():
     wl = synth.Workload("tw", 1, 2, 128, 6, 10, 20, 2, 1, "bf16", True, seed=synth.BASE_SEED + 86)
     x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
