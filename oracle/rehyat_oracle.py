@@ -103,6 +103,43 @@ def phi_param_count(n_heads, d, D_h, D_out, with_bias=False):
 
 
 # ----------------------------------------------------------------------------------------
+# what a DiT block does to q and k before the attention operator (the block of Eq. 1 around
+# A_l; the paper takes it over from the pretrained model and does not restate it)
+# ----------------------------------------------------------------------------------------
+
+def rms_norm(x, weight=None, eps=1e-6):
+    """x / sqrt(mean(x^2 over the last axis) + eps) * weight, the RMS normalisation applied to the
+    queries and keys of each head (weight [d] or broadcastable; None: ones)."""
+    x = np.asarray(x, np.float64)
+    y = x / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + eps)
+    return y if weight is None else y * np.asarray(weight, np.float64)
+
+
+def rope_rotate(x, cos, sin):
+    """Rotary position embedding with caller-supplied tables: the pair (x[..., n, 2i], x[..., n, 2i+1]) of token n
+    is rotated by the angle whose cosine and sine are cos[n, i], sin[n, i] (x [..., N, d]; cos, sin [N, d/2])."""
+    x = np.asarray(x, np.float64)
+    cos = np.asarray(cos, np.float64); sin = np.asarray(sin, np.float64)
+    a, b = x[..., 0::2], x[..., 1::2]
+    out = np.empty_like(x)
+    out[..., 0::2] = a * cos - b * sin
+    out[..., 1::2] = a * sin + b * cos
+    return out
+
+
+def qk_transform(q, k, q_weight=None, k_weight=None, eps=1e-6, cos=None, sin=None, norm=True):
+    """q, k [B, n_h, N, d] as the block hands them over -> what the attention operator sees: per-head RMS norm
+    (weights [n_h, d] or None) followed by the rotation.  Either step can be left out (norm=False; cos=None)."""
+    q = np.asarray(q, np.float64); k = np.asarray(k, np.float64)
+    if norm:
+        q = rms_norm(q, None if q_weight is None else np.asarray(q_weight, np.float64)[None, :, None, :], eps)
+        k = rms_norm(k, None if k_weight is None else np.asarray(k_weight, np.float64)[None, :, None, :], eps)
+    if cos is not None:
+        q, k = rope_rotate(q, cos, sin), rope_rotate(k, cos, sin)
+    return q, k
+
+
+# ----------------------------------------------------------------------------------------
 # token sets
 # ----------------------------------------------------------------------------------------
 

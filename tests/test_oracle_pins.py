@@ -400,3 +400,66 @@ def test_stored_rows_are_reproduced_by_the_recurrent_form():
         assert np.max(np.abs(y[0, h, r] - want)) < 1e-13
         n += 1
     assert n == 22
+
+
+# ------------------------------------------------------------------ q/k normalisation and rotation
+def test_rms_norm_by_hand():
+    y = orc.rms_norm(np.array([3.0, 4.0]), eps=0.0)
+    assert np.allclose(y, np.array([3.0, 4.0]) / math.sqrt(12.5), atol=1e-15)          # mean square (9 + 16) / 2
+    assert np.allclose(orc.rms_norm(np.array([3.0, 4.0]), weight=np.array([2.0, -1.0]), eps=0.0),
+                       [6.0 / math.sqrt(12.5), -4.0 / math.sqrt(12.5)], atol=1e-15)
+    assert np.allclose(orc.rms_norm(np.array([1.0, 1.0, 1.0, 1.0]), eps=3.0), 0.5)     # 1 / sqrt(1 + 3)
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((5, 7, 16))
+    y = orc.rms_norm(x, eps=0.0)
+    assert np.allclose(np.sqrt((y * y).mean(-1)), 1.0)                                 # unit RMS, any scale of the input
+    assert np.allclose(orc.rms_norm(10.0 * x, eps=0.0), y)
+    assert np.allclose(orc.rms_norm(x, eps=0.0), torch.nn.functional.rms_norm(torch.from_numpy(x), (16,), eps=0.0).numpy())
+
+
+def test_rope_by_hand_and_its_invariants():
+    # a quarter turn maps (1, 0) to (0, 1) and (0, 1) to (-1, 0); angle 0 is the identity
+    x = np.array([[1.0, 0.0, 0.0, 1.0]])
+    cos = np.array([[0.0, 0.0]]); sin = np.array([[1.0, 1.0]])
+    assert np.allclose(orc.rope_rotate(x, cos, sin), [[0.0, 1.0, -1.0, 0.0]], atol=1e-15)
+    assert np.allclose(orc.rope_rotate(x, np.ones((1, 2)), np.zeros((1, 2))), x)
+    # 30 degrees on (2, 0): (sqrt 3, 1)
+    assert np.allclose(orc.rope_rotate(np.array([[2.0, 0.0]]), [[math.sqrt(3) / 2]], [[0.5]]), [[math.sqrt(3.0), 1.0]], atol=1e-15)
+    rng = np.random.default_rng(4)
+    N, d = 9, 8
+    theta = 1.0 / 100.0 ** (np.arange(d // 2) / (d // 2))
+    ang = np.arange(N)[:, None] * theta[None, :]
+    q, k = rng.standard_normal((N, d)), rng.standard_normal((N, d))
+    rq, rk = orc.rope_rotate(q, np.cos(ang), np.sin(ang)), orc.rope_rotate(k, np.cos(ang), np.sin(ang))
+    # the same thing as a complex multiplication of the pairs
+    zq = (q[:, 0::2] + 1j * q[:, 1::2]) * np.exp(1j * ang)
+    assert np.allclose(rq[:, 0::2], zq.real) and np.allclose(rq[:, 1::2], zq.imag)
+    # a rotation: pair norms are kept
+    assert np.allclose(rq[:, 0::2] ** 2 + rq[:, 1::2] ** 2, q[:, 0::2] ** 2 + q[:, 1::2] ** 2)
+    # relative positions: <R_m q, R_n k> depends on n - m only
+    q0, k0 = q[0], k[0]
+    dots = np.array([[orc.rope_rotate(q0[None], np.cos(ang[m:m + 1]), np.sin(ang[m:m + 1]))[0] @
+                      orc.rope_rotate(k0[None], np.cos(ang[n:n + 1]), np.sin(ang[n:n + 1]))[0] for n in range(N)] for m in range(N)])
+    for s_ in range(1, N - 1):
+        assert np.allclose(np.diag(dots, s_), np.diag(dots, s_)[0])
+    assert not np.allclose(np.diag(dots, 1), np.diag(dots, 2)[:1])
+
+
+def test_qk_transform_composes_norm_then_rotation():
+    rng = np.random.default_rng(6)
+    B, nh, N, d = 2, 3, 5, 4
+    q, k = rng.standard_normal((B, nh, N, d)), rng.standard_normal((B, nh, N, d))
+    wq, wk = rng.standard_normal((nh, d)), rng.standard_normal((nh, d))
+    ang = rng.standard_normal((N, d // 2))
+    tq, tk = orc.qk_transform(q, k, wq, wk, 1e-6, np.cos(ang), np.sin(ang))
+    for b in range(B):
+        for h in range(nh):
+            assert np.allclose(tq[b, h], orc.rope_rotate(orc.rms_norm(q[b, h], wq[h], 1e-6), np.cos(ang), np.sin(ang)))
+            assert np.allclose(tk[b, h], orc.rope_rotate(orc.rms_norm(k[b, h], wk[h], 1e-6), np.cos(ang), np.sin(ang)))
+    # the order matters when the weight is not constant inside a pair (norm first, as the block does)
+    other = orc.rms_norm(orc.rope_rotate(q[0, 0], np.cos(ang), np.sin(ang)), wq[0], 1e-6)
+    assert not np.allclose(tq[0, 0], other)
+    nq, _ = orc.qk_transform(q, k, None, None, 0.0, None, None)
+    assert np.allclose(np.sqrt((nq * nq).mean(-1)), 1.0)
+    rq, _ = orc.qk_transform(q, k, cos=np.cos(ang), sin=np.sin(ang), norm=False)
+    assert np.allclose(rq, orc.rope_rotate(q, np.cos(ang), np.sin(ang)))
