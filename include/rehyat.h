@@ -106,6 +106,11 @@ typedef struct rehyat_config {
                                    (Section 4.3 varies the "transformation complexity" of phi).
                                    Deeper maps run on the SIMT kernels (the softmax window stays
                                    on the tensor cores).                                       */
+  int32_t qk_transform;         /* 1: the context can normalise and rotate q and k ahead of the
+                                   operator (rehyat_set_qk_transform); rehyat_create then also
+                                   allocates room for the transformed q and k of max_frames
+                                   frames (max_frames >= 1 required).  0: q and k are used as
+                                   given.                                                      */
   int32_t window_tiles;         /* tensor-core window kernel: 128-row query tiles per work
                                    item.  0 = chosen per launch from how many items there are
                                    for the SMs; 1 or 2 fixes it (same results up to the order
@@ -227,6 +232,31 @@ int rehyat_forward_static(const rehyat_config* cfg, const void* q, const void* k
                           int32_t chunk, int32_t overlap, void* cuda_stream);
 size_t rehyat_static_scratch_bytes(void);
 
+/* What a DiT block does to q and k between its projections and the attention operator (the block of Eq. 1
+ * around A_l, which the paper takes over from the pretrained model): per-head RMS normalisation
+ *   x <- x / sqrt(mean_d(x^2) + norm_eps) * weight        (weight [n_heads, head_dim], or NULL for none)
+ * followed by the rotary embedding from caller-supplied tables: the pair (x[2i], x[2i+1]) of token n is turned by
+ * the angle with cosine rope_cos[n*head_dim/2 + i] and sine rope_sin[n*head_dim/2 + i] (how the angles follow from
+ * the frame / row / column of a token is the caller's business).  Either step can be left out (rms_norm = 0;
+ * rope_cos = NULL).  All pointers are device pointers that must stay valid while the transform is set; the
+ * tables are fp32 and cover the frames*H*W tokens of every forward call that follows.
+ *
+ * rehyat_set_qk_transform(ctx, t) switches it on for the rehyat_forward calls that follow (a context made with
+ * qk_transform = 1, frames <= max_frames; q, k must be laid out so that the last element of the batch lies
+ * within max_batch*n_heads*max_frames*max_tokens_per_frame*head_dim elements of the first), t = NULL switches
+ * it off.  Each call then runs one more kernel, bound by HBM, that writes the transformed q and k into the
+ * context's buffers; both branches (softmax window and phi) see the transformed tensors; v is untouched.
+ * rehyat_forward_host and rehyat_stream_step return REHYAT_ERR_UNSUPPORTED while a transform is set. */
+typedef struct rehyat_qk_transform {
+  const void* q_norm_weight;    /* [n_heads, head_dim], operator dtype, or NULL */
+  const void* k_norm_weight;
+  int32_t rms_norm;             /* 1: normalise, 0: skip the normalisation (the weights are then ignored) */
+  float norm_eps;
+  const float* rope_cos;        /* [frames*H*W, head_dim/2] fp32, or NULL: no rotation */
+  const float* rope_sin;
+} rehyat_qk_transform;
+int rehyat_set_qk_transform(rehyat_ctx* ctx, const rehyat_qk_transform* t);
+
 /* Frees the workspace.  NULL is a no-op returning REHYAT_OK. */
 int rehyat_destroy(rehyat_ctx* ctx);
 
@@ -275,7 +305,8 @@ int rehyat_set_linear_share_output(rehyat_ctx* ctx, float* share);
 #define REHYAT_PROF_SCAN    1   /* running sum along the chunk axis (Eq. 14-15) */
 #define REHYAT_PROF_READOUT 2   /* phi_q + linear read-out (Eq. 7, 9)            */
 #define REHYAT_PROF_WINDOW  3   /* softmax window + joint normaliser (Eq. 5-8)   */
-#define REHYAT_PROF_KINDS   4
+#define REHYAT_PROF_QKPREP  4   /* q/k normalisation + rotation, when set         */
+#define REHYAT_PROF_KINDS   5
 int rehyat_profile_enable(rehyat_ctx* ctx, int on);
 int rehyat_profile_read(rehyat_ctx* ctx, double* ms, int32_t* launches);
 

@@ -22,16 +22,16 @@ EXPORTS = ["rehyat_create", "rehyat_forward", "rehyat_forward_host", "rehyat_for
            "rehyat_stream_begin", "rehyat_stream_step", "rehyat_stream_state_bytes", "rehyat_stream_export",
            "rehyat_stream_import",
            "rehyat_workspace_bytes", "rehyat_status", "rehyat_set_wait_limit", "rehyat_last_launches", "rehyat_last_impl",
-           "rehyat_last_window_tiles", "rehyat_set_linear_share_output",
+           "rehyat_last_window_tiles", "rehyat_set_linear_share_output", "rehyat_set_qk_transform",
            "rehyat_profile_enable", "rehyat_profile_read", "rehyat_strerror", "rehyat_version"]
-PROF_KINDS = ("state", "scan", "readout", "window")
+PROF_KINDS = ("state", "scan", "readout", "window", "qk_prep")
 
 
 class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "device", "dtype", "n_heads", "head_dim", "phi_hidden", "phi_dim", "poly_degree", "act_hidden",
         "act_out", "c_mode", "impl", "max_batch", "max_tokens_per_frame", "max_chunk_frames", "group_tokens",
-        "bidirectional", "max_frames", "exp_poly", "phi_layers", "window_tiles")]
+        "bidirectional", "max_frames", "exp_poly", "phi_layers", "qk_transform", "window_tiles")]
 
 
 # Values of the tuning fields of rehyat_config that a Rehyat(...) call does not name (0 = the library's choice).
@@ -40,6 +40,11 @@ TUNING_DEFAULTS = {"exp_poly": 0, "window_tiles": 0}
 
 class Layout(C.Structure):
     _fields_ = [("stride_batch", C.c_int64), ("stride_head", C.c_int64), ("stride_token", C.c_int64)]
+
+
+class QkTransform(C.Structure):
+    _fields_ = [("q_norm_weight", C.c_void_p), ("k_norm_weight", C.c_void_p), ("rms_norm", C.c_int32),
+                ("norm_eps", C.c_float), ("rope_cos", C.c_void_p), ("rope_sin", C.c_void_p)]
 
 
 class PhiParams(C.Structure):
@@ -83,6 +88,7 @@ def lib():
         L.rehyat_last_impl.argtypes = [C.c_void_p]
         L.rehyat_last_window_tiles.argtypes = [C.c_void_p]
         L.rehyat_set_linear_share_output.argtypes = [C.c_void_p, C.c_void_p]
+        L.rehyat_set_qk_transform.argtypes = [C.c_void_p, C.POINTER(QkTransform)]
         L.rehyat_profile_enable.argtypes = [C.c_void_p, C.c_int]
         L.rehyat_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int32)]
         L.rehyat_strerror.argtypes = [C.c_int]
@@ -115,7 +121,7 @@ class Rehyat:
     def __init__(self, *, n_heads, head_dim, dtype="bf16", phi_hidden=None, phi_dim=None, poly_degree=2,
                  act_hidden="relu", act_out="relu", c_mode="rowmax", impl="auto", max_batch=1,
                  max_tokens_per_frame=1560, max_chunk_frames=3, group_tokens=0, device=0, bidirectional=False,
-                 max_frames=0, phi_layers=2, **tuning):
+                 max_frames=0, phi_layers=2, qk_transform=False, **tuning):
         unknown = set(tuning) - set(TUNING_DEFAULTS)
         if unknown:
             raise TypeError(f"unknown arguments {sorted(unknown)}")
@@ -123,7 +129,8 @@ class Rehyat:
         self.cfg = Config(device, DTYPE[dtype], n_heads, head_dim, phi_hidden or 2 * head_dim,
                           phi_dim or 2 * head_dim, poly_degree, ACT[act_hidden], ACT[act_out], C_MODE[c_mode],
                           IMPL[impl], max_batch, max_tokens_per_frame, max_chunk_frames, group_tokens,
-                          int(bool(bidirectional)), max_frames, int(tune["exp_poly"]), phi_layers, int(tune["window_tiles"]))
+                          int(bool(bidirectional)), max_frames, int(tune["exp_poly"]), phi_layers, int(bool(qk_transform)),
+                          int(tune["window_tiles"]))
         self.dtype = dtype
         self._h = C.c_void_p(None)
         _check(lib().rehyat_create(C.byref(self._h), C.byref(self.cfg)), "rehyat_create")
@@ -158,6 +165,17 @@ class Rehyat:
     def set_linear_share_output(self, share):
         """share: float32 CUDA tensor [B, n_heads, N] the window kernels fill with nL / (nS + nL), or None."""
         _check(lib().rehyat_set_linear_share_output(self._h, _ptr(share)), "rehyat_set_linear_share_output")
+
+    def set_qk_transform(self, *, q_weight=None, k_weight=None, rms_norm=True, eps=1e-6, cos=None, sin=None, off=False):
+        """rehyat_set_qk_transform: per-head RMS normalisation (weights [n_heads, d] CUDA tensors in the operator
+        dtype, or None) and / or the rotary embedding from fp32 CUDA tables cos, sin [N, d/2].  off=True: as given."""
+        if off:
+            _check(lib().rehyat_set_qk_transform(self._h, None), "rehyat_set_qk_transform")
+            self._qk_keep = None
+            return
+        t = QkTransform(_ptr(q_weight), _ptr(k_weight), int(bool(rms_norm)), float(eps), _ptr(cos), _ptr(sin))
+        _check(lib().rehyat_set_qk_transform(self._h, C.byref(t)), "rehyat_set_qk_transform")
+        self._qk_keep = (q_weight, k_weight, cos, sin)         # the library keeps the pointers, not the tensors
 
     @staticmethod
     def phi_struct(phi_q, phi_k):
@@ -257,7 +275,7 @@ def forward_static(q, k, v, phi_q, phi_k, frames, H, W, chunk, overlap, *, dtype
     if out is None:
         out = torch.empty_like(q)
     cfg = Config(q.device.index or 0, DTYPE[dtype], nh, d, phi_hidden or 2 * d, phi_dim or 2 * d, poly_degree,
-                 ACT[act_hidden], ACT[act_out], C_MODE[c_mode], 0, 1, 1, 1, 0, 0, 0, 0, phi_layers, 0)
+                 ACT[act_hidden], ACT[act_out], C_MODE[c_mode], 0, 1, 1, 1, 0, 0, 0, 0, phi_layers, 0, 0)
     lay = Layout(nh * N * d, N * d, d)
     st = stream if stream is not None else torch.cuda.current_stream(q.device)
     phi = Rehyat.phi_struct(phi_q, phi_k)

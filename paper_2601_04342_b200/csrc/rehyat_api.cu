@@ -66,6 +66,11 @@ struct rehyat_ctx {
   int epoch = 0;               // number of the last tensor-core launch, 1, 2, ... (see ptx::WaitCtx)
   unsigned wait_limit_us = 1000000u;   // bound of every device-side wait
   int withhold_loads = 0;      // test hook of rehyat_set_wait_limit
+  void* qprep = nullptr;       // q and k after rehyat_set_qk_transform (cfg.qk_transform), same layout as the inputs
+  void* kprep = nullptr;
+  size_t prep_elems = 0;       // elements each of the two holds
+  bool qk_on = false;
+  rehyat_qk_transform qk = {};
   float* share_out = nullptr;  // rehyat_set_linear_share_output
   float* share_now = nullptr;  // what the window launches of the call in progress write (null in chunk-by-chunk steps)
   // chunk-by-chunk processing (rehyat_stream_*): the running state lives in slot 0 of `state`; k and v of the
@@ -120,6 +125,7 @@ int check_config(const rehyat_config* c) {
   if (c->max_frames < 0 || c->max_frames > (1 << 20) || (c->bidirectional && c->max_frames < 1)) return REHYAT_ERR_INVALID_ARG;
   if (c->exp_poly < -1 || c->exp_poly > 3) return REHYAT_ERR_INVALID_ARG;
   if (c->phi_layers != 0 && (c->phi_layers < 2 || c->phi_layers > 4)) return REHYAT_ERR_INVALID_ARG;
+  if (c->qk_transform != 0 && (c->qk_transform != 1 || c->max_frames < 1)) return REHYAT_ERR_INVALID_ARG;
   if (c->window_tiles < 0 || c->window_tiles > 2) return REHYAT_ERR_INVALID_ARG;
   if (c->head_dim != 64 && c->head_dim != 128) return REHYAT_ERR_UNSUPPORTED;
   return REHYAT_OK;
@@ -300,6 +306,7 @@ int check_sizes(const rehyat_ctx* ctx, int batch, int frames, int H, int W, int 
   if (HW * frames > INT_MAX / 2) return REHYAT_ERR_INVALID_ARG;
   if ((chunk < frames ? chunk : frames) > c.max_chunk_frames) return REHYAT_ERR_INVALID_ARG;   // one chunk covers everything beyond `frames`
   if (c.bidirectional && frames + 1 > ctx->cum_frames) return REHYAT_ERR_INVALID_ARG;
+  if (ctx->qk_on && frames > c.max_frames) return REHYAT_ERR_INVALID_ARG;
   return REHYAT_OK;
 }
 
@@ -383,6 +390,12 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
   bool ok = cudaMalloc(&ctx->state, b_state) == cudaSuccess && cudaMalloc(&ctx->partial, b_partial) == cudaSuccess &&
             cudaMalloc(&ctx->readout, b_rd) == cudaSuccess && cudaMalloc(&ctx->status_dev, 256) == cudaSuccess;
   ctx->ws_bytes = b_state + b_partial + b_rd + 256;
+  if (ok && c.qk_transform) {
+    ctx->prep_elems = (size_t)ctx->bh_max * c.max_frames * c.max_tokens_per_frame * c.head_dim;
+    const size_t b_prep = ctx->prep_elems * elem_size(c.dtype);
+    ok = cudaMalloc(&ctx->qprep, b_prep) == cudaSuccess && cudaMalloc(&ctx->kprep, b_prep) == cudaSuccess;
+    ctx->ws_bytes += 2 * b_prep;
+  }
   if (ok && c.bidirectional) {
     // Eq. 10-12 is not a recurrence: one running state per latent frame, sized here so that forward never allocates
     const size_t b_cum = slot * ((size_t)c.max_frames + 1);
@@ -412,6 +425,7 @@ int rehyat_destroy(rehyat_ctx* ctx) {
   if (!ctx) return REHYAT_OK;
   DeviceGuard guard(ctx->cfg.device);
   cudaFree(ctx->state); cudaFree(ctx->partial); cudaFree(ctx->readout); cudaFree(ctx->status_dev); cudaFree(ctx->cum);
+  cudaFree(ctx->qprep); cudaFree(ctx->kprep);
   tc_workspace_destroy(&ctx->tc);
   ctx->prof.clear();
   for (void* p : ctx->stage) cudaFree(p);
@@ -475,6 +489,19 @@ int rehyat_status(rehyat_ctx* ctx, void* cuda_stream) {
   return REHYAT_OK;
 }
 
+int rehyat_set_qk_transform(rehyat_ctx* ctx, const rehyat_qk_transform* t) {
+  if (!ctx) return REHYAT_ERR_INVALID_ARG;
+  if (!t) { ctx->qk_on = false; return REHYAT_OK; }
+  if (!ctx->cfg.qk_transform) return REHYAT_ERR_UNSUPPORTED;     // the context was made without room for it
+  const void* ptrs[] = {t->q_norm_weight, t->k_norm_weight, t->rope_cos, t->rope_sin};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return REHYAT_ERR_INVALID_ARG;
+  if ((t->rope_cos == nullptr) != (t->rope_sin == nullptr) || !(t->norm_eps >= 0.f)) return REHYAT_ERR_INVALID_ARG;
+  ctx->qk = *t;
+  ctx->qk_on = true;
+  return REHYAT_OK;
+}
+
 int rehyat_set_wait_limit(rehyat_ctx* ctx, int32_t wait_limit_us, int32_t withhold_loads) {
   if (!ctx || wait_limit_us < 0) return REHYAT_ERR_INVALID_ARG;
   ctx->wait_limit_us = wait_limit_us > 0 ? (unsigned)wait_limit_us : 1000000u;
@@ -535,6 +562,29 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   ctx->last_launches = 0;
   ctx->last_impl = ctx->tensor_ok ? 1 : 0;
   ctx->stream.active = false;                 // the workspace is about to be overwritten
+  if (ctx->qk_on) {
+    // q and k are normalised and rotated into the context's buffers, in the layout they came in
+    const long long last = (batch - 1) * g.stride_b + (g.n_heads - 1) * g.stride_h + (N - 1) * g.stride_n + c.head_dim;
+    if (ctx->head_count > 0 || (size_t)last > ctx->prep_elems) return REHYAT_ERR_INVALID_ARG;
+    QkPrepArgs pa = {ctx->qk.q_norm_weight, ctx->qk.k_norm_weight, ctx->qk.rope_cos, ctx->qk.rope_sin, ctx->qk.norm_eps,
+                     ctx->qk.rms_norm};
+    const int rows_per_block = 256 / (c.head_dim / 8);
+    const unsigned blocks = (unsigned)((N + rows_per_block - 1) / rows_per_block < 2048 ? (N + rows_per_block - 1) / rows_per_block : 2048);
+    const dim3 grid(blocks, g.BH, 2);
+    ctx->prof.begin(REHYAT_PROF_QKPREP, st);
+    if (c.dtype == REHYAT_DTYPE_FP32) {
+      if (c.head_dim == 64) qk_prepare<float, 64><<<grid, 256, 0, st>>>((const float*)q, (const float*)k, (float*)ctx->qprep, (float*)ctx->kprep, g, pa);
+      else qk_prepare<float, 128><<<grid, 256, 0, st>>>((const float*)q, (const float*)k, (float*)ctx->qprep, (float*)ctx->kprep, g, pa);
+    } else {
+      using B = __nv_bfloat16;
+      if (c.head_dim == 64) qk_prepare<B, 64><<<grid, 256, 0, st>>>((const B*)q, (const B*)k, (B*)ctx->qprep, (B*)ctx->kprep, g, pa);
+      else qk_prepare<B, 128><<<grid, 256, 0, st>>>((const B*)q, (const B*)k, (B*)ctx->qprep, (B*)ctx->kprep, g, pa);
+    }
+    ctx->prof.end(REHYAT_PROF_QKPREP, st);
+    ctx->last_launches += 1;
+    q = ctx->qprep;
+    k = ctx->kprep;
+  }
   ctx->share_now = ctx->head_count > 0 ? nullptr : ctx->share_out;   // not through rehyat_forward_host
   if (c.bidirectional && n_chunks > 1) {
     // Eq. 10-12: the linear set of a chunk is everything outside its window.  Pass 1 sums the state frame by
@@ -585,6 +635,7 @@ int rehyat_forward_host(rehyat_ctx* ctx, const void* q_host, const void* k_host,
                         void* out_host, const rehyat_phi_params* phi, int32_t batch, int32_t frames, int32_t H,
                         int32_t W, int32_t chunk, int32_t overlap, void* cuda_stream) {
   if (!ctx || !q_host || !k_host || !v_host || !out_host || !phi) return REHYAT_ERR_INVALID_ARG;
+  if (ctx->qk_on) return REHYAT_ERR_UNSUPPORTED;
   // every argument is checked before the first copy is enqueued
   if (const int bad = check_sizes(ctx, batch, frames, H, W, chunk, overlap)) return bad;
   const rehyat_config& c = ctx->cfg;
@@ -737,6 +788,7 @@ int rehyat_stream_step(rehyat_ctx* ctx, const void* q_chunk, const void* k_chunk
   if (!ctx || !q_chunk || !k_chunk || !v_chunk || !out_chunk || !lay || !phi) return REHYAT_ERR_INVALID_ARG;
   rehyat_ctx::Stream& s = ctx->stream;
   if (!s.active || frames_in_chunk < 1 || frames_in_chunk > s.chunk) return REHYAT_ERR_INVALID_ARG;
+  if (ctx->qk_on) return REHYAT_ERR_UNSUPPORTED;
   const rehyat_config& c = ctx->cfg;
   if (out_chunk == q_chunk || out_chunk == k_chunk || out_chunk == v_chunk) return REHYAT_ERR_INVALID_ARG;
   const void* ptrs[] = {q_chunk, k_chunk, v_chunk, out_chunk};

@@ -298,6 +298,61 @@ readout_simt(const T* __restrict__ q, PhiPtrs<T> wq, PhiDims pd, Geo g, const fl
   }
 }
 
+// What a DiT block does to q and k before the attention operator (the block of Eq. 1 around A_l): per-head RMS
+// normalisation x / sqrt(mean(x^2) + eps) * weight, then the rotary embedding with caller-supplied tables (the
+// pair (x[2i], x[2i+1]) of token n turned by the angle of cos[n][i], sin[n][i]).  One pass over q and k, bound by
+// HBM: every element is read once and written once, in the layout it came in.
+// grid (row blocks, BH, 2: q / k), 256 threads; a row of d elements is shared by d/8 lanes, eight elements each.
+struct QkPrepArgs {
+  const void* wq; const void* wk;       // [n_heads][d] in the operator dtype, or null
+  const float* cos; const float* sin;   // [N][d/2], or null
+  float eps;
+  int rms_norm;
+};
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+qk_prepare(const T* __restrict__ q, const T* __restrict__ k, T* __restrict__ qo, T* __restrict__ ko, Geo g, QkPrepArgs a) {
+  constexpr int LPR = D / 8;                                        // lanes per row
+  const T* __restrict__ src = blockIdx.z ? k : q;
+  T* __restrict__ dst = blockIdx.z ? ko : qo;
+  const T* __restrict__ wgt = static_cast<const T*>(blockIdx.z ? a.wk : a.wq);
+  const int bh = blockIdx.y, head = bh % g.n_heads;
+  const long long hoff = head_offset(g, bh);
+  const int lane_in_row = threadIdx.x % LPR, col = lane_in_row * 8;
+  const int rows_per_block = 256 / LPR;
+  for (int row = blockIdx.x * rows_per_block + threadIdx.x / LPR; row < g.N; row += gridDim.x * rows_per_block) {
+    const T* p = src + hoff + (long long)row * g.stride_n + col;
+    const float4 x0 = ld4(p), x1 = ld4(p + 4);
+    float x[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+    if (a.rms_norm) {
+      float ss = 0.f;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) ss = fmaf(x[e], x[e], ss);
+#pragma unroll
+      for (int o = 1; o < LPR; o <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      const float inv = rsqrtf(ss * (1.f / D) + a.eps);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) x[e] *= inv;
+      if (wgt != nullptr) {
+        const float4 w0 = ld4(wgt + (size_t)head * D + col), w1 = ld4(wgt + (size_t)head * D + col + 4);
+        x[0] *= w0.x; x[1] *= w0.y; x[2] *= w0.z; x[3] *= w0.w; x[4] *= w1.x; x[5] *= w1.y; x[6] *= w1.z; x[7] *= w1.w;
+      }
+    }
+    if (a.cos != nullptr) {
+      const float4 c = *reinterpret_cast<const float4*>(a.cos + (size_t)row * (D / 2) + col / 2);
+      const float4 s = *reinterpret_cast<const float4*>(a.sin + (size_t)row * (D / 2) + col / 2);
+      const float cs[4] = {c.x, c.y, c.z, c.w}, sn[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float u = x[2 * e], v = x[2 * e + 1];
+        x[2 * e] = u * cs[e] - v * sn[e];
+        x[2 * e + 1] = u * sn[e] + v * cs[e];
+      }
+    }
+    st8(dst + hoff + (long long)row * g.stride_n + col, x);
+  }
+}
+
 // grid (tiles per chunk of WIN_BM rows, G, BH), 128 threads.  Softmax window of Eq. 6 and 8 with a
 // running row maximum, then the joint normalisation of Eq. 5 with the linear read-out `rd`.
 constexpr int WIN_BM = 32, WIN_BN = 64, WIN_THREADS = 128;
