@@ -253,6 +253,37 @@ def bidirectional_timing(wl, dev, phi_q, phi_k, stream, causal_ms):
     return res
 
 
+def qk_transform_timing(wl, dev, phi_q, phi_k, stream, plain_ms, peaks):
+    """The same layer with q and k normalised and rotated ahead of the operator by the library's own pass
+    (per-head RMS norm with weights, rotary tables of one-dimensional positions): the pass is bound by HBM, it
+    reads q, k and writes the transformed q, k once."""
+    from paper_2601_04342_b200 import binding
+    op = binding.for_workload(wl, qk_transform=True)
+    w = torch.ones((wl.n_heads, wl.head_dim), device="cuda", dtype=dev["q"].dtype)
+    half = wl.head_dim // 2
+    ang = torch.arange(wl.N, device="cuda", dtype=torch.float32)[:, None] * \
+        (10000.0 ** (-torch.arange(half, device="cuda", dtype=torch.float32) / half))[None, :]
+    cos, sin = torch.cos(ang).contiguous(), torch.sin(ang).contiguous()
+    op.set_qk_transform(q_weight=w, k_weight=w, cos=cos, sin=sin)
+    out = torch.empty_like(dev["q"])
+    run = lambda: op.forward(dev["q"], dev["k"], dev["v"], phi_q, phi_k, wl.T, wl.H, wl.W, wl.Tc, wl.To, out=out, stream=stream)
+    for _ in range(3):
+        run()
+    op.profile_enable(True)
+    ms = _time_ms(run, stream, 0, 20)
+    prof = op.profile_read()
+    op.profile_enable(False)
+    assert op.status() == 0
+    prep_ms = prof["qk_prep"][0] / max(prof["qk_prep"][1], 1)
+    nbytes = 4 * wl.B * wl.n_heads * wl.N * wl.head_dim * dev["q"].element_size()      # q, k read; q', k' written
+    res = {"ms_per_step": ms, "plain_ms_per_step": plain_ms, "prepass_ms": prep_ms, "prepass_algorithmic_bytes": nbytes,
+           "prepass_gbs": nbytes / (prep_ms * 1e-3) / 1e9 if prep_ms > 0 else None,
+           "prepass_frac_of_hbm_peak": nbytes / (prep_ms * 1e-3) / 1e9 / peaks["hbm_gbs"] if prep_ms > 0 else None,
+           "workspace_bytes": op.workspace_bytes}
+    op.close()
+    return res
+
+
 def lib_state_bytes(op):
     from paper_2601_04342_b200 import binding
     return binding.lib().rehyat_stream_state_bytes(op._h)
@@ -554,6 +585,8 @@ def main():
     if world == 1:
         extras["workspace_bytes_by_latent_frames"] = workspace_by_frames(wl, local_rank)
         extras["chunk_by_chunk"] = stream_timing(wl, dev, phi_q, phi_k, stream, flops)
+    if world == 1 and wl.dtype == "bf16":
+        extras["qk_transform_same_shape"] = qk_transform_timing(wl, dev, phi_q, phi_k, stream, ms_step, peaks)
     if world == 1 and args.all_configs:
         extras["bidirectional_same_shape"] = bidirectional_timing(wl, dev, phi_q, phi_k, stream, ms_step)
     if world == 1:
