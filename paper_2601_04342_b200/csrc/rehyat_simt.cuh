@@ -320,6 +320,12 @@ qk_prepare(const T* __restrict__ q, const T* __restrict__ k, T* __restrict__ qo,
   const long long hoff = head_offset(g, bh);
   const int lane_in_row = threadIdx.x % LPR, col = lane_in_row * 8;
   const int rows_per_block = 256 / LPR;
+  // a thread keeps its eight columns for all its rows: their norm weights are loaded once
+  float wv[8] = {1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f, 1.f};
+  if (a.rms_norm && wgt != nullptr) {
+    const float4 w0 = ld4(wgt + (size_t)head * D + col), w1 = ld4(wgt + (size_t)head * D + col + 4);
+    wv[0] = w0.x; wv[1] = w0.y; wv[2] = w0.z; wv[3] = w0.w; wv[4] = w1.x; wv[5] = w1.y; wv[6] = w1.z; wv[7] = w1.w;
+  }
   for (int row = blockIdx.x * rows_per_block + threadIdx.x / LPR; row < g.N; row += gridDim.x * rows_per_block) {
     const T* p = src + hoff + (long long)row * g.stride_n + col;
     const float4 x0 = ld4(p), x1 = ld4(p + 4);
@@ -332,11 +338,7 @@ qk_prepare(const T* __restrict__ q, const T* __restrict__ k, T* __restrict__ qo,
       for (int o = 1; o < LPR; o <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
       const float inv = rsqrtf(ss * (1.f / D) + a.eps);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) x[e] *= inv;
-      if (wgt != nullptr) {
-        const float4 w0 = ld4(wgt + (size_t)head * D + col), w1 = ld4(wgt + (size_t)head * D + col + 4);
-        x[0] *= w0.x; x[1] *= w0.y; x[2] *= w0.z; x[3] *= w0.w; x[4] *= w1.x; x[5] *= w1.y; x[6] *= w1.z; x[7] *= w1.w;
-      }
+      for (int e = 0; e < 8; ++e) x[e] *= inv * wv[e];
     }
     if (a.cos != nullptr) {
       const float4 c = *reinterpret_cast<const float4*>(a.cos + (size_t)row * (D / 2) + col / 2);
