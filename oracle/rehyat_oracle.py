@@ -43,7 +43,9 @@ Readings taken where the paper is silent or garbled (each is restated in the des
     two (the widths and activation of the two-layer map, nothing new to choose).
 
 Parity unpinned (the paper prints no numbers that would decide them): rowmax vs zero,
-the activation functions, which chunk is the short one.
+the activation functions, which chunk is the short one, which deeper phi maps the authors
+tried, and the convention of the block's q/k normalisation and rotation (rms_norm,
+rope_rotate: the block is taken over from the pretrained model and not restated).
 """
 from __future__ import annotations
 
