@@ -222,11 +222,14 @@ class Rehyat:
                "rehyat_stream_begin")
 
     def stream_step(self, q, k, v, phi_q, phi_k, frames_in_chunk, out=None, stream=None):
-        """q, k, v: contiguous CUDA tensors [B, n_heads, frames_in_chunk*H*W, d] of the next chunk."""
+        """q, k, v: CUDA tensors [B, n_heads, frames_in_chunk*H*W, d] of the next chunk, contiguous or views that
+        share their strides (head_dim contiguous), e.g. slices of the whole sequence; `out` likewise."""
         if out is None:
             out = torch.empty_like(q)
-        B, nh, N, d = q.shape
-        lay = Layout(nh * N * d, N * d, d)
+        sb, sh, sn, sd = q.stride()
+        if sd != 1 or any(t.stride() != q.stride() or t.shape != q.shape for t in (k, v, out)):
+            raise ValueError("q, k, v, out must share shape and strides, with head_dim contiguous")
+        lay = Layout(sb, sh, sn)
         st = stream if stream is not None else torch.cuda.current_stream(q.device)
         phi = self.phi_struct(phi_q, phi_k)
         _check(lib().rehyat_stream_step(self._h, _ptr(q), _ptr(k), _ptr(v), _ptr(out), C.byref(lay), C.byref(phi),

@@ -146,3 +146,34 @@ def test_zero_strides_of_one_element_axes_and_bad_strides():
     assert call(binding.Layout(2 * N * dd, 0, dd)) == binding.ERR_INVALID_ARG
     assert call(binding.Layout(2 * N * dd, N * dd, dd - 8)) == binding.ERR_INVALID_ARG
     op.close()
+
+
+def test_a_layer_split_over_three_ranks_equals_the_layer_in_one_call():
+    """binding.ShardedRehyat with the ranks run one after the other on this GPU (independent launches, nothing
+    waits on another rank): every rank writes only its own (batch, head) blocks, and together they give, bit for
+    bit, what one call on all heads gives."""
+    from paper_2601_04342_b200 import binding, geometry
+    wl = synth.Workload("shard", 2, 4, 128, 5, 10, 20, 2, 1, "bf16", True, seed=synth.BASE_SEED + 75)
+    x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
+    d = _dev(x)
+    op = binding.for_workload(wl, window_tiles=2)
+    whole = op.forward(d["q"], d["k"], d["v"], d["phi_q"], d["phi_k"], wl.T, wl.H, wl.W, wl.Tc, wl.To)
+    assert op.status() == binding.OK
+    op.close()
+    assert np.abs(whole.double().cpu().numpy() - _oracle(wl, x)).max() <= 2e-2
+    out = torch.full_like(d["q"], float("nan"))
+    world = 3                                                 # 8 problems over 3 ranks: 3, 3, 2, with cuts inside batch items
+    for rank in range(world):
+        sh = binding.ShardedRehyat(world, rank, batch=wl.B, n_heads=wl.n_heads, head_dim=wl.head_dim, dtype=wl.dtype,
+                                   phi_hidden=wl.D_h, phi_dim=wl.D_out, poly_degree=wl.P, max_tokens_per_frame=wl.HW,
+                                   max_chunk_frames=wl.Tc, window_tiles=2)
+        before = out.clone()
+        sh.forward(d["q"], d["k"], d["v"], out, d["phi_q"], d["phi_k"], wl.T, wl.H, wl.W, wl.Tc, wl.To)
+        assert sh.status() == binding.OK and sh.last_launches > 0
+        mine = torch.zeros((wl.B, wl.n_heads), dtype=torch.bool)
+        for (b0, nb, h0, nh) in geometry.shard_rects(wl.B, wl.n_heads, world, rank):
+            mine[b0:b0 + nb, h0:h0 + nh] = True
+        changed = ~(torch.isnan(out) == torch.isnan(before)).flatten(2).all(dim=2).cpu()
+        assert torch.equal(changed, mine)                     # exactly this rank's blocks were written
+        sh.close()
+    assert torch.equal(out, whole)

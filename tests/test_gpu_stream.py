@@ -134,3 +134,33 @@ def test_stream_argument_checks():
     with pytest.raises(binding.RehyatError):            # a damaged blob
         op.stream_import(b"\x00" * len(blob))
     op.close()
+
+
+@pytest.mark.parametrize("layout", ["bhnd", "bnhd"])
+def test_chunks_as_views_of_the_whole_sequence(layout):
+    """q is read and out is written in place, with the caller's strides: the chunks are passed as views of the
+    whole [B, heads, N, d] (or token-major [B, N, heads, d]) tensors, nothing is made contiguous."""
+    from paper_2601_04342_b200 import binding
+    wl = synth.Workload("views", 2, 3, 128, 7, 9, 17, 2, 1, "bf16", True, seed=synth.BASE_SEED + 97)
+    x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
+    f = synth.to_f64(x)
+    ref = orc.hybrid_rnn(f["q"], f["k"], f["v"], f["phi_q"], f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To, P=wl.P)
+    d = _dev(x)
+    if layout == "bnhd":                                     # token-major storage, seen as [B, heads, N, d]
+        full = {n: d[n].transpose(1, 2).contiguous().transpose(1, 2) for n in ("q", "k", "v")}
+    else:
+        full = {n: d[n] for n in ("q", "k", "v")}
+    out = torch.full_like(full["q"], float("nan"))
+    assert out.stride() == full["q"].stride()
+    op = binding.for_workload(wl)
+    op.stream_begin(wl.B, wl.H, wl.W, wl.Tc, wl.To)
+    for t in range(-(-wl.T // wl.Tc)):
+        f0, f1 = t * wl.Tc, min((t + 1) * wl.Tc, wl.T)
+        sl = slice(f0 * wl.HW, f1 * wl.HW)
+        q, k, v = (full[n][:, :, sl] for n in ("q", "k", "v"))
+        o = out[:, :, sl]
+        assert not q.is_contiguous()
+        op.stream_step(q, k, v, d["phi_q"], d["phi_k"], f1 - f0, out=o)
+        assert op.status() == 0
+    op.close()
+    gate(out.double().cpu().numpy(), ref, "bf16")
