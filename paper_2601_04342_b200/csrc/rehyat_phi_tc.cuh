@@ -212,26 +212,27 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       };
       // one 128x128 half of an MLP GEMM: A tile [128 x 64*nks] K-major at a_base, B tiles from the ring
       auto mlp_half = [&](uint32_t a_base, int nks) -> bool {
-        for (int ks = 0; ks < nks; ++ks) {
+        uint64_t da = smem_desc_sw128(a_base, 16, 1024);             // advanced by one 64-column sub-tile per ring tile
+        for (int ks = 0; ks < nks; ++ks, da = smem_desc_advance(da, PH_SUB)) {
           if (!wait(&bars->ring_full[ring_i % RING], (ring_i / RING) & 1)) return false;
-          const uint32_t bt = ring_addr(ring_i % RING);
+          const uint64_t db = smem_desc_sw128(ring_addr(ring_i % RING), 16, 1024);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
-            umma_ss(tmem + T_SCR, smem_desc_sw128(a_base + ks * PH_SUB + kk * 32, 16, 1024),
-                    smem_desc_sw128(bt + kk * 32, 16, 1024), id_kk, (ks | kk) != 0);
+            umma_ss(tmem + T_SCR, smem_desc_advance(da, kk * 32), smem_desc_advance(db, kk * 32), id_kk, (ks | kk) != 0);
           ring_release();
         }
         umma_commit(smem_u32(&bars->acc_ready));
         return true;
       };
       // contraction that consumes phi half `c` (its tile is at phi_base)
+      const uint64_t d_v = smem_desc_sw128(sV, PH_SUB, 1024), d_ones = smem_desc_sw128(sOnes, 16, 1024);
       auto consume_half = [&](int c, uint32_t phi_base, bool first_tile) {
+        const uint64_t d_phi = smem_desc_sw128(phi_base, PH_SUB, 1024);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {                            // 16 tokens per step
-          const uint64_t ad = smem_desc_sw128(phi_base + kk * 2048, PH_SUB, 1024);
-          umma_ss(tmem + T_ACC + c * 128, ad, smem_desc_sw128(sV + kk * 2048, PH_SUB, 1024), id_st,
-                  (!first_tile || kk > 0) ? 1u : 0u);
-          umma_ss(tmem + T_Z + c * 16, ad, smem_desc_sw128(sOnes + (kk >> 2) * 2048 + (kk & 3) * 32, 16, 1024), id_z,
+          const uint64_t ad = smem_desc_advance(d_phi, kk * 2048);
+          umma_ss(tmem + T_ACC + c * 128, ad, smem_desc_advance(d_v, kk * 2048), id_st, (!first_tile || kk > 0) ? 1u : 0u);
+          umma_ss(tmem + T_Z + c * 16, ad, smem_desc_advance(d_ones, (kk >> 2) * 2048 + (kk & 3) * 32), id_z,
                   (!first_tile || kk > 0) ? 1u : 0u);
         }
       };

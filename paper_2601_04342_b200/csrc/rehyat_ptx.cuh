@@ -266,6 +266,13 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
          ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// The descriptor of the same layout `byte_off` bytes further on (a multiple of 16; the tile stays below the 256 KB
+// the address field spans): only the start-address field moves, so one 64-bit add replaces building it again.
+// The thread that issues the MMAs is a single thread; what it computes between two MMAs is issue time.
+__device__ __forceinline__ uint64_t smem_desc_advance(uint64_t desc, uint32_t byte_off) {
+  return desc + (uint64_t)(byte_off >> 4);
+}
+
 // Instruction descriptor of tcgen05.mma kind::f16, bf16 x bf16 -> fp32:
 //   [4,6) D format (1 = f32), [7,10) A format (1 = bf16), [10,13) B format (1 = bf16),
 //   [15] A major (0 = K), [16] B major (0 = K, 1 = MN), [17,23) N >> 3, [24,29) M >> 4.

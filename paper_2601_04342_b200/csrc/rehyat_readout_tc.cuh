@@ -155,6 +155,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       constexpr uint32_t id_kk = idesc_bf16(128, 128, 0, 0);       // A K-major (smem or TMEM), B K-major: the MLP GEMMs
       constexpr uint32_t id_rd = idesc_bf16(128, 128, 0, 1);       // A = phi (K-major), B = state (MN-major)
       uint32_t ring_i = 0, n_epi[2] = {0, 0};
+      const uint64_t d_x = smem_desc_sw128(sX, 16, 1024);
       // A wait that is given up ends the role at once: the helpers return false and run() returns, so nothing
       // further is issued.  No flag is carried along; the hot path pays one predicated branch per wait.
       auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
@@ -179,10 +180,10 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         for (int ks = 0; ks < 2; ++ks) {
           const uint32_t bt = ring_wait();
           if (!bt) return false;
+          const uint64_t da = smem_desc_advance(d_x, ks * PH_SUB), db = smem_desc_sw128(bt, 16, 1024);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
-            umma_ss(tmem + T_SCR + b * 128, smem_desc_sw128(sX + ks * PH_SUB + kk * 32, 16, 1024),
-                    smem_desc_sw128(bt + kk * 32, 16, 1024), id_kk, (ks | kk) != 0);
+            umma_ss(tmem + T_SCR + b * 128, smem_desc_advance(da, kk * 32), smem_desc_advance(db, kk * 32), id_kk, (ks | kk) != 0);
           ring_release();
         }
         umma_commit(smem_u32(&bars->acc_ready[b]));
@@ -192,10 +193,10 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         for (int ks = 0; ks < 4; ++ks) {
           const uint32_t bt = ring_wait();
           if (!bt) return false;
+          const uint64_t db = smem_desc_sw128(bt, 16, 1024);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
-            umma_ts(tmem + T_SCR + b * 128, tmem + T_H + (ks * 4 + kk) * 8, smem_desc_sw128(bt + kk * 32, 16, 1024), id_kk,
-                    (ks | kk) != 0);
+            umma_ts(tmem + T_SCR + b * 128, tmem + T_H + (ks * 4 + kk) * 8, smem_desc_advance(db, kk * 32), id_kk, (ks | kk) != 0);
           ring_release();
         }
         umma_commit(smem_u32(&bars->acc_ready[b]));
@@ -205,10 +206,10 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         for (int f = 0; f < 2; ++f) {
           const uint32_t bt = ring_wait();
           if (!bt) return false;
+          const uint64_t da = smem_desc_sw128(phi_base + f * PH_SUB, 16, 1024), db = smem_desc_sw128(bt, 8192, 1024);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
-            umma_ss(tmem + T_R, smem_desc_sw128(phi_base + f * PH_SUB + kk * 32, 16, 1024),
-                    smem_desc_sw128(bt + kk * 2048, 8192, 1024), id_rd, (c | f | kk) != 0);
+            umma_ss(tmem + T_R, smem_desc_advance(da, kk * 32), smem_desc_advance(db, kk * 2048), id_rd, (c | f | kk) != 0);
           ring_release();
         }
         return true;
