@@ -73,6 +73,130 @@ __device__ __forceinline__ bool win_item(const Geo& g, int item, int pairs, WinI
   return true;
 }
 
+// The MMAs of both window kernels, issued by one thread.  TMEM: S slots at columns 0 and 128, O slots at 256 and
+// 384.  Descriptors differ only in the start-address field (low word): built once, offsets added per MMA.
+struct WinMma {
+  static constexpr uint32_t idesc_qk = ptx::idesc_bf16(TC_BM, TC_BN, 0, 0);   // A = Q (K-major), B = K (K-major)
+  static constexpr uint32_t idesc_pv = ptx::idesc_bf16(TC_BM, TC_D, 0, 1);    // A = P (TMEM),    B = V (MN-major)
+  uint32_t tmem, q_lo, q_hi, k_lo, k_hi, v_lo, v_hi;
+  __device__ __forceinline__ WinMma(uint32_t tmem_base, uint32_t sQ, uint32_t sK, uint32_t sV) : tmem(tmem_base) {
+    ptx::upk2u(ptx::smem_desc_sw128(sQ, 16, 1024), q_lo, q_hi);
+    ptx::upk2u(ptx::smem_desc_sw128(sK, 16, 1024), k_lo, k_hi);
+    ptx::upk2u(ptx::smem_desc_sw128(sV, TC_SUB_BYTES, 1024), v_lo, v_hi);
+  }
+  // S[slot] = Q[q_tile] K[stage]^T
+  __device__ __forceinline__ void qk(int slot, int q_tile, int stage) const {
+    const uint32_t a0 = q_lo + q_tile * (TC_TILE_BYTES >> 4), b0 = k_lo + stage * (TC_TILE_BYTES >> 4);
+#pragma unroll
+    for (int kk = 0; kk < TC_D / 16; ++kk) {
+      const uint32_t off = ((kk >> 2) * TC_SUB_BYTES + (kk & 3) * 32) >> 4;
+      ptx::umma_ss(tmem + slot * TC_BN, ptx::pk2u(a0 + off, q_hi), ptx::pk2u(b0 + off, k_hi), idesc_qk, kk > 0);
+    }
+  }
+  // O[slot] (+)= P[slot][:, keys 64*half .. +64) V[stage][those keys, :]
+  __device__ __forceinline__ void pv(int slot, int stage, int half, bool acc) const {
+    const uint32_t b0 = v_lo + stage * (TC_TILE_BYTES >> 4);
+#pragma unroll
+    for (int kk = half * 4; kk < half * 4 + 4; ++kk)
+      ptx::umma_ts(tmem + 256 + slot * TC_D, tmem + slot * TC_BN + kk * 8, ptx::pk2u(b0 + kk * (16 * 128 >> 4), v_hi), idesc_pv,
+                   (acc || kk > half * 4) ? 1u : 0u);
+  }
+};
+
+// Running softmax state of one query row over the key tiles of a TMEM slot: the true maximum so far, the
+// reference the exponentials are taken against (it follows the maximum lazily), four partial row sums.
+struct SoftmaxRow {
+  float m_true = -INFINITY, m_used = -INFINITY;
+  uint64_t l2a = 0ull, l2b = 0ull;
+  __device__ __forceinline__ float sum() const {
+    float a0, a1, b0, b1;
+    ptx::upk2(l2a, a0, a1);
+    ptx::upk2(l2b, b0, b1);
+    return (a0 + a1) + (b0 + b1);
+  }
+};
+
+// One 128-key tile of one query row (this thread's TMEM lane), shared by both window kernels (Eq. 6, 8): S is
+// read from the 128 columns at tS, keys beyond n_valid are masked, the reference maximum is moved (and O at tO and
+// the row sums rescaled) only when the maximum grew by more than 2^8, P = 2^((s - m_used) c) goes back to the
+// first 64 columns of S as bf16 in two halves, each announced on its barrier.  `has_previous`: the slot already
+// holds a P V of this item (O may then need the rescale); `wait_previous_pv()` waits for it and returns false if
+// the wait was given up, which is also what this function then returns.
+// EMU: of every four pairs of exponentials, how many are evaluated on the FMA pipe.
+template <int EMU, typename WaitPv>
+__device__ __forceinline__ bool softmax_key_tile(uint32_t tS, uint32_t tO, int n_valid, float c, bool has_previous,
+                                                 SoftmaxRow& st, uint32_t bar_half0, uint32_t bar_half1, int lane,
+                                                 WaitPv&& wait_previous_pv) {
+  using namespace ptx;
+  uint32_t sr[4][32];
+#pragma unroll
+  for (int cc = 0; cc < 4; ++cc) tmem_ld32(tS + cc * 32, sr[cc]);
+  tmem_wait_ld();
+  if (n_valid < TC_BN) {
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+      for (int e = 0; e < 32; ++e)
+        if (cc * 32 + e >= n_valid) sr[cc][e] = 0xff800000u;   // -inf
+  }
+  // row maximum: four independent chains of three-input max
+  float mx[4] = {st.m_true, st.m_true, st.m_true, st.m_true};
+#pragma unroll
+  for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+    for (int e = 0; e < 32; e += 2)
+      mx[cc] = fmax3(mx[cc], __uint_as_float(sr[cc][e]), __uint_as_float(sr[cc][e + 1]));
+  st.m_true = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+  const bool need = (st.m_true - st.m_used) * c > 8.f;               // true on the first tile (m_used = -inf)
+  if (__any_sync(0xffffffffu, need)) {
+    const float m_new = need ? st.m_true : st.m_used;
+    if (has_previous) {
+      // S of this tile follows the completion of the slot's previous P V, so O may be touched
+      if (!wait_previous_pv()) return false;
+      tc_fence_after();
+      const float f = ex2((st.m_used - m_new) * c);                  // 1 for lanes that keep their reference
+      const uint64_t f2 = pk2(f, f);
+      st.l2a = mul2(st.l2a, f2);
+      st.l2b = mul2(st.l2b, f2);
+#pragma unroll 1
+      for (int cc = 0; cc < TC_D / 8; ++cc) {                        // rare: small pieces keep the register peak low
+        uint32_t o[8];
+        tmem_ld8(tO + cc * 8, o);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
+        tmem_st8(tO + cc * 8, o);
+      }
+    }
+    st.m_used = m_new;
+  }
+  const float mc = -st.m_used * c;
+  const uint64_t c2 = pk2(c, c), mc2 = pk2(mc, mc);
+#pragma unroll
+  for (int cc = 0; cc < 4; ++cc) {
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+      float t0, t1, p0, p1;
+      upk2(fma2(pk2u(sr[cc][e], sr[cc][e + 1]), c2, mc2), t0, t1);
+      if (((e >> 1) & 3) < EMU) {                                    // EMU of every 4 pairs on the FMA pipe
+        ex2_poly2(t0, t1, p0, p1);
+      } else {
+        p0 = ex2(t0);
+        p1 = ex2(t1);
+      }
+      if ((e >> 1) & 1) st.l2b = add2(st.l2b, pk2(p0, p1)); else st.l2a = add2(st.l2a, pk2(p0, p1));
+      sr[cc >> 1][(cc & 1) * 16 + (e >> 1)] = pack_bf16(p0, p1);
+    }
+    if (cc & 1) {
+      tmem_st32(tS + (cc >> 1) * 32, sr[cc >> 1]);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive_warp((cc >> 1) ? bar_half1 : bar_half0, lane);     // P of 64 keys is in place
+    }
+  }
+  return true;
+}
+
 // Persistent: gridDim.x CTAs (one per SM) walk the items blockIdx.x, blockIdx.x + gridDim.x, ...  Barriers,
 // TMEM and the K/V rings live across items; every role keeps running counts of the phases it has used.
 // EMU: of every four pairs of exponentials, how many are evaluated on the FMA pipe.
@@ -173,28 +297,9 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
   } else if (warp == 1) {
     // ------------------------------------------------------------------ UMMA issuer
     if (elect_one()) {
-      constexpr uint32_t idesc_qk = idesc_bf16(TC_BM, TC_BN, 0, 0);   // A = Q (K-major), B = K (K-major)
-      constexpr uint32_t idesc_pv = idesc_bf16(TC_BM, TC_D, 0, 1);    // A = P (TMEM),    B = V (MN-major)
-      // Descriptors differ only in the start-address field (low word): build them once and add offsets.
-      uint32_t q_lo, q_hi, k_lo, k_hi, v_lo, v_hi;
-      upk2u(smem_desc_sw128(sQ, 16, 1024), q_lo, q_hi);
-      upk2u(smem_desc_sw128(sK, 16, 1024), k_lo, k_hi);
-      upk2u(smem_desc_sw128(sV, TC_SUB_BYTES, 1024), v_lo, v_hi);
-      auto issue_qk = [&](int i, int s) {
-        const uint32_t a0 = q_lo + i * (TC_TILE_BYTES >> 4), b0 = k_lo + s * (TC_TILE_BYTES >> 4);
-#pragma unroll
-        for (int kk = 0; kk < TC_D / 16; ++kk) {
-          const uint32_t off = ((kk >> 2) * TC_SUB_BYTES + (kk & 3) * 32) >> 4;
-          umma_ss(tmem + i * TC_BN, pk2u(a0 + off, q_hi), pk2u(b0 + off, k_hi), idesc_qk, kk > 0);
-        }
-      };
-      auto issue_pv = [&](int i, int s, int half, bool acc) {        // keys [64*half, 64*half+64) of the tile
-        const uint32_t b0 = v_lo + s * (TC_TILE_BYTES >> 4);
-#pragma unroll
-        for (int kk = half * 4; kk < half * 4 + 4; ++kk)
-          umma_ts(tmem + 256 + i * TC_D, tmem + i * TC_BN + kk * 8, pk2u(b0 + kk * (16 * 128 >> 4), v_hi), idesc_pv,
-                  (acc || kk > half * 4) ? 1u : 0u);
-      };
+      const WinMma mma(tmem, sQ, sK, sV);
+      auto issue_qk = [&](int i, int s) { mma.qk(i, i, s); };         // query tile i into its own slot
+      auto issue_pv = [&](int i, int s, int half, bool acc) { mma.pv(i, s, half, acc); };
       uint32_t kv_it = 0, n_done = 0;                                // K/V tiles consumed, items done
       uint32_t n_p[TC_QT] = {0, 0}, n_o[TC_QT] = {0, 0};             // P hand-overs and items per query tile
       bool alive = true;                                             // false once a wait has been given up: issue nothing more
@@ -271,84 +376,17 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       WinItem w;
       if (!win_item(g, item, pairs, w) || i >= w.ntiles) continue;
       const int n_kv = w.n_kv, lo = w.lo, hi = w.hi;
-      float m_true = -INFINITY, m_used = -INFINITY;
-      uint64_t l2a = 0ull, l2b = 0ull;                               // four partial row sums as two fp32 pairs
+      SoftmaxRow st;
       for (int j = 0; j < n_kv; ++j) {
         if (!wait(&bars->s_ready[i], (n_s + j) & 1)) break;
         tc_fence_after();
-        uint32_t sr[4][32];
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) tmem_ld32(tS + cc * 32, sr[cc]);
-        tmem_wait_ld();
-        const int n_valid = hi - (lo + j * TC_BN);                   // >= 1
-        if (n_valid < TC_BN) {
-#pragma unroll
-          for (int cc = 0; cc < 4; ++cc)
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (cc * 32 + e >= n_valid) sr[cc][e] = 0xff800000u;   // -inf
-        }
-        // row maximum: four independent chains of three-input max
-        float mx[4] = {m_true, m_true, m_true, m_true};
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc)
-#pragma unroll
-          for (int e = 0; e < 32; e += 2)
-            mx[cc] = fmax3(mx[cc], __uint_as_float(sr[cc][e]), __uint_as_float(sr[cc][e + 1]));
-        m_true = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-        const bool need = (m_true - m_used) * c > 8.f;               // true on the first tile (m_used = -inf)
-        if (__any_sync(0xffffffffu, need)) {
-          const float m_new = need ? m_true : m_used;
-          if (j > 0) {
-            // s_ready(j) follows the completion of P V of tile j-1, so O may be touched
-            if (!wait(&bars->pv_done[i], (n_s + j - 1) & 1)) break;
-            tc_fence_after();
-            const float f = ex2((m_used - m_new) * c);               // 1 for lanes that keep their reference
-            const uint64_t f2 = pk2(f, f);
-            l2a = mul2(l2a, f2);
-            l2b = mul2(l2b, f2);
-#pragma unroll 1
-            for (int cc = 0; cc < TC_D / 8; ++cc) {                   // rare: small pieces keep the register peak low
-              uint32_t o[8];
-              tmem_ld8(tO + cc * 8, o);
-              tmem_wait_ld();
-#pragma unroll
-              for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
-              tmem_st8(tO + cc * 8, o);
-            }
-          }
-          m_used = m_new;
-        }
-        const float mc = -m_used * c;
-        const uint64_t c2 = pk2(c, c), mc2 = pk2(mc, mc);
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            float t0, t1, p0, p1;
-            upk2(fma2(pk2u(sr[cc][e], sr[cc][e + 1]), c2, mc2), t0, t1);
-            if (((e >> 1) & 3) < EMU) {                              // EMU of every 4 pairs on the FMA pipe
-              ex2_poly2(t0, t1, p0, p1);
-            } else {
-              p0 = ex2(t0);
-              p1 = ex2(t1);
-            }
-            if ((e >> 1) & 1) l2b = add2(l2b, pk2(p0, p1)); else l2a = add2(l2a, pk2(p0, p1));
-            sr[cc >> 1][(cc & 1) * 16 + (e >> 1)] = pack_bf16(p0, p1);
-          }
-          if (cc & 1) {
-            tmem_st32(tS + (cc >> 1) * 32, sr[cc >> 1]);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive_warp(smem_u32(&bars->p_half[i][cc >> 1]), lane);       // P of 64 keys is in place
-          }
-        }
+        if (!softmax_key_tile<EMU>(tS, tO, hi - (lo + j * TC_BN), c, j > 0, st, smem_u32(&bars->p_half[i][0]),
+                                   smem_u32(&bars->p_half[i][1]), lane,
+                                   [&]() { return wait(&bars->pv_done[i], (n_s + j - 1) & 1); }))
+          break;
       }
       if (!alive) break;
-      float la0, la1, lb0, lb1;
-      upk2(l2a, la0, la1);
-      upk2(l2b, lb0, lb1);
-      const float l = (la0 + la1) + (lb0 + lb1);
+      const float m_true = st.m_true, m_used = st.m_used, l = st.sum();
 
       // Eq. 5: bring O and l to the final row maximum, add the linear read-out, divide, store.
       const int row = w.row_base + i * TC_BM + (warp & 3) * 32 + lane;

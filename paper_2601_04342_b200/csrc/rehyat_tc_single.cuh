@@ -149,27 +149,9 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   } else if (warp == 1) {
     // ------------------------------------------------------------------ UMMA issuer
     if (elect_one()) {
-      constexpr uint32_t idesc_qk = idesc_bf16(TC_BM, TC_BN, 0, 0);   // A = Q (K-major), B = K (K-major)
-      constexpr uint32_t idesc_pv = idesc_bf16(TC_BM, TC_D, 0, 1);    // A = P (TMEM),    B = V (MN-major)
-      uint32_t q_lo, q_hi, k_lo, k_hi, v_lo, v_hi;
-      upk2u(smem_desc_sw128(sQ, 16, 1024), q_lo, q_hi);
-      upk2u(smem_desc_sw128(sK, 16, 1024), k_lo, k_hi);
-      upk2u(smem_desc_sw128(sV, TC_SUB_BYTES, 1024), v_lo, v_hi);
-      auto issue_qk = [&](int i, int s) {                            // Q times K stage s into slot i
-        const uint32_t b0 = k_lo + s * (TC_TILE_BYTES >> 4);
-#pragma unroll
-        for (int kk = 0; kk < TC_D / 16; ++kk) {
-          const uint32_t off = ((kk >> 2) * TC_SUB_BYTES + (kk & 3) * 32) >> 4;
-          umma_ss(tmem + i * TC_BN, pk2u(q_lo + off, q_hi), pk2u(b0 + off, k_hi), idesc_qk, kk > 0);
-        }
-      };
-      auto issue_pv = [&](int i, int s, int half, bool acc) {        // keys [64*half, 64*half+64) of the tile
-        const uint32_t b0 = v_lo + s * (TC_TILE_BYTES >> 4);
-#pragma unroll
-        for (int kk = half * 4; kk < half * 4 + 4; ++kk)
-          umma_ts(tmem + 256 + i * TC_D, tmem + i * TC_BN + kk * 8, pk2u(b0 + kk * (16 * 128 >> 4), v_hi), idesc_pv,
-                  (acc || kk > half * 4) ? 1u : 0u);
-      };
+      const WinMma mma(tmem, sQ, sK, sV);
+      auto issue_qk = [&](int i, int s) { mma.qk(i, 0, s); };         // the one query tile into slot i
+      auto issue_pv = [&](int i, int s, int half, bool acc) { mma.pv(i, s, half, acc); };
       uint32_t kv_it = 0, n_done = 0;                                // K/V tiles consumed, items done
       uint32_t n_p[2] = {0, 0};                                      // P hand-overs per slot
       bool alive = true;                                             // false once a wait has been given up: issue nothing more
@@ -241,85 +223,18 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       if (!win_item1(g, item, tiles, w)) continue;
       const int n_kv = w.n_kv, lo = w.lo, hi = w.hi;
       const int cnt0 = (n_kv + 1) >> 1, cnt1 = n_kv >> 1, cnt = i == 0 ? cnt0 : cnt1;   // this slot: tiles i, i+2, ...
-      float m_true = -INFINITY, m_used = -INFINITY;
-      uint64_t l2a = 0ull, l2b = 0ull;                               // four partial row sums as two fp32 pairs
+      SoftmaxRow st;
       for (int t = 0; t < cnt; ++t) {
         const int j = i + 2 * t;
         if (!wait(&bars->s_ready[i], (n_s[i] + t) & 1)) break;
         tc_fence_after();
-        uint32_t sr[4][32];
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) tmem_ld32(tS + cc * 32, sr[cc]);
-        tmem_wait_ld();
-        const int n_valid = hi - (lo + j * TC_BN);                   // >= 1
-        if (n_valid < TC_BN) {
-#pragma unroll
-          for (int cc = 0; cc < 4; ++cc)
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (cc * 32 + e >= n_valid) sr[cc][e] = 0xff800000u;   // -inf
-        }
-        // row maximum: four independent chains of three-input max
-        float mx[4] = {m_true, m_true, m_true, m_true};
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc)
-#pragma unroll
-          for (int e = 0; e < 32; e += 2)
-            mx[cc] = fmax3(mx[cc], __uint_as_float(sr[cc][e]), __uint_as_float(sr[cc][e + 1]));
-        m_true = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-        const bool need = (m_true - m_used) * c > 8.f;               // true on the slot's first tile (m_used = -inf)
-        if (__any_sync(0xffffffffu, need)) {
-          const float m_new = need ? m_true : m_used;
-          if (t > 0) {
-            // s_ready follows the completion of P V of this slot's previous tile, so O may be touched
-            if (!wait(&bars->pv_done[i], (n_s[i] + t - 1) & 1)) break;
-            tc_fence_after();
-            const float f = ex2((m_used - m_new) * c);               // 1 for lanes that keep their reference
-            const uint64_t f2 = pk2(f, f);
-            l2a = mul2(l2a, f2);
-            l2b = mul2(l2b, f2);
-#pragma unroll 1
-            for (int cc = 0; cc < TC_D / 8; ++cc) {                   // rare: small pieces keep the register peak low
-              uint32_t o[8];
-              tmem_ld8(tO + cc * 8, o);
-              tmem_wait_ld();
-#pragma unroll
-              for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
-              tmem_st8(tO + cc * 8, o);
-            }
-          }
-          m_used = m_new;
-        }
-        const float mc = -m_used * c;
-        const uint64_t c2 = pk2(c, c), mc2 = pk2(mc, mc);
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            float t0, t1, p0, p1;
-            upk2(fma2(pk2u(sr[cc][e], sr[cc][e + 1]), c2, mc2), t0, t1);
-            if (((e >> 1) & 3) < EMU) {                              // EMU of every 4 pairs on the FMA pipe
-              ex2_poly2(t0, t1, p0, p1);
-            } else {
-              p0 = ex2(t0);
-              p1 = ex2(t1);
-            }
-            if ((e >> 1) & 1) l2b = add2(l2b, pk2(p0, p1)); else l2a = add2(l2a, pk2(p0, p1));
-            sr[cc >> 1][(cc & 1) * 16 + (e >> 1)] = pack_bf16(p0, p1);
-          }
-          if (cc & 1) {
-            tmem_st32(tS + (cc >> 1) * 32, sr[cc >> 1]);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive_warp(smem_u32(&bars->p_half[i][cc >> 1]), lane);       // P of 64 keys is in place
-          }
-        }
+        if (!softmax_key_tile<EMU>(tS, tO, hi - (lo + j * TC_BN), c, t > 0, st, smem_u32(&bars->p_half[i][0]),
+                                   smem_u32(&bars->p_half[i][1]), lane,
+                                   [&]() { return wait(&bars->pv_done[i], (n_s[i] + t - 1) & 1); }))
+          break;
       }
       if (!alive) break;
-      float la0, la1, lb0, lb1;
-      upk2(l2a, la0, la1);
-      upk2(l2b, lb0, lb1);
-      const float l = (la0 + la1) + (lb0 + lb1);
+      const float m_true = st.m_true, m_used = st.m_used, l = st.sum();
 
       // Exchange the slots' maxima and row sums (a slot without key tiles contributes m = -inf, l = 0).  The
       // buffer alternates with the item: a warpgroup can be at most one item ahead of the other, because the
