@@ -569,8 +569,8 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
     QkPrepArgs pa = {ctx->qk.q_norm_weight, ctx->qk.k_norm_weight, ctx->qk.rope_cos, ctx->qk.rope_sin, ctx->qk.norm_eps,
                      ctx->qk.rms_norm};
     const int rows_per_block = 256 / (c.head_dim / 8);
-    // about eight CTAs per SM over the whole grid, every thread walking several rows of its columns
-    const long long want = (8LL * ctx->tc.n_sm + 2 * g.BH - 1) / (2 * g.BH), need = (N + rows_per_block - 1) / rows_per_block;
+    // about thirty-two CTAs per SM over the whole grid, every thread walking several pairs of rows of its columns
+    const long long want = (32LL * ctx->tc.n_sm + 2 * g.BH - 1) / (2 * g.BH), need = (N + 2 * rows_per_block - 1) / (2 * rows_per_block);
     const unsigned blocks = (unsigned)(need < want ? need : (want > 0 ? want : 1));
     const dim3 grid(blocks, g.BH, 2);
     ctx->prof.begin(REHYAT_PROF_QKPREP, st);

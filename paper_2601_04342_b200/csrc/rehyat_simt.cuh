@@ -326,32 +326,52 @@ qk_prepare(const T* __restrict__ q, const T* __restrict__ k, T* __restrict__ qo,
     const float4 w0 = ld4(wgt + (size_t)head * D + col), w1 = ld4(wgt + (size_t)head * D + col + 4);
     wv[0] = w0.x; wv[1] = w0.y; wv[2] = w0.z; wv[3] = w0.w; wv[4] = w1.x; wv[5] = w1.y; wv[6] = w1.z; wv[7] = w1.w;
   }
-  for (int row = blockIdx.x * rows_per_block + threadIdx.x / LPR; row < g.N; row += gridDim.x * rows_per_block) {
-    const T* p = src + hoff + (long long)row * g.stride_n + col;
-    const float4 x0 = ld4(p), x1 = ld4(p + 4);
-    float x[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-    if (a.rms_norm) {
-      float ss = 0.f;
+  // the lanes that share a row reduce among themselves: row groups of one warp may leave the loop at different times
+  const unsigned row_lanes = (LPR >= 32 ? 0xffffffffu : ((1u << LPR) - 1u) << ((threadIdx.x & 31) / LPR * LPR));
+  // two rows per step, both loaded before either is worked on: twice the bytes in flight per thread
+  const int stride = gridDim.x * rows_per_block;
+  for (int row0 = blockIdx.x * rows_per_block + threadIdx.x / LPR; row0 < g.N; row0 += 2 * stride) {
+    float x[2][8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) ss = fmaf(x[e], x[e], ss);
+    for (int u = 0; u < 2; ++u) {
+      const int row = row0 + u * stride;
+      if (row < g.N) {
+        const T* p = src + hoff + (long long)row * g.stride_n + col;
+        const float4 x0 = ld4(p), x1 = ld4(p + 4);
+        x[u][0] = x0.x; x[u][1] = x0.y; x[u][2] = x0.z; x[u][3] = x0.w;
+        x[u][4] = x1.x; x[u][5] = x1.y; x[u][6] = x1.z; x[u][7] = x1.w;
+      } else {
 #pragma unroll
-      for (int o = 1; o < LPR; o <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      const float inv = rsqrtf(ss * (1.f / D) + a.eps);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) x[e] *= inv * wv[e];
-    }
-    if (a.cos != nullptr) {
-      const float4 c = *reinterpret_cast<const float4*>(a.cos + (size_t)row * (D / 2) + col / 2);
-      const float4 s = *reinterpret_cast<const float4*>(a.sin + (size_t)row * (D / 2) + col / 2);
-      const float cs[4] = {c.x, c.y, c.z, c.w}, sn[4] = {s.x, s.y, s.z, s.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float u = x[2 * e], v = x[2 * e + 1];
-        x[2 * e] = u * cs[e] - v * sn[e];
-        x[2 * e + 1] = u * sn[e] + v * cs[e];
+        for (int e = 0; e < 8; ++e) x[u][e] = 0.f;
       }
     }
-    st8(dst + hoff + (long long)row * g.stride_n + col, x);
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int row = row0 + u * stride;                 // rows beyond the end take part in the shuffles, nothing else
+      if (a.rms_norm) {
+        float ss = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ss = fmaf(x[u][e], x[u][e], ss);
+#pragma unroll
+        for (int o = 1; o < LPR; o <<= 1) ss += __shfl_xor_sync(row_lanes, ss, o);
+        const float inv = rsqrtf(ss * (1.f / D) + a.eps);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[u][e] *= inv * wv[e];
+      }
+      if (row >= g.N) continue;
+      if (a.cos != nullptr) {
+        const float4 c = *reinterpret_cast<const float4*>(a.cos + (size_t)row * (D / 2) + col / 2);
+        const float4 s = *reinterpret_cast<const float4*>(a.sin + (size_t)row * (D / 2) + col / 2);
+        const float cs[4] = {c.x, c.y, c.z, c.w}, sn[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float p0 = x[u][2 * e], p1 = x[u][2 * e + 1];
+          x[u][2 * e] = p0 * cs[e] - p1 * sn[e];
+          x[u][2 * e + 1] = p0 * sn[e] + p1 * cs[e];
+        }
+      }
+      st8(dst + hoff + (long long)row * g.stride_n + col, x[u]);
+    }
   }
 }
 

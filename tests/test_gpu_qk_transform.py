@@ -84,6 +84,8 @@ def _check(y, ref, dtype):
 CASES = [
     synth.Workload("qk_bf16", 2, 2, 128, 5, 10, 20, 2, 1, "bf16", False, seed=synth.BASE_SEED + 95),
     synth.Workload("qk_fp32", 1, 2, 64, 4, 8, 8, 1, 1, "fp32", False, seed=synth.BASE_SEED + 96),
+    # an odd number of tokens (1071): the last row of the pass has no neighbour in its warp
+    synth.Workload("qk_bf16_odd", 1, 2, 128, 7, 9, 17, 3, 1, "bf16", False, seed=synth.BASE_SEED + 98),
 ]
 
 
