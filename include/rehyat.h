@@ -246,7 +246,11 @@ size_t rehyat_static_scratch_bytes(void);
  * within max_batch*n_heads*max_frames*max_tokens_per_frame*head_dim elements of the first), t = NULL switches
  * it off.  Each call then runs one more kernel, bound by HBM, that writes the transformed q and k into the
  * context's buffers; both branches (softmax window and phi) see the transformed tensors; v is untouched.
- * rehyat_forward_host and rehyat_stream_step return REHYAT_ERR_UNSUPPORTED while a transform is set. */
+ * rehyat_stream_step applies it chunk by chunk: k is normalised and rotated on its way into the window buffer
+ * (in place of the copy it needs anyway), q into a buffer of one chunk; the tables are read at the positions
+ * that follow the tokens of the chunks processed so far, so they must cover the whole sequence, and the kept
+ * frames inside an exported state are the transformed ones (resume with the same transform set).
+ * rehyat_forward_host returns REHYAT_ERR_UNSUPPORTED while a transform is set. */
 typedef struct rehyat_qk_transform {
   const void* q_norm_weight;    /* [n_heads, head_dim], operator dtype, or NULL */
   const void* k_norm_weight;

@@ -86,8 +86,11 @@ struct rehyat_ctx {
     long long chunks_done = 0;
     int cap_tokens = 0;           // tokens per (batch, head) each buffer holds
     int start = 0;                // token index of the window's first token
+    long long tokens_done = 0;    // tokens per (batch, head) of the chunks processed so far (position of the next chunk)
     void* kbuf = nullptr;
     void* vbuf = nullptr;
+    void* qbuf = nullptr;         // the chunk's q after the q/k transform (contexts made with qk_transform only)
+    int chunk_cap = 0;            // tokens per (batch, head) qbuf holds
     size_t bytes = 0;
   } stream;
 };
@@ -310,6 +313,31 @@ int check_sizes(const rehyat_ctx* ctx, int batch, int frames, int H, int W, int 
   return REHYAT_OK;
 }
 
+// Enqueues the q/k transform set with rehyat_set_qk_transform: `rows` token rows per (batch, head) of q and k (source
+// strides in `pa.s*`) into qo and ko (strides in `pa.q*`, `pa.k*`), rotation tables read from position pa.pos0 on.
+void launch_qk_prepare(rehyat_ctx* ctx, const void* q, const void* k, void* qo, void* ko, QkPrepArgs pa, int BH, cudaStream_t st) {
+  const rehyat_config& c = ctx->cfg;
+  pa.wq = ctx->qk.q_norm_weight; pa.wk = ctx->qk.k_norm_weight;
+  pa.cos = ctx->qk.rope_cos; pa.sin = ctx->qk.rope_sin;
+  pa.eps = ctx->qk.norm_eps; pa.rms_norm = ctx->qk.rms_norm;
+  const int rows_per_block = 256 / (c.head_dim / 8);
+  // about thirty-two CTAs per SM over the whole grid, every thread walking several pairs of rows of its columns
+  const long long want = (32LL * ctx->tc.n_sm + 2 * BH - 1) / (2 * BH), need = (pa.rows + 2 * rows_per_block - 1) / (2 * rows_per_block);
+  const unsigned blocks = (unsigned)(need < want ? need : (want > 0 ? want : 1));
+  const dim3 grid(blocks, BH, 2);
+  ctx->prof.begin(REHYAT_PROF_QKPREP, st);
+  if (c.dtype == REHYAT_DTYPE_FP32) {
+    if (c.head_dim == 64) qk_prepare<float, 64><<<grid, 256, 0, st>>>((const float*)q, (const float*)k, (float*)qo, (float*)ko, pa);
+    else qk_prepare<float, 128><<<grid, 256, 0, st>>>((const float*)q, (const float*)k, (float*)qo, (float*)ko, pa);
+  } else {
+    using B = __nv_bfloat16;
+    if (c.head_dim == 64) qk_prepare<B, 64><<<grid, 256, 0, st>>>((const B*)q, (const B*)k, (B*)qo, (B*)ko, pa);
+    else qk_prepare<B, 128><<<grid, 256, 0, st>>>((const B*)q, (const B*)k, (B*)qo, (B*)ko, pa);
+  }
+  ctx->prof.end(REHYAT_PROF_QKPREP, st);
+  ctx->last_launches += 1;
+}
+
 // Copies `rows` token rows of `row_bytes` bytes for each of BH (batch, head) problems between two strided
 // layouts (byte strides; rows are contiguous and 16-byte aligned).  grid (row tiles, BH), 256 threads.
 __global__ void copy_rows(uint8_t* __restrict__ dst0, uint8_t* __restrict__ dst1, long long dst_b, long long dst_h, long long dst_n,
@@ -432,7 +460,7 @@ int rehyat_destroy(rehyat_ctx* ctx) {
   if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
   if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
   for (cudaEvent_t e : ctx->host_events) cudaEventDestroy(e);
-  cudaFree(ctx->stream.kbuf); cudaFree(ctx->stream.vbuf);
+  cudaFree(ctx->stream.kbuf); cudaFree(ctx->stream.vbuf); cudaFree(ctx->stream.qbuf);
   delete ctx;
   return REHYAT_OK;
 }
@@ -549,6 +577,7 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   if (g.stride_h == 0) g.stride_h = g.stride_n * N;
   if (g.stride_b == 0) g.stride_b = g.stride_h * g.n_heads;
   g.qstride_b = g.stride_b; g.qstride_h = g.stride_h; g.qstride_n = g.stride_n;   // q and out: laid out like k and v
+  g.ostride_b = g.stride_b; g.ostride_h = g.stride_h; g.ostride_n = g.stride_n;
   g.q_off = 0; g.Nq = g.N;
   const int n_chunks = (frames + chunk_eff - 1) / chunk_eff;
   g.q_shift = 0;
@@ -566,24 +595,10 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
     // q and k are normalised and rotated into the context's buffers, in the layout they came in
     const long long last = (batch - 1) * g.stride_b + (g.n_heads - 1) * g.stride_h + (N - 1) * g.stride_n + c.head_dim;
     if (ctx->head_count > 0 || (size_t)last > ctx->prep_elems) return REHYAT_ERR_INVALID_ARG;
-    QkPrepArgs pa = {ctx->qk.q_norm_weight, ctx->qk.k_norm_weight, ctx->qk.rope_cos, ctx->qk.rope_sin, ctx->qk.norm_eps,
-                     ctx->qk.rms_norm};
-    const int rows_per_block = 256 / (c.head_dim / 8);
-    // about thirty-two CTAs per SM over the whole grid, every thread walking several pairs of rows of its columns
-    const long long want = (32LL * ctx->tc.n_sm + 2 * g.BH - 1) / (2 * g.BH), need = (N + 2 * rows_per_block - 1) / (2 * rows_per_block);
-    const unsigned blocks = (unsigned)(need < want ? need : (want > 0 ? want : 1));
-    const dim3 grid(blocks, g.BH, 2);
-    ctx->prof.begin(REHYAT_PROF_QKPREP, st);
-    if (c.dtype == REHYAT_DTYPE_FP32) {
-      if (c.head_dim == 64) qk_prepare<float, 64><<<grid, 256, 0, st>>>((const float*)q, (const float*)k, (float*)ctx->qprep, (float*)ctx->kprep, g, pa);
-      else qk_prepare<float, 128><<<grid, 256, 0, st>>>((const float*)q, (const float*)k, (float*)ctx->qprep, (float*)ctx->kprep, g, pa);
-    } else {
-      using B = __nv_bfloat16;
-      if (c.head_dim == 64) qk_prepare<B, 64><<<grid, 256, 0, st>>>((const B*)q, (const B*)k, (B*)ctx->qprep, (B*)ctx->kprep, g, pa);
-      else qk_prepare<B, 128><<<grid, 256, 0, st>>>((const B*)q, (const B*)k, (B*)ctx->qprep, (B*)ctx->kprep, g, pa);
-    }
-    ctx->prof.end(REHYAT_PROF_QKPREP, st);
-    ctx->last_launches += 1;
+    QkPrepArgs pa = {};
+    pa.rows = (int)N; pa.n_heads = g.n_heads; pa.pos0 = 0;
+    pa.sb = pa.qb = pa.kb = g.stride_b; pa.sh = pa.qh = pa.kh = g.stride_h; pa.sn = pa.qn = pa.kn = g.stride_n;
+    launch_qk_prepare(ctx, q, k, ctx->qprep, ctx->kprep, pa, g.BH, st);
     q = ctx->qprep;
     k = ctx->kprep;
   }
@@ -727,6 +742,7 @@ struct StreamHeader {          // first bytes of an exported state
   uint32_t magic, version;
   int32_t dtype, n_heads, head_dim, phi_dim, batch, H, W, chunk, overlap, halo, has_state, reserved;
   int64_t chunks_done;
+  int64_t tokens_done;         // position of the next chunk's first token (rotation tables of a q/k transform)
 };
 constexpr uint32_t kStreamMagic = 0x52485953u;   // "RHYS"
 
@@ -744,7 +760,7 @@ void launch_copy_rows2(void* dst0, void* dst1, long long dst_b, long long dst_h,
   if (rows <= 0) return;
   const long long total = (long long)rows * (row_bytes / 16);
   const unsigned blocks = (unsigned)((total + 255) / 256 < 256 ? (total + 255) / 256 : 256);
-  copy_rows<<<dim3(blocks, BH, 2), 256, 0, st>>>((uint8_t*)dst0, (uint8_t*)dst1, dst_b, dst_h, dst_n, (const uint8_t*)src0,
+  copy_rows<<<dim3(blocks, BH, dst1 ? 2 : 1), 256, 0, st>>>((uint8_t*)dst0, (uint8_t*)dst1, dst_b, dst_h, dst_n, (const uint8_t*)src0,
                                                  (const uint8_t*)src1, src_b, src_h, src_n, rows, row_bytes, n_heads);
 }
 
@@ -768,19 +784,21 @@ int rehyat_stream_begin(rehyat_ctx* ctx, int32_t batch, int32_t H, int32_t W, in
   cudaStream_t st = (cudaStream_t)cuda_stream;
   rehyat_ctx::Stream& s = ctx->stream;
   const size_t one = (size_t)batch * c.n_heads * cap * c.head_dim * elem_size(c.dtype);
-  if (one * 2 > s.bytes) {                          // grow the two buffers (the only allocation of this API)
+  const size_t qone = c.qk_transform ? (size_t)batch * c.n_heads * chunk * HW * c.head_dim * elem_size(c.dtype) : 0;
+  if (one * 2 + qone > s.bytes) {                   // grow the buffers (the only allocation of this API)
     if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
-    void** all[2] = {&s.kbuf, &s.vbuf};
+    void** all[3] = {&s.kbuf, &s.vbuf, &s.qbuf};
     for (void** p : all) { cudaFree(*p); *p = nullptr; }
     s.bytes = 0;
-    for (void** p : all)
-      if (cudaMalloc(p, one) != cudaSuccess) { cudaGetLastError(); return REHYAT_ERR_ALLOC; }
-    s.bytes = one * 2;
+    if (cudaMalloc(&s.kbuf, one) != cudaSuccess || cudaMalloc(&s.vbuf, one) != cudaSuccess ||
+        (qone && cudaMalloc(&s.qbuf, qone) != cudaSuccess)) { cudaGetLastError(); return REHYAT_ERR_ALLOC; }
+    s.bytes = one * 2 + qone;
   }
+  s.chunk_cap = (int)(chunk * HW);
   s.active = true;
   s.batch = batch; s.H = H; s.W = W; s.chunk = chunk; s.overlap = overlap;
   s.cap_tokens = (int)cap;
-  s.halo = 0; s.has_state = 0; s.chunks_done = 0; s.start = 0;
+  s.halo = 0; s.has_state = 0; s.chunks_done = 0; s.start = 0; s.tokens_done = 0;
   return REHYAT_OK;
 }
 
@@ -790,7 +808,6 @@ int rehyat_stream_step(rehyat_ctx* ctx, const void* q_chunk, const void* k_chunk
   if (!ctx || !q_chunk || !k_chunk || !v_chunk || !out_chunk || !lay || !phi) return REHYAT_ERR_INVALID_ARG;
   rehyat_ctx::Stream& s = ctx->stream;
   if (!s.active || frames_in_chunk < 1 || frames_in_chunk > s.chunk) return REHYAT_ERR_INVALID_ARG;
-  if (ctx->qk_on) return REHYAT_ERR_UNSUPPORTED;
   const rehyat_config& c = ctx->cfg;
   if (out_chunk == q_chunk || out_chunk == k_chunk || out_chunk == v_chunk) return REHYAT_ERR_INVALID_ARG;
   const void* ptrs[] = {q_chunk, k_chunk, v_chunk, out_chunk};
@@ -821,23 +838,40 @@ int rehyat_stream_step(rehyat_ctx* ctx, const void* q_chunk, const void* k_chunk
   }
   uint8_t* kwin = (uint8_t*)s.kbuf + (long long)s.start * sn * es;     // first token of the softmax window
   uint8_t* vwin = (uint8_t*)s.vbuf + (long long)s.start * sn * es;
-  // 1. k and v of the chunk go behind the kept frames (they have to outlive the call); q and out stay where they are
-  launch_copy_rows2(kwin + (long long)h * sn * es, vwin + (long long)h * sn * es, sb * es, sh * es, sn * es, k_chunk, v_chunk,
-                    lay->stride_batch * es, lay->stride_head * es, lay->stride_token * es, Np, row_bytes, BH, c.n_heads, st);
+  // 1. k and v of the chunk go behind the kept frames (they have to outlive the call); q and out stay where they are.
+  //    With a q/k transform set, k is normalised and rotated on its way into the window (instead of being copied)
+  //    and q into a buffer of its own, both at the positions that follow the chunks processed so far.
+  ctx->last_launches = 0;
+  const void* q_used = q_chunk;
+  if (ctx->qk_on) {
+    QkPrepArgs pa = {};
+    pa.rows = Np; pa.n_heads = c.n_heads; pa.pos0 = (int)s.tokens_done;
+    pa.sb = lay->stride_batch; pa.sh = lay->stride_head; pa.sn = lay->stride_token;
+    pa.qn = c.head_dim; pa.qh = (long long)s.chunk_cap * c.head_dim; pa.qb = pa.qh * c.n_heads;
+    pa.kb = sb; pa.kh = sh; pa.kn = sn;
+    launch_qk_prepare(ctx, q_chunk, k_chunk, s.qbuf, kwin + (long long)h * sn * es, pa, BH, st);
+    launch_copy_rows2(vwin + (long long)h * sn * es, nullptr, sb * es, sh * es, sn * es, v_chunk, nullptr,
+                      lay->stride_batch * es, lay->stride_head * es, lay->stride_token * es, Np, row_bytes, BH, c.n_heads, st);
+    q_used = s.qbuf;
+  } else {
+    launch_copy_rows2(kwin + (long long)h * sn * es, vwin + (long long)h * sn * es, sb * es, sh * es, sn * es, k_chunk, v_chunk,
+                      lay->stride_batch * es, lay->stride_head * es, lay->stride_token * es, Np, row_bytes, BH, c.n_heads, st);
+  }
   // 2. Eq. 16 for this chunk: one chunk whose queries are rows [h, h + Np) of the window and whose softmax set
   //    is the whole window
   Geo g;
   g.N = h + Np; g.Np = Np; g.ToHW = h; g.t0 = 0; g.G = 1; g.n_heads = c.n_heads; g.BH = BH;
   g.stride_b = sb; g.stride_h = sh; g.stride_n = sn;
   g.q_shift = h; g.prefix = s.has_state;
-  g.qstride_b = lay->stride_batch; g.qstride_h = lay->stride_head; g.qstride_n = lay->stride_token;
-  if (g.qstride_h == 0) g.qstride_h = g.qstride_n * Np;
-  if (g.qstride_b == 0) g.qstride_b = g.qstride_h * c.n_heads;
+  g.ostride_b = lay->stride_batch; g.ostride_h = lay->stride_head; g.ostride_n = lay->stride_token;
+  if (g.ostride_h == 0) g.ostride_h = g.ostride_n * Np;
+  if (g.ostride_b == 0) g.ostride_b = g.ostride_h * c.n_heads;
+  g.qstride_b = g.ostride_b; g.qstride_h = g.ostride_h; g.qstride_n = g.ostride_n;
+  if (ctx->qk_on) { g.qstride_n = c.head_dim; g.qstride_h = (long long)s.chunk_cap * c.head_dim; g.qstride_b = g.qstride_h * c.n_heads; }
   g.q_off = h; g.Nq = Np;
   ctx->share_now = nullptr;
-  ctx->last_launches = 0;
   ctx->last_impl = ctx->tensor_ok ? 1 : 0;
-  int rc = run_parts(ctx, q_chunk, kwin, vwin, out_chunk, phi, g, s.batch, 1, -1, (s.has_state ? PART_READOUT : 0) | PART_WINDOW, st);
+  int rc = run_parts(ctx, q_used, kwin, vwin, out_chunk, phi, g, s.batch, 1, -1, (s.has_state ? PART_READOUT : 0) | PART_WINDOW, st);
   if (rc != REHYAT_OK) return rc;
   // 3. Eq. 17-18: the tokens that leave the window before the next chunk enter the running state
   const int keep = (long long)s.overlap * HW < (long long)h + Np ? s.overlap * HW : h + Np;
@@ -853,6 +887,7 @@ int rehyat_stream_step(rehyat_ctx* ctx, const void* q_chunk, const void* k_chunk
   // 4. the window moves on: the frames that stay are addressed, not copied
   s.start += leave;
   s.halo = keep;
+  s.tokens_done += Np;
   ++s.chunks_done;
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
@@ -871,8 +906,8 @@ int rehyat_stream_export(rehyat_ctx* ctx, void* host_buf, size_t capacity, void*
   if (!guard.ok) return REHYAT_ERR_CUDA;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   if (cudaStreamSynchronize(st) != cudaSuccess) return REHYAT_ERR_CUDA;
-  StreamHeader hd = {kStreamMagic, 1, c.dtype, c.n_heads, c.head_dim, c.phi_dim, s.batch, s.H, s.W, s.chunk, s.overlap,
-                     s.halo, s.has_state, 0, s.chunks_done};
+  StreamHeader hd = {kStreamMagic, 2, c.dtype, c.n_heads, c.head_dim, c.phi_dim, s.batch, s.H, s.W, s.chunk, s.overlap,
+                     s.halo, s.has_state, 0, s.chunks_done, s.tokens_done};
   uint8_t* p = (uint8_t*)host_buf;
   memcpy(p, &hd, sizeof(hd));
   p += sizeof(hd);
@@ -899,14 +934,14 @@ int rehyat_stream_import(rehyat_ctx* ctx, const void* host_buf, size_t bytes, vo
   const rehyat_config& c = ctx->cfg;
   StreamHeader hd;
   memcpy(&hd, host_buf, sizeof(hd));
-  if (hd.magic != kStreamMagic || hd.version != 1 || hd.dtype != c.dtype || hd.n_heads != c.n_heads ||
+  if (hd.magic != kStreamMagic || hd.version != 2 || hd.dtype != c.dtype || hd.n_heads != c.n_heads ||
       hd.head_dim != c.head_dim || hd.phi_dim != c.phi_dim)
     return REHYAT_ERR_INVALID_ARG;
   if (hd.halo < 0 || (long long)hd.halo > (long long)hd.overlap * hd.H * hd.W) return REHYAT_ERR_INVALID_ARG;
   int rc = rehyat_stream_begin(ctx, hd.batch, hd.H, hd.W, hd.chunk, hd.overlap, cuda_stream);
   if (rc != REHYAT_OK) return rc;
   rehyat_ctx::Stream& s = ctx->stream;
-  s.halo = hd.halo; s.has_state = hd.has_state ? 1 : 0; s.chunks_done = hd.chunks_done;
+  s.halo = hd.halo; s.has_state = hd.has_state ? 1 : 0; s.chunks_done = hd.chunks_done; s.tokens_done = hd.tokens_done;
   if (bytes < rehyat_stream_state_bytes(ctx)) { s.active = false; return REHYAT_ERR_INVALID_ARG; }
   DeviceGuard guard(c.device);
   if (!guard.ok) return REHYAT_ERR_CUDA;

@@ -33,6 +33,7 @@ struct Geo {
   // have Nq rows and their own strides.  A whole-sequence call has q_off = 0, Nq = N and the strides of k, v.
   long long qstride_b, qstride_h, qstride_n;
   int q_off, Nq;
+  long long ostride_b, ostride_h, ostride_n;   // out: the rows of q, strides of its own (a step may read a transformed copy of q)
 };
 
 __host__ __device__ inline int geo_q0(const Geo& g, int t) { return t * g.Np + g.q_shift; }
@@ -86,10 +87,14 @@ __device__ __forceinline__ float2 unpack_f16(uint32_t pair) {
 __device__ __forceinline__ long long head_offset(const Geo& g, int bh) {
   return (long long)(bh / g.n_heads) * g.stride_b + (long long)(bh % g.n_heads) * g.stride_h;
 }
-// Element offset of buffer row `row` (a query row) of (batch*head) bh inside q or out.
+// Element offset of buffer row `row` (a query row) of (batch*head) bh inside q, and inside out.
 __device__ __forceinline__ long long q_row_offset(const Geo& g, int bh, int row) {
   return (long long)(bh / g.n_heads) * g.qstride_b + (long long)(bh % g.n_heads) * g.qstride_h +
          (long long)(row - g.q_off) * g.qstride_n;
+}
+__device__ __forceinline__ long long out_row_offset(const Geo& g, int bh, int row) {
+  return (long long)(bh / g.n_heads) * g.ostride_b + (long long)(bh % g.n_heads) * g.ostride_h +
+         (long long)(row - g.q_off) * g.ostride_n;
 }
 
 __device__ __forceinline__ float ldf(const float* p) { return *p; }

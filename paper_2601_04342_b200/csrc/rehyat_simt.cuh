@@ -305,19 +305,26 @@ readout_simt(const T* __restrict__ q, PhiPtrs<T> wq, PhiDims pd, Geo g, const fl
 // grid (row blocks, BH, 2: q / k), 256 threads; a row of d elements is shared by d/8 lanes, eight elements each.
 struct QkPrepArgs {
   const void* wq; const void* wk;       // [n_heads][d] in the operator dtype, or null
-  const float* cos; const float* sin;   // [N][d/2], or null
+  const float* cos; const float* sin;   // [positions][d/2], or null
   float eps;
   int rms_norm;
+  int rows, n_heads;                    // token rows per (batch, head), heads
+  int pos0;                             // position of row 0 in the rotation tables (tokens of earlier chunks)
+  long long sb, sh, sn;                 // element strides of the sources (q and k share them)
+  long long qb, qh, qn;                 // ... of the transformed q
+  long long kb, kh, kn;                 // ... of the transformed k
 };
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
-qk_prepare(const T* __restrict__ q, const T* __restrict__ k, T* __restrict__ qo, T* __restrict__ ko, Geo g, QkPrepArgs a) {
+qk_prepare(const T* __restrict__ q, const T* __restrict__ k, T* __restrict__ qo, T* __restrict__ ko, QkPrepArgs a) {
   constexpr int LPR = D / 8;                                        // lanes per row
   const T* __restrict__ src = blockIdx.z ? k : q;
   T* __restrict__ dst = blockIdx.z ? ko : qo;
   const T* __restrict__ wgt = static_cast<const T*>(blockIdx.z ? a.wk : a.wq);
-  const int bh = blockIdx.y, head = bh % g.n_heads;
-  const long long hoff = head_offset(g, bh);
+  const int bh = blockIdx.y, head = bh % a.n_heads, bat = bh / a.n_heads;
+  const long long hoff = (long long)bat * a.sb + (long long)head * a.sh;
+  const long long doff = blockIdx.z ? (long long)bat * a.kb + (long long)head * a.kh : (long long)bat * a.qb + (long long)head * a.qh;
+  const long long dn = blockIdx.z ? a.kn : a.qn;
   const int lane_in_row = threadIdx.x % LPR, col = lane_in_row * 8;
   const int rows_per_block = 256 / LPR;
   // a thread keeps its eight columns for all its rows: their norm weights are loaded once
@@ -330,13 +337,13 @@ qk_prepare(const T* __restrict__ q, const T* __restrict__ k, T* __restrict__ qo,
   const unsigned row_lanes = (LPR >= 32 ? 0xffffffffu : ((1u << LPR) - 1u) << ((threadIdx.x & 31) / LPR * LPR));
   // two rows per step, both loaded before either is worked on: twice the bytes in flight per thread
   const int stride = gridDim.x * rows_per_block;
-  for (int row0 = blockIdx.x * rows_per_block + threadIdx.x / LPR; row0 < g.N; row0 += 2 * stride) {
+  for (int row0 = blockIdx.x * rows_per_block + threadIdx.x / LPR; row0 < a.rows; row0 += 2 * stride) {
     float x[2][8];
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
       const int row = row0 + u * stride;
-      if (row < g.N) {
-        const T* p = src + hoff + (long long)row * g.stride_n + col;
+      if (row < a.rows) {
+        const T* p = src + hoff + (long long)row * a.sn + col;
         const float4 x0 = ld4(p), x1 = ld4(p + 4);
         x[u][0] = x0.x; x[u][1] = x0.y; x[u][2] = x0.z; x[u][3] = x0.w;
         x[u][4] = x1.x; x[u][5] = x1.y; x[u][6] = x1.z; x[u][7] = x1.w;
@@ -358,10 +365,10 @@ qk_prepare(const T* __restrict__ q, const T* __restrict__ k, T* __restrict__ qo,
 #pragma unroll
         for (int e = 0; e < 8; ++e) x[u][e] *= inv * wv[e];
       }
-      if (row >= g.N) continue;
+      if (row >= a.rows) continue;
       if (a.cos != nullptr) {
-        const float4 c = *reinterpret_cast<const float4*>(a.cos + (size_t)row * (D / 2) + col / 2);
-        const float4 s = *reinterpret_cast<const float4*>(a.sin + (size_t)row * (D / 2) + col / 2);
+        const float4 c = *reinterpret_cast<const float4*>(a.cos + (size_t)(a.pos0 + row) * (D / 2) + col / 2);
+        const float4 s = *reinterpret_cast<const float4*>(a.sin + (size_t)(a.pos0 + row) * (D / 2) + col / 2);
         const float cs[4] = {c.x, c.y, c.z, c.w}, sn[4] = {s.x, s.y, s.z, s.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -370,7 +377,7 @@ qk_prepare(const T* __restrict__ q, const T* __restrict__ k, T* __restrict__ qo,
           x[u][2 * e + 1] = p0 * sn[e] + p1 * cs[e];
         }
       }
-      st8(dst + hoff + (long long)row * g.stride_n + col, x[u]);
+      st8(dst + doff + (long long)row * dn + col, x[u]);
     }
   }
 }
@@ -509,7 +516,7 @@ window_simt(const T* __restrict__ q, const T* __restrict__ k, const T* __restric
     }
     const float inv = 1.f / (l[i] * ws + lam * nL);
     if (share != nullptr && tx == 0) share[(size_t)bh * g.N + row] = lam * nL * inv;   // part of the normaliser that is linear
-    T* orow = out + q_row_offset(g, bh, row) + tx * DC;
+    T* orow = out + out_row_offset(g, bh, row) + tx * DC;
 #pragma unroll
     for (int c = 0; c < DC; ++c) {
       const float aL = linear ? rd[rd_index(g, rd_rows, D, bh, ci, row - q0, (tx * DC + c) >> 2) + ((tx * DC + c) & 3)] : 0.f;

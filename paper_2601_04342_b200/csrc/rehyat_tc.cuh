@@ -414,7 +414,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           lam = __expf(-r);
         }
       }
-      __nv_bfloat16* orow = out + q_row_offset(g, w.bh, row);
+      __nv_bfloat16* orow = out + out_row_offset(g, w.bh, row);
       if (!wait(&bars->pv_done[i], (n_s + n_kv - 1) & 1)) break;
       tc_fence_after();
       n_s += n_kv;

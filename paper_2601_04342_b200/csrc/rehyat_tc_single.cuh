@@ -272,7 +272,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           lam = __expf(-rr);
         }
       }
-      __nv_bfloat16* orow = out + q_row_offset(g, w.bh, row) + i * (TC_D / 2);
+      __nv_bfloat16* orow = out + out_row_offset(g, w.bh, row) + i * (TC_D / 2);
       if (!wait(&bars->pv_done[0], (n_s[0] + cnt0 - 1) & 1)) break;
       if (cnt1 > 0 && !wait(&bars->pv_done[1], (n_s[1] + cnt1 - 1) & 1)) break;
       tc_fence_after();

@@ -120,3 +120,45 @@ def test_transform_needs_a_context_made_for_it_and_respects_max_frames():
         op.forward(d["q"], d["k"], d["v"], pq, pk, wl.T, wl.H, wl.W, wl.Tc, wl.To)
     assert e.value.code == binding.ERR_INVALID_ARG
     op.close()
+
+
+@pytest.mark.parametrize("resume_after", [None, 2])
+def test_transform_chunk_by_chunk(resume_after):
+    """rehyat_stream_step with a transform set: k is transformed on its way into the window buffer, q into a buffer
+    of one chunk, rotation tables read at the running position.  All steps together equal the oracle on the whole
+    transformed sequence; a sequence resumed from an exported state continues bit for bit."""
+    from paper_2601_04342_b200 import binding
+    wl = synth.Workload("qk_stream", 2, 2, 128, 7, 9, 17, 2, 1, "bf16", False, seed=synth.BASE_SEED + 99)
+    x, wq, wk, cos, sin = _case(wl, 19)
+    ref, _ = _oracle(wl, x, wq, wk, cos, sin)
+    d = {n: x[n].cuda() for n in ("q", "k", "v")}
+    pq = {n: t.cuda() for n, t in x["phi_q"].items()}
+    pk = {n: t.cuda() for n, t in x["phi_k"].items()}
+    keep = [wq.cuda(), wk.cuda(), cos.cuda(), sin.cuda()]
+
+    def make():
+        op = binding.for_workload(wl, qk_transform=True)
+        op.set_qk_transform(q_weight=keep[0], k_weight=keep[1], eps=1e-6, cos=keep[2], sin=keep[3])
+        return op
+
+    def run(resume):
+        op = make()
+        out = torch.full_like(d["q"], float("nan"))
+        op.stream_begin(wl.B, wl.H, wl.W, wl.Tc, wl.To)
+        for t in range(-(-wl.T // wl.Tc)):
+            f0, f1 = t * wl.Tc, min((t + 1) * wl.Tc, wl.T)
+            sl = slice(f0 * wl.HW, f1 * wl.HW)
+            op.stream_step(d["q"][:, :, sl], d["k"][:, :, sl], d["v"][:, :, sl], pq, pk, f1 - f0, out=out[:, :, sl])
+            assert op.status() == 0
+            if resume is not None and t + 1 == resume:
+                blob = op.stream_export()
+                op.close()
+                op = make()
+                op.stream_import(blob)
+        op.close()
+        return out
+
+    y = run(None)
+    _check(y.double().cpu().numpy(), ref, "bf16")
+    if resume_after is not None:
+        assert torch.equal(run(resume_after), y)
