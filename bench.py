@@ -327,7 +327,7 @@ def time_config(wl, device, stream, full_softmax=False, steps=20, rms_norm=True)
     ms = _time_ms(run, stream, 3, steps)
     assert op.status() == 0
     fl = geometry.flop_model(wl.B, wl.n_heads, wl.head_dim, wl.T, wl.HW, wl.Tc, wl.To, wl.D_h, wl.D_out)
-    res = {"workload": wl.name, "batch": wl.B, "tokens": wl.N, "chunk_frames": wl.Tc, "overlap_frames": wl.To,
+    res = {"workload": wl.name, "batch": wl.B, "heads": wl.n_heads, "head_dim": wl.head_dim, "tokens": wl.N, "chunk_frames": wl.Tc, "overlap_frames": wl.To,
            "steps": steps, "ms_per_step": ms, "tflops": fl["total"] / (ms * 1e-3) / 1e12,
            "tokens_per_s": wl.B * wl.N / (ms * 1e-3), "workspace_bytes": op.workspace_bytes, "launches_per_step": op.last_launches,
            "window_tiles_per_item": op.last_window_tiles, "full_softmax_flop_ratio": fl["full_softmax"] / fl["total"],
@@ -597,6 +597,9 @@ def main():
         extras["other_configs"] = [time_config(synth.CONFIGS[n], local_rank, stream, steps=10,
                                                full_softmax=(args.all_configs and n == "cfg_long"))
                                    for n in ("cfg_long", "long_constant_memory", "wan13b_320x480")]
+        # the same tokens and model width with heads of 64 channels: tensor-core window, fp32 kernels for phi
+        extras["other_configs"].append(time_config(wl.with_(name="heads_of_64", n_heads=2 * wl.n_heads, head_dim=wl.head_dim // 2),
+                                                   local_rank, stream, steps=5))
         extras["chunk_overlap_sweep"] = [time_config(w, local_rank, stream, steps=5) for w in synth.sweep_configs()]
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -244,8 +244,11 @@ int run_parts(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void
   if (ctx->tensor_ok) {
     using B = __nv_bfloat16;
     if (!ctx->tc.phi_ok) {
-      rc = launch_group_simt<B, 128>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot,
-                                     parts & (PART_STATE | PART_READOUT), st);
+      rc = c.head_dim == 64
+               ? launch_group_simt<B, 64>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot,
+                                          parts & (PART_STATE | PART_READOUT), st)
+               : launch_group_simt<B, 128>(ctx, (const B*)q, (const B*)k, (const B*)v, (B*)out, phi, g, n_split, carry_slot,
+                                           parts & (PART_STATE | PART_READOUT), st);
     } else {
       if (parts & PART_STATE) {
         ctx->prof.begin(REHYAT_PROF_STATE, st);
@@ -399,7 +402,8 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
   if ((c.impl == REHYAT_IMPL_TENSOR || c.impl == REHYAT_IMPL_TENSOR_WINDOW) && !ctx->tensor_ok) { delete ctx; return REHYAT_ERR_UNSUPPORTED; }
   if (c.impl == REHYAT_IMPL_SIMT) ctx->tensor_ok = false;
   ctx->tc.phi_ok = ctx->tensor_ok && c.impl != REHYAT_IMPL_TENSOR_WINDOW && c.phi_layers <= 2 &&
-                   tc_phi_supported(c.phi_hidden, c.phi_dim, c.poly_degree);
+                   tc_phi_supported(c.head_dim, c.phi_hidden, c.phi_dim, c.poly_degree);
+  ctx->tc.head_dim = c.head_dim;
 
   const int np_max = c.max_tokens_per_frame * c.max_chunk_frames;
   const int want = c.group_tokens > 0 ? c.group_tokens : 32768;
@@ -411,9 +415,9 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
   const size_t SD = c.head_dim + 4;
   const size_t slot = (size_t)ctx->bh_max * c.phi_dim * SD * sizeof(float);
   const size_t b_state = slot * ctx->Gmax, b_partial = slot * ctx->partial_units;
-  // read-out of one chunk group: fp32 rows of d + 4 for the SIMT window kernel, RDH_PIECES 16-byte pieces per row
-  // (bf16) for the tensor-core ones
-  const size_t b_rd = ctx->tensor_ok ? (size_t)ctx->bh_max * ctx->rd_cap * RDH_PIECES * 16
+  // read-out of one chunk group: fp32 rows of d + 4 for the SIMT window kernel, d/8 + 1 16-byte pieces per row
+  // (fp16 ratios) for the tensor-core ones
+  const size_t b_rd = ctx->tensor_ok ? (size_t)ctx->bh_max * ctx->rd_cap * rdh_pieces(c.head_dim) * 16
                                      : (size_t)ctx->bh_max * ctx->rd_cap * SD * sizeof(float);
   bool ok = cudaMalloc(&ctx->state, b_state) == cudaSuccess && cudaMalloc(&ctx->partial, b_partial) == cudaSuccess &&
             cudaMalloc(&ctx->readout, b_rd) == cudaSuccess && cudaMalloc(&ctx->status_dev, 256) == cudaSuccess;

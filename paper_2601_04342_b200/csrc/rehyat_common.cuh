@@ -61,17 +61,17 @@ __host__ __device__ inline size_t rd_index(const Geo& g, int rd_rows, int d, int
 
 // The same workspace as the tensor-core kernels keep it (bf16 operator, head_dim 128): nL_i = phi_q(q_i) z_t in
 // fp32 and the d columns of the RATIO aL_i / nL_i = phi_q(q_i) s_t / nL_i in fp16, eight to a 16-byte piece:
-// RDH_PIECES pieces per 128-row tile (the last one holds nL in its first word), each with the tile's rows
+// rdh_pieces(d) = d/8 + 1 pieces per 128-row tile (the last one holds nL in its first word), each with the tile's rows
 // contiguous.  For non-negative features the ratio is a weighted mean of the v_j, so it fits fp16 whatever the
 // size of the sums, and its rounding (2^-11 relative) is below the bf16 rounding of the output; a ratio beyond the
 // fp16 range (features of both signs, nL near zero: Eq. 5 is then indefinite anyway) is clamped.  The workspace
 // and the traffic between the read-out and the window kernel are half of the fp32 form.  Returns the index of
 // the 16-byte piece `piece` of the row.
-constexpr int RDH_PIECES = 128 / 8 + 1;
-__host__ __device__ inline size_t rdh_index(const Geo& g, int rd_rows, int bh, int ci, int row_in_chunk, int piece) {
+__host__ __device__ constexpr int rdh_pieces(int d) { return d / 8 + 1; }
+__host__ __device__ inline size_t rdh_index(const Geo& g, int rd_rows, int d, int bh, int ci, int row_in_chunk, int piece) {
   const int tiles = (g.Np + 127) >> 7;
   const size_t tile = (size_t)bh * (size_t)(rd_rows >> 7) + (size_t)ci * tiles + (size_t)(row_in_chunk >> 7);
-  return (tile * (size_t)RDH_PIECES + (size_t)piece) * 128 + (size_t)(row_in_chunk & 127);
+  return (tile * (size_t)rdh_pieces(d) + (size_t)piece) * 128 + (size_t)(row_in_chunk & 127);
 }
 
 // Packs two ratios (see rdh_index) into one fp16 pair, clamped to the finite fp16 range.

@@ -313,7 +313,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         if (tok_valid) {
 #pragma unroll
           for (int e = 0; e < 32; e += 8)
-            rdh[rdh_index(g, a.rd_rows, bh, ci, ric, (ch * 64 + cb * 32 + e) >> 3)] =
+            rdh[rdh_index(g, a.rd_rows, PH_D, bh, ci, ric, (ch * 64 + cb * 32 + e) >> 3)] =
                 make_uint4(pack_ratio_f16(__uint_as_float(x[e]) * inv_nl, __uint_as_float(x[e + 1]) * inv_nl),
                            pack_ratio_f16(__uint_as_float(x[e + 2]) * inv_nl, __uint_as_float(x[e + 3]) * inv_nl),
                            pack_ratio_f16(__uint_as_float(x[e + 4]) * inv_nl, __uint_as_float(x[e + 5]) * inv_nl),
@@ -321,7 +321,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         }
       }
       if (tok_valid && ch == 1)
-        rdh[rdh_index(g, a.rd_rows, bh, ci, ric, RDH_PIECES - 1)] = make_uint4(__float_as_uint(nl_row), 0u, 0u, 0u);
+        rdh[rdh_index(g, a.rd_rows, PH_D, bh, ci, ric, rdh_pieces(PH_D) - 1)] = make_uint4(__float_as_uint(nl_row), 0u, 0u, 0u);
       tc_fence_before();
       mbar_arrive_warp(smem_u32(&bars->out_read), lane);
     };

@@ -268,7 +268,7 @@ readout_simt(const T* __restrict__ q, PhiPtrs<T> wq, PhiDims pd, Geo g, const fl
       float acc = 0.f;
       for (int ff = 0; ff < pd.Dp; ++ff) acc = fmaf(Fs[r * pd.Dp + ff], S[(size_t)ff * SD + D], acc);
       nl_s[r] = acc;
-      if (tok0 + r < q1) rd[rdh_index(g, rd_rows, bh, ci, tok0 + r - q0, RDH_PIECES - 1) * 4] = acc;
+      if (tok0 + r < q1) rd[rdh_index(g, rd_rows, D, bh, ci, tok0 + r - q0, rdh_pieces(D) - 1) * 4] = acc;
     }
     __syncthreads();
   }
@@ -291,7 +291,7 @@ readout_simt(const T* __restrict__ q, PhiPtrs<T> wq, PhiDims pd, Geo g, const fl
         rd[rd_index(g, rd_rows, D, bh, ci, tok - q0, c >> 2) + (c & 3)] = acc[r];
       } else {
         const float nl = nl_s[r0 + r], ratio = nl != 0.f ? acc[r] / nl : 0.f;
-        reinterpret_cast<__half*>(rd)[rdh_index(g, rd_rows, bh, ci, tok - q0, c >> 3) * 8 + (c & 7)] =
+        reinterpret_cast<__half*>(rd)[rdh_index(g, rd_rows, D, bh, ci, tok - q0, c >> 3) * 8 + (c & 7)] =
             __float2half_rn(fminf(fmaxf(ratio, -65504.f), 65504.f));
       }
     }

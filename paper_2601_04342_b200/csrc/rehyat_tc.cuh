@@ -26,7 +26,6 @@
 
 namespace rehyat {
 
-constexpr int TC_D = 128;             // head_dim
 constexpr int TC_BM = 128;            // rows per query tile
 constexpr int TC_QT = 2;              // query tiles per CTA
 constexpr int TC_BN = 128;            // keys per tile
@@ -34,9 +33,18 @@ constexpr int TC_STAGES = 2;          // K ring and V ring depth
 constexpr int TC_THREADS = 384;
 constexpr int TC_REGS_SOFTMAX = 200;   // registers per thread of the softmax warps (setmaxnreg)
 constexpr int TC_REGS_OTHER = 96;       // ... of the producer / issuer warpgroup
-constexpr int TC_TILE_BYTES = TC_BN * TC_D * 2;       // 32 KB: two [128 x 64] swizzled sub-tiles
-constexpr int TC_SUB_BYTES = TC_TILE_BYTES / 2;
-constexpr int TC_WIN_SMEM = (TC_QT + 2 * TC_STAGES) * TC_TILE_BYTES + 1024 /*barriers*/ + 1024 /*align*/;
+// Sizes that follow from the head dimension D (128 or 64).  A Q, K or V tile of 128 rows is D/64 swizzled
+// [128 x 64] sub-tiles of 16 KB.  TMEM keeps the map of D = 128 for both: S slots at columns 0 and 128, O slots at
+// 256 and 384 (D = 64 uses the first 64 columns of each O slot).
+template <int D>
+struct WinShape {
+  static_assert(D == 64 || D == 128, "head_dim of the tensor-core window kernels");
+  static constexpr int SUBS = D / 64;
+  static constexpr int SUB_BYTES = TC_BN * 64 * 2;
+  static constexpr int TILE_BYTES = SUBS * SUB_BYTES;
+  static constexpr int SMEM = (TC_QT + 2 * TC_STAGES) * TILE_BYTES + 1024 /*barriers*/ + 1024 /*align*/;      // window_tc
+  static constexpr int SMEM1 = (1 + 2 * TC_STAGES) * TILE_BYTES + 8192 /*barriers, merge buffer*/ + 1024;   // window_tc1
+};
 
 enum TcErr : int { TC_ERR_LOAD = 1, TC_ERR_MMA = 2, TC_ERR_SOFTMAX = 4 };
 
@@ -75,30 +83,32 @@ __device__ __forceinline__ bool win_item(const Geo& g, int item, int pairs, WinI
 
 // The MMAs of both window kernels, issued by one thread.  TMEM: S slots at columns 0 and 128, O slots at 256 and
 // 384.  Descriptors differ only in the start-address field (low word): built once, offsets added per MMA.
+template <int D>
 struct WinMma {
+  using SH = WinShape<D>;
   static constexpr uint32_t idesc_qk = ptx::idesc_bf16(TC_BM, TC_BN, 0, 0);   // A = Q (K-major), B = K (K-major)
-  static constexpr uint32_t idesc_pv = ptx::idesc_bf16(TC_BM, TC_D, 0, 1);    // A = P (TMEM),    B = V (MN-major)
+  static constexpr uint32_t idesc_pv = ptx::idesc_bf16(TC_BM, D, 0, 1);       // A = P (TMEM),    B = V (MN-major)
   uint32_t tmem, q_lo, q_hi, k_lo, k_hi, v_lo, v_hi;
   __device__ __forceinline__ WinMma(uint32_t tmem_base, uint32_t sQ, uint32_t sK, uint32_t sV) : tmem(tmem_base) {
     ptx::upk2u(ptx::smem_desc_sw128(sQ, 16, 1024), q_lo, q_hi);
     ptx::upk2u(ptx::smem_desc_sw128(sK, 16, 1024), k_lo, k_hi);
-    ptx::upk2u(ptx::smem_desc_sw128(sV, TC_SUB_BYTES, 1024), v_lo, v_hi);
+    ptx::upk2u(ptx::smem_desc_sw128(sV, SH::SUB_BYTES, 1024), v_lo, v_hi);
   }
   // S[slot] = Q[q_tile] K[stage]^T
   __device__ __forceinline__ void qk(int slot, int q_tile, int stage) const {
-    const uint32_t a0 = q_lo + q_tile * (TC_TILE_BYTES >> 4), b0 = k_lo + stage * (TC_TILE_BYTES >> 4);
+    const uint32_t a0 = q_lo + q_tile * (SH::TILE_BYTES >> 4), b0 = k_lo + stage * (SH::TILE_BYTES >> 4);
 #pragma unroll
-    for (int kk = 0; kk < TC_D / 16; ++kk) {
-      const uint32_t off = ((kk >> 2) * TC_SUB_BYTES + (kk & 3) * 32) >> 4;
+    for (int kk = 0; kk < D / 16; ++kk) {
+      const uint32_t off = ((kk >> 2) * SH::SUB_BYTES + (kk & 3) * 32) >> 4;
       ptx::umma_ss(tmem + slot * TC_BN, ptx::pk2u(a0 + off, q_hi), ptx::pk2u(b0 + off, k_hi), idesc_qk, kk > 0);
     }
   }
   // O[slot] (+)= P[slot][:, keys 64*half .. +64) V[stage][those keys, :]
   __device__ __forceinline__ void pv(int slot, int stage, int half, bool acc) const {
-    const uint32_t b0 = v_lo + stage * (TC_TILE_BYTES >> 4);
+    const uint32_t b0 = v_lo + stage * (SH::TILE_BYTES >> 4);
 #pragma unroll
     for (int kk = half * 4; kk < half * 4 + 4; ++kk)
-      ptx::umma_ts(tmem + 256 + slot * TC_D, tmem + slot * TC_BN + kk * 8, ptx::pk2u(b0 + kk * (16 * 128 >> 4), v_hi), idesc_pv,
+      ptx::umma_ts(tmem + 256 + slot * 128, tmem + slot * TC_BN + kk * 8, ptx::pk2u(b0 + kk * (16 * 128 >> 4), v_hi), idesc_pv,
                    (acc || kk > half * 4) ? 1u : 0u);
   }
 };
@@ -123,7 +133,7 @@ struct SoftmaxRow {
 // holds a P V of this item (O may then need the rescale); `wait_previous_pv()` waits for it and returns false if
 // the wait was given up, which is also what this function then returns.
 // EMU: of every four pairs of exponentials, how many are evaluated on the FMA pipe.
-template <int EMU, typename WaitPv>
+template <int EMU, int D, typename WaitPv>
 __device__ __forceinline__ bool softmax_key_tile(uint32_t tS, uint32_t tO, int n_valid, float c, bool has_previous,
                                                  SoftmaxRow& st, uint32_t bar_half0, uint32_t bar_half1, int lane,
                                                  WaitPv&& wait_previous_pv) {
@@ -159,7 +169,7 @@ __device__ __forceinline__ bool softmax_key_tile(uint32_t tS, uint32_t tO, int n
       st.l2a = mul2(st.l2a, f2);
       st.l2b = mul2(st.l2b, f2);
 #pragma unroll 1
-      for (int cc = 0; cc < TC_D / 8; ++cc) {                        // rare: small pieces keep the register peak low
+      for (int cc = 0; cc < D / 8; ++cc) {                           // rare: small pieces keep the register peak low
         uint32_t o[8];
         tmem_ld8(tO + cc * 8, o);
         tmem_wait_ld();
@@ -199,14 +209,16 @@ __device__ __forceinline__ bool softmax_key_tile(uint32_t tS, uint32_t tO, int n
 
 // Persistent: gridDim.x CTAs (one per SM) walk the items blockIdx.x, blockIdx.x + gridDim.x, ...  Barriers,
 // TMEM and the K/V rings live across items; every role keeps running counts of the phases it has used.
-// EMU: of every four pairs of exponentials, how many are evaluated on the FMA pipe.
-template <int EMU>
+// EMU: of every four pairs of exponentials, how many are evaluated on the FMA pipe.  D: head_dim.
+template <int EMU, int D>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
           const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ out, Geo g,
           const float* __restrict__ rd, int rd_rows, float scale, int c_mode, ptx::WaitArgs wa,
           int n_items, int pairs, float* __restrict__ share) {
   using namespace ptx;
+  using SH = WinShape<D>;
+  constexpr int TC_TILE_BYTES = SH::TILE_BYTES, TC_SUB_BYTES = SH::SUB_BYTES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -214,6 +226,11 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
   const uint32_t sK = sQ + TC_QT * TC_TILE_BYTES;                  // TC_STAGES tiles
   const uint32_t sV = sK + TC_STAGES * TC_TILE_BYTES;              // TC_STAGES tiles
   WinBars* bars = reinterpret_cast<WinBars*>(smem + (TC_QT + 2 * TC_STAGES) * TC_TILE_BYTES);
+  // one tile = SH::SUBS boxes of 64 columns
+  auto load_tile = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int row, int h, int b) {
+#pragma unroll
+    for (int sb = 0; sb < SH::SUBS; ++sb) tma_load_4d(dst + sb * TC_SUB_BYTES, tm, bar, sb * 64, row, h, b);
+  };
   const uint32_t wc = smem_u32(&bars->wctx);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -259,10 +276,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         if (!alive) break;
         const uint32_t qf = smem_u32(&bars->q_full);
         mbar_expect_tx(qf, w.ntiles * TC_TILE_BYTES);
-        for (int i = 0; i < w.ntiles; ++i) {
-          tma_load_4d(sQ + i * TC_TILE_BYTES, &tm_q, qf, 0, w.row_base - g.q_off + i * TC_BM, w.h_idx, w.b_idx);
-          tma_load_4d(sQ + i * TC_TILE_BYTES + TC_SUB_BYTES, &tm_q, qf, 64, w.row_base - g.q_off + i * TC_BM, w.h_idx, w.b_idx);
-        }
+        for (int i = 0; i < w.ntiles; ++i) load_tile(sQ + i * TC_TILE_BYTES, &tm_q, qf, w.row_base - g.q_off + i * TC_BM, w.h_idx, w.b_idx);
         ++n_q;
         for (int j = 0; j < w.n_kv && alive; ++j) {
           const int s = n_k % TC_STAGES;
@@ -272,15 +286,13 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           if (!alive) break;
           const uint32_t kf = smem_u32(&bars->k_full[s]);
           mbar_expect_tx(kf, TC_TILE_BYTES);
-          tma_load_4d(sK + s * TC_TILE_BYTES, &tm_k, kf, 0, key0, w.h_idx, w.b_idx);
-          tma_load_4d(sK + s * TC_TILE_BYTES + TC_SUB_BYTES, &tm_k, kf, 64, key0, w.h_idx, w.b_idx);
+          load_tile(sK + s * TC_TILE_BYTES, &tm_k, kf, key0, w.h_idx, w.b_idx);
           ++n_k;
           alive = mbar_wait(smem_u32(&bars->v_empty[s]), ph ^ 1, wc, TC_ERR_LOAD);
           if (!alive) break;
           const uint32_t vf = smem_u32(&bars->v_full[s]);
           mbar_expect_tx(vf, TC_TILE_BYTES);
-          tma_load_4d(sV + s * TC_TILE_BYTES, &tm_v, vf, 0, key0, w.h_idx, w.b_idx);
-          tma_load_4d(sV + s * TC_TILE_BYTES + TC_SUB_BYTES, &tm_v, vf, 64, key0, w.h_idx, w.b_idx);
+          load_tile(sV + s * TC_TILE_BYTES, &tm_v, vf, key0, w.h_idx, w.b_idx);
           ++n_v;
         }
       }
@@ -297,7 +309,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
   } else if (warp == 1) {
     // ------------------------------------------------------------------ UMMA issuer
     if (elect_one()) {
-      const WinMma mma(tmem, sQ, sK, sV);
+      const WinMma<D> mma(tmem, sQ, sK, sV);
       auto issue_qk = [&](int i, int s) { mma.qk(i, i, s); };         // query tile i into its own slot
       auto issue_pv = [&](int i, int s, int half, bool acc) { mma.pv(i, s, half, acc); };
       uint32_t kv_it = 0, n_done = 0;                                // K/V tiles consumed, items done
@@ -362,7 +374,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     setmaxnreg_inc<TC_REGS_SOFTMAX>();
     const int i = (warp - 4) >> 2;                                   // query tile of this warpgroup
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tS = tmem + lane_off + i * TC_BN, tO = tmem + lane_off + 256 + i * TC_D;
+    const uint32_t tS = tmem + lane_off + i * TC_BN, tO = tmem + lane_off + 256 + i * 128;
     const float c = scale * 1.4426950408889634f;                     // logits -> log2 domain
     uint32_t n_s = 0;                                                // key tiles this query tile has been through
     // A wait that was given up ends the role.  The warp decides together (tcgen05.ld / st and the votes below
@@ -380,7 +392,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       for (int j = 0; j < n_kv; ++j) {
         if (!wait(&bars->s_ready[i], (n_s + j) & 1)) break;
         tc_fence_after();
-        if (!softmax_key_tile<EMU>(tS, tO, hi - (lo + j * TC_BN), c, j > 0, st, smem_u32(&bars->p_half[i][0]),
+        if (!softmax_key_tile<EMU, D>(tS, tO, hi - (lo + j * TC_BN), c, j > 0, st, smem_u32(&bars->p_half[i][0]),
                                    smem_u32(&bars->p_half[i][1]), lane,
                                    [&]() { return wait(&bars->pv_done[i], (n_s + j - 1) & 1); }))
           break;
@@ -392,17 +404,17 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       const int row = w.row_base + i * TC_BM + (warp & 3) * 32 + lane;
       const bool valid = row < w.q1;
       // the whole read-out row is requested before the wait for the last P V, which hides its latency
-      uint4 rdv[TC_D / 8];                                           // fp16 pairs of aL / nL
+      uint4 rdv[D / 8];                                              // fp16 pairs of aL / nL
       float nL = 0.f;
       if (w.linear) {
         const int ric = (valid ? row : w.q0) - w.q0, ci = w.ci;      // row inside the chunk: consecutive threads, consecutive pieces
         const uint4* rdh = reinterpret_cast<const uint4*>(rd);
 #pragma unroll
-        for (int u = 0; u < TC_D / 8; ++u) rdv[u] = __ldg(rdh + rdh_index(g, rd_rows, w.bh, ci, ric, u));
-        nL = __ldg(reinterpret_cast<const float*>(rdh + rdh_index(g, rd_rows, w.bh, ci, ric, RDH_PIECES - 1)));
+        for (int u = 0; u < D / 8; ++u) rdv[u] = __ldg(rdh + rdh_index(g, rd_rows, D, w.bh, ci, ric, u));
+        nL = __ldg(reinterpret_cast<const float*>(rdh + rdh_index(g, rd_rows, D, w.bh, ci, ric, rdh_pieces(D) - 1)));
       } else {
 #pragma unroll
-        for (int u = 0; u < TC_D / 8; ++u) rdv[u] = make_uint4(0u, 0u, 0u, 0u);
+        for (int u = 0; u < D / 8; ++u) rdv[u] = make_uint4(0u, 0u, 0u, 0u);
       }
       const float fin = ex2((m_used - m_true) * c);
       float ws = fin, lam = 0.f;
@@ -422,11 +434,11 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       const float wsi = ws * inv, lami = lam * inv * nL;               // the read-out comes as the ratio aL / nL
       if (share != nullptr && valid) share[(size_t)w.bh * g.N + row] = lami;       // part of the normaliser that is linear
 #pragma unroll
-      for (int hh = 0; hh < 4; ++hh) {                               // 32 columns of O at a time
+      for (int hh = 0; hh < D / 32; ++hh) {                          // 32 columns of O at a time
         uint32_t o[32];
         tmem_ld32(tO + hh * 32, o);
         tmem_wait_ld();
-        if (hh == 3) {                                               // O has been read: TMEM is free for the next item
+        if (hh == D / 32 - 1) {                                      // O has been read: TMEM is free for the next item
           tc_fence_before();
           mbar_arrive_warp(smem_u32(&bars->o_free[i]), lane);
         }
@@ -468,12 +480,13 @@ struct TcWorkspace {
   bool phi_ok = false;                  // the linear branch runs on the tensor-core kernels too
   int n_sm = 148;                       // SMs of the device
   int exp_poly = 1;                     // of every 4 pairs of exponentials, how many the FMA pipe evaluates
+  int head_dim = 128;                   // 128 or 64
   int item_tiles = 0;                   // query tiles per window item: 1, 2, or 0 = chosen per launch
   int last_item_tiles = 0;              // what the last window launch used
 };
 
-inline bool tc_shape_supported(bool bf16, int d, int, int, int, int, int) { return bf16 && d == TC_D; }
-inline bool tc_phi_supported(int Dh, int Dp, int P) { return Dh == PH_DH && Dp == PH_DP && P != 3; }
+inline bool tc_shape_supported(bool bf16, int d, int, int, int, int, int) { return bf16 && (d == 128 || d == 64); }
+inline bool tc_phi_supported(int d, int Dh, int Dp, int P) { return d == PH_D && Dh == PH_DH && Dp == PH_DP && P != 3; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -497,17 +510,21 @@ inline bool tc_workspace_create(TcWorkspace* w, int bh_max, int Gmax, int d, int
 inline void tc_workspace_destroy(TcWorkspace* w) { cudaFree(w->state_bf16); w->state_bf16 = nullptr; }
 
 // window_tc1 (one query tile per item) and its launcher live in rehyat_tc_single.cuh
-inline int tc_launch_window1(int exp_poly, int n_sm, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+inline int tc_launch_window1(int head_dim, int exp_poly, int n_sm, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                              __nv_bfloat16* o, const Geo& g, const float* rd, int rd_rows, float scale, int c_mode,
                              const ptx::WaitArgs& wa, float* share, cudaStream_t st);
 inline bool tc_set_attributes1();
 
 inline int tc_set_attributes() {
   bool ok = tc_set_attributes1() &&
-            cudaFuncSetAttribute(window_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(window_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(window_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
-            cudaFuncSetAttribute(window_tc<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN_SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(window_tc<0, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<128>::SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(window_tc<1, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<128>::SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(window_tc<2, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<128>::SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(window_tc<3, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<128>::SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(window_tc<0, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<64>::SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(window_tc<1, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<64>::SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(window_tc<2, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<64>::SMEM) == cudaSuccess &&
+            cudaFuncSetAttribute(window_tc<3, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<64>::SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(phi_tc<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(phi_tc<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
             cudaFuncSetAttribute(phi_tc<false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PH_SMEM) == cudaSuccess &&
@@ -529,14 +546,14 @@ inline bool tc_encode(const TcWorkspace* w, CUtensorMap* tm, const void* base, i
 // Tensor map over one of q, k, v: dims (d, N, heads, batch), box [64 x 128 rows], 128-byte swizzle,
 // out-of-range rows read as zero.
 inline bool tc_make_tmap(const TcWorkspace* w, CUtensorMap* tm, const void* base, const Geo& g, int batch) {
-  const cuuint64_t dims[4] = {(cuuint64_t)TC_D, (cuuint64_t)g.N, (cuuint64_t)g.n_heads, (cuuint64_t)batch};
+  const cuuint64_t dims[4] = {(cuuint64_t)w->head_dim, (cuuint64_t)g.N, (cuuint64_t)g.n_heads, (cuuint64_t)batch};
   const cuuint64_t strides[3] = {(cuuint64_t)g.stride_n * 2, (cuuint64_t)g.stride_h * 2, (cuuint64_t)g.stride_b * 2};
   const cuuint32_t box[4] = {64, (cuuint32_t)TC_BN, 1, 1};
   return tc_encode(w, tm, base, 4, dims, strides, box);
 }
 // The same over q: its own row count and strides (see Geo).
 inline bool tc_make_tmap_q(const TcWorkspace* w, CUtensorMap* tm, const void* base, const Geo& g, int batch) {
-  const cuuint64_t dims[4] = {(cuuint64_t)TC_D, (cuuint64_t)g.Nq, (cuuint64_t)g.n_heads, (cuuint64_t)batch};
+  const cuuint64_t dims[4] = {(cuuint64_t)w->head_dim, (cuuint64_t)g.Nq, (cuuint64_t)g.n_heads, (cuuint64_t)batch};
   const cuuint64_t strides[3] = {(cuuint64_t)g.qstride_n * 2, (cuuint64_t)g.qstride_h * 2, (cuuint64_t)g.qstride_b * 2};
   const cuuint32_t box[4] = {64, (cuuint32_t)TC_BN, 1, 1};
   return tc_encode(w, tm, base, 4, dims, strides, box);
@@ -560,7 +577,7 @@ inline int tc_launch_window(TcWorkspace* w, const void* q, const void* k, const 
   const int pairs = (g.Np + TC_QT * TC_BM - 1) / (TC_QT * TC_BM);
   const int n_items = pairs * g.G * g.BH;
   const dim3 grid(n_items < w->n_sm ? n_items : w->n_sm);
-  const float scale = 1.0f / sqrtf((float)TC_D);
+  const float scale = 1.0f / sqrtf((float)w->head_dim);
   __nv_bfloat16* o = (__nv_bfloat16*)out;
   // Items of two query tiles share their K/V tiles in shared memory; items of one tile (window_tc1) take half
   // as long each and fill the SMs better when there are few of them, as in a chunk-by-chunk step.  Whole waves
@@ -569,17 +586,20 @@ inline int tc_launch_window(TcWorkspace* w, const void* q, const void* k, const 
   const double cost2 = 2.0 * (double)((n_items + w->n_sm - 1) / w->n_sm), cost1 = 1.08 * (double)((n1 + w->n_sm - 1) / w->n_sm);
   if (w->item_tiles == 1 || (w->item_tiles == 0 && cost1 < 0.93 * cost2)) {
     w->last_item_tiles = 1;
-    return tc_launch_window1(w->exp_poly, w->n_sm, tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, share, st);
+    return tc_launch_window1(w->head_dim, w->exp_poly, w->n_sm, tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, share, st);
   }
   w->last_item_tiles = 2;
-#define REHYAT_LAUNCH_WINDOW(E) \
-  window_tc<E><<<grid, TC_THREADS, TC_WIN_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, n_items, pairs, share)
-  switch (w->exp_poly) {
-    case 0: REHYAT_LAUNCH_WINDOW(0); break;
-    case 2: REHYAT_LAUNCH_WINDOW(2); break;
-    case 3: REHYAT_LAUNCH_WINDOW(3); break;
-    default: REHYAT_LAUNCH_WINDOW(1); break;
+#define REHYAT_LAUNCH_WINDOW(E, D) \
+  window_tc<E, D><<<grid, TC_THREADS, WinShape<D>::SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, n_items, pairs, share)
+#define REHYAT_LAUNCH_WINDOW_D(D)                \
+  switch (w->exp_poly) {                         \
+    case 0: REHYAT_LAUNCH_WINDOW(0, D); break;   \
+    case 2: REHYAT_LAUNCH_WINDOW(2, D); break;   \
+    case 3: REHYAT_LAUNCH_WINDOW(3, D); break;   \
+    default: REHYAT_LAUNCH_WINDOW(1, D); break;  \
   }
+  if (w->head_dim == 64) { REHYAT_LAUNCH_WINDOW_D(64) } else { REHYAT_LAUNCH_WINDOW_D(128) }
+#undef REHYAT_LAUNCH_WINDOW_D
 #undef REHYAT_LAUNCH_WINDOW
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }

@@ -26,7 +26,6 @@ struct WinBars1 {
   ptx::WaitCtx wctx;
   float mrg[2][2][3][TC_BM];   // [item parity][slot]: reference maximum, true maximum and row sum of every row
 };
-constexpr int TC_WIN1_SMEM = (1 + 2 * TC_STAGES) * TC_TILE_BYTES + 8192 /*barriers, merge buffer*/ + 1024 /*align*/;
 static_assert(sizeof(WinBars1) <= 8192, "barrier block");
 
 // Items are numbered (batch*head, chunk, query tile), query tile fastest; `tiles` = tiles of a full chunk.
@@ -47,14 +46,16 @@ __device__ __forceinline__ bool win_item1(const Geo& g, int item, int tiles, Win
 }
 
 // Persistent like window_tc: gridDim.x CTAs walk the items blockIdx.x, blockIdx.x + gridDim.x, ...
-// EMU: of every four pairs of exponentials, how many are evaluated on the FMA pipe.
-template <int EMU>
+// EMU: of every four pairs of exponentials, how many are evaluated on the FMA pipe.  D: head_dim.
+template <int EMU, int D>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ out, Geo g,
            const float* __restrict__ rd, int rd_rows, float scale, int c_mode, ptx::WaitArgs wa,
            int n_items, int tiles, float* __restrict__ share) {
   using namespace ptx;
+  using SH = WinShape<D>;
+  constexpr int TC_TILE_BYTES = SH::TILE_BYTES, TC_SUB_BYTES = SH::SUB_BYTES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -109,8 +110,8 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         if (!alive) break;
         const uint32_t qf = smem_u32(&bars->q_full);
         mbar_expect_tx(qf, TC_TILE_BYTES);
-        tma_load_4d(sQ, &tm_q, qf, 0, w.row_base - g.q_off, w.h_idx, w.b_idx);
-        tma_load_4d(sQ + TC_SUB_BYTES, &tm_q, qf, 64, w.row_base - g.q_off, w.h_idx, w.b_idx);
+#pragma unroll
+        for (int sb = 0; sb < SH::SUBS; ++sb) tma_load_4d(sQ + sb * TC_SUB_BYTES, &tm_q, qf, sb * 64, w.row_base - g.q_off, w.h_idx, w.b_idx);
         ++n_q;
         auto load_tile = [&](bool is_v, int j) {                     // key tile j of the item into its ring stage
           const uint32_t it = kv_it + j;
@@ -123,8 +124,8 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           const uint32_t dst = (is_v ? sV : sK) + s * TC_TILE_BYTES;
           const CUtensorMap* tm = is_v ? &tm_v : &tm_k;
           mbar_expect_tx(full, TC_TILE_BYTES);
-          tma_load_4d(dst, tm, full, 0, key0, w.h_idx, w.b_idx);
-          tma_load_4d(dst + TC_SUB_BYTES, tm, full, 64, key0, w.h_idx, w.b_idx);
+#pragma unroll
+          for (int sb = 0; sb < SH::SUBS; ++sb) tma_load_4d(dst + sb * TC_SUB_BYTES, tm, full, sb * 64, key0, w.h_idx, w.b_idx);
           if (is_v) ++n_v; else ++n_k;
           return true;
         };
@@ -149,7 +150,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   } else if (warp == 1) {
     // ------------------------------------------------------------------ UMMA issuer
     if (elect_one()) {
-      const WinMma mma(tmem, sQ, sK, sV);
+      const WinMma<D> mma(tmem, sQ, sK, sV);
       auto issue_qk = [&](int i, int s) { mma.qk(i, 0, s); };         // the one query tile into slot i
       auto issue_pv = [&](int i, int s, int half, bool acc) { mma.pv(i, s, half, acc); };
       uint32_t kv_it = 0, n_done = 0;                                // K/V tiles consumed, items done
@@ -207,7 +208,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     setmaxnreg_inc<TC_REGS_SOFTMAX>();
     const int i = (warp - 4) >> 2;                                   // TMEM slot of this warpgroup
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tS = tmem + lane_off + i * TC_BN, tO = tmem + lane_off + 256 + i * TC_D;
+    const uint32_t tS = tmem + lane_off + i * TC_BN, tO = tmem + lane_off + 256 + i * 128;
     const float c = scale * 1.4426950408889634f;                     // logits -> log2 domain
     const int r = (warp & 3) * 32 + lane;                            // row of the query tile
     uint32_t n_s[2] = {0, 0};                                        // key tiles each slot has been through
@@ -228,7 +229,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const int j = i + 2 * t;
         if (!wait(&bars->s_ready[i], (n_s[i] + t) & 1)) break;
         tc_fence_after();
-        if (!softmax_key_tile<EMU>(tS, tO, hi - (lo + j * TC_BN), c, t > 0, st, smem_u32(&bars->p_half[i][0]),
+        if (!softmax_key_tile<EMU, D>(tS, tO, hi - (lo + j * TC_BN), c, t > 0, st, smem_u32(&bars->p_half[i][0]),
                                    smem_u32(&bars->p_half[i][1]), lane,
                                    [&]() { return wait(&bars->pv_done[i], (n_s[i] + t - 1) & 1); }))
           break;
@@ -251,17 +252,17 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const int row = w.row_base + r;
       const bool valid = row < w.q1;
       // this warpgroup's half of the read-out row is requested before the wait for the last P V
-      uint4 rdv[TC_D / 16];                                          // fp16 pairs of aL / nL
+      uint4 rdv[D / 16];                                             // fp16 pairs of aL / nL
       float nL = 0.f;
       if (w.linear) {
         const int ric = (valid ? row : w.q0) - w.q0, ci = w.ci;
         const uint4* rdh = reinterpret_cast<const uint4*>(rd);
 #pragma unroll
-        for (int u = 0; u < TC_D / 16; ++u) rdv[u] = __ldg(rdh + rdh_index(g, rd_rows, w.bh, ci, ric, i * (TC_D / 16) + u));
-        nL = __ldg(reinterpret_cast<const float*>(rdh + rdh_index(g, rd_rows, w.bh, ci, ric, RDH_PIECES - 1)));
+        for (int u = 0; u < D / 16; ++u) rdv[u] = __ldg(rdh + rdh_index(g, rd_rows, D, w.bh, ci, ric, i * (D / 16) + u));
+        nL = __ldg(reinterpret_cast<const float*>(rdh + rdh_index(g, rd_rows, D, w.bh, ci, ric, rdh_pieces(D) - 1)));
       } else {
 #pragma unroll
-        for (int u = 0; u < TC_D / 16; ++u) rdv[u] = make_uint4(0u, 0u, 0u, 0u);
+        for (int u = 0; u < D / 16; ++u) rdv[u] = make_uint4(0u, 0u, 0u, 0u);
       }
       float f0 = ex2((mu0 - m_fin) * c), f1 = cnt1 > 0 ? ex2((mu1 - m_fin) * c) : 0.f, lam = 0.f;
       if (w.linear) {
@@ -272,7 +273,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           lam = __expf(-rr);
         }
       }
-      __nv_bfloat16* orow = out + out_row_offset(g, w.bh, row) + i * (TC_D / 2);
+      __nv_bfloat16* orow = out + out_row_offset(g, w.bh, row) + i * (D / 2);
       if (!wait(&bars->pv_done[0], (n_s[0] + cnt0 - 1) & 1)) break;
       if (cnt1 > 0 && !wait(&bars->pv_done[1], (n_s[1] + cnt1 - 1) & 1)) break;
       tc_fence_after();
@@ -280,19 +281,19 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const float inv = 1.f / (l0 * f0 + l1 * f1 + lam * nL);
       const float w0 = f0 * inv, w1 = f1 * inv, lami = lam * inv * nL;   // the read-out comes as the ratio aL / nL
       if (share != nullptr && valid && i == 0) share[(size_t)w.bh * g.N + row] = lami;   // part of the normaliser that is linear
-      const uint32_t tO0 = tmem + lane_off + 256 + i * (TC_D / 2);
+      const uint32_t tO0 = tmem + lane_off + 256 + i * (D / 2);
 #pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {                               // 32 columns at a time
+      for (int hh = 0; hh < D / 64; ++hh) {                          // 32 of this warpgroup's D/2 columns at a time
         uint32_t o0[32], o1[32];
         tmem_ld32(tO0 + hh * 32, o0);
         if (cnt1 > 0) {
-          tmem_ld32(tO0 + TC_D + hh * 32, o1);
+          tmem_ld32(tO0 + 128 + hh * 32, o1);
         } else {
 #pragma unroll
           for (int e = 0; e < 32; ++e) o1[e] = 0u;                   // slot 1 was not used
         }
         tmem_wait_ld();
-        if (hh == 1) {                                               // this warpgroup has read both slots
+        if (hh == D / 64 - 1) {                                      // this warpgroup has read both slots
           tc_fence_before();
           mbar_arrive_warp(smem_u32(&bars->o_free[i]), lane);
         }
@@ -326,29 +327,36 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 }
 
 // Launches window_tc1 with the tensor maps and arguments tc_launch_window has prepared.
-inline int tc_launch_window1(int exp_poly, int n_sm, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+inline int tc_launch_window1(int head_dim, int exp_poly, int n_sm, const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
                              __nv_bfloat16* o, const Geo& g, const float* rd, int rd_rows, float scale, int c_mode,
                              const ptx::WaitArgs& wa, float* share, cudaStream_t st) {
   const int tiles = (g.Np + TC_BM - 1) / TC_BM;
   const int n_items = tiles * g.G * g.BH;
   const dim3 grid(n_items < n_sm ? n_items : n_sm);
-#define REHYAT_LAUNCH_WINDOW1(E) \
-  window_tc1<E><<<grid, TC_THREADS, TC_WIN1_SMEM, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, n_items, tiles, share)
-  switch (exp_poly) {
-    case 0: REHYAT_LAUNCH_WINDOW1(0); break;
-    case 2: REHYAT_LAUNCH_WINDOW1(2); break;
-    case 3: REHYAT_LAUNCH_WINDOW1(3); break;
-    default: REHYAT_LAUNCH_WINDOW1(1); break;
+#define REHYAT_LAUNCH_WINDOW1(E, D) \
+  window_tc1<E, D><<<grid, TC_THREADS, WinShape<D>::SMEM1, st>>>(tq, tk, tv, o, g, rd, rd_rows, scale, c_mode, wa, n_items, tiles, share)
+#define REHYAT_LAUNCH_WINDOW1_D(D)               \
+  switch (exp_poly) {                            \
+    case 0: REHYAT_LAUNCH_WINDOW1(0, D); break;  \
+    case 2: REHYAT_LAUNCH_WINDOW1(2, D); break;  \
+    case 3: REHYAT_LAUNCH_WINDOW1(3, D); break;  \
+    default: REHYAT_LAUNCH_WINDOW1(1, D); break; \
   }
+  if (head_dim == 64) { REHYAT_LAUNCH_WINDOW1_D(64) } else { REHYAT_LAUNCH_WINDOW1_D(128) }
+#undef REHYAT_LAUNCH_WINDOW1_D
 #undef REHYAT_LAUNCH_WINDOW1
   return cudaGetLastError() == cudaSuccess ? REHYAT_OK : REHYAT_ERR_CUDA;
 }
 
 inline bool tc_set_attributes1() {
-  return cudaFuncSetAttribute(window_tc1<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN1_SMEM) == cudaSuccess &&
-         cudaFuncSetAttribute(window_tc1<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN1_SMEM) == cudaSuccess &&
-         cudaFuncSetAttribute(window_tc1<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN1_SMEM) == cudaSuccess &&
-         cudaFuncSetAttribute(window_tc1<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_WIN1_SMEM) == cudaSuccess;
+  return cudaFuncSetAttribute(window_tc1<0, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<128>::SMEM1) == cudaSuccess &&
+         cudaFuncSetAttribute(window_tc1<1, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<128>::SMEM1) == cudaSuccess &&
+         cudaFuncSetAttribute(window_tc1<2, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<128>::SMEM1) == cudaSuccess &&
+         cudaFuncSetAttribute(window_tc1<3, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<128>::SMEM1) == cudaSuccess &&
+         cudaFuncSetAttribute(window_tc1<0, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<64>::SMEM1) == cudaSuccess &&
+         cudaFuncSetAttribute(window_tc1<1, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<64>::SMEM1) == cudaSuccess &&
+         cudaFuncSetAttribute(window_tc1<2, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<64>::SMEM1) == cudaSuccess &&
+         cudaFuncSetAttribute(window_tc1<3, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, WinShape<64>::SMEM1) == cudaSuccess;
 }
 
 }  // namespace rehyat

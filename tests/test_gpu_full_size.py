@@ -157,6 +157,16 @@ def test_320x480_layer_every_element():
     gate(y.double().numpy(), ref)
 
 
+@pytest.mark.parametrize("tiles", [1, 2], ids=["one_tile_items", "two_tile_items"])
+def test_head_dim_64_full_length_sampled(tiles):
+    """The same 32,760 tokens with heads of 64 channels (24 heads): the softmax window runs on the tensor
+    cores with 64-column tiles, phi, state and read-out on the fp32 kernels."""
+    wl = synth.CONFIGS["wan13b_layer"].with_(name="d64_layer", n_heads=24, head_dim=64, seed=synth.BASE_SEED + 57)
+    x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
+    y, _, _ = gpu_forward(wl, x, window_tiles=tiles)
+    check_sampled(wl, x, y, [(0, 0), (0, 23)], seed=57)
+
+
 # ------------------------------------------------------------------ CFG batch, longer video
 def test_cfg_long_sampled_rows():
     wl = synth.CONFIGS["cfg_long"]                 # B=2, 41 frames: 14 chunks, the last one 2 frames
