@@ -285,7 +285,9 @@ int rehyat_set_wait_limit(rehyat_ctx* ctx, int32_t wait_limit_us, int32_t withho
 /* Number of kernel launches the last rehyat_forward on this context enqueued. */
 int rehyat_last_launches(const rehyat_ctx* ctx);
 
-/* 1 if the last forward ran the tensor-core kernels, 0 for the SIMT kernels. */
+/* Kernels of the last forward: 2 = every step on the tensor cores, 1 = the softmax window on the tensor cores
+ * and phi, state and read-out on the fp32 SIMT kernels (a phi map the tensor-core kernels do not cover: more
+ * than two layers, widths that are not multiples of 32), 0 = SIMT kernels throughout. */
 int rehyat_last_impl(const rehyat_ctx* ctx);
 
 /* Query tiles per work item of the last tensor-core window launch: 2 (window_tc) or 1 (window_tc1);

@@ -159,6 +159,11 @@ class Rehyat:
         return "tensor" if lib().rehyat_last_impl(self._h) else "simt"
 
     @property
+    def last_phi_impl(self):
+        """Kernels of phi, state and read-out in the last forward."""
+        return "tensor" if lib().rehyat_last_impl(self._h) == 2 else "simt"
+
+    @property
     def last_window_tiles(self):
         return lib().rehyat_last_window_tiles(self._h)
 

@@ -252,7 +252,7 @@ int run_parts(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void
     } else {
       if (parts & PART_STATE) {
         ctx->prof.begin(REHYAT_PROF_STATE, st);
-        rc = tc_launch_state(&ctx->tc, k, v, phi, g, batch, c.poly_degree, c.act_hidden, c.act_out, n_split,
+        rc = tc_launch_state(&ctx->tc, k, v, phi, g, batch, c.phi_hidden, c.phi_dim, c.poly_degree, c.act_hidden, c.act_out, n_split,
                              ctx->partial, next_wait(ctx), st);
         ctx->prof.end(REHYAT_PROF_STATE, st);
         const size_t per_slot = (size_t)g.BH * c.phi_dim * (c.head_dim + 4);
@@ -264,7 +264,7 @@ int run_parts(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void
       }
       if (rc == REHYAT_OK && (parts & PART_READOUT)) {
         ctx->prof.begin(REHYAT_PROF_READOUT, st);
-        rc = tc_launch_readout(&ctx->tc, q, phi, g, batch, c.poly_degree, c.act_hidden, c.act_out, ctx->state,
+        rc = tc_launch_readout(&ctx->tc, q, phi, g, batch, c.phi_hidden, c.phi_dim, c.poly_degree, c.act_hidden, c.act_out, ctx->state,
                                ctx->readout, ctx->rd_cap, next_wait(ctx), st);
         ctx->prof.end(REHYAT_PROF_READOUT, st);
         ctx->last_launches += 1;
@@ -593,7 +593,7 @@ int rehyat_forward(rehyat_ctx* ctx, const void* q, const void* k, const void* v,
   const int n_split = pick_state_split(ctx, g, G < n_chunks ? G : n_chunks, g.Np);
 
   ctx->last_launches = 0;
-  ctx->last_impl = ctx->tensor_ok ? 1 : 0;
+  ctx->last_impl = ctx->tensor_ok ? (ctx->tc.phi_ok ? 2 : 1) : 0;
   ctx->stream.active = false;                 // the workspace is about to be overwritten
   if (ctx->qk_on) {
     // q and k are normalised and rotated into the context's buffers, in the layout they came in
@@ -874,7 +874,7 @@ int rehyat_stream_step(rehyat_ctx* ctx, const void* q_chunk, const void* k_chunk
   if (ctx->qk_on) { g.qstride_n = c.head_dim; g.qstride_h = (long long)s.chunk_cap * c.head_dim; g.qstride_b = g.qstride_h * c.n_heads; }
   g.q_off = h; g.Nq = Np;
   ctx->share_now = nullptr;
-  ctx->last_impl = ctx->tensor_ok ? 1 : 0;
+  ctx->last_impl = ctx->tensor_ok ? (ctx->tc.phi_ok ? 2 : 1) : 0;
   int rc = run_parts(ctx, q_used, kwin, vwin, out_chunk, phi, g, s.batch, 1, -1, (s.has_state ? PART_READOUT : 0) | PART_WINDOW, st);
   if (rc != REHYAT_OK) return rc;
   // 3. Eq. 17-18: the tokens that leave the window before the next chunk enter the running state

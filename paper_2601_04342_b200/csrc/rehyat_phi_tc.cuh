@@ -1,4 +1,4 @@
-// Tensor-core kernel of the chunk-state increments for bf16, head_dim 128, phi widths D_h = D' = 256.
+// Tensor-core kernel of the chunk-state increments for bf16, head_dim 64 or 128, phi widths up to 256.
 //
 // phi_tc evaluates the feature map phi_k of Section 3.2 ("Characterization of phi") on tiles of 128 keys with
 // tcgen05.mma and feeds it straight into the contraction that consumes it: phi_k(K tile)^T [V | 1] accumulated
@@ -13,6 +13,12 @@
 //   warp 9     UMMA issuer
 // The phi tile is written once in the 128-byte-swizzled [token][feature] image; the state GEMM reads
 // it as an MN-major A operand (features are M).
+//
+// The schedule is laid out for head_dim 128 and D_h = D' = 256 (GEN = false: every extent a constant).  With
+// GEN = true the extents come from the arguments: head_dim 64 halves the K extent of the first GEMM and the N
+// extent of the state GEMM, a width of at most 128 drops the second half of its GEMM, and a width that is not
+// a multiple of 128 (or 64) relies on the tensor maps, which read rows and columns beyond the matrix as zero:
+// hidden units beyond D_h meet zero columns of W2, features beyond D' are zero (or masked) and never stored.
 #pragma once
 
 #include <cuda.h>
@@ -51,11 +57,12 @@ struct PhBars {
 };
 
 struct PhiTcArgs {
-  const __nv_bfloat16* b1;     // [heads][256]
-  const __nv_bfloat16* b2;     // [heads][256]
+  const __nv_bfloat16* b1;     // [heads][D_h]
+  const __nv_bfloat16* b2;     // [heads][D']
   int P, act_hidden, act_out;
+  int d, Dh, Dp;               // head_dim (64 or 128), phi widths (read by the GEN = true kernels)
   int n_split;                 // state kernel: splits of a chunk's increment
-  float* partial;              // state kernel: [G][n_split][BH][256][132]
+  float* partial;              // state kernel: [G][n_split][BH][D'][d + 4]
   const float* state;          // read-out kernel: fp32 states (z column is read)
   float* rd;                   // read-out kernel: the read-out workspace (see rdh_index)
   int rd_rows;
@@ -63,9 +70,21 @@ struct PhiTcArgs {
   ptx::WaitArgs wa;            // status word, launch epoch, wait limit
 };
 
-// tm_x: K, tm_v: V, 4-D like the window kernel's maps.  tm_w1: (128, 256, heads), tm_w2: (256, 256, heads),
-// boxes [64 x 128].  PC: polynomial degree known at compile time (0: read it from the arguments).
-template <bool RELU, int PC>
+// Extents of one launch: constants for the default shape, read from the arguments otherwise.
+template <bool GEN>
+struct PhiExtents {
+  int d, Dh, Dp;
+  __device__ explicit PhiExtents(const PhiTcArgs& a) : d(GEN ? a.d : PH_D), Dh(GEN ? a.Dh : PH_DH), Dp(GEN ? a.Dp : PH_DP) {}
+  __device__ int sd() const { return d + 4; }              // row of a state: d columns of s, then z, padded
+  __device__ int ks1() const { return d / 64; }            // 64-column K blocks of the first GEMM
+  __device__ int ks2() const { return (Dh + 63) / 64; }    // ... of the second
+  __device__ int nh() const { return (Dh + 127) / 128; }   // 128-column halves of H
+  __device__ int nu() const { return (Dp + 127) / 128; }   // ... of U
+};
+
+// tm_x: K, tm_v: V, 4-D like the window kernel's maps.  tm_w1: (d, D_h, heads), tm_w2: (D_h, D', heads),
+// boxes [64 x 128].  PC: polynomial degree known at compile time (0: read it from the arguments; 2 needs D' = 256).
+template <bool RELU, int PC, bool GEN>
 __global__ void __launch_bounds__(PH_THREADS, 1)
 phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_v,
        const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2, Geo g, PhiTcArgs a) {
@@ -81,6 +100,8 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
   const int b_idx = bh / g.n_heads, h_idx = bh % g.n_heads;
+  const PhiExtents<GEN> ex(a);
+  const int Dp = ex.Dp, SD = ex.sd(), ks1 = ex.ks1(), ks2 = ex.ks2(), nh = ex.nh(), nu = ex.nu();
 
   // token range [tok_a, tok_b) of this CTA
   const int lo_prev = t > 0 ? geo_lo(g, t - 1) : 0, lo = geo_lo(g, t);
@@ -91,8 +112,8 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   const int n_tiles = (tok_b - tok_a + 127) / 128;
 
   if (n_tiles == 0) {                          // nothing admitted: the partial is zero
-    float* dst = a.partial + (((size_t)ci * a.n_split + blockIdx.x) * g.BH + bh) * PH_DP * PH_SD;
-    for (int i = threadIdx.x; i < PH_DP * PH_SD / 4; i += PH_THREADS)
+    float* dst = a.partial + (((size_t)ci * a.n_split + blockIdx.x) * g.BH + bh) * Dp * SD;
+    for (int i = threadIdx.x; i < Dp * SD / 4; i += PH_THREADS)
       reinterpret_cast<float4*>(dst)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     return;
   }
@@ -110,9 +131,9 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     fence_mbar_init();
   }
   // biases as fp32; the ones tile: row 0 of both 64-column sub-tiles is 1, the rest 0
-  for (int i = threadIdx.x; i < 256; i += PH_THREADS) {
-    s_b1[i] = __bfloat162float(a.b1[(size_t)h_idx * 256 + i]);
-    s_b2[i] = __bfloat162float(a.b2[(size_t)h_idx * 256 + i]);
+  for (int i = threadIdx.x; i < 256; i += PH_THREADS) {          // zero beyond the widths
+    s_b1[i] = i < ex.Dh ? __bfloat162float(a.b1[(size_t)h_idx * ex.Dh + i]) : 0.f;
+    s_b2[i] = i < Dp ? __bfloat162float(a.b2[(size_t)h_idx * Dp + i]) : 0.f;
   }
   {
     uint32_t* ones = reinterpret_cast<uint32_t*>(smem + PH_OFF_ONES);
@@ -159,23 +180,21 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
         alive = mbar_wait(smem_u32(&bars->x_empty), (j & 1) ^ 1, wc, PH_ERR_LOAD);
         if (!alive) break;
         const uint32_t xf = smem_u32(&bars->x_full);
-        mbar_expect_tx(xf, PH_TILE_BYTES);
-        tma_load_4d(sX, &tm_x, xf, 0, tok0, h_idx, b_idx);
-        tma_load_4d(sX + PH_SUB, &tm_x, xf, 64, tok0, h_idx, b_idx);
+        mbar_expect_tx(xf, PH_SUB * ks1);
+        for (int ks = 0; ks < ks1; ++ks) tma_load_4d(sX + ks * PH_SUB, &tm_x, xf, ks * 64, tok0, h_idx, b_idx);
         ++n_x;
-        for (int nh = 0; nh < 2; ++nh)
-          for (int ks = 0; ks < 2; ++ks) ring_load(&tm_w1, ks * 64, nh * 128, h_idx);
+        for (int half = 0; half < nh; ++half)
+          for (int ks = 0; ks < ks1; ++ks) ring_load(&tm_w1, ks * 64, half * 128, h_idx);
         {
           alive = alive && mbar_wait(smem_u32(&bars->v_empty), (j & 1) ^ 1, wc, PH_ERR_LOAD);
           if (!alive) break;
           const uint32_t vf = smem_u32(&bars->v_full);
-          mbar_expect_tx(vf, PH_TILE_BYTES);
-          tma_load_4d(sV, &tm_v, vf, 0, tok0, h_idx, b_idx);
-          tma_load_4d(sV + PH_SUB, &tm_v, vf, 64, tok0, h_idx, b_idx);
+          mbar_expect_tx(vf, PH_SUB * ks1);
+          for (int ks = 0; ks < ks1; ++ks) tma_load_4d(sV + ks * PH_SUB, &tm_v, vf, ks * 64, tok0, h_idx, b_idx);
           ++n_v;
         }
-        for (int ks = 0; ks < 4; ++ks) ring_load(&tm_w2, ks * 64, 0, h_idx);
-        for (int ks = 0; ks < 4; ++ks) ring_load(&tm_w2, ks * 64, 128, h_idx);
+        for (int half = 0; half < nu; ++half)
+          for (int ks = 0; ks < ks2; ++ks) ring_load(&tm_w2, ks * 64, half * 128, h_idx);
       }
       if (!alive) {
         // Given up: wait for the last load issued into every buffer before the CTA exits (the full barriers
@@ -191,7 +210,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     // ------------------------------------------------------------------ UMMA issuer
     if (elect_one()) {
       constexpr uint32_t id_kk = idesc_bf16(128, 128, 0, 0);       // A K-major, B K-major   (the two MLP GEMMs)
-      constexpr uint32_t id_st = idesc_bf16(128, 128, 1, 1);       // A = phi^T (MN-major), B = V (MN-major)
+      const uint32_t id_st = idesc_bf16(128, ex.d, 1, 1);          // A = phi^T (MN-major), B = V (MN-major)
       constexpr uint32_t id_z = idesc_bf16(128, 16, 1, 0);         // A = phi^T (MN-major), B = ones (K-major)
       uint32_t ring_i = 0, n_epi = 0;
       // A wait that is given up ends the role at once: the helpers return false and run() returns, so nothing
@@ -239,25 +258,28 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       auto run = [&]() {
         for (int j = 0; j < n_tiles; ++j) {
           if (!wait(&bars->x_full, j & 1)) return;
-          if (j > 0) {
+          if (j > 0 && nu == 2) {
             if (!wait_epi()) return;                                  // scratch free: phi half 1 of tile j-1 written
             if (!wait(&bars->v_full, (j - 1) & 1)) return;            // ... and consumed
             consume_half(1, sHb, j == 1);
             umma_commit(smem_u32(&bars->v_empty));
           }
-          if (!mlp_half(sX, 2)) return;                               // H[:, 0:128]
+          if (!mlp_half(sX, ks1)) return;                             // H[:, 0:128]
           if (!wait_epi()) return;
-          if (!mlp_half(sX, 2)) return;                               // H[:, 128:256]
+          if (nh == 2 && !mlp_half(sX, ks1)) return;                  // H[:, 128:256]
           umma_commit(smem_u32(&bars->x_empty));
+          if (nh == 2 && !wait_epi()) return;
+          if (!mlp_half(sHb, ks2)) return;                            // U[:, 0:128]
           if (!wait_epi()) return;
-          if (!mlp_half(sHb, 4)) return;                              // U[:, 0:128]
-          if (!wait_epi()) return;
-          if (!mlp_half(sHb, 4)) return;                              // U[:, 128:256]
+          if (nu == 2 && !mlp_half(sHb, ks2)) return;                 // U[:, 128:256]
           if (!wait(&bars->v_full, j & 1)) return;
           consume_half(0, sPhi0, j == 0);
+          if (nu == 1) umma_commit(smem_u32(&bars->v_empty));         // no second half: V is free once these have run
         }
-        if (!wait_epi()) return;
-        consume_half(1, sHb, n_tiles == 1);
+        if (nu == 2) {
+          if (!wait_epi()) return;
+          consume_half(1, sHb, n_tiles == 1);
+        }
         umma_commit(smem_u32(&bars->out_ready));
       };
       run();
@@ -274,7 +296,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     const int r = qd * 32 + lane;
     const uint32_t lane_off = (uint32_t)(qd * 32) << 16;
     uint32_t n_acc = 0;
-    const int part_w = PH_DP / (PC ? PC : a.P);                     // a multiple of 32 (P in {1,2,4})
+    const int part_w = Dp / (PC ? PC : a.P);                        // RELU: a multiple of 32
     // After a wait has been given up anywhere in the CTA every later wait returns at once.  These warps then run
     // through the rest of the current tile on whatever the accumulators hold (tcgen05.ld needs all 32 lanes, so
     // nothing is skipped lane by lane; every address stays inside the CTA's TMEM and shared memory) and leave
@@ -286,11 +308,12 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       const bool tok_valid = tok_a + j * 128 + r < tok_b;
 #pragma unroll
       for (int step = 0; step < 4; ++step) {                        // H half 0, H half 1, U half 0, U half 1
+        const int half = step & 1;
+        const bool is_u = step >= 2;
+        if (half >= (is_u ? nu : nh)) continue;                     // a width of at most 128 has no second half
         wait(&bars->acc_ready, n_acc & 1);
         ++n_acc;
         tc_fence_after();
-        const int half = step & 1;
-        const bool is_u = step >= 2;
         const uint32_t dst = !is_u ? sHb : (half == 0 ? sPhi0 : sHb);
         const int dst_col0 = !is_u ? half * 128 : 0;
         const float* bias = (is_u ? s_b2 : s_b1) + half * 128;
@@ -324,12 +347,23 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
             }
           } else {
             const int act = is_u ? a.act_out : a.act_hidden;
-            const int part = is_u ? (half * 128 + col0) / part_w : 0;
+            if (GEN && is_u) {                                      // parts end anywhere; features beyond D' are zero
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-              float y0 = apply_act(__uint_as_float(x[cb][e]) + bias[col0 + e], act);
-              float y1 = apply_act(__uint_as_float(x[cb][e + 1]) + bias[col0 + e + 1], act);
-              w[e >> 1] = pack_bf16(poly_power(y0, part), poly_power(y1, part));
+              for (int e = 0; e < 32; e += 2) {
+                const int f0 = half * 128 + col0 + e;
+                const float y0 = apply_act(__uint_as_float(x[cb][e]) + bias[col0 + e], act);
+                const float y1 = apply_act(__uint_as_float(x[cb][e + 1]) + bias[col0 + e + 1], act);
+                w[e >> 1] = pack_bf16(f0 < Dp ? poly_power(y0, f0 / part_w) : 0.f,
+                                      f0 + 1 < Dp ? poly_power(y1, (f0 + 1) / part_w) : 0.f);
+              }
+            } else {
+              const int part = is_u ? (half * 128 + col0) / part_w : 0;
+#pragma unroll
+              for (int e = 0; e < 32; e += 2) {
+                float y0 = apply_act(__uint_as_float(x[cb][e]) + bias[col0 + e], act);
+                float y1 = apply_act(__uint_as_float(x[cb][e + 1]) + bias[col0 + e + 1], act);
+                w[e >> 1] = pack_bf16(poly_power(y0, part), poly_power(y1, part));
+              }
             }
           }
           if (is_u && !tok_valid) {
@@ -349,28 +383,34 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     }
     wait(&bars->out_ready, 0);
     if (!aborted()) {
-      // flush: lane r holds feature c*128 + r of half c; this thread writes its 64 columns
+      // flush: lane r holds feature c*128 + r of half c; this thread writes its share of the d columns
       tc_fence_after();
-      float* base = a.partial + (((size_t)ci * a.n_split + blockIdx.x) * g.BH + bh) * PH_DP * PH_SD;
+      float* base = a.partial + (((size_t)ci * a.n_split + blockIdx.x) * g.BH + bh) * Dp * SD;
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
-        float* dst = base + (size_t)(c * 128 + r) * PH_SD;
+        if (c >= nu) continue;
+        const bool feat_valid = c * 128 + r < Dp;
+        float* dst = base + (size_t)(c * 128 + r) * SD;
 #pragma unroll
         for (int cb = 0; cb < 2; ++cb) {
+          const int col = ch * 64 + cb * 32;
+          if (col >= ex.d) continue;                                // the same for the whole warp
           uint32_t x[32];
-          tmem_ld32(tmem + lane_off + T_ACC + c * 128 + ch * 64 + cb * 32, x);
+          tmem_ld32(tmem + lane_off + T_ACC + c * 128 + col, x);
           tmem_wait_ld();
+          if (feat_valid) {
 #pragma unroll
-          for (int e = 0; e < 32; e += 4)
-            *reinterpret_cast<float4*>(dst + ch * 64 + cb * 32 + e) =
-                make_float4(__uint_as_float(x[e]), __uint_as_float(x[e + 1]), __uint_as_float(x[e + 2]),
-                            __uint_as_float(x[e + 3]));
+            for (int e = 0; e < 32; e += 4)
+              *reinterpret_cast<float4*>(dst + col + e) =
+                  make_float4(__uint_as_float(x[e]), __uint_as_float(x[e + 1]), __uint_as_float(x[e + 2]),
+                              __uint_as_float(x[e + 3]));
+          }
         }
         if (ch == 1) {
           uint32_t zc[16];
           tmem_ld16(tmem + lane_off + T_Z + c * 16, zc);
           tmem_wait_ld();
-          *reinterpret_cast<float4*>(dst + PH_D) = make_float4(__uint_as_float(zc[0]), 0.f, 0.f, 0.f);
+          if (feat_valid) *reinterpret_cast<float4*>(dst + ex.d) = make_float4(__uint_as_float(zc[0]), 0.f, 0.f, 0.f);
         }
       }
     }

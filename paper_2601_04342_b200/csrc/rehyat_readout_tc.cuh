@@ -1,4 +1,5 @@
-// Tensor-core kernel of the linear read-out for bf16, head_dim 128, phi widths D_h = D' = 256:
+// Tensor-core kernel of the linear read-out for bf16, head_dim 64 or 128, phi widths up to 256 (the schedule is
+// laid out for 128 / 256 / 256; GEN = true reads the extents from the arguments as phi_tc does):
 //   phi_q on tiles of 128 queries (Section 3.2 "Characterization of phi"), then phi_q(Q tile) s_t on the
 //   tensor core and phi_q(Q tile) z_t on the ALUs (Eq. 7, 9, 16), written as the fp32 read-out of the tile.
 //
@@ -40,10 +41,10 @@ struct RdBars {
   ptx::WaitCtx wctx;
 };
 
-// tm_x: Q, 4-D like the window kernel's maps.  tm_w1: (128, 256, heads), tm_w2: (256, 256, heads), boxes
-// [64 x 128].  tm_s: bf16 states (128, 256, G*BH), box [64 x 64].  PC: polynomial degree known at compile time
-// (0: read it from the arguments).
-template <bool RELU, int PC>
+// tm_x: Q, 4-D like the window kernel's maps.  tm_w1: (d, D_h, heads), tm_w2: (D_h, D', heads), boxes
+// [64 x 128].  tm_s: bf16 states (d, D', G*BH), box [64 x 64].  PC: polynomial degree known at compile time
+// (0: read it from the arguments; 2 needs D' = 256).
+template <bool RELU, int PC, bool GEN>
 __global__ void __launch_bounds__(PH_THREADS, 1)
 readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w1,
            const __grid_constant__ CUtensorMap tm_w2, const __grid_constant__ CUtensorMap tm_s, Geo g, PhiTcArgs a) {
@@ -62,6 +63,9 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
   const int ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
   const int b_idx = bh / g.n_heads, h_idx = bh % g.n_heads;
   if (!geo_linear(g, t)) return;                                    // empty linear set
+  const PhiExtents<GEN> ex(a);
+  const int d = ex.d, Dp = ex.Dp, SD = ex.sd(), ks1 = ex.ks1(), ks2 = ex.ks2(), nh = ex.nh(), nu = ex.nu();
+  const int nf = (Dp + 63) / 64;                                    // 64-feature blocks of the state
   const int q0 = geo_q0(g, t), q1 = geo_q1(g, t);
   const int tok_a = min(q0 + (int)blockIdx.x * a.tiles_per_cta * 128, q1);
   const int tok_b = min(tok_a + a.tiles_per_cta * 128, q1);
@@ -79,10 +83,10 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
     wait_ctx_init(&bars->wctx, a.wa);
     fence_mbar_init();
   }
-  for (int i = threadIdx.x; i < 256; i += PH_THREADS) {             // biases and z_t as fp32
-    s_b1[i] = __bfloat162float(a.b1[(size_t)h_idx * 256 + i]);
-    s_b2[i] = __bfloat162float(a.b2[(size_t)h_idx * 256 + i]);
-    s_z[i] = a.state[(((size_t)ci * g.BH + bh) * PH_DP + i) * PH_SD + PH_D];
+  for (int i = threadIdx.x; i < 256; i += PH_THREADS) {             // biases and z_t as fp32, zero beyond the widths
+    s_b1[i] = i < ex.Dh ? __bfloat162float(a.b1[(size_t)h_idx * ex.Dh + i]) : 0.f;
+    s_b2[i] = i < Dp ? __bfloat162float(a.b2[(size_t)h_idx * Dp + i]) : 0.f;
+    s_z[i] = i < Dp ? a.state[(((size_t)ci * g.BH + bh) * Dp + i) * SD + d] : 0.f;
   }
   if (warp == 9) {
     tmem_alloc(smem_u32(&bars->tmem_base), 512);
@@ -101,45 +105,47 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_w1); prefetch_tensormap(&tm_w2); prefetch_tensormap(&tm_s);
       uint32_t ring_i = 0, n_x = 0;                                 // ring tiles and X tiles issued so far
       bool alive = true;
-      auto ring_slot = [&](uint32_t& full) -> uint32_t {            // waits for the next stage to be free; 0 on abort
+      auto ring_slot = [&](uint32_t& full, uint32_t bytes) -> uint32_t {   // waits for the next stage to be free; 0 on abort
         const int s = ring_i % RD_RING;
         alive = alive && mbar_wait(smem_u32(&bars->ring_empty[s]), ((ring_i / RD_RING) & 1) ^ 1, wc, PH_ERR_LOAD);
         if (!alive) return 0u;
         full = smem_u32(&bars->ring_full[s]);
-        mbar_expect_tx(full, RD_WT_BYTES);
+        mbar_expect_tx(full, bytes);
         ++ring_i;
         return sRing + s * RD_WT_BYTES;
       };
       auto weight_load = [&](const CUtensorMap* tm, int x, int y) {
         uint32_t full = 0;
-        const uint32_t dst = ring_slot(full);
+        const uint32_t dst = ring_slot(full, RD_WT_BYTES);
         if (dst) tma_load_3d(dst, tm, full, x, y, h_idx);
       };
-      auto state_load = [&](int f) {                                // [64 features x 128 d] as two 64-column boxes
+      auto state_load = [&](int f) {                                // [64 features x d] as 64-column boxes
         uint32_t full = 0;
-        const uint32_t dst = ring_slot(full);
-        if (dst) {
-          tma_load_3d(dst, &tm_s, full, 0, f * 64, ci * g.BH + bh);
-          tma_load_3d(dst + 8192, &tm_s, full, 64, f * 64, ci * g.BH + bh);
-        }
+        const uint32_t dst = ring_slot(full, 8192u * ks1);
+        if (dst)
+          for (int ks = 0; ks < ks1; ++ks) tma_load_3d(dst + ks * 8192, &tm_s, full, ks * 64, f * 64, ci * g.BH + bh);
+      };
+      auto state_half = [&](int c) {                                // the blocks of features [128 c, 128 c + 128)
+        for (int f = 2 * c; f < 2 * c + 2 && f < nf; ++f) state_load(f);
       };
       for (int j = 0; j < n_tiles && alive; ++j) {
         alive = mbar_wait(smem_u32(&bars->x_empty), (j & 1) ^ 1, wc, PH_ERR_LOAD);
         if (!alive) break;
         const uint32_t xf = smem_u32(&bars->x_full);
-        mbar_expect_tx(xf, PH_TILE_BYTES);
-        tma_load_4d(sX, &tm_x, xf, 0, tok_a - g.q_off + j * 128, h_idx, b_idx);
-        tma_load_4d(sX + PH_SUB, &tm_x, xf, 64, tok_a - g.q_off + j * 128, h_idx, b_idx);
+        mbar_expect_tx(xf, PH_SUB * ks1);
+        for (int ks = 0; ks < ks1; ++ks)
+          tma_load_4d(sX + ks * PH_SUB, &tm_x, xf, ks * 64, tok_a - g.q_off + j * 128, h_idx, b_idx);
         ++n_x;
         // the ring follows the issue order of the MMAs: read-out of the previous tile between this tile's H halves
-        for (int ks = 0; ks < 2; ++ks) weight_load(&tm_w1, ks * 64, 0);
-        if (j > 0) { state_load(0); state_load(1); }
-        for (int ks = 0; ks < 2; ++ks) weight_load(&tm_w1, ks * 64, 128);
-        if (j > 0) { state_load(2); state_load(3); }
-        for (int ks = 0; ks < 4; ++ks) weight_load(&tm_w2, ks * 64, 0);
-        for (int ks = 0; ks < 4; ++ks) weight_load(&tm_w2, ks * 64, 128);
+        for (int ks = 0; ks < ks1; ++ks) weight_load(&tm_w1, ks * 64, 0);
+        if (j > 0) state_half(0);
+        if (nh == 2)
+          for (int ks = 0; ks < ks1; ++ks) weight_load(&tm_w1, ks * 64, 128);
+        if (j > 0 && nu == 2) state_half(1);
+        for (int half = 0; half < nu; ++half)
+          for (int ks = 0; ks < ks2; ++ks) weight_load(&tm_w2, ks * 64, half * 128);
       }
-      for (int f = 0; f < 4 && alive; ++f) state_load(f);
+      for (int c = 0; c < nu && alive; ++c) state_half(c);
       if (!alive) {
         // Given up: wait for the last load issued into every buffer before the CTA exits (the full barriers
         // complete by byte count, whatever the consumers do).
@@ -153,7 +159,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
     // ------------------------------------------------------------------ UMMA issuer
     if (elect_one()) {
       constexpr uint32_t id_kk = idesc_bf16(128, 128, 0, 0);       // A K-major (smem or TMEM), B K-major: the MLP GEMMs
-      constexpr uint32_t id_rd = idesc_bf16(128, 128, 0, 1);       // A = phi (K-major), B = state (MN-major)
+      const uint32_t id_rd = idesc_bf16(128, d, 0, 1);             // A = phi (K-major), B = state (MN-major)
       uint32_t ring_i = 0, n_epi[2] = {0, 0};
       const uint64_t d_x = smem_desc_sw128(sX, 16, 1024);
       // A wait that is given up ends the role at once: the helpers return false and run() returns, so nothing
@@ -177,7 +183,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         return true;
       };
       auto h_half = [&](int b) -> bool {                            // H[:, 128 b : 128 b + 128] = X W1[...]^T into scratch b
-        for (int ks = 0; ks < 2; ++ks) {
+        for (int ks = 0; ks < ks1; ++ks) {
           const uint32_t bt = ring_wait();
           if (!bt) return false;
           const uint64_t da = smem_desc_advance(d_x, ks * PH_SUB), db = smem_desc_sw128(bt, 16, 1024);
@@ -190,7 +196,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         return true;
       };
       auto u_half = [&](int b) -> bool {                            // U[:, 128 b : ...] = H W2[...]^T with H read from TMEM
-        for (int ks = 0; ks < 4; ++ks) {
+        for (int ks = 0; ks < ks2; ++ks) {
           const uint32_t bt = ring_wait();
           if (!bt) return false;
           const uint64_t db = smem_desc_sw128(bt, 16, 1024);
@@ -203,7 +209,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         return true;
       };
       auto readout_half = [&](int c, uint32_t phi_base) -> bool {   // R (+)= phi[:, 128 c : ...] s_t[128 c : ..., :]
-        for (int f = 0; f < 2; ++f) {
+        for (int f = 0; f < 2 && 2 * c + f < nf; ++f) {
           const uint32_t bt = ring_wait();
           if (!bt) return false;
           const uint64_t da = smem_desc_sw128(phi_base + f * PH_SUB, 16, 1024), db = smem_desc_sw128(bt, 8192, 1024);
@@ -222,22 +228,24 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
           if (j > 0) {
             if (j > 1 && !wait(&bars->out_read, (j - 2) & 1)) return; // the read-out of tile j-2 has left TMEM
             if (!readout_half(0, sPhi0)) return;
-            if (!wait_epi(1)) return;                                 // U half 1 of tile j-1
+            if (nu == 2 && !wait_epi(1)) return;                      // U half 1 of tile j-1
           }
-          if (!h_half(1)) return;
+          if (nh == 2 && !h_half(1)) return;
           umma_commit(smem_u32(&bars->x_empty));
           if (j > 0) {
-            if (!readout_half(1, sPhi1)) return;
+            if (nu == 2 && !readout_half(1, sPhi1)) return;
             umma_commit(smem_u32(&bars->out_ready));
           }
-          if (!wait_epi(0) || !wait_epi(1)) return;                   // all of H is in TMEM
-          if (!u_half(0) || !u_half(1)) return;
+          if (!wait_epi(0) || (nh == 2 && !wait_epi(1))) return;      // all of H is in TMEM
+          if (!u_half(0) || (nu == 2 && !u_half(1))) return;
         }
         if (!wait_epi(0)) return;
         if (n_tiles > 1 && !wait(&bars->out_read, (n_tiles - 2) & 1)) return;
         if (!readout_half(0, sPhi0)) return;
-        if (!wait_epi(1)) return;
-        if (!readout_half(1, sPhi1)) return;
+        if (nu == 2) {
+          if (!wait_epi(1)) return;
+          if (!readout_half(1, sPhi1)) return;
+        }
         umma_commit(smem_u32(&bars->out_ready));
       };
       run();
@@ -254,7 +262,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
     const int r = qd * 32 + lane;
     const uint32_t lane_off = (uint32_t)(qd * 32) << 16;
     uint32_t n_acc[2] = {0, 0};
-    const int part_w = PH_DP / (PC ? PC : a.P);                     // a multiple of 32 (P in {1,2,4})
+    const int part_w = Dp / (PC ? PC : a.P);                        // RELU: a multiple of 32
     // After a wait has been given up anywhere in the CTA every later wait returns at once.  These warps then run
     // through the rest of the current tile on whatever the accumulators hold (tcgen05.ld / st need all 32 lanes,
     // so nothing is skipped lane by lane; every address stays inside the CTA's TMEM and shared memory) and leave
@@ -285,12 +293,23 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         }
       } else {
         const int act = is_u ? a.act_out : a.act_hidden;
-        const int part = is_u ? col0 / part_w : 0;
+        if (GEN && is_u) {                                          // parts end anywhere; features beyond D' are zero
 #pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          const float y0 = apply_act(__uint_as_float(x[e]) + bias[e], act);
-          const float y1 = apply_act(__uint_as_float(x[e + 1]) + bias[e + 1], act);
-          w[e >> 1] = pack_bf16(poly_power(y0, part), poly_power(y1, part));
+          for (int e = 0; e < 32; e += 2) {
+            const int f0 = col0 + e;
+            const float y0 = apply_act(__uint_as_float(x[e]) + bias[e], act);
+            const float y1 = apply_act(__uint_as_float(x[e + 1]) + bias[e + 1], act);
+            w[e >> 1] = pack_bf16(f0 < Dp ? poly_power(y0, f0 / part_w) : 0.f,
+                                  f0 + 1 < Dp ? poly_power(y1, (f0 + 1) / part_w) : 0.f);
+          }
+        } else {
+          const int part = is_u ? col0 / part_w : 0;
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float y0 = apply_act(__uint_as_float(x[e]) + bias[e], act);
+            const float y1 = apply_act(__uint_as_float(x[e + 1]) + bias[e + 1], act);
+            w[e >> 1] = pack_bf16(poly_power(y0, part), poly_power(y1, part));
+          }
         }
       }
     };
@@ -307,13 +326,14 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       const float inv_nl = nl_row != 0.f ? 1.f / nl_row : 0.f;       // the read-out is stored as the ratio aL / nL
 #pragma unroll
       for (int cb = 0; cb < 2; ++cb) {
+        if (ch * 64 + cb * 32 >= d) continue;                        // the same for the whole warp
         uint32_t x[32];
         tmem_ld32(tmem + lane_off + T_R + ch * 64 + cb * 32, x);
         tmem_wait_ld();
         if (tok_valid) {
 #pragma unroll
           for (int e = 0; e < 32; e += 8)
-            rdh[rdh_index(g, a.rd_rows, PH_D, bh, ci, ric, (ch * 64 + cb * 32 + e) >> 3)] =
+            rdh[rdh_index(g, a.rd_rows, d, bh, ci, ric, (ch * 64 + cb * 32 + e) >> 3)] =
                 make_uint4(pack_ratio_f16(__uint_as_float(x[e]) * inv_nl, __uint_as_float(x[e + 1]) * inv_nl),
                            pack_ratio_f16(__uint_as_float(x[e + 2]) * inv_nl, __uint_as_float(x[e + 3]) * inv_nl),
                            pack_ratio_f16(__uint_as_float(x[e + 4]) * inv_nl, __uint_as_float(x[e + 5]) * inv_nl),
@@ -321,7 +341,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         }
       }
       if (tok_valid && ch == 1)
-        rdh[rdh_index(g, a.rd_rows, PH_D, bh, ci, ric, rdh_pieces(PH_D) - 1)] = make_uint4(__float_as_uint(nl_row), 0u, 0u, 0u);
+        rdh[rdh_index(g, a.rd_rows, d, bh, ci, ric, rdh_pieces(d) - 1)] = make_uint4(__float_as_uint(nl_row), 0u, 0u, 0u);
       tc_fence_before();
       mbar_arrive_warp(smem_u32(&bars->out_read), lane);
     };
@@ -331,6 +351,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       // H halves: bias, activation, bf16, back to TMEM as the A operand of the second GEMM
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
+        if (half >= nh) continue;                                   // a width of at most 128 has no second half
         wait(&bars->acc_ready[half], n_acc[half] & 1);
         ++n_acc[half];
         tc_fence_after();
@@ -354,6 +375,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       float nl = 0.f;
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
+        if (half >= nu) continue;
         wait(&bars->acc_ready[half], n_acc[half] & 1);
         ++n_acc[half];
         tc_fence_after();
@@ -385,7 +407,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
             st_tile_chunk_sw128(dst, PH_SUB, r, ch * 64 + cb * 32 + e, w4);
           }
         }
-        if (half == 1) {
+        if (half == nu - 1) {
           // The buffer alternates with the tile.  It is free: its last reader (read-out store of tile j-2)
           // precedes, for every thread, that thread's arrival for U half 0 of tile j-1, which the issuer
           // waited for before the MMAs of this tile could start.

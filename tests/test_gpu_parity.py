@@ -42,6 +42,7 @@ def run_gpu(wl, x, *, impl="auto", c_mode="rowmax", layout="bhnd", **kw):
     if layout == "bnhd":
         y = y.transpose(1, 2)
     used = op.last_impl
+    run_gpu.phi_kernels = op.last_phi_impl          # kernels of phi, state and read-out in this call
     op.close()
     return y.double().cpu().numpy(), used
 
@@ -126,7 +127,7 @@ def test_small_cases_every_element(case, c_mode):
     x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
     ref, frac = oracle_full(wl, x, c_mode)
     y, used = run_gpu(wl, x, c_mode=c_mode)
-    assert used == ("tensor" if dtype == "bf16" else "simt")    # bf16: the softmax window runs on the tensor cores for d = 64 and 128
+    assert used == run_gpu.phi_kernels == ("tensor" if dtype == "bf16" else "simt")   # bf16: every step on the tensor cores, d = 64 and 128
     check(y, ref, dtype)
     if To < T - Tc and c_mode == "rowmax":
         assert frac.max() > 0.05
@@ -253,13 +254,17 @@ def test_host_buffer_entry_point_matches_device_entry_point():
 
 # ------------------------------------------------------------------ other feature maps (activations, degree, widths)
 PHI_VARIANTS = [
-    # id, P, act_hidden, act_out, phi_hidden, phi_dim, kernels expected for bf16 d=128
+    # id, P, act_hidden, act_out, phi_hidden, phi_dim, kernels of phi, state and read-out expected for bf16
     ("degree1_relu", 1, "relu", "relu", 0, 0, "tensor"),
     ("degree4_relu", 4, "relu", "relu", 0, 0, "tensor"),
     ("degree2_gelu_softplus", 2, "gelu", "softplus", 0, 0, "tensor"),
     ("degree2_identity_elu1", 2, "identity", "elu1", 0, 0, "tensor"),
-    ("degree3_width192", 3, "relu", "relu", 128, 192, "tensor"),      # phi on the SIMT kernels, window on the tensor cores
-    ("degree2_narrow", 2, "relu", "softplus", 64, 96, "tensor"),
+    ("degree3_width192", 3, "relu", "relu", 128, 192, "tensor"),      # one half of H, one and a half of U; parts of 64
+    ("degree2_narrow", 2, "relu", "softplus", 64, 96, "tensor"),      # parts of 48 features: they end inside a 32-column block
+    ("degree3_relu_parts_of_32", 3, "relu", "relu", 192, 96, "tensor"),
+    ("degree4_hidden96_width128", 4, "gelu", "relu", 96, 128, "tensor"),   # K extent of the second GEMM ends inside a 64-column block
+    ("degree2_hidden256_width64", 2, "relu", "elu1", 0, 64, "tensor"),
+    ("degree2_widths_not_multiples_of_32", 2, "relu", "relu", 72, 104, "simt"),
 ]
 
 
@@ -275,8 +280,25 @@ def test_other_feature_maps(variant, dtype):
     ref = orc.hybrid_direct(f["q"], f["k"], f["v"], f["phi_q"], f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To, P=P,
                             act_hidden=ah, act_out=ao)
     y, used = run_gpu(wl, x, act_hidden=ah, act_out=ao)
-    assert used == (expect if dtype == "bf16" else "simt")
+    assert used == ("tensor" if dtype == "bf16" else "simt")
+    assert run_gpu.phi_kernels == (expect if dtype == "bf16" else "simt")
     check(y, ref, dtype)
+
+
+@pytest.mark.parametrize("variant", [v for v in PHI_VARIANTS if v[6] == "tensor"], ids=[v[0] for v in PHI_VARIANTS if v[6] == "tensor"])
+def test_other_feature_maps_with_heads_of_64(variant):
+    """The same maps on heads of 64 channels (bf16): half the K extent of the first GEMM, 64-column state and
+    read-out accumulators.  Default widths are 2 d = 128 here."""
+    _, P, ah, ao, Dh, Dp, _ = variant
+    wl = synth.Workload("phi64", 1, 3, 64, 5, 10, 20, 2, 1, "bf16", True, P=P, seed=synth.BASE_SEED + 87,
+                        phi_hidden=Dh, phi_dim=Dp)
+    x = synth.make_inputs(wl, phi_scale=1.5 if ao == "relu" else 1.0, v_frame_offsets=True)
+    f = synth.to_f64(x)
+    ref = orc.hybrid_direct(f["q"], f["k"], f["v"], f["phi_q"], f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To, P=P,
+                            act_hidden=ah, act_out=ao)
+    y, used = run_gpu(wl, x, act_hidden=ah, act_out=ao)
+    assert used == run_gpu.phi_kernels == "tensor"
+    check(y, ref, "bf16")
 
 
 @pytest.mark.parametrize("layers", [3, 4])
@@ -296,7 +318,7 @@ def test_deeper_feature_maps(layers, dtype):
     two = {n: t for n, t in f["phi_q"].items() if n not in ("Wmid", "bmid")}
     assert np.abs(orc.hybrid_direct(f["q"], f["k"], f["v"], two, f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To) - ref).max() > 1e-2
     y, used = run_gpu(wl, x)
-    assert used == ("tensor" if dtype == "bf16" else "simt")
+    assert used == ("tensor" if dtype == "bf16" else "simt") and run_gpu.phi_kernels == "simt"
     check(y, ref, dtype)
 
 
