@@ -252,7 +252,8 @@ int run_parts(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void
     } else {
       if (parts & PART_STATE) {
         ctx->prof.begin(REHYAT_PROF_STATE, st);
-        rc = tc_launch_state(&ctx->tc, k, v, phi, g, batch, c.phi_hidden, c.phi_dim, c.poly_degree, c.act_hidden, c.act_out, n_split,
+        rc = tc_launch_state(&ctx->tc, k, v, phi, g, batch, c.phi_hidden, c.phi_dim, c.poly_degree,
+                             c.phi_layers > 2 ? c.phi_layers - 2 : 0, c.act_hidden, c.act_out, n_split,
                              ctx->partial, next_wait(ctx), st);
         ctx->prof.end(REHYAT_PROF_STATE, st);
         const size_t per_slot = (size_t)g.BH * c.phi_dim * (c.head_dim + 4);
@@ -264,7 +265,8 @@ int run_parts(rehyat_ctx* ctx, const void* q, const void* k, const void* v, void
       }
       if (rc == REHYAT_OK && (parts & PART_READOUT)) {
         ctx->prof.begin(REHYAT_PROF_READOUT, st);
-        rc = tc_launch_readout(&ctx->tc, q, phi, g, batch, c.phi_hidden, c.phi_dim, c.poly_degree, c.act_hidden, c.act_out, ctx->state,
+        rc = tc_launch_readout(&ctx->tc, q, phi, g, batch, c.phi_hidden, c.phi_dim, c.poly_degree,
+                               c.phi_layers > 2 ? c.phi_layers - 2 : 0, c.act_hidden, c.act_out, ctx->state,
                                ctx->readout, ctx->rd_cap, next_wait(ctx), st);
         ctx->prof.end(REHYAT_PROF_READOUT, st);
         ctx->last_launches += 1;
@@ -401,8 +403,8 @@ int rehyat_create(rehyat_ctx** out, const rehyat_config* cfg) {
                                       c.poly_degree, c.act_hidden, c.act_out);
   if ((c.impl == REHYAT_IMPL_TENSOR || c.impl == REHYAT_IMPL_TENSOR_WINDOW) && !ctx->tensor_ok) { delete ctx; return REHYAT_ERR_UNSUPPORTED; }
   if (c.impl == REHYAT_IMPL_SIMT) ctx->tensor_ok = false;
-  ctx->tc.phi_ok = ctx->tensor_ok && c.impl != REHYAT_IMPL_TENSOR_WINDOW && c.phi_layers <= 2 &&
-                   tc_phi_supported(c.head_dim, c.phi_hidden, c.phi_dim, c.poly_degree);
+  ctx->tc.phi_ok = ctx->tensor_ok && c.impl != REHYAT_IMPL_TENSOR_WINDOW &&
+                   tc_phi_supported(c.head_dim, c.phi_hidden, c.phi_dim, c.poly_degree, c.phi_layers > 2 ? c.phi_layers - 2 : 0);
   ctx->tc.head_dim = c.head_dim;
 
   const int np_max = c.max_tokens_per_frame * c.max_chunk_frames;

@@ -19,6 +19,9 @@
 // extent of the state GEMM, a width of at most 128 drops the second half of its GEMM, and a width that is not
 // a multiple of 128 (or 64) relies on the tensor maps, which read rows and columns beyond the matrix as zero:
 // hidden units beyond D_h meet zero columns of W2, features beyond D' are zero (or masked) and never stored.
+// A map of more than two layers (GEN only) runs its hidden layers h <- act(Wmid h + bmid) between the two: the
+// hidden activations alternate between the H buffer and a second one made of the X tile and the phi half 0
+// tile, both idle at that point (the next X tile is then requested later, after the last reader of that buffer).
 #pragma once
 
 #include <cuda.h>
@@ -41,8 +44,9 @@ constexpr int PH_OFF_HB = PH_OFF_V + PH_TILE_BYTES;            // 64 KB; its fir
 constexpr int PH_OFF_PHI0 = PH_OFF_HB + 2 * PH_TILE_BYTES;
 constexpr int PH_OFF_RING = PH_OFF_PHI0 + PH_TILE_BYTES;
 constexpr int PH_OFF_ONES = PH_OFF_RING + PH_RING * PH_WT_BYTES; // [16 x 128] K-major, row 0 = 1
-constexpr int PH_OFF_BIAS = PH_OFF_ONES + 4096;                 // b1[256], b2[256] fp32
-constexpr int PH_OFF_BARS = PH_OFF_BIAS + 2 * 256 * 4;
+constexpr int PH_OFF_BIAS = PH_OFF_ONES + 4096;                 // b1[256], b2[256], bmid[2][256] fp32
+constexpr int PH_MAX_MID = 2;                                   // hidden layers between the first and the last
+constexpr int PH_OFF_BARS = PH_OFF_BIAS + (2 + PH_MAX_MID) * 256 * 4;
 constexpr int PH_SMEM = PH_OFF_BARS + 512 + 1024;
 
 enum PhErr : int { PH_ERR_LOAD = 16, PH_ERR_MMA = 32, PH_ERR_EPI = 64 };
@@ -61,6 +65,8 @@ struct PhiTcArgs {
   const __nv_bfloat16* b2;     // [heads][D']
   int P, act_hidden, act_out;
   int d, Dh, Dp;               // head_dim (64 or 128), phi widths (read by the GEN = true kernels)
+  int n_mid;                   // hidden layers between the first and the last (GEN = true kernels), at most PH_MAX_MID
+  const __nv_bfloat16* bm;     // [heads][n_mid][D_h]
   int n_split;                 // state kernel: splits of a chunk's increment
   float* partial;              // state kernel: [G][n_split][BH][D'][d + 4]
   const float* state;          // read-out kernel: fp32 states (z column is read)
@@ -73,8 +79,9 @@ struct PhiTcArgs {
 // Extents of one launch: constants for the default shape, read from the arguments otherwise.
 template <bool GEN>
 struct PhiExtents {
-  int d, Dh, Dp;
-  __device__ explicit PhiExtents(const PhiTcArgs& a) : d(GEN ? a.d : PH_D), Dh(GEN ? a.Dh : PH_DH), Dp(GEN ? a.Dp : PH_DP) {}
+  int d, Dh, Dp, n_mid;
+  __device__ explicit PhiExtents(const PhiTcArgs& a)
+      : d(GEN ? a.d : PH_D), Dh(GEN ? a.Dh : PH_DH), Dp(GEN ? a.Dp : PH_DP), n_mid(GEN ? a.n_mid : 0) {}
   __device__ int sd() const { return d + 4; }              // row of a state: d columns of s, then z, padded
   __device__ int ks1() const { return d / 64; }            // 64-column K blocks of the first GEMM
   __device__ int ks2() const { return (Dh + 63) / 64; }    // ... of the second
@@ -83,11 +90,13 @@ struct PhiExtents {
 };
 
 // tm_x: K, tm_v: V, 4-D like the window kernel's maps.  tm_w1: (d, D_h, heads), tm_w2: (D_h, D', heads),
-// boxes [64 x 128].  PC: polynomial degree known at compile time (0: read it from the arguments; 2 needs D' = 256).
+// tm_wm: (D_h, D_h, heads * n_mid) (any valid map when n_mid = 0), boxes [64 x 128].  PC: polynomial degree known
+// at compile time (0: read it from the arguments; 2 needs D' = 256).
 template <bool RELU, int PC, bool GEN>
 __global__ void __launch_bounds__(PH_THREADS, 1)
 phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_v,
-       const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2, Geo g, PhiTcArgs a) {
+       const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2,
+       const __grid_constant__ CUtensorMap tm_wm, Geo g, PhiTcArgs a) {
   using namespace ptx;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sb = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -101,7 +110,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   const int ci = blockIdx.y, bh = blockIdx.z, t = g.t0 + ci;
   const int b_idx = bh / g.n_heads, h_idx = bh % g.n_heads;
   const PhiExtents<GEN> ex(a);
-  const int Dp = ex.Dp, SD = ex.sd(), ks1 = ex.ks1(), ks2 = ex.ks2(), nh = ex.nh(), nu = ex.nu();
+  const int Dp = ex.Dp, SD = ex.sd(), ks1 = ex.ks1(), ks2 = ex.ks2(), nh = ex.nh(), nu = ex.nu(), n_mid = ex.n_mid;
 
   // token range [tok_a, tok_b) of this CTA
   const int lo_prev = t > 0 ? geo_lo(g, t - 1) : 0, lo = geo_lo(g, t);
@@ -134,6 +143,8 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   for (int i = threadIdx.x; i < 256; i += PH_THREADS) {          // zero beyond the widths
     s_b1[i] = i < ex.Dh ? __bfloat162float(a.b1[(size_t)h_idx * ex.Dh + i]) : 0.f;
     s_b2[i] = i < Dp ? __bfloat162float(a.b2[(size_t)h_idx * Dp + i]) : 0.f;
+    for (int m = 0; m < n_mid; ++m)
+      s_b2[(1 + m) * 256 + i] = i < ex.Dh ? __bfloat162float(a.bm[((size_t)h_idx * n_mid + m) * ex.Dh + i]) : 0.f;
   }
   {
     uint32_t* ones = reinterpret_cast<uint32_t*>(smem + PH_OFF_ONES);
@@ -158,11 +169,19 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   const uint32_t sX = sb + PH_OFF_X, sV = sb + PH_OFF_V, sHb = sb + PH_OFF_HB, sPhi0 = sb + PH_OFF_PHI0,
                  sRing = sb + PH_OFF_RING, sOnes = sb + PH_OFF_ONES;
   auto ring_addr = [&](int s) -> uint32_t { return sRing + s * PH_WT_BYTES; };
+  // The two buffers of hidden activations, each four [128 x 64] sub-tiles: 0 = the H buffer, 1 = the X tile
+  // followed by the phi half 0 tile.  The first layer writes buffer 0, hidden layer m reads m % 2 and writes the other.
+  auto hid_sub = [&](int buf, int sub) -> uint32_t {
+    return buf == 0 ? sHb + sub * PH_SUB : (sub < 2 ? sX + sub * PH_SUB : sPhi0 + (sub - 2) * PH_SUB);
+  };
+  const int last_hid = n_mid & 1;                                   // where the last hidden activations are
+  const uint32_t sPhiHalf0 = last_hid ? sHb + 2 * PH_SUB : sPhi0;   // phi half 0: away from the buffer the last GEMMs read
 
   if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
     if (elect_one() && !a.wa.withhold_loads) {
       prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_w1); prefetch_tensormap(&tm_w2);
+      if (n_mid > 0) prefetch_tensormap(&tm_wm);
       uint32_t ring_i = 0, n_x = 0, n_v = 0;                       // ring tiles, X tiles and V tiles issued so far
       bool alive = true;
       auto ring_load = [&](const CUtensorMap* tm, int x, int y, int z) {
@@ -185,6 +204,9 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
         ++n_x;
         for (int half = 0; half < nh; ++half)
           for (int ks = 0; ks < ks1; ++ks) ring_load(&tm_w1, ks * 64, half * 128, h_idx);
+        for (int m = 0; m < n_mid; ++m)
+          for (int half = 0; half < nh; ++half)
+            for (int ks = 0; ks < ks2; ++ks) ring_load(&tm_wm, ks * 64, half * 128, h_idx * n_mid + m);
         {
           alive = alive && mbar_wait(smem_u32(&bars->v_empty), (j & 1) ^ 1, wc, PH_ERR_LOAD);
           if (!alive) break;
@@ -229,10 +251,11 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
         ++n_epi;
         return true;
       };
-      // one 128x128 half of an MLP GEMM: A tile [128 x 64*nks] K-major at a_base, B tiles from the ring
-      auto mlp_half = [&](uint32_t a_base, int nks) -> bool {
-        uint64_t da = smem_desc_sw128(a_base, 16, 1024);             // advanced by one 64-column sub-tile per ring tile
-        for (int ks = 0; ks < nks; ++ks, da = smem_desc_advance(da, PH_SUB)) {
+      // one 128x128 half of an MLP GEMM: A = the X tile (buf < 0) or a buffer of hidden activations, [128 x 64*nks]
+      // K-major in 64-column sub-tiles, B tiles from the ring
+      auto mlp_half = [&](int buf, int nks) -> bool {
+        for (int ks = 0; ks < nks; ++ks) {
+          const uint64_t da = smem_desc_sw128(buf < 0 ? sX + ks * PH_SUB : hid_sub(buf, ks), 16, 1024);
           if (!wait(&bars->ring_full[ring_i % RING], (ring_i / RING) & 1)) return false;
           const uint64_t db = smem_desc_sw128(ring_addr(ring_i % RING), 16, 1024);
 #pragma unroll
@@ -264,16 +287,25 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
             consume_half(1, sHb, j == 1);
             umma_commit(smem_u32(&bars->v_empty));
           }
-          if (!mlp_half(sX, ks1)) return;                             // H[:, 0:128]
+          if (!mlp_half(-1, ks1)) return;                             // H[:, 0:128]
           if (!wait_epi()) return;
-          if (nh == 2 && !mlp_half(sX, ks1)) return;                  // H[:, 128:256]
-          umma_commit(smem_u32(&bars->x_empty));
+          if (nh == 2 && !mlp_half(-1, ks1)) return;                  // H[:, 128:256]
+          // The X tile is free after its last reader: the first layer, or the last GEMMs that read hidden buffer 1.
+          if (n_mid == 0) umma_commit(smem_u32(&bars->x_empty));
           if (nh == 2 && !wait_epi()) return;
-          if (!mlp_half(sHb, ks2)) return;                            // U[:, 0:128]
+          for (int m = 0; m < n_mid; ++m) {                           // hidden layer m: buffer m % 2 -> the other
+            if (!mlp_half(m & 1, ks2)) return;
+            if (!wait_epi()) return;
+            if (nh == 2 && !mlp_half(m & 1, ks2)) return;
+            if (m == n_mid - 1 && last_hid == 0) umma_commit(smem_u32(&bars->x_empty));
+            if (nh == 2 && !wait_epi()) return;
+          }
+          if (!mlp_half(last_hid, ks2)) return;                       // U[:, 0:128]
           if (!wait_epi()) return;
-          if (nu == 2 && !mlp_half(sHb, ks2)) return;                 // U[:, 128:256]
+          if (nu == 2 && !mlp_half(last_hid, ks2)) return;            // U[:, 128:256]
+          if (last_hid == 1) umma_commit(smem_u32(&bars->x_empty));
           if (!wait(&bars->v_full, j & 1)) return;
-          consume_half(0, sPhi0, j == 0);
+          consume_half(0, sPhiHalf0, j == 0);
           if (nu == 1) umma_commit(smem_u32(&bars->v_empty));         // no second half: V is free once these have run
         }
         if (nu == 2) {
@@ -303,20 +335,14 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
     // at the head of the next tile, where the whole warp looks at the flag together.
     auto aborted = [&]() -> bool { return __any_sync(0xffffffffu, wait_ctx_aborted(wc) != 0); };
     auto wait = [&](uint64_t* bar, uint32_t parity) { mbar_wait(smem_u32(bar), parity, wc, PH_ERR_EPI); };
-    for (int j = 0; j < n_tiles; ++j) {
-      if (aborted()) break;
-      const bool tok_valid = tok_a + j * 128 + r < tok_b;
-#pragma unroll
-      for (int step = 0; step < 4; ++step) {                        // H half 0, H half 1, U half 0, U half 1
-        const int half = step & 1;
-        const bool is_u = step >= 2;
-        if (half >= (is_u ? nu : nh)) continue;                     // a width of at most 128 has no second half
+    bool tok_valid = false;
+    // One 128-column half of a layer leaves the scratch accumulator: bias (`bias` points at this half's first
+    // column), activation, for the last layer (is_u) the power of its polynomial part, bf16, into columns
+    // [64 ch, 64 ch + 64) of the half's destination, the swizzled [128 x 64] sub-tile at dst_sub.
+    auto epi_step = [&](const bool is_u, const int half, const float* bias, const uint32_t dst_sub) {
         wait(&bars->acc_ready, n_acc & 1);
         ++n_acc;
         tc_fence_after();
-        const uint32_t dst = !is_u ? sHb : (half == 0 ? sPhi0 : sHb);
-        const int dst_col0 = !is_u ? half * 128 : 0;
-        const float* bias = (is_u ? s_b2 : s_b1) + half * 128;
         uint32_t x[2][32];
         tmem_ld32(tmem + lane_off + T_SCR + ch * 64, x[0]);
         tmem_ld32(tmem + lane_off + T_SCR + ch * 64 + 32, x[1]);
@@ -373,13 +399,27 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
 #pragma unroll
           for (int e = 0; e < 32; e += 8) {
             const uint4 w4 = make_uint4(w[e >> 1], w[(e >> 1) + 1], w[(e >> 1) + 2], w[(e >> 1) + 3]);
-            st_tile_chunk_sw128(dst, PH_SUB, r, dst_col0 + col0 + e, w4);
+            st_tile_chunk_sw128(dst_sub, PH_SUB, r, cb * 32 + e, w4);
           }
         }
         fence_proxy_async_smem();
         tc_fence_before();
         mbar_arrive_warp(smem_u32(&bars->epi_done), lane);
-      }
+    };
+    for (int j = 0; j < n_tiles; ++j) {
+      if (aborted()) break;
+      tok_valid = tok_a + j * 128 + r < tok_b;
+      // a width of at most 128 has no second half
+#pragma unroll
+      for (int half = 0; half < 2; ++half)                          // first layer -> hidden buffer 0
+        if (half < nh) epi_step(false, half, s_b1 + half * 128, hid_sub(0, half * 2 + ch));
+      for (int m = 0; m < n_mid; ++m)                               // hidden layer m -> the buffer it does not read
+#pragma unroll
+        for (int half = 0; half < 2; ++half)
+          if (half < nh) epi_step(false, half, s_b2 + (1 + m) * 256 + half * 128, hid_sub((m & 1) ^ 1, half * 2 + ch));
+#pragma unroll
+      for (int half = 0; half < 2; ++half)                          // last layer -> the phi tiles
+        if (half < nu) epi_step(true, half, s_b2 + half * 128, (half == 0 ? sPhiHalf0 : sHb) + ch * PH_SUB);
     }
     wait(&bars->out_ready, 0);
     if (!aborted()) {

@@ -27,8 +27,8 @@ constexpr int RD_OFF_X = 0;
 constexpr int RD_OFF_PHI0 = RD_OFF_X + PH_TILE_BYTES;
 constexpr int RD_OFF_PHI1 = RD_OFF_PHI0 + PH_TILE_BYTES;
 constexpr int RD_OFF_RING = RD_OFF_PHI1 + PH_TILE_BYTES;
-constexpr int RD_OFF_BIAS = RD_OFF_RING + RD_RING * RD_WT_BYTES;  // b1[256], b2[256], z[256], two partial phi.z sums per token (x2: by tile parity)
-constexpr int RD_OFF_BARS = RD_OFF_BIAS + 5 * 256 * 4;
+constexpr int RD_OFF_BIAS = RD_OFF_RING + RD_RING * RD_WT_BYTES;  // b1[256], b2[256], z[256], two partial phi.z sums per token (x2: by tile parity), bmid[2][256]
+constexpr int RD_OFF_BARS = RD_OFF_BIAS + (5 + PH_MAX_MID) * 256 * 4;
 constexpr int RD_SMEM = RD_OFF_BARS + 512 + 1024;
 
 struct RdBars {
@@ -41,13 +41,16 @@ struct RdBars {
   ptx::WaitCtx wctx;
 };
 
-// tm_x: Q, 4-D like the window kernel's maps.  tm_w1: (d, D_h, heads), tm_w2: (D_h, D', heads), boxes
-// [64 x 128].  tm_s: bf16 states (d, D', G*BH), box [64 x 64].  PC: polynomial degree known at compile time
-// (0: read it from the arguments; 2 needs D' = 256).
+// tm_x: Q, 4-D like the window kernel's maps.  tm_w1: (d, D_h, heads), tm_w2: (D_h, D', heads), tm_wm: (D_h, D_h,
+// heads * n_mid) (any valid map when n_mid = 0), boxes [64 x 128].  tm_s: bf16 states (d, D', G*BH), box [64 x 64].
+// PC: polynomial degree known at compile time (0: read it from the arguments; 2 needs D' = 256).
+// A hidden layer of a deeper map (GEN only) reads H from TMEM and writes it back there: both halves of its GEMM
+// have completed before the first column of H is overwritten.
 template <bool RELU, int PC, bool GEN>
 __global__ void __launch_bounds__(PH_THREADS, 1)
 readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w1,
-           const __grid_constant__ CUtensorMap tm_w2, const __grid_constant__ CUtensorMap tm_s, Geo g, PhiTcArgs a) {
+           const __grid_constant__ CUtensorMap tm_w2, const __grid_constant__ CUtensorMap tm_wm,
+           const __grid_constant__ CUtensorMap tm_s, Geo g, PhiTcArgs a) {
   using namespace ptx;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sb = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -57,6 +60,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
   float* s_b2 = s_b1 + 256;
   float* s_z = s_b2 + 256;
   float* s_nl = s_z + 256;
+  float* s_bm = s_nl + 512;
   const uint32_t wc = smem_u32(&bars->wctx);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -66,6 +70,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
   const PhiExtents<GEN> ex(a);
   const int d = ex.d, Dp = ex.Dp, SD = ex.sd(), ks1 = ex.ks1(), ks2 = ex.ks2(), nh = ex.nh(), nu = ex.nu();
   const int nf = (Dp + 63) / 64;                                    // 64-feature blocks of the state
+  const int n_mid = ex.n_mid;
   const int q0 = geo_q0(g, t), q1 = geo_q1(g, t);
   const int tok_a = min(q0 + (int)blockIdx.x * a.tiles_per_cta * 128, q1);
   const int tok_b = min(tok_a + a.tiles_per_cta * 128, q1);
@@ -87,6 +92,8 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
     s_b1[i] = i < ex.Dh ? __bfloat162float(a.b1[(size_t)h_idx * ex.Dh + i]) : 0.f;
     s_b2[i] = i < Dp ? __bfloat162float(a.b2[(size_t)h_idx * Dp + i]) : 0.f;
     s_z[i] = i < Dp ? a.state[(((size_t)ci * g.BH + bh) * Dp + i) * SD + d] : 0.f;
+    for (int m = 0; m < n_mid; ++m)
+      s_bm[m * 256 + i] = i < ex.Dh ? __bfloat162float(a.bm[((size_t)h_idx * n_mid + m) * ex.Dh + i]) : 0.f;
   }
   if (warp == 9) {
     tmem_alloc(smem_u32(&bars->tmem_base), 512);
@@ -103,6 +110,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
     // ------------------------------------------------------------------ TMA producer
     if (elect_one() && !a.wa.withhold_loads) {
       prefetch_tensormap(&tm_x); prefetch_tensormap(&tm_w1); prefetch_tensormap(&tm_w2); prefetch_tensormap(&tm_s);
+      if (n_mid > 0) prefetch_tensormap(&tm_wm);
       uint32_t ring_i = 0, n_x = 0;                                 // ring tiles and X tiles issued so far
       bool alive = true;
       auto ring_slot = [&](uint32_t& full, uint32_t bytes) -> uint32_t {   // waits for the next stage to be free; 0 on abort
@@ -114,10 +122,10 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         ++ring_i;
         return sRing + s * RD_WT_BYTES;
       };
-      auto weight_load = [&](const CUtensorMap* tm, int x, int y) {
+      auto weight_load = [&](const CUtensorMap* tm, int x, int y, int plane) {
         uint32_t full = 0;
         const uint32_t dst = ring_slot(full, RD_WT_BYTES);
-        if (dst) tma_load_3d(dst, tm, full, x, y, h_idx);
+        if (dst) tma_load_3d(dst, tm, full, x, y, plane);
       };
       auto state_load = [&](int f) {                                // [64 features x d] as 64-column boxes
         uint32_t full = 0;
@@ -137,13 +145,16 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
           tma_load_4d(sX + ks * PH_SUB, &tm_x, xf, ks * 64, tok_a - g.q_off + j * 128, h_idx, b_idx);
         ++n_x;
         // the ring follows the issue order of the MMAs: read-out of the previous tile between this tile's H halves
-        for (int ks = 0; ks < ks1; ++ks) weight_load(&tm_w1, ks * 64, 0);
+        for (int ks = 0; ks < ks1; ++ks) weight_load(&tm_w1, ks * 64, 0, h_idx);
         if (j > 0) state_half(0);
         if (nh == 2)
-          for (int ks = 0; ks < ks1; ++ks) weight_load(&tm_w1, ks * 64, 128);
+          for (int ks = 0; ks < ks1; ++ks) weight_load(&tm_w1, ks * 64, 128, h_idx);
         if (j > 0 && nu == 2) state_half(1);
+        for (int m = 0; m < n_mid; ++m)
+          for (int half = 0; half < nh; ++half)
+            for (int ks = 0; ks < ks2; ++ks) weight_load(&tm_wm, ks * 64, half * 128, h_idx * n_mid + m);
         for (int half = 0; half < nu; ++half)
-          for (int ks = 0; ks < ks2; ++ks) weight_load(&tm_w2, ks * 64, half * 128);
+          for (int ks = 0; ks < ks2; ++ks) weight_load(&tm_w2, ks * 64, half * 128, h_idx);
       }
       for (int c = 0; c < nu && alive; ++c) state_half(c);
       if (!alive) {
@@ -237,6 +248,10 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
             umma_commit(smem_u32(&bars->out_ready));
           }
           if (!wait_epi(0) || (nh == 2 && !wait_epi(1))) return;      // all of H is in TMEM
+          for (int m = 0; m < n_mid; ++m) {                           // hidden layers: H -> scratch -> H
+            if (!u_half(0) || (nh == 2 && !u_half(1))) return;
+            if (!wait_epi(0) || (nh == 2 && !wait_epi(1))) return;
+          }
           if (!u_half(0) || (nu == 2 && !u_half(1))) return;
         }
         if (!wait_epi(0)) return;
@@ -371,6 +386,34 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         mbar_arrive_warp(smem_u32(&bars->epi_done[half]), lane);
       }
       if (j > 0) readout_store(j - 1);
+      // hidden layers of a deeper map: both halves of the GEMM are complete before H is overwritten
+      for (int m = 0; m < n_mid; ++m) {
+        wait(&bars->acc_ready[0], n_acc[0] & 1);
+        ++n_acc[0];
+        if (nh == 2) {
+          wait(&bars->acc_ready[1], n_acc[1] & 1);
+          ++n_acc[1];
+        }
+        tc_fence_after();
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          if (half >= nh) continue;
+          uint32_t x[2][32];
+          tmem_ld32(tmem + lane_off + T_SCR + half * 128 + ch * 64, x[0]);
+          tmem_ld32(tmem + lane_off + T_SCR + half * 128 + ch * 64 + 32, x[1]);
+          tmem_wait_ld();
+#pragma unroll
+          for (int cb = 0; cb < 2; ++cb) {
+            const int col0 = half * 128 + ch * 64 + cb * 32;
+            uint32_t w[16];
+            activate(x[cb], s_bm + m * 256 + col0, false, col0, w);
+            tmem_st16(tmem + lane_off + T_H + (col0 >> 1), w);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive_warp(smem_u32(&bars->epi_done[half]), lane);
+        }
+      }
       // U halves: bias, activation, power, bf16, to the swizzled phi tiles; phi . z_t on the way
       float nl = 0.f;
 #pragma unroll

@@ -487,16 +487,17 @@ struct TcWorkspace {
 
 inline bool tc_shape_supported(bool bf16, int d, int, int, int, int, int) { return bf16 && (d == 128 || d == 64); }
 // The phi kernels: head_dim 64 or 128, widths that are multiples of 32 between 64 (32 for D') and 256.
-inline bool tc_phi_supported(int d, int Dh, int Dp, int P) {
+// Up to PH_MAX_MID hidden layers between the first and the last.
+inline bool tc_phi_supported(int d, int Dh, int Dp, int P, int n_mid) {
   return (d == 64 || d == 128) && Dh >= 64 && Dh <= PH_DH && Dh % 32 == 0 && Dp >= 32 && Dp <= PH_DP && Dp % 32 == 0 &&
-         P >= 1 && Dp % P == 0;
+         P >= 1 && Dp % P == 0 && n_mid >= 0 && n_mid <= PH_MAX_MID;
 }
-// Which instantiation serves a map: the fixed-shape kernels for 128 / 256 / 256, the ones that read their
-// extents otherwise; the ReLU fast path needs polynomial parts that end on 32-column blocks.
+// Which instantiation serves a map: the fixed-shape kernels for the two-layer map of 128 / 256 / 256, the ones
+// that read their extents otherwise; the ReLU fast path needs polynomial parts that end on 32-column blocks.
 struct PhiKernelChoice { bool gen, relu; int pc; };
-inline PhiKernelChoice tc_phi_choice(int d, int Dh, int Dp, int P, int act_hidden, int act_out) {
+inline PhiKernelChoice tc_phi_choice(int d, int Dh, int Dp, int P, int n_mid, int act_hidden, int act_out) {
   PhiKernelChoice c;
-  c.gen = !(d == PH_D && Dh == PH_DH && Dp == PH_DP);
+  c.gen = !(d == PH_D && Dh == PH_DH && Dp == PH_DP && n_mid == 0);
   c.relu = act_hidden == ACT_RELU && act_out == ACT_RELU && (Dp / P) % 32 == 0;
   c.pc = (!c.gen && c.relu && P == 2) ? 2 : 0;
   return c;
@@ -624,22 +625,24 @@ inline int tc_launch_window(TcWorkspace* w, const void* q, const void* k, const 
 
 // phi_k + chunk-state partial sums of one group (Eq. 17-18).
 inline int tc_launch_state(const TcWorkspace* w, const void* k, const void* v, const rehyat_phi_params* phi,
-                           const Geo& g, int batch, int Dh, int Dp, int P, int act_hidden, int act_out, int n_split,
-                           float* partial, const ptx::WaitArgs& wa, cudaStream_t st) {
+                           const Geo& g, int batch, int Dh, int Dp, int P, int n_mid, int act_hidden, int act_out,
+                           int n_split, float* partial, const ptx::WaitArgs& wa, cudaStream_t st) {
   const int d = w->head_dim;
-  CUtensorMap tk, tv, tw1, tw2;
+  CUtensorMap tk, tv, tw1, tw2, twm;
   if (!tc_make_tmap(w, &tk, k, g, batch) || !tc_make_tmap(w, &tv, v, g, batch) ||
       !tc_make_tmap_3d(w, &tw1, phi->k_W1, d, Dh, g.n_heads, 128) ||
       !tc_make_tmap_3d(w, &tw2, phi->k_W2, Dh, Dp, g.n_heads, 128))
     return REHYAT_ERR_CUDA;
+  twm = tw2;                                                        // not read without hidden layers in between
+  if (n_mid > 0 && !tc_make_tmap_3d(w, &twm, phi->k_Wmid, Dh, Dh, g.n_heads * n_mid, 128)) return REHYAT_ERR_CUDA;
   PhiTcArgs a = {};
-  a.b1 = (const __nv_bfloat16*)phi->k_b1; a.b2 = (const __nv_bfloat16*)phi->k_b2;
+  a.b1 = (const __nv_bfloat16*)phi->k_b1; a.b2 = (const __nv_bfloat16*)phi->k_b2; a.bm = (const __nv_bfloat16*)phi->k_bmid;
   a.P = P; a.act_hidden = act_hidden; a.act_out = act_out;
-  a.d = d; a.Dh = Dh; a.Dp = Dp;
+  a.d = d; a.Dh = Dh; a.Dp = Dp; a.n_mid = n_mid;
   a.n_split = n_split; a.partial = partial; a.wa = wa;
-  const PhiKernelChoice ch = tc_phi_choice(d, Dh, Dp, P, act_hidden, act_out);
+  const PhiKernelChoice ch = tc_phi_choice(d, Dh, Dp, P, n_mid, act_hidden, act_out);
   const dim3 grid(n_split, g.G, g.BH);
-#define REHYAT_LAUNCH_PHI(R, PC, GEN) phi_tc<R, PC, GEN><<<grid, PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, g, a)
+#define REHYAT_LAUNCH_PHI(R, PC, GEN) phi_tc<R, PC, GEN><<<grid, PH_THREADS, PH_SMEM, st>>>(tk, tv, tw1, tw2, twm, g, a)
   if (ch.gen) { if (ch.relu) REHYAT_LAUNCH_PHI(true, 0, true); else REHYAT_LAUNCH_PHI(false, 0, true); }
   else if (ch.pc == 2) REHYAT_LAUNCH_PHI(true, 2, false);
   else if (ch.relu) REHYAT_LAUNCH_PHI(true, 0, false);
@@ -650,18 +653,20 @@ inline int tc_launch_state(const TcWorkspace* w, const void* k, const void* v, c
 
 // phi_q + linear read-out of one group's queries (Eq. 7, 9, 16).
 inline int tc_launch_readout(const TcWorkspace* w, const void* q, const rehyat_phi_params* phi, const Geo& g, int batch,
-                             int Dh, int Dp, int P, int act_hidden, int act_out, const float* state, float* rd, int rd_rows,
-                             const ptx::WaitArgs& wa, cudaStream_t st) {
+                             int Dh, int Dp, int P, int n_mid, int act_hidden, int act_out, const float* state, float* rd,
+                             int rd_rows, const ptx::WaitArgs& wa, cudaStream_t st) {
   const int d = w->head_dim;
-  CUtensorMap tq, tw1, tw2, ts;
+  CUtensorMap tq, tw1, tw2, twm, ts;
   if (!tc_make_tmap_q(w, &tq, q, g, batch) || !tc_make_tmap_3d(w, &tw1, phi->q_W1, d, Dh, g.n_heads, 128) ||
       !tc_make_tmap_3d(w, &tw2, phi->q_W2, Dh, Dp, g.n_heads, 128) ||
       !tc_make_tmap_3d(w, &ts, w->state_bf16, d, Dp, g.G * g.BH, 64))
     return REHYAT_ERR_CUDA;
   PhiTcArgs a = {};
-  a.b1 = (const __nv_bfloat16*)phi->q_b1; a.b2 = (const __nv_bfloat16*)phi->q_b2;
+  twm = tw2;                                                        // not read without hidden layers in between
+  if (n_mid > 0 && !tc_make_tmap_3d(w, &twm, phi->q_Wmid, Dh, Dh, g.n_heads * n_mid, 128)) return REHYAT_ERR_CUDA;
+  a.b1 = (const __nv_bfloat16*)phi->q_b1; a.b2 = (const __nv_bfloat16*)phi->q_b2; a.bm = (const __nv_bfloat16*)phi->q_bmid;
   a.P = P; a.act_hidden = act_hidden; a.act_out = act_out;
-  a.d = d; a.Dh = Dh; a.Dp = Dp;
+  a.d = d; a.Dh = Dh; a.Dp = Dp; a.n_mid = n_mid;
   a.state = state; a.rd = rd; a.rd_rows = rd_rows; a.wa = wa;
   // One CTA per SM: split a chunk's query tiles over as many CTAs as costs the fewest tile-times over all waves.
   const int tiles = (g.Np + 127) / 128;
@@ -676,9 +681,9 @@ inline int tc_launch_readout(const TcWorkspace* w, const void* q, const rehyat_p
   }
   a.tiles_per_cta = (tiles + best_s - 1) / best_s;
   const int ctas = (tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
-  const PhiKernelChoice ch = tc_phi_choice(d, Dh, Dp, P, act_hidden, act_out);
+  const PhiKernelChoice ch = tc_phi_choice(d, Dh, Dp, P, n_mid, act_hidden, act_out);
   const dim3 grid(ctas, g.G, g.BH);
-#define REHYAT_LAUNCH_RD(R, PC, GEN) readout_tc<R, PC, GEN><<<grid, PH_THREADS, RD_SMEM, st>>>(tq, tw1, tw2, ts, g, a)
+#define REHYAT_LAUNCH_RD(R, PC, GEN) readout_tc<R, PC, GEN><<<grid, PH_THREADS, RD_SMEM, st>>>(tq, tw1, tw2, twm, ts, g, a)
   if (ch.gen) { if (ch.relu) REHYAT_LAUNCH_RD(true, 0, true); else REHYAT_LAUNCH_RD(false, 0, true); }
   else if (ch.pc == 2) REHYAT_LAUNCH_RD(true, 2, false);
   else if (ch.relu) REHYAT_LAUNCH_RD(true, 0, false);

@@ -302,15 +302,17 @@ def test_other_feature_maps_with_heads_of_64(variant):
 
 
 @pytest.mark.parametrize("layers", [3, 4])
-@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
-def test_deeper_feature_maps(layers, dtype):
-    """phi with one or two further hidden layers (rehyat_config.phi_layers): the linear branch runs on the SIMT
-    kernels, the softmax window of the bf16 case on the tensor cores."""
-    wl = synth.Workload("deep", 1, 2, 128, 5, 10, 20, 2, 1, dtype, dtype == "bf16", seed=synth.BASE_SEED + 89,
-                        phi_layers=layers)
+@pytest.mark.parametrize("dtype,d,Dh", [("bf16", 128, 0), ("fp32", 128, 0), ("bf16", 64, 0), ("bf16", 128, 160)],
+                         ids=["bf16", "fp32", "bf16_d64", "bf16_hidden160"])
+def test_deeper_feature_maps(layers, dtype, d, Dh):
+    """phi with one or two further hidden layers (rehyat_config.phi_layers); bf16 runs them on the tensor cores,
+    the hidden activations going from one buffer to the other."""
+    wl = synth.Workload("deep", 1, 2, d, 5, 10, 20, 2, 1, dtype, dtype == "bf16", seed=synth.BASE_SEED + 89,
+                        phi_layers=layers, phi_hidden=Dh)
     # every further layer of std-0.02 parameters shrinks the features: scaled so that about half of the normaliser is linear
-    x = synth.make_inputs(wl, phi_scale={3: 2.0, 4: 2.5}[layers], v_frame_offsets=True)
-    assert x["phi_q"]["Wmid"].shape == (2, layers - 2, 256, 256)
+    scale = {3: 2.0, 4: 2.5}[layers] * ({3: 1.25, 4: 1.5}[layers] if wl.D_h == 128 else 1.0)
+    x = synth.make_inputs(wl, phi_scale=scale, v_frame_offsets=True)
+    assert x["phi_q"]["Wmid"].shape == (2, layers - 2, wl.D_h, wl.D_h)
     f = synth.to_f64(x)
     ref, frac = orc.hybrid_direct(f["q"], f["k"], f["v"], f["phi_q"], f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To,
                                   return_parts=True)
@@ -318,7 +320,7 @@ def test_deeper_feature_maps(layers, dtype):
     two = {n: t for n, t in f["phi_q"].items() if n not in ("Wmid", "bmid")}
     assert np.abs(orc.hybrid_direct(f["q"], f["k"], f["v"], two, f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To) - ref).max() > 1e-2
     y, used = run_gpu(wl, x)
-    assert used == ("tensor" if dtype == "bf16" else "simt") and run_gpu.phi_kernels == "simt"
+    assert used == run_gpu.phi_kernels == ("tensor" if dtype == "bf16" else "simt")
     check(y, ref, dtype)
 
 
