@@ -57,9 +57,10 @@ typedef enum {
  * ("typically the maximum exponent").  ZERO: c = 0 (evaluated stably). */
 typedef enum { REHYAT_C_ROWMAX = 0, REHYAT_C_ZERO = 1 } rehyat_c_mode;
 
-/* Kernel family.  AUTO: tensor-core (tcgen05) kernels when dtype is bf16 and the shape is one
- * they cover (head_dim 128 for the softmax window; D_h = D' = 256 as well for the linear branch),
- * SIMT fp32 kernels otherwise.  SIMT / TENSOR force one (TENSOR fails with REHYAT_ERR_UNSUPPORTED
+/* Kernel family.  AUTO: tensor-core (tcgen05) kernels when dtype is bf16 (head_dim 64 or 128 for
+ * the softmax window; for phi, state and read-out also D_h and D' multiples of 32 with
+ * 64 <= D_h <= 256, 32 <= D' <= 256; other widths keep the window on the tensor cores and run
+ * the linear branch on the fp32 kernels), SIMT fp32 kernels otherwise.  SIMT / TENSOR force one (TENSOR fails with REHYAT_ERR_UNSUPPORTED
  * where it does not apply).  TENSOR_WINDOW: tensor-core window, SIMT linear branch (a cross-check). */
 typedef enum {
   REHYAT_IMPL_AUTO = 0, REHYAT_IMPL_SIMT = 1, REHYAT_IMPL_TENSOR = 2, REHYAT_IMPL_TENSOR_WINDOW = 3
@@ -104,8 +105,7 @@ typedef struct rehyat_config {
                                    experiments; 3 or 4 = one or two further hidden layers
                                    h <- act_hidden(Wmid h + bmid) of width D_h between the two
                                    (Section 4.3 varies the "transformation complexity" of phi).
-                                   Deeper maps run on the SIMT kernels (the softmax window stays
-                                   on the tensor cores).                                       */
+                                   The tensor-core kernels cover them too.                     */
   int32_t qk_transform;         /* 1: the context can normalise and rotate q and k ahead of the
                                    operator (rehyat_set_qk_transform); rehyat_create then also
                                    allocates room for the transformed q and k of max_frames
@@ -286,8 +286,8 @@ int rehyat_set_wait_limit(rehyat_ctx* ctx, int32_t wait_limit_us, int32_t withho
 int rehyat_last_launches(const rehyat_ctx* ctx);
 
 /* Kernels of the last forward: 2 = every step on the tensor cores, 1 = the softmax window on the tensor cores
- * and phi, state and read-out on the fp32 SIMT kernels (a phi map the tensor-core kernels do not cover: more
- * than two layers, widths that are not multiples of 32), 0 = SIMT kernels throughout. */
+ * and phi, state and read-out on the fp32 SIMT kernels (phi widths the tensor-core kernels do not cover, or
+ * REHYAT_IMPL_TENSOR_WINDOW), 0 = SIMT kernels throughout. */
 int rehyat_last_impl(const rehyat_ctx* ctx);
 
 /* Query tiles per work item of the last tensor-core window launch: 2 (window_tc) or 1 (window_tc1);
