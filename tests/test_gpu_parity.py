@@ -238,9 +238,10 @@ def test_invalid_arguments_are_rejected_before_launch():
     assert e.value.code == binding.ERR_UNSUPPORTED
 
 
-def test_host_buffer_entry_point_matches_device_entry_point():
+@pytest.mark.parametrize("d", [128, 64])
+def test_host_buffer_entry_point_matches_device_entry_point(d):
     from paper_2601_04342_b200 import binding
-    wl = synth.Workload("host", 1, 2, 128, 4, 10, 20, 2, 1, "bf16", True, seed=synth.BASE_SEED + 84)
+    wl = synth.Workload("host", 1, 2, d, 4, 10, 20, 2, 1, "bf16", True, seed=synth.BASE_SEED + 84)
     x = synth.make_inputs(wl, phi_scale=1.5)
     y_dev, _ = run_gpu(wl, x)
     op = binding.for_workload(wl)

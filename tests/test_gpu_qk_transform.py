@@ -86,6 +86,7 @@ CASES = [
     synth.Workload("qk_fp32", 1, 2, 64, 4, 8, 8, 1, 1, "fp32", False, seed=synth.BASE_SEED + 96),
     # an odd number of tokens (1071): the last row of the pass has no neighbour in its warp
     synth.Workload("qk_bf16_odd", 1, 2, 128, 7, 9, 17, 3, 1, "bf16", False, seed=synth.BASE_SEED + 98),
+    synth.Workload("qk_bf16_d64", 1, 3, 64, 5, 10, 20, 2, 1, "bf16", False, seed=synth.BASE_SEED + 94),
 ]
 
 

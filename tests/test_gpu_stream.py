@@ -65,7 +65,8 @@ CASES = [
     ("bf16_multi_tile", 1, 2, 128, 7, 10, 20, 2, 1, "bf16"),            # last chunk 1 frame
     ("bf16_no_overlap", 1, 3, 128, 6, 13, 11, 2, 0, "bf16"),
     ("bf16_overlap_ge_chunk", 1, 2, 128, 6, 12, 12, 1, 3, "bf16"),
-    ("bf16_d64_simt", 1, 2, 64, 5, 10, 13, 2, 1, "bf16"),
+    ("bf16_d64", 1, 2, 64, 5, 10, 13, 2, 1, "bf16"),
+    ("bf16_d64_multi_tile", 2, 3, 64, 7, 10, 20, 2, 1, "bf16"),
 ]
 
 
