@@ -43,7 +43,7 @@ def gpu_forward(wl, x, **kw):
     free_before = torch.cuda.mem_get_info()[0]
     op.forward(q, k, v, pq, pk, wl.T, wl.H, wl.W, wl.Tc, wl.To, out=out)
     assert op.status() == 0
-    assert op.last_impl == "tensor" and op.last_launches > 0
+    assert op.last_impl == "tensor" and op.last_phi_impl == "tensor" and op.last_launches > 0
     extra = max(torch.cuda.max_memory_allocated() - before, free_before - torch.cuda.mem_get_info()[0])
     ws = op.workspace_bytes
     op.close()
@@ -165,6 +165,17 @@ def test_head_dim_64_full_length_sampled(tiles):
     x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
     y, _, _ = gpu_forward(wl, x, window_tiles=tiles)
     check_sampled(wl, x, y, [(0, 0), (0, 23)], seed=57)
+
+
+@pytest.mark.parametrize("variant", ["three_layers", "degree3_width192"])
+def test_other_feature_maps_full_length_sampled(variant):
+    """Feature maps other than the default at the full 32,760 tokens, on the tensor-core kernels that read their
+    extents from the arguments: a three-layer map, and P = 3 with D_h = 128, D' = 192 (one and a half halves)."""
+    kw = dict(phi_layers=3) if variant == "three_layers" else dict(P=3, phi_hidden=128, phi_dim=192)
+    wl = synth.CONFIGS["wan13b_layer"].with_(name=variant, seed=synth.BASE_SEED + 58, **kw)
+    x = synth.make_inputs(wl, phi_scale=2.0 if variant == "three_layers" else 1.5, v_frame_offsets=True)
+    y, _, _ = gpu_forward(wl, x)
+    assert check_sampled(wl, x, y, [(0, 1), (0, 10)], seed=58) > 0.05     # the linear branch carries weight
 
 
 # ------------------------------------------------------------------ CFG batch, longer video
