@@ -337,13 +337,21 @@ qk_prepare(const T* __restrict__ q, const T* __restrict__ k, T* __restrict__ qo,
   const unsigned row_lanes = (LPR >= 32 ? 0xffffffffu : ((1u << LPR) - 1u) << ((threadIdx.x & 31) / LPR * LPR));
   // two rows per step, both loaded before either is worked on: twice the bytes in flight per thread
   const int stride = gridDim.x * rows_per_block;
-  for (int row0 = blockIdx.x * rows_per_block + threadIdx.x / LPR; row0 < a.rows; row0 += 2 * stride) {
+  const int first = blockIdx.x * rows_per_block + threadIdx.x / LPR;
+  // the addresses of a thread's rows advance by constants: pointers of the first of the two rows, stepped per turn
+  const T* sp = src + hoff + (long long)first * a.sn + col;
+  T* dp = dst + doff + (long long)first * dn + col;
+  const float* cp = a.cos != nullptr ? a.cos + (size_t)(a.pos0 + first) * (D / 2) + col / 2 : nullptr;
+  const float* np_ = a.cos != nullptr ? a.sin + (size_t)(a.pos0 + first) * (D / 2) + col / 2 : nullptr;
+  const long long s_row = (long long)stride * a.sn, d_row = (long long)stride * dn;       // one row group further
+  const size_t t_row = (size_t)stride * (D / 2);
+  for (int row0 = first; row0 < a.rows; row0 += 2 * stride, sp += 2 * s_row, dp += 2 * d_row, cp += 2 * t_row, np_ += 2 * t_row) {
     float x[2][8];
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
       const int row = row0 + u * stride;
       if (row < a.rows) {
-        const T* p = src + hoff + (long long)row * a.sn + col;
+        const T* p = sp + u * s_row;
         const float4 x0 = ld4(p), x1 = ld4(p + 4);
         x[u][0] = x0.x; x[u][1] = x0.y; x[u][2] = x0.z; x[u][3] = x0.w;
         x[u][4] = x1.x; x[u][5] = x1.y; x[u][6] = x1.z; x[u][7] = x1.w;
@@ -367,8 +375,8 @@ qk_prepare(const T* __restrict__ q, const T* __restrict__ k, T* __restrict__ qo,
       }
       if (row >= a.rows) continue;
       if (a.cos != nullptr) {
-        const float4 c = *reinterpret_cast<const float4*>(a.cos + (size_t)(a.pos0 + row) * (D / 2) + col / 2);
-        const float4 s = *reinterpret_cast<const float4*>(a.sin + (size_t)(a.pos0 + row) * (D / 2) + col / 2);
+        const float4 c = *reinterpret_cast<const float4*>(cp + u * t_row);
+        const float4 s = *reinterpret_cast<const float4*>(np_ + u * t_row);
         const float cs[4] = {c.x, c.y, c.z, c.w}, sn[4] = {s.x, s.y, s.z, s.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -377,7 +385,7 @@ qk_prepare(const T* __restrict__ q, const T* __restrict__ k, T* __restrict__ qo,
           x[u][2 * e + 1] = p0 * sn[e] + p1 * cs[e];
         }
       }
-      st8(dst + doff + (long long)row * dn + col, x[u]);
+      st8(dp + u * d_row, x[u]);
     }
   }
 }
