@@ -34,18 +34,21 @@ def _oracle(wl, x, **kw):
     return orc.hybrid_rnn(f["q"], f["k"], f["v"], f["phi_q"], f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To, P=wl.P, **kw)
 
 
-def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(both_window_kernels):
+@pytest.mark.parametrize("shape", ["default", "heads_of_64", "three_layers"])
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(both_window_kernels, shape):
     """All four tensor-core kernels (state, read-out and either window kernel) run into their wait limit, the
     host reads REHYAT_ERR_DEVICE_TIMEOUT exactly once, and the next forward on the same context gives the bits
-    it gave before."""
+    it gave before.  The default shape runs the fixed-extent phi kernels, the other two the ones that read their
+    extents (64-column tiles; hidden layers in between)."""
     from paper_2601_04342_b200 import binding
-    wl = synth.Workload("timeout", 1, 2, 128, 6, 10, 20, 2, 1, "bf16", True, seed=synth.BASE_SEED + 70)
-    x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
+    d, layers = {"default": (128, 2), "heads_of_64": (64, 2), "three_layers": (128, 3)}[shape]
+    wl = synth.Workload("timeout", 1, 2, d, 6, 10, 20, 2, 1, "bf16", True, seed=synth.BASE_SEED + 70, phi_layers=layers)
+    x = synth.make_inputs(wl, phi_scale=1.5 if layers == 2 else 2.0, v_frame_offsets=True)
     d = _dev(x)
     op = binding.for_workload(wl)
     args = (d["q"], d["k"], d["v"], d["phi_q"], d["phi_k"], wl.T, wl.H, wl.W, wl.Tc, wl.To)
     before = op.forward(*args).clone()
-    assert op.status() == binding.OK and op.last_impl == "tensor"
+    assert op.status() == binding.OK and op.last_impl == op.last_phi_impl == "tensor"
     assert np.abs(before.double().cpu().numpy() - _oracle(wl, x)).max() <= 2e-2
 
     op.set_wait_limit(2000, withhold_loads=True)              # 2 ms per wait, no loads: every launch gives up
