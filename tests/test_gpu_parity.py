@@ -359,3 +359,33 @@ def test_window_items_of_one_tile_edge_shapes():
             y, used = run_gpu(wl, x, c_mode=c_mode)
             assert used == "tensor"
             check(y, ref, "bf16")
+
+
+# ------------------------------------------------------------------ seeded random geometries
+def _random_case(seed):
+    """A small random problem: geometry (chunk and overlap against the frame count, ragged tiles), head size, phi
+    widths and degree, c mode, layout.  Widths are multiples of 32 so that bf16 runs every step on the tensor cores."""
+    rng = np.random.default_rng(1000 + seed)
+    d = int(rng.choice([64, 128]))
+    T = int(rng.integers(2, 9))
+    Tc = int(rng.integers(1, min(T, 4) + 1))
+    To = int(rng.integers(0, 4))
+    H, W = int(rng.integers(3, 13)), int(rng.integers(5, 21))
+    P = int(rng.choice([1, 2, 3, 4]))
+    Dp = int(rng.choice([w for w in (96, 128, 192, 256) if w % P == 0 and (w // P) % 8 == 0]))
+    Dh = int(rng.choice([64, 96, 128, 192, 256]))
+    layers = int(rng.choice([2, 2, 3, 4]))
+    wl = synth.Workload(f"rand{seed}", int(rng.integers(1, 3)), int(rng.integers(1, 4)), d, T, H, W, Tc, To, "bf16", True,
+                        P=P, seed=synth.BASE_SEED + 300 + seed, phi_hidden=Dh, phi_dim=Dp, phi_layers=layers)
+    return wl, str(rng.choice(["rowmax", "zero"])), str(rng.choice(["bhnd", "bnhd"])), {2: 1.5, 3: 2.0, 4: 2.5}[layers]
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_geometries(seed):
+    wl, c_mode, layout, scale = _random_case(seed)
+    x = synth.make_inputs(wl, phi_scale=scale, v_frame_offsets=True)
+    f = synth.to_f64(x)
+    ref = orc.hybrid_direct(f["q"], f["k"], f["v"], f["phi_q"], f["phi_k"], wl.T, wl.HW, wl.Tc, wl.To, P=wl.P, c_mode=c_mode)
+    y, used = run_gpu(wl, x, c_mode=c_mode, layout=layout)
+    assert used == run_gpu.phi_kernels == "tensor", (wl, c_mode, layout)
+    check(y, ref, "bf16")
