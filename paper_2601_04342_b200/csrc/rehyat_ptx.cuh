@@ -54,6 +54,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The same with a suspend-time hint: the thread may stay suspended for up to `hint_ns` before the instruction
+// returns false (it still returns at once when the phase completes).  A role that waits long and often then
+// leaves the issue slots of its scheduler to the warps that share it.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
 
 // Bounded waits.  Every spin on an mbarrier in the tensor-core kernels goes through mbar_wait: it gives up after
 // `limit_ns` of wall time, records `code` in the sticky status word status[0] and publishes the launch's epoch in
@@ -97,10 +111,10 @@ __device__ __forceinline__ int wait_ctx_aborted(uint32_t wctx) {     // abort_fl
 // The slow path is on the critical path of the roles that wait often (a try_wait that fails returns within a few
 // hundred cycles), so it polls the barrier and the CTA's abort flag only; the global epoch and the timer are
 // looked at once per 1024 polls (some tens of microseconds).
-__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t wctx, int code) {
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint32_t wctx, int code, uint32_t hint_ns) {
   const unsigned long long t0 = global_timer_ns();
   for (uint32_t i = 1;; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (hint_ns ? mbar_try_wait_hint(bar, parity, hint_ns) : mbar_try_wait(bar, parity)) return true;
     if (wait_ctx_aborted(wctx)) return false;
     if ((i & 1023u) == 0u) {
       volatile WaitCtx* w = reinterpret_cast<volatile WaitCtx*>(__cvta_shared_to_generic(wctx));
@@ -115,9 +129,11 @@ __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, ui
     }
   }
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t wctx, int code) {
+// hint_ns: suspend-time hint of the polls after the first (0: none); the time limit is then looked at once per
+// 1024 * hint_ns at most.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t wctx, int code, uint32_t hint_ns = 0) {
   if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, wctx, code);
+  return mbar_wait_slow(bar, parity, wctx, code, hint_ns);
 }
 // Wait of a role for what it has itself put in flight (its TMA loads, its tcgen05.mma through a commit) before
 // the CTA may free TMEM and exit.  The abort flag does not cut it short; only the time limit does.

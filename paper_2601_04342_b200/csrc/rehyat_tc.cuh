@@ -47,6 +47,12 @@ struct WinShape {
 };
 
 enum TcErr : int { TC_ERR_LOAD = 1, TC_ERR_MMA = 2, TC_ERR_SOFTMAX = 4 };
+// Suspend-time hints (ns) of the waits of the TMA producer, of the MMA issuer and of the softmax warps.  The first
+// two roles wait most of the time; without a hint their polling takes issue slots from the softmax warps that share
+// their schedulers, whose tiles then end 140 - 210 cycles after those of the other two schedulers (measured with
+// clock64 stamps), and the hand-over waits for the slowest warp.  With the hints the window kernel is 1.5 % faster;
+// longer hints (10, 100 us) and a hint on the softmax warps' own waits change nothing more.
+constexpr uint32_t TC_HINT_P = 1000, TC_HINT_I = 1000, TC_HINT_S = 0;
 
 struct WinBars {   // offsets (bytes) inside the barrier block
   uint64_t q_full, q_empty;
@@ -272,7 +278,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         WinItem w;
         if (!win_item(g, item, pairs, w)) continue;
         // Q of the previous item has been read by its last Q K^T
-        if (n_q > 0) alive = mbar_wait(smem_u32(&bars->q_empty), (n_q - 1) & 1, wc, TC_ERR_LOAD);
+        if (n_q > 0) alive = mbar_wait(smem_u32(&bars->q_empty), (n_q - 1) & 1, wc, TC_ERR_LOAD, TC_HINT_P);
         if (!alive) break;
         const uint32_t qf = smem_u32(&bars->q_full);
         mbar_expect_tx(qf, w.ntiles * TC_TILE_BYTES);
@@ -282,13 +288,13 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           const int s = n_k % TC_STAGES;
           const uint32_t ph = (n_k / TC_STAGES) & 1;
           const int key0 = w.lo + j * TC_BN;
-          alive = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1, wc, TC_ERR_LOAD);
+          alive = mbar_wait(smem_u32(&bars->k_empty[s]), ph ^ 1, wc, TC_ERR_LOAD, TC_HINT_P);
           if (!alive) break;
           const uint32_t kf = smem_u32(&bars->k_full[s]);
           mbar_expect_tx(kf, TC_TILE_BYTES);
           load_tile(sK + s * TC_TILE_BYTES, &tm_k, kf, key0, w.h_idx, w.b_idx);
           ++n_k;
-          alive = mbar_wait(smem_u32(&bars->v_empty[s]), ph ^ 1, wc, TC_ERR_LOAD);
+          alive = mbar_wait(smem_u32(&bars->v_empty[s]), ph ^ 1, wc, TC_ERR_LOAD, TC_HINT_P);
           if (!alive) break;
           const uint32_t vf = smem_u32(&bars->v_full[s]);
           mbar_expect_tx(vf, TC_TILE_BYTES);
@@ -316,7 +322,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       uint32_t n_p[TC_QT] = {0, 0}, n_o[TC_QT] = {0, 0};             // P hand-overs and items per query tile
       bool alive = true;                                             // false once a wait has been given up: issue nothing more
       auto wait = [&](uint64_t* bar, uint32_t parity) {
-        alive = alive && mbar_wait(smem_u32(bar), parity, wc, TC_ERR_MMA);
+        alive = alive && mbar_wait(smem_u32(bar), parity, wc, TC_ERR_MMA, TC_HINT_I);
         return alive;
       };
       for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
@@ -381,7 +387,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     // need all 32 lanes), so every wait is followed by a vote.
     bool alive = true;
     auto wait = [&](uint64_t* bar, uint32_t parity) {
-      alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, wc, TC_ERR_SOFTMAX));
+      alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, wc, TC_ERR_SOFTMAX, TC_HINT_S));
       return alive;
     };
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {

@@ -106,7 +106,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         WinItem w;
         if (!win_item1(g, item, tiles, w)) continue;
         // Q of the previous item has been read by its last Q K^T
-        if (n_q > 0) alive = mbar_wait(smem_u32(&bars->q_empty), (n_q - 1) & 1, wc, TC_ERR_LOAD);
+        if (n_q > 0) alive = mbar_wait(smem_u32(&bars->q_empty), (n_q - 1) & 1, wc, TC_ERR_LOAD, TC_HINT_P);
         if (!alive) break;
         const uint32_t qf = smem_u32(&bars->q_full);
         mbar_expect_tx(qf, TC_TILE_BYTES);
@@ -118,7 +118,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           const int s = it % TC_STAGES;
           const uint32_t ph = (it / TC_STAGES) & 1;
           const int key0 = w.lo + j * TC_BN;
-          if (!mbar_wait(smem_u32(is_v ? &bars->v_empty[s] : &bars->k_empty[s]), ph ^ 1, wc, TC_ERR_LOAD))
+          if (!mbar_wait(smem_u32(is_v ? &bars->v_empty[s] : &bars->k_empty[s]), ph ^ 1, wc, TC_ERR_LOAD, TC_HINT_P))
             return false;
           const uint32_t full = smem_u32(is_v ? &bars->v_full[s] : &bars->k_full[s]);
           const uint32_t dst = (is_v ? sV : sK) + s * TC_TILE_BYTES;
@@ -157,7 +157,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       uint32_t n_p[2] = {0, 0};                                      // P hand-overs per slot
       bool alive = true;                                             // false once a wait has been given up: issue nothing more
       auto wait = [&](uint64_t* bar, uint32_t parity) {
-        alive = alive && mbar_wait(smem_u32(bar), parity, wc, TC_ERR_MMA);
+        alive = alive && mbar_wait(smem_u32(bar), parity, wc, TC_ERR_MMA, TC_HINT_I);
         return alive;
       };
       for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
@@ -216,7 +216,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     // A wait that was given up ends the role; the warp decides together (tcgen05.ld / st need all 32 lanes).
     bool alive = true;
     auto wait = [&](uint64_t* bar, uint32_t parity) {
-      alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, wc, TC_ERR_SOFTMAX));
+      alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(bar), parity, wc, TC_ERR_SOFTMAX, TC_HINT_S));
       return alive;
     };
     for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
