@@ -156,13 +156,13 @@ __device__ __forceinline__ bool softmax_key_tile(uint32_t tS, uint32_t tO, int n
         if (cc * 32 + e >= n_valid) sr[cc][e] = 0xff800000u;   // -inf
   }
   // row maximum: four independent chains of three-input max
-  float mx[4] = {st.m_true, st.m_true, st.m_true, st.m_true};
+  float mx[8] = {st.m_true, st.m_true, st.m_true, st.m_true, st.m_true, st.m_true, st.m_true, st.m_true};
 #pragma unroll
   for (int cc = 0; cc < 4; ++cc)
 #pragma unroll
     for (int e = 0; e < 32; e += 2)
-      mx[cc] = fmax3(mx[cc], __uint_as_float(sr[cc][e]), __uint_as_float(sr[cc][e + 1]));
-  st.m_true = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+      mx[cc * 2 + ((e >> 1) & 1)] = fmax3(mx[cc * 2 + ((e >> 1) & 1)], __uint_as_float(sr[cc][e]), __uint_as_float(sr[cc][e + 1]));
+  st.m_true = fmaxf(fmax3(mx[0], mx[1], mx[2]), fmax3(fmaxf(mx[3], mx[4]), fmaxf(mx[5], mx[6]), mx[7]));
   const bool need = (st.m_true - st.m_used) * c > 8.f;               // true on the first tile (m_used = -inf)
   if (__any_sync(0xffffffffu, need)) {
     const float m_new = need ? st.m_true : st.m_used;
