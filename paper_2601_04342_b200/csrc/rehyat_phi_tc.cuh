@@ -40,7 +40,7 @@ constexpr int PH_SUB = PH_TILE_BYTES / 2;
 // shared memory map (bytes from the 1024-aligned base)
 constexpr int PH_OFF_X = 0;
 constexpr int PH_OFF_V = PH_OFF_X + PH_TILE_BYTES;
-constexpr int PH_OFF_HB = PH_OFF_V + PH_TILE_BYTES;            // 64 KB; its first half doubles as phi half 1
+constexpr int PH_OFF_HB = PH_OFF_V + PH_TILE_BYTES;            // 64 KB; one of its halves doubles as phi half 1
 constexpr int PH_OFF_PHI0 = PH_OFF_HB + 2 * PH_TILE_BYTES;
 constexpr int PH_OFF_RING = PH_OFF_PHI0 + PH_TILE_BYTES;
 constexpr int PH_OFF_ONES = PH_OFF_RING + PH_RING * PH_WT_BYTES; // [16 x 128] K-major, row 0 = 1
@@ -176,6 +176,10 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
   };
   const int last_hid = n_mid & 1;                                   // where the last hidden activations are
   const uint32_t sPhiHalf0 = last_hid ? sHb + 2 * PH_SUB : sPhi0;   // phi half 0: away from the buffer the last GEMMs read
+  // phi half 1 takes a half of the H buffer once the last GEMM has read it.  Where the first layer writes that
+  // buffer again (last_hid == 0) it is the second half: the first half-GEMM of the next tile and its epilogue (which
+  // writes the first half) then need not wait for the state GEMM that reads phi half 1.
+  const uint32_t sPhiHalf1 = last_hid ? sHb : sHb + 2 * PH_SUB;
 
   if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
@@ -281,13 +285,19 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
       auto run = [&]() {
         for (int j = 0; j < n_tiles; ++j) {
           if (!wait(&bars->x_full, j & 1)) return;
-          if (j > 0 && nu == 2) {
-            if (!wait_epi()) return;                                  // scratch free: phi half 1 of tile j-1 written
-            if (!wait(&bars->v_full, (j - 1) & 1)) return;            // ... and consumed
-            consume_half(1, sHb, j == 1);
+          const bool owe_half1 = j > 0 && nu == 2;                    // phi half 1 of tile j-1 is not yet in the state
+          if (owe_half1 && !wait_epi()) return;                       // scratch free: phi half 1 of tile j-1 written
+          if (owe_half1 && last_hid == 1) {
+            if (!wait(&bars->v_full, (j - 1) & 1)) return;
+            consume_half(1, sPhiHalf1, j == 1);
             umma_commit(smem_u32(&bars->v_empty));
           }
           if (!mlp_half(-1, ks1)) return;                             // H[:, 0:128]
+          if (owe_half1 && last_hid == 0) {                           // behind the half-GEMM: it runs during that half's epilogue
+            if (!wait(&bars->v_full, (j - 1) & 1)) return;
+            consume_half(1, sPhiHalf1, j == 1);
+            umma_commit(smem_u32(&bars->v_empty));
+          }
           if (!wait_epi()) return;
           if (nh == 2 && !mlp_half(-1, ks1)) return;                  // H[:, 128:256]
           // The X tile is free after its last reader: the first layer, or the last GEMMs that read hidden buffer 1.
@@ -310,7 +320,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
         }
         if (nu == 2) {
           if (!wait_epi()) return;
-          consume_half(1, sHb, n_tiles == 1);
+          consume_half(1, sPhiHalf1, n_tiles == 1);
         }
         umma_commit(smem_u32(&bars->out_ready));
       };
@@ -419,7 +429,7 @@ phi_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtenso
           if (half < nh) epi_step(false, half, s_b2 + (1 + m) * 256 + half * 128, hid_sub((m & 1) ^ 1, half * 2 + ch));
 #pragma unroll
       for (int half = 0; half < 2; ++half)                          // last layer -> the phi tiles
-        if (half < nu) epi_step(true, half, s_b2 + half * 128, (half == 0 ? sPhiHalf0 : sHb) + ch * PH_SUB);
+        if (half < nu) epi_step(true, half, s_b2 + half * 128, (half == 0 ? sPhiHalf0 : sPhiHalf1) + ch * PH_SUB);
     }
     wait(&bars->out_ready, 0);
     if (!aborted()) {
