@@ -415,7 +415,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
       }
       // U halves: bias, activation, power, bf16, to the swizzled phi tiles; phi . z_t on the way
       const bool tok_valid = tok_a + j * 128 + r < tok_b;
-      float nl = 0.f;
+      float nl4[4] = {0.f, 0.f, 0.f, 0.f};                          // four chains: the sum is not one dependent sequence
 #pragma unroll 1
       for (int half = 0; half < nu; ++half) {
         wait_acc(half);
@@ -439,8 +439,8 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
             const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-              nl = fmaf(__uint_as_float(ww[u] << 16), zz[2 * u], nl);
-              nl = fmaf(__uint_as_float(ww[u] & 0xffff0000u), zz[2 * u + 1], nl);
+              nl4[u] = fmaf(__uint_as_float(ww[u] << 16), zz[2 * u], nl4[u]);
+              nl4[u] = fmaf(__uint_as_float(ww[u] & 0xffff0000u), zz[2 * u + 1], nl4[u]);
             }
             st_tile_chunk_sw128(dst, PH_SUB, r, ch * 64 + cb * 16 + e, w4);
           }
@@ -449,7 +449,7 @@ readout_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
           // The buffer alternates with the tile.  It is free: its last reader (read-out store of tile j-2)
           // precedes, for every thread, that thread's arrival for U half 0 of tile j-1, which the issuer
           // waited for before the MMAs of this tile could start.
-          s_nl[(j & 1) * 256 + ch * 128 + r] = nl;
+          s_nl[(j & 1) * 256 + ch * 128 + r] = (nl4[0] + nl4[1]) + (nl4[2] + nl4[3]);
           mbar_arrive_warp(smem_u32(&bars->nl_ready), lane);
         }
         fence_proxy_async_smem();
