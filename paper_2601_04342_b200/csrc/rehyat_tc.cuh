@@ -47,6 +47,11 @@ struct WinShape {
 };
 
 enum TcErr : int { TC_ERR_LOAD = 1, TC_ERR_MMA = 2, TC_ERR_SOFTMAX = 4 };
+// One 32-byte store (a whole sector) of sixteen bf16; the address must be 32-byte aligned.
+__device__ __forceinline__ void st_global_32B(void* p, uint4 a, uint4 b) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
+}
 // Suspend-time hints (ns) of the waits of the TMA producer, of the MMA issuer and of the softmax warps.  The first
 // two roles wait most of the time; without a hint their polling takes issue slots from the softmax warps that share
 // their schedulers, whose tiles then end 140 - 210 cycles after those of the other two schedulers (measured with
@@ -382,6 +387,8 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_off + i * TC_BN, tO = tmem + lane_off + 256 + i * 128;
     const float c = scale * 1.4426950408889634f;                     // logits -> log2 domain
+    const bool out_32B = ((reinterpret_cast<uintptr_t>(out) | (uintptr_t)(g.ostride_b * 2) | (uintptr_t)(g.ostride_h * 2) |
+                           (uintptr_t)(g.ostride_n * 2)) & 31u) == 0;   // every row of out starts on a 32-byte boundary
     uint32_t n_s = 0;                                                // key tiles this query tile has been through
     // A wait that was given up ends the role.  The warp decides together (tcgen05.ld / st and the votes below
     // need all 32 lanes), so every wait is followed by a vote.
@@ -449,6 +456,7 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           mbar_arrive_warp(smem_u32(&bars->o_free[i]), lane);
         }
         if (valid) {
+          uint4 v4[4];
 #pragma unroll
           for (int e = 0; e < 32; e += 8) {
             const uint4 x = rdv[hh * 4 + (e >> 3)];                  // eight columns of aL / nL as fp16 pairs
@@ -456,12 +464,19 @@ window_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
               const float2 rr = unpack_f16(pair);
               return pack_bf16(__uint_as_float(o[q]) * wsi + lami * rr.x, __uint_as_float(o[q + 1]) * wsi + lami * rr.y);
             };
-            uint4 v4;
-            v4.x = fin(e + 0, x.x);
-            v4.y = fin(e + 2, x.y);
-            v4.z = fin(e + 4, x.z);
-            v4.w = fin(e + 6, x.w);
-            *reinterpret_cast<uint4*>(orow + hh * 32 + e) = v4;
+            v4[e >> 3].x = fin(e + 0, x.x);
+            v4[e >> 3].y = fin(e + 2, x.y);
+            v4[e >> 3].z = fin(e + 4, x.z);
+            v4[e >> 3].w = fin(e + 6, x.w);
+          }
+          // a thread writes its own row: whole 32-byte sectors where the output allows it (every lane of a store
+          // touches another row, so nothing merges on the way)
+          if (out_32B) {
+            st_global_32B(orow + hh * 32, v4[0], v4[1]);
+            st_global_32B(orow + hh * 32 + 16, v4[2], v4[3]);
+          } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) *reinterpret_cast<uint4*>(orow + hh * 32 + u * 8) = v4[u];
           }
         }
       }

@@ -180,3 +180,25 @@ def test_a_layer_split_over_three_ranks_equals_the_layer_in_one_call():
         assert torch.equal(changed, mine)                     # exactly this rank's blocks were written
         sh.close()
     assert torch.equal(out, whole)
+
+
+def test_output_that_starts_off_a_32_byte_boundary(both_window_kernels):
+    """The window kernel writes whole 32-byte sectors where every output row starts on a 32-byte boundary and
+    16-byte pieces otherwise (the ABI asks for 16-byte alignment only): both forms give the same bits."""
+    from paper_2601_04342_b200 import binding
+    wl = synth.Workload("align", 1, 2, 128, 5, 10, 20, 2, 1, "bf16", True, seed=synth.BASE_SEED + 76)
+    x = synth.make_inputs(wl, phi_scale=1.5, v_frame_offsets=True)
+    d = _dev(x)
+    op = binding.for_workload(wl)
+    args = (d["q"], d["k"], d["v"], d["phi_q"], d["phi_k"], wl.T, wl.H, wl.W, wl.Tc, wl.To)
+    aligned = op.forward(*args).clone()
+    assert aligned.data_ptr() % 32 == 0
+    flat = torch.full((d["q"].numel() + 16,), float("nan"), device="cuda", dtype=d["q"].dtype)
+    shifted = flat[8:8 + d["q"].numel()].view_as(d["q"])          # 16 bytes further: rows no longer start on 32 bytes
+    assert shifted.data_ptr() % 32 == 16
+    op.forward(*args, out=shifted)
+    assert op.status() == binding.OK
+    assert torch.equal(shifted, aligned)
+    assert bool(torch.isnan(flat[:8]).all()) and bool(torch.isnan(flat[8 + d["q"].numel():]).all())
+    assert np.abs(aligned.double().cpu().numpy() - _oracle(wl, x)).max() <= 2e-2
+    op.close()
