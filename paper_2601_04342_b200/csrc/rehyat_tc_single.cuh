@@ -210,6 +210,8 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_off + i * TC_BN, tO = tmem + lane_off + 256 + i * 128;
     const float c = scale * 1.4426950408889634f;                     // logits -> log2 domain
+    const bool out_32B = ((reinterpret_cast<uintptr_t>(out) | (uintptr_t)(g.ostride_b * 2) | (uintptr_t)(g.ostride_h * 2) |
+                           (uintptr_t)(g.ostride_n * 2)) & 31u) == 0;   // every row of out starts on a 32-byte boundary
     const int r = (warp & 3) * 32 + lane;                            // row of the query tile
     uint32_t n_s[2] = {0, 0};                                        // key tiles each slot has been through
     uint32_t n_items_done = 0;
@@ -298,6 +300,7 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           mbar_arrive_warp(smem_u32(&bars->o_free[i]), lane);
         }
         if (valid) {
+          uint4 v4[4];
 #pragma unroll
           for (int e = 0; e < 32; e += 8) {
             const uint4 x = rdv[hh * 4 + (e >> 3)];                  // eight columns of aL / nL as fp16 pairs
@@ -306,12 +309,17 @@ window_tc1(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               return pack_bf16(__uint_as_float(o0[q]) * w0 + __uint_as_float(o1[q]) * w1 + lami * rr.x,
                                __uint_as_float(o0[q + 1]) * w0 + __uint_as_float(o1[q + 1]) * w1 + lami * rr.y);
             };
-            uint4 v4;
-            v4.x = fin(e + 0, x.x);
-            v4.y = fin(e + 2, x.y);
-            v4.z = fin(e + 4, x.z);
-            v4.w = fin(e + 6, x.w);
-            *reinterpret_cast<uint4*>(orow + hh * 32 + e) = v4;
+            v4[e >> 3].x = fin(e + 0, x.x);
+            v4[e >> 3].y = fin(e + 2, x.y);
+            v4[e >> 3].z = fin(e + 4, x.z);
+            v4[e >> 3].w = fin(e + 6, x.w);
+          }
+          if (out_32B) {                                             // whole 32-byte sectors, as in window_tc
+            st_global_32B(orow + hh * 32, v4[0], v4[1]);
+            st_global_32B(orow + hh * 32 + 16, v4[2], v4[3]);
+          } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) *reinterpret_cast<uint4*>(orow + hh * 32 + u * 8) = v4[u];
           }
         }
       }
